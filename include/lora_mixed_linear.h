@@ -1,0 +1,189 @@
+/*
+ * lora_mixed_linear.h — C ABI of the B200 (sm_100a) mixed-adapter LoRA linear layer.
+ *
+ * The operation.  A batch of T tokens from several agents shares one frozen base weight W0
+ * and every token is bound to one resident (adapter, version) entry of an adapter slot
+ * table, or to none:
+ *
+ *     y[t][n] = sum_k x[t][k] W0[n][k]  +  scale_s * sum_j ( sum_k x[t][k] A_s[j][k] ) B_s[n][j]
+ *
+ * with s the entry of token t; a token bound to no adapter (slot -1) gets the first sum only.
+ * Source of the problem statement: the paper's Section 2 ("LoRA adapters": low-rank modules
+ * on a shared frozen base; requests routed to the correct adapter; updates published
+ * atomically, never partially visible), Section 4.2 (inference binds the last committed
+ * adapter version, staged state stays private until published), Section 5.1 (validity key:
+ * the adapter names the LoRA slot, the adapter version the committed state) and Section 5.3
+ * (an old version keeps serving while work for the newly trained version already runs, so
+ * both are resident at once).  One physical slot of the table = one resident
+ * (adapter_id, version) pair; two versions of one adapter occupy two slots.
+ *
+ * Conventions for every call below
+ *   - All matrices are row-major bf16:  x[T][d_in], W0[d_out][d_in], A[rank][d_in],
+ *     B[d_out][rank], y[T][d_out].  Accumulation is fp32; y is rounded once to bf16 (nearest
+ *     even).  The shrink result u = scale*(x.A^T) is rounded to bf16 before the expand.
+ *   - "device pointer" = memory of the table's CUDA device; "host pointer" = ordinary host
+ *     memory.  Device pointers must be 16-byte aligned; d_in and d_out are multiples of 8.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - The library never allocates, frees or keeps x, W0, y or the workspace: the caller owns
+ *     them and must keep them alive until the stream work has finished.  The table owns only
+ *     its own packed copy of the registered adapters and a status word.
+ *   - Errors are return codes; nothing throws, aborts or traps.  An error detected on the
+ *     host returns before anything is launched and leaves the table unchanged.  Errors only
+ *     visible on the device (an unknown or retired slot id in slot_ids, malformed
+ *     seg_offsets, a perm entry outside [0,T), a bounded wait that ran out) set a sticky bit
+ *     in the table's device status word; the affected tokens get the base output only
+ *     (malformed seg_offsets: every token of that call), and the kernels finish normally.
+ *   - lora_mixed_linear, lml_segment_tokens and lora_mixed_linear_host neither allocate nor
+ *     synchronise nor read device memory from the host.
+ *   - Calls that use the same workspace, or the same table from different streams without
+ *     ordering between them, race; one table may be shared by ordered streams.
+ *   - Same inputs give bitwise the same y on every run (no atomics touch y).
+ */
+#ifndef LORA_MIXED_LINEAR_H_
+#define LORA_MIXED_LINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lml_table lml_table; /* adapter slot table of ONE linear site (fixed d_in, d_out) */
+
+typedef enum {
+    LML_OK = 0,
+    LML_ERR_INVALID_ARG = 1, /* null / misaligned pointer, negative size, rank outside [1,64], ... */
+    LML_ERR_BAD_SLOT = 2,
+    LML_ERR_TABLE_FULL = 3,
+    LML_ERR_DUPLICATE = 4,   /* (adapter_id, version) already resident */
+    LML_ERR_NOT_FOUND = 5,
+    LML_ERR_UNSUPPORTED = 6, /* device is not sm_100 */
+    LML_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed */
+    LML_ERR_TIMEOUT = 8,
+    LML_ERR_WORKSPACE = 9    /* workspace missing, misaligned or smaller than lml_workspace_bytes */
+} lml_status;
+
+/* bits of the device status word (lml_device_status) */
+#define LML_FLAG_BAD_SLOT 1u    /* slot id >= max_slots or not live: tokens got base output only  */
+#define LML_FLAG_BAD_OFFSETS 2u /* seg_offsets not 0-based / monotone / ending at T: base only     */
+#define LML_FLAG_BAD_PERM 4u    /* perm entry outside [0,T): that position was skipped             */
+#define LML_FLAG_TIMEOUT 8u     /* a bounded in-kernel wait gave up                                */
+
+#define LML_MAX_SLOTS 64  /* upper bound for max_slots */
+#define LML_MAX_RANK 64   /* upper bound for an adapter's rank */
+#define LML_DECODE_MAX_TOKENS 16 /* T <= this takes the bandwidth-bound decode kernels */
+
+const char* lml_status_string(lml_status s);
+
+/*
+ * Create the slot table of one linear site on CUDA device `device`.
+ * Allocates (once, here) the packed adapter arena: max_slots * 64 * (d_in + d_out) bf16, plus
+ * a few hundred bytes.  1 <= max_slots <= LML_MAX_SLOTS; d_in, d_out > 0 and multiples of 8.
+ * Errors: INVALID_ARG, UNSUPPORTED (not compute capability 10.x), CUDA.
+ */
+lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, int max_slots);
+
+/* Free the table and its arena.  The caller makes sure no enqueued work still uses it. */
+lml_status lml_table_destroy(lml_table* t);
+
+/*
+ * register_adapter — make (adapter_id, version) resident (the paper's "publish a staged
+ * version": Section 4.2 / 5.3; a newer version is registered while the older one still
+ * serves).  A: device bf16 [rank][d_in]; B: device bf16 [d_out][rank]; 1 <= rank <= 64;
+ * scale is the final multiplier (the library never divides by rank).  The adapter is copied
+ * into the table's arena in the layout the kernels read (rows zero-padded to rank 64) by a
+ * small kernel enqueued on `stream`; A and B may be released once that stream work is done.
+ * The new entry is visible to calls issued after this returns; work on OTHER streams must be
+ * ordered after `stream` by the caller.  *slot_out receives the physical slot index to use in
+ * slot_ids / token_slots (lowest free index).  A rejected call changes nothing: no
+ * half-registered entry is ever visible.
+ * Errors: INVALID_ARG, DUPLICATE, TABLE_FULL, CUDA.
+ */
+lml_status register_adapter(lml_table* t, int adapter_id, int version, const void* A, const void* B,
+                            int rank, float scale, void* stream, int* slot_out);
+
+/*
+ * retire_version — drop a resident (adapter_id, version) entry (Section 5.3: the old version
+ * goes away once in-flight work bound to it is done).  Host-side and immediate for later
+ * calls; work already enqueued keeps the slot description it was launched with, but the
+ * slot's arena space may be reused by the next register_adapter, so retire only after work
+ * bound to that slot has been ordered before the registering stream.  Other slots keep their
+ * indices.  Errors: INVALID_ARG, NOT_FOUND.
+ */
+lml_status retire_version(lml_table* t, int adapter_id, int version);
+
+/* Slot index of a resident (adapter_id, version).  Errors: INVALID_ARG, NOT_FOUND. */
+lml_status lml_lookup(const lml_table* t, int adapter_id, int version, int* slot_out);
+
+/* rank / scale / (adapter_id, version) of a slot; any out pointer may be NULL.
+ * Errors: INVALID_ARG, BAD_SLOT (index out of range or slot free). */
+lml_status lml_slot_info(const lml_table* t, int slot, int* adapter_id, int* version, int* rank,
+                         float* scale);
+
+/*
+ * Bytes of device workspace lora_mixed_linear needs for T <= max_tokens and G <= max_segments
+ * (with or without perm).  Contents need no initialisation and carry nothing between calls.
+ * Returns 0 on invalid arguments.
+ */
+size_t lml_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
+
+/*
+ * lml_segment_tokens — the token-segmentation pass: group T tokens by slot.
+ * token_slots: device int32[T], physical slot per token or -1 (no adapter).
+ * Outputs (device): perm int32[T] (position -> token row); seg_offsets int32[max_slots + 2];
+ * seg_slot_ids int32[max_slots + 1].  Always exactly G = max_slots + 1 segments are produced:
+ * segment i < max_slots holds the tokens of slot i (possibly none), the last segment holds
+ * the -1 tokens; so G is known on the host without reading device memory.  The grouping is
+ * stable: tokens keep their relative order inside a segment.  Ids outside [-1, max_slots)
+ * or naming a free slot go to the -1 group and set LML_FLAG_BAD_SLOT.
+ * T == 0 is valid (all offsets 0).  Errors: INVALID_ARG, CUDA.
+ */
+lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, int32_t* perm,
+                              int32_t* seg_offsets, int32_t* seg_slot_ids, void* stream);
+
+/*
+ * lora_mixed_linear — the layer.  x: device bf16 [T][d_in]; W0: device bf16 [d_out][d_in];
+ * y: device bf16 [T][d_out], overwritten.  seg_offsets: device int32[G+1] with
+ * seg_offsets[0] = 0 <= ... <= seg_offsets[G] = T; slot_ids: device int32[G], physical slot
+ * or -1 per segment (repeated slots, empty segments and any order are fine).  Segment g
+ * covers positions [seg_offsets[g], seg_offsets[g+1]); position p is row perm[p] of x and y
+ * if perm (device int32[T], a permutation) is given, else row p.  G == 0 means "no adapter
+ * anywhere".  T == 0 returns LML_OK without launching.
+ * T <= 16 runs the bandwidth-bound decode kernels (W0 read once with 128-bit loads); larger
+ * T runs the TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
+ * Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
+                             const int32_t* seg_offsets, const int32_t* slot_ids, int G,
+                             const int32_t* perm, void* y, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
+ * Host-buffer form of the same call, for callers whose activations live in host memory.
+ * x_host, seg_offsets_host, slot_ids_host, perm_host (may be NULL), y_host are HOST pointers
+ * (pinned memory makes the copies asynchronous); W0 stays a device pointer (resident
+ * weight).  The call enqueues on `stream`: copies in, the layer, the copy of y out.  The
+ * device staging lives in `workspace`, which must hold lml_host_workspace_bytes().  y_host
+ * is valid once the stream has been synchronised.  Errors as lora_mixed_linear.
+ */
+size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
+lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* W0, int T,
+                                  const int32_t* seg_offsets_host, const int32_t* slot_ids_host,
+                                  int G, const int32_t* perm_host, void* y_host, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
+/*
+ * Read and clear the sticky device status word (LML_FLAG_* bits).  Synchronises `stream`.
+ * Errors: INVALID_ARG, CUDA.
+ */
+lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream);
+
+/* Number of kernels the last lora_mixed_linear / lml_segment_tokens call on this table
+ * launched (for launch accounting in benchmarks). */
+int lml_last_launch_count(const lml_table* t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORA_MIXED_LINEAR_H_ */

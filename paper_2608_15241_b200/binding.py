@@ -1,0 +1,274 @@
+"""Thin ctypes binding of the C-ABI library (include/lora_mixed_linear.h).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.
+PyTorch supplies device memory and streams.  There is no CPU fallback: if the shared
+library is missing, or a call returns an error status, this module raises.
+
+Module-level functions carry the C names (lml_table_create, register_adapter,
+retire_version, lml_segment_tokens, lora_mixed_linear, ...) and take raw pointers/ints;
+`Table` wraps them for torch tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblora_mixed_linear.so")
+
+LML_OK = 0
+STATUS_NAMES = {0: "LML_OK", 1: "LML_ERR_INVALID_ARG", 2: "LML_ERR_BAD_SLOT", 3: "LML_ERR_TABLE_FULL",
+                4: "LML_ERR_DUPLICATE", 5: "LML_ERR_NOT_FOUND", 6: "LML_ERR_UNSUPPORTED",
+                7: "LML_ERR_CUDA", 8: "LML_ERR_TIMEOUT", 9: "LML_ERR_WORKSPACE"}
+FLAG_BAD_SLOT, FLAG_BAD_OFFSETS, FLAG_BAD_PERM, FLAG_TIMEOUT = 1, 2, 4, 8
+MAX_SLOTS, MAX_RANK, DECODE_MAX_TOKENS = 64, 64, 16
+
+EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "register_adapter",
+           "retire_version", "lml_lookup", "lml_slot_info", "lml_workspace_bytes",
+           "lml_segment_tokens", "lora_mixed_linear", "lml_host_workspace_bytes",
+           "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count")
+
+
+class LmlError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with "
+                              "`python -m paper_2608_15241_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.lml_status_string.restype = ctypes.c_char_p
+        L.lml_status_string.argtypes = [i32]
+        L.lml_table_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32]
+        L.lml_table_destroy.argtypes = [vp]
+        L.register_adapter.argtypes = [vp, i32, i32, vp, vp, i32, ctypes.c_float, vp, ctypes.POINTER(i32)]
+        L.retire_version.argtypes = [vp, i32, i32]
+        L.lml_lookup.argtypes = [vp, i32, i32, ctypes.POINTER(i32)]
+        L.lml_slot_info.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                    ctypes.POINTER(ctypes.c_float)]
+        L.lml_workspace_bytes.restype = sz
+        L.lml_workspace_bytes.argtypes = [vp, i32, i32]
+        L.lml_host_workspace_bytes.restype = sz
+        L.lml_host_workspace_bytes.argtypes = [vp, i32, i32]
+        L.lml_segment_tokens.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.lora_mixed_linear.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.lora_mixed_linear_host.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.lml_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+        L.lml_last_launch_count.argtypes = [vp]
+        for name in EXPORTS:
+            if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes"):
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != LML_OK:
+        raise LmlError(status, where)
+
+
+# ---- C names, raw arguments ---------------------------------------------------------------------
+
+def lml_status_string(status: int) -> str:
+    return lib().lml_status_string(status).decode()
+
+
+def lml_table_create(device: int, d_in: int, d_out: int, max_slots: int) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().lml_table_create(ctypes.byref(h), device, d_in, d_out, max_slots), "lml_table_create")
+    return h.value
+
+
+def lml_table_destroy(table: int) -> None:
+    _check(lib().lml_table_destroy(table), "lml_table_destroy")
+
+
+def register_adapter(table: int, adapter_id: int, version: int, A_ptr: int, B_ptr: int, rank: int,
+                     scale: float, stream: int = 0) -> int:
+    slot = ctypes.c_int(-1)
+    _check(lib().register_adapter(table, adapter_id, version, A_ptr, B_ptr, rank, scale, stream,
+                                  ctypes.byref(slot)), "register_adapter")
+    return slot.value
+
+
+def retire_version(table: int, adapter_id: int, version: int) -> None:
+    _check(lib().retire_version(table, adapter_id, version), "retire_version")
+
+
+def lml_lookup(table: int, adapter_id: int, version: int) -> int:
+    slot = ctypes.c_int(-1)
+    _check(lib().lml_lookup(table, adapter_id, version, ctypes.byref(slot)), "lml_lookup")
+    return slot.value
+
+
+def lml_slot_info(table: int, slot: int) -> Tuple[int, int, int, float]:
+    a, v, r, s = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_float()
+    _check(lib().lml_slot_info(table, slot, ctypes.byref(a), ctypes.byref(v), ctypes.byref(r), ctypes.byref(s)),
+           "lml_slot_info")
+    return a.value, v.value, r.value, s.value
+
+
+def lml_workspace_bytes(table: int, max_tokens: int, max_segments: int) -> int:
+    return int(lib().lml_workspace_bytes(table, max_tokens, max_segments))
+
+
+def lml_host_workspace_bytes(table: int, max_tokens: int, max_segments: int) -> int:
+    return int(lib().lml_host_workspace_bytes(table, max_tokens, max_segments))
+
+
+def lml_segment_tokens(table: int, token_slots_ptr: int, T: int, perm_ptr: int, seg_offsets_ptr: int,
+                       seg_slot_ids_ptr: int, stream: int = 0) -> None:
+    _check(lib().lml_segment_tokens(table, token_slots_ptr, T, perm_ptr, seg_offsets_ptr, seg_slot_ids_ptr,
+                                    stream), "lml_segment_tokens")
+
+
+def lora_mixed_linear(table: int, x_ptr: int, W0_ptr: int, T: int, seg_offsets_ptr: int, slot_ids_ptr: int,
+                      G: int, perm_ptr: int, y_ptr: int, workspace_ptr: int, workspace_bytes: int,
+                      stream: int = 0) -> None:
+    _check(lib().lora_mixed_linear(table, x_ptr, W0_ptr, T, seg_offsets_ptr, slot_ids_ptr, G, perm_ptr, y_ptr,
+                                   workspace_ptr, workspace_bytes, stream), "lora_mixed_linear")
+
+
+def lora_mixed_linear_host(table: int, x_host_ptr: int, W0_ptr: int, T: int, seg_offsets_host_ptr: int,
+                           slot_ids_host_ptr: int, G: int, perm_host_ptr: int, y_host_ptr: int,
+                           workspace_ptr: int, workspace_bytes: int, stream: int = 0) -> None:
+    _check(lib().lora_mixed_linear_host(table, x_host_ptr, W0_ptr, T, seg_offsets_host_ptr, slot_ids_host_ptr, G,
+                                        perm_host_ptr, y_host_ptr, workspace_ptr, workspace_bytes, stream),
+           "lora_mixed_linear_host")
+
+
+def lml_device_status(table: int, stream: int = 0) -> int:
+    f = ctypes.c_uint32(0)
+    _check(lib().lml_device_status(table, ctypes.byref(f), stream), "lml_device_status")
+    return int(f.value)
+
+
+def lml_last_launch_count(table: int) -> int:
+    return int(lib().lml_last_launch_count(table))
+
+
+# ---- torch convenience ------------------------------------------------------------------------------
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _stream(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Table:
+    """Adapter slot table of one linear site, for torch tensors (bf16 CUDA, contiguous)."""
+
+    def __init__(self, d_in: int, d_out: int, max_slots: int = MAX_SLOTS, device: int = 0):
+        self.d_in, self.d_out, self.max_slots, self.device = d_in, d_out, max_slots, device
+        self.handle = lml_table_create(device, d_in, d_out, max_slots)
+        self._ws = None
+
+    def close(self) -> None:
+        if self.handle:
+            lml_table_destroy(self.handle)
+            self.handle = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def register_adapter(self, adapter_id: int, version: int, A, B, scale: float, stream=None) -> int:
+        import torch
+        assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.is_cuda and B.is_cuda
+        assert A.is_contiguous() and B.is_contiguous()
+        rank = int(A.shape[0])
+        assert A.shape == (rank, self.d_in) and B.shape == (self.d_out, rank), (A.shape, B.shape)
+        return register_adapter(self.handle, adapter_id, version, _ptr(A), _ptr(B), rank, float(scale),
+                                _stream(stream))
+
+    def retire_version(self, adapter_id: int, version: int) -> None:
+        retire_version(self.handle, adapter_id, version)
+
+    def lookup(self, adapter_id: int, version: int) -> int:
+        return lml_lookup(self.handle, adapter_id, version)
+
+    def slot_info(self, slot: int):
+        return lml_slot_info(self.handle, slot)
+
+    def workspace_bytes(self, max_tokens: int, max_segments: int) -> int:
+        return lml_workspace_bytes(self.handle, max_tokens, max_segments)
+
+    def workspace(self, T: int, G: int, host: bool = False):
+        """A cached torch byte buffer large enough for (T, G); grown on demand (outside the hot call)."""
+        import torch
+        need = (lml_host_workspace_bytes if host else lml_workspace_bytes)(self.handle, T, G)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(max(need, 1024), dtype=torch.uint8, device=f"cuda:{self.device}")
+        return self._ws
+
+    def segment_tokens(self, token_slots, stream=None):
+        """token_slots int32[T] (cuda) -> (perm int32[T], seg_offsets int32[max_slots+2],
+        seg_slot_ids int32[max_slots+1]); G = max_slots + 1."""
+        import torch
+        assert token_slots.dtype == torch.int32 and token_slots.is_cuda and token_slots.is_contiguous()
+        T = int(token_slots.shape[0])
+        dev = token_slots.device
+        perm = torch.empty(max(T, 1), dtype=torch.int32, device=dev)
+        seg_offsets = torch.empty(self.max_slots + 2, dtype=torch.int32, device=dev)
+        seg_slot_ids = torch.empty(self.max_slots + 1, dtype=torch.int32, device=dev)
+        lml_segment_tokens(self.handle, _ptr(token_slots), T, _ptr(perm), _ptr(seg_offsets), _ptr(seg_slot_ids),
+                           _stream(stream))
+        return perm[:T], seg_offsets, seg_slot_ids
+
+    def lora_mixed_linear(self, x, W0, seg_offsets, slot_ids, perm=None, y=None, workspace=None, stream=None):
+        import torch
+        assert x.dtype == torch.bfloat16 and W0.dtype == torch.bfloat16 and x.is_cuda and W0.is_cuda
+        assert x.is_contiguous() and W0.is_contiguous()
+        T = int(x.shape[0])
+        assert x.shape[1] == self.d_in and W0.shape == (self.d_out, self.d_in)
+        G = 0 if slot_ids is None else int(slot_ids.shape[0])
+        if G:
+            assert seg_offsets.dtype == torch.int32 and slot_ids.dtype == torch.int32
+            assert seg_offsets.shape[0] == G + 1 and seg_offsets.is_cuda and slot_ids.is_cuda
+        if perm is not None:
+            assert perm.dtype == torch.int32 and perm.shape[0] == T and perm.is_cuda
+        if y is None:
+            y = torch.empty((T, self.d_out), dtype=torch.bfloat16, device=x.device)
+        if workspace is None:
+            workspace = self.workspace(T, G)
+        lora_mixed_linear(self.handle, _ptr(x), _ptr(W0), T, _ptr(seg_offsets) if G else 0,
+                          _ptr(slot_ids) if G else 0, G, _ptr(perm), _ptr(y), _ptr(workspace),
+                          int(workspace.numel()), _stream(stream))
+        return y
+
+    def lora_mixed_linear_host(self, x_host, W0, seg_offsets_host, slot_ids_host, y_host, perm_host=None,
+                               workspace=None, stream=None):
+        """x_host / y_host: CPU bf16 tensors (pinned for asynchronous copies); W0 on the device."""
+        T = int(x_host.shape[0])
+        G = 0 if slot_ids_host is None else int(slot_ids_host.shape[0])
+        assert not x_host.is_cuda and not y_host.is_cuda and W0.is_cuda
+        if workspace is None:
+            workspace = self.workspace(T, G, host=True)
+        lora_mixed_linear_host(self.handle, _ptr(x_host), _ptr(W0), T, _ptr(seg_offsets_host) if G else 0,
+                               _ptr(slot_ids_host) if G else 0, G, _ptr(perm_host), _ptr(y_host),
+                               _ptr(workspace), int(workspace.numel()), _stream(stream))
+        return y_host
+
+    def device_status(self, stream=None) -> int:
+        return lml_device_status(self.handle, _stream(stream))
+
+    def last_launch_count(self) -> int:
+        return lml_last_launch_count(self.handle)

@@ -1,0 +1,366 @@
+// Host side of the C ABI: the adapter slot table, argument validation, workspace layout and
+// dispatch to the decode / prefill kernels.  See include/lora_mixed_linear.h for the contract.
+#include <mutex>
+#include <new>
+
+#include "lml_internal.cuh"
+
+using namespace lml;
+
+struct lml_table {
+    int device = 0, d_in = 0, d_out = 0, max_slots = 0, num_sms = 0;
+    struct Entry {
+        bool live = false;
+        int adapter_id = 0, version = 0, rank = 0;
+        float scale = 0.f;
+    } entries[kMaxSlots];
+    Arena arena{};
+    CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
+    int last_launches = 0;
+    mutable std::mutex mu;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+SlotSnapshot snapshot(const lml_table* t)
+{
+    SlotSnapshot s;
+    for (int i = 0; i < kMaxSlots; ++i) {
+        const bool live = i < t->max_slots && t->entries[i].live;
+        s.rank[i] = live ? (uint8_t)t->entries[i].rank : 0;
+        s.scale[i] = live ? t->entries[i].scale : 0.f;
+    }
+    s.max_slots = t->max_slots;
+    return s;
+}
+
+// Workspace layout of the prefill path: [PlanWord][u blocks][gathered x (perm form only)];
+// the decode path uses [PlanWord][u fp32 16x64][row_slot 16].
+struct WsLayout {
+    size_t plan_off, u_off, xg_off, total;
+};
+WsLayout ws_layout(const lml_table* t, int T, int G)
+{
+    WsLayout w;
+    w.plan_off = 0;
+    w.u_off = round_up(sizeof(PlanWord), 1024);
+    const size_t num_m = (size_t)(T + kTileM - 1) / kTileM;
+    size_t u_bytes = (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
+    const size_t dec_bytes = (size_t)kDecodeMaxT * kRankPad * sizeof(float) + kDecodeMaxT * sizeof(int32_t);
+    if (u_bytes < dec_bytes) u_bytes = dec_bytes;
+    w.xg_off = w.u_off + round_up(u_bytes, 1024);
+    w.total = w.xg_off + round_up((size_t)T * t->d_in * sizeof(__nv_bfloat16), 1024);
+    return w;
+}
+
+const int kMaxTokens = kTileM * 32768;   // keeps every grid dimension and int index in range
+
+}  // namespace
+
+extern "C" {
+
+const char* lml_status_string(lml_status s)
+{
+    switch (s) {
+        case LML_OK: return "ok";
+        case LML_ERR_INVALID_ARG: return "invalid argument";
+        case LML_ERR_BAD_SLOT: return "bad slot";
+        case LML_ERR_TABLE_FULL: return "slot table full";
+        case LML_ERR_DUPLICATE: return "adapter version already resident";
+        case LML_ERR_NOT_FOUND: return "adapter version not resident";
+        case LML_ERR_UNSUPPORTED: return "device is not sm_100";
+        case LML_ERR_CUDA: return "CUDA call failed";
+        case LML_ERR_TIMEOUT: return "device wait timed out";
+        case LML_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    }
+    return "unknown status";
+}
+
+lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, int max_slots)
+{
+    if (!out) return LML_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (device < 0 || d_in <= 0 || d_out <= 0 || (d_in % 8) || (d_out % 8) || max_slots < 1 ||
+        max_slots > kMaxSlots)
+        return LML_ERR_INVALID_ARG;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    if (device >= count) return LML_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    if (prop.major != 10) return LML_ERR_UNSUPPORTED;
+    DeviceGuard guard(device);
+    if (!guard.ok) return LML_ERR_CUDA;
+
+    lml_table* t = new (std::nothrow) lml_table();
+    if (!t) return LML_ERR_CUDA;
+    t->device = device; t->d_in = d_in; t->d_out = d_out; t->max_slots = max_slots;
+    t->num_sms = prop.multiProcessorCount;
+    const size_t a_bytes = (size_t)max_slots * kRankPad * d_in * sizeof(__nv_bfloat16);
+    const size_t b_bytes = (size_t)max_slots * d_out * kRankPad * sizeof(__nv_bfloat16);
+    bool ok = cudaMalloc(&t->arena.A, a_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->arena.B, b_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->arena.status, 256) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.A, 0, a_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.B, 0, b_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
+    ok = ok && gemm_sm100_init(device) == cudaSuccess;
+    ok = ok && encode_tmap_3d(&t->tmap_B256, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
+                              kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status);
+        delete t;
+        return LML_ERR_CUDA;
+    }
+    *out = t;
+    return LML_OK;
+}
+
+lml_status lml_table_destroy(lml_table* t)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    {
+        DeviceGuard guard(t->device);
+        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status);
+    }
+    delete t;
+    return LML_OK;
+}
+
+lml_status register_adapter(lml_table* t, int adapter_id, int version, const void* A, const void* B, int rank,
+                            float scale, void* stream, int* slot_out)
+{
+    if (!t || !A || !B || !slot_out || rank < 1 || rank > LML_MAX_RANK || !aligned16(A) || !aligned16(B) ||
+        !(scale == scale))
+        return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    int free_slot = -1;
+    for (int i = 0; i < t->max_slots; ++i) {
+        const auto& e = t->entries[i];
+        if (e.live && e.adapter_id == adapter_id && e.version == version) return LML_ERR_DUPLICATE;
+        if (!e.live && free_slot < 0) free_slot = i;
+    }
+    if (free_slot < 0) return LML_ERR_TABLE_FULL;
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    if (launch_pack_adapter(t->arena, free_slot, A, B, rank, t->d_in, t->d_out, (cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
+    auto& e = t->entries[free_slot];
+    e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
+    e.live = true;   // published last: the entry is complete before it becomes visible
+    *slot_out = free_slot;
+    return LML_OK;
+}
+
+lml_status retire_version(lml_table* t, int adapter_id, int version)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    for (int i = 0; i < t->max_slots; ++i) {
+        auto& e = t->entries[i];
+        if (e.live && e.adapter_id == adapter_id && e.version == version) { e.live = false; return LML_OK; }
+    }
+    return LML_ERR_NOT_FOUND;
+}
+
+lml_status lml_lookup(const lml_table* t, int adapter_id, int version, int* slot_out)
+{
+    if (!t || !slot_out) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    for (int i = 0; i < t->max_slots; ++i) {
+        const auto& e = t->entries[i];
+        if (e.live && e.adapter_id == adapter_id && e.version == version) { *slot_out = i; return LML_OK; }
+    }
+    return LML_ERR_NOT_FOUND;
+}
+
+lml_status lml_slot_info(const lml_table* t, int slot, int* adapter_id, int* version, int* rank, float* scale)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (slot < 0 || slot >= t->max_slots || !t->entries[slot].live) return LML_ERR_BAD_SLOT;
+    const auto& e = t->entries[slot];
+    if (adapter_id) *adapter_id = e.adapter_id;
+    if (version) *version = e.version;
+    if (rank) *rank = e.rank;
+    if (scale) *scale = e.scale;
+    return LML_OK;
+}
+
+size_t lml_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
+{
+    if (!t || max_tokens < 0 || max_segments < 0 || max_tokens > kMaxTokens) return 0;
+    return ws_layout(t, max_tokens, max_segments).total;
+}
+
+lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, int32_t* perm, int32_t* seg_offsets,
+                              int32_t* seg_slot_ids, void* stream)
+{
+    if (!t || T < 0 || T > kMaxTokens || !seg_offsets || !seg_slot_ids || (T > 0 && (!token_slots || !perm)))
+        return LML_ERR_INVALID_ARG;
+    SlotSnapshot snap;
+    {
+        std::lock_guard<std::mutex> lock(t->mu);
+        snap = snapshot(t);
+    }
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    if (launch_segment_tokens(t->arena, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, (cudaStream_t)stream) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
+    t->last_launches = 1;
+    return LML_OK;
+}
+
+lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T, const int32_t* seg_offsets,
+                             const int32_t* slot_ids, int G, const int32_t* perm, void* y, void* workspace,
+                             size_t workspace_bytes, void* stream_v)
+{
+    if (!t || T < 0 || G < 0 || T > kMaxTokens || G > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x || !W0 || !y || !aligned16(x) || !aligned16(W0) || !aligned16(y)) return LML_ERR_INVALID_ARG;
+    if (G > 0 && (!seg_offsets || !slot_ids)) return LML_ERR_INVALID_ARG;
+    if (G == 0) perm = nullptr;   // without adapters the row order is irrelevant
+    const WsLayout ws = ws_layout(t, T, G);
+    const bool decode = T <= kDecodeMaxT;
+    const size_t need = decode ? ws.xg_off : (perm ? ws.total : ws.xg_off);
+    const bool need_ws = G > 0 || (!decode && perm);
+    if (need_ws && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) || workspace_bytes < need))
+        return LML_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    SlotSnapshot snap;
+    {
+        std::lock_guard<std::mutex> lock(t->mu);
+        snap = snapshot(t);
+    }
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    uint8_t* wsb = static_cast<uint8_t*>(workspace);
+    int launches = 0;
+    cudaError_t e = cudaSuccess;
+
+    if (decode) {
+        DecodeArgs a;
+        a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
+        a.u = G > 0 ? reinterpret_cast<float*>(wsb + ws.u_off) : nullptr;
+        a.row_slot = G > 0 ? reinterpret_cast<int32_t*>(wsb + ws.u_off + (size_t)kDecodeMaxT * kRankPad * sizeof(float))
+                           : nullptr;
+        a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G;
+        e = launch_decode(t->arena, snap, a, stream, &launches);
+    } else {
+        const void* xg = x;
+        if (perm) {
+            e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, t->arena.status, stream);
+            if (e == cudaSuccess) { ++launches; xg = wsb + ws.xg_off; }
+        }
+        PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
+        __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
+        if (e == cudaSuccess && G > 0) {
+            e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids, G, nullptr, plan, u_blocks,
+                                     stream);
+            if (e == cudaSuccess) ++launches;
+        }
+        if (e == cudaSuccess) {
+            GemmArgs a;
+            a.x = xg; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
+            a.plan = plan; a.u_blocks = u_blocks ? u_blocks : reinterpret_cast<const __nv_bfloat16*>(x);
+            a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
+            if (G == 0) a.u_blocks = reinterpret_cast<const __nv_bfloat16*>(W0);   // never read; map needs a valid base
+            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
+            if (e == cudaSuccess) ++launches;
+        }
+    }
+    t->last_launches = launches;
+    if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    return LML_OK;
+}
+
+size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
+{
+    if (!t || max_tokens < 0 || max_segments < 0 || max_tokens > kMaxTokens) return 0;
+    size_t n = ws_layout(t, max_tokens, max_segments).total;
+    n += round_up((size_t)max_tokens * t->d_in * 2, 1024);    // x staging
+    n += round_up((size_t)max_tokens * t->d_out * 2, 1024);   // y staging
+    n += round_up((size_t)(max_segments + 1) * 4, 1024) + round_up((size_t)max_segments * 4 + 4, 1024);
+    n += round_up((size_t)max_tokens * 4 + 4, 1024);          // perm staging
+    return n;
+}
+
+lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* W0, int T,
+                                  const int32_t* seg_offsets_host, const int32_t* slot_ids_host, int G,
+                                  const int32_t* perm_host, void* y_host, void* workspace, size_t workspace_bytes,
+                                  void* stream_v)
+{
+    if (!t || T < 0 || G < 0 || T > kMaxTokens || G > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x_host || !W0 || !y_host || (G > 0 && (!seg_offsets_host || !slot_ids_host))) return LML_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||
+        workspace_bytes < lml_host_workspace_bytes(t, T, G))
+        return LML_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    uint8_t* p = static_cast<uint8_t*>(workspace);
+    const size_t inner = ws_layout(t, T, G).total;
+    uint8_t* xs = p + inner;
+    uint8_t* ys = xs + round_up((size_t)T * t->d_in * 2, 1024);
+    uint8_t* so = ys + round_up((size_t)T * t->d_out * 2, 1024);
+    uint8_t* si = so + round_up((size_t)(G + 1) * 4, 1024);
+    uint8_t* pm = si + round_up((size_t)G * 4 + 4, 1024);
+    bool ok = cudaMemcpyAsync(xs, x_host, (size_t)T * t->d_in * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (G > 0) {
+        ok = ok && cudaMemcpyAsync(so, seg_offsets_host, (size_t)(G + 1) * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(si, slot_ids_host, (size_t)G * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    }
+    if (perm_host)
+        ok = ok && cudaMemcpyAsync(pm, perm_host, (size_t)T * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
+    lml_status st = lora_mixed_linear(t, xs, W0, T, reinterpret_cast<int32_t*>(so), reinterpret_cast<int32_t*>(si), G,
+                                      perm_host ? reinterpret_cast<int32_t*>(pm) : nullptr, ys, p, inner, stream);
+    if (st != LML_OK) return st;
+    if (cudaMemcpyAsync(y_host, ys, (size_t)T * t->d_out * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
+    return LML_OK;
+}
+
+lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
+{
+    if (!t || !flags_out) return LML_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    uint32_t v = 0;
+    bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(t->arena.status, 0, sizeof v, stream) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
+    *flags_out = v;
+    return LML_OK;
+}
+
+int lml_last_launch_count(const lml_table* t) { return t ? t->last_launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,159 @@
+// Small helper kernels: adapter packing (register_adapter), token segmentation, row gather.
+#include "lml_internal.cuh"
+
+namespace lml {
+
+// ---------------------------------------------------------------------------------------------
+// register_adapter: copy A[rank][d_in] and B[d_out][rank] into the arena, zero-padded to rank 64,
+// so that every kernel can read fixed-shape, 16-byte aligned rows.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_adapter_kernel(__nv_bfloat16* __restrict__ dstA,
+                                                           __nv_bfloat16* __restrict__ dstB,
+                                                           const __nv_bfloat16* __restrict__ A,
+                                                           const __nv_bfloat16* __restrict__ B,
+                                                           int rank, int d_in, int d_out)
+{
+    const long long nA8 = (long long)kRankPad * (d_in / 8);   // uint4 chunks of the padded A
+    const long long nB = (long long)d_out * kRankPad;         // elements of the padded B
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int k8 = d_in / 8;
+    for (long long i = tid; i < nA8; i += stride) {
+        int j = (int)(i / k8);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (j < rank) v = reinterpret_cast<const uint4*>(A)[i];   // same linear index: rows are contiguous
+        reinterpret_cast<uint4*>(dstA)[i] = v;
+    }
+    const unsigned short* Bs = reinterpret_cast<const unsigned short*>(B);
+    unsigned short* Bd = reinterpret_cast<unsigned short*>(dstB);
+    for (long long i = tid; i < nB; i += stride) {
+        int j = (int)(i % kRankPad);
+        long long n = i / kRankPad;
+        Bd[i] = (j < rank) ? Bs[n * rank + j] : (unsigned short)0;
+    }
+}
+
+cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const void* B, int rank,
+                                int d_in, int d_out, cudaStream_t stream)
+{
+    __nv_bfloat16* dstA = ar.A + (size_t)slot * kRankPad * d_in;
+    __nv_bfloat16* dstB = ar.B + (size_t)slot * d_out * kRankPad;
+    long long work = (long long)d_out * kRankPad;
+    int blocks = (int)((work + 255) / 256);
+    if (blocks > 1184) blocks = 1184;
+    pack_adapter_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, (const __nv_bfloat16*)A,
+                                                    (const __nv_bfloat16*)B, rank, d_in, d_out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Token segmentation: stable counting sort of T tokens by slot (keys 0..max_slots-1, then -1).
+// One CTA of 32 warps.  Warp w owns a contiguous range of tokens; pass 1 counts keys per warp,
+// a scan turns the counts into (key-major, warp-minor) start positions, pass 2 walks the same
+// range in order and places each token, using match_any to rank equal keys inside a 32-token
+// chunk.  Everything is order-deterministic.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSegWarps = 32;
+
+__global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
+    const __grid_constant__ SlotSnapshot snap, const int32_t* __restrict__ token_slots, int T,
+    int32_t* __restrict__ perm, int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_slot_ids,
+    uint32_t* __restrict__ status)
+{
+    __shared__ int hist[kSegWarps][kMaxSlots + 1];
+    __shared__ int base[kMaxSlots + 2];
+    const int nk = snap.max_slots + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < kSegWarps * (kMaxSlots + 1); i += blockDim.x) (&hist[0][0])[i] = 0;
+    __syncthreads();
+
+    int per = (T + kSegWarps - 1) / kSegWarps;
+    per = (per + 31) & ~31;
+    const int begin = min(T, warp * per);
+    const int end = min(T, begin + per);
+    bool bad = false;
+
+    for (int c = begin; c < end; c += 32) {
+        int i = c + lane;
+        if (i < end) {
+            int s = __ldg(token_slots + i);
+            if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) { bad = true; s = -1; }
+            int key = s < 0 ? snap.max_slots : s;
+            atomicAdd(&hist[warp][key], 1);
+        }
+    }
+    if (bad) atomicOr(status, LML_FLAG_BAD_SLOT);
+    __syncthreads();
+    if ((int)threadIdx.x < nk) {
+        int run = 0;
+        for (int w = 0; w < kSegWarps; ++w) { int c = hist[w][threadIdx.x]; hist[w][threadIdx.x] = run; run += c; }
+        base[threadIdx.x] = run;   // total of this key for now
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int k = 0; k < nk; ++k) {
+            int c = base[k];
+            base[k] = run;
+            seg_offsets[k] = run;
+            seg_slot_ids[k] = k < snap.max_slots ? k : -1;
+            run += c;
+        }
+        seg_offsets[nk] = run;
+    }
+    __syncthreads();
+
+    for (int c = begin; c < end; c += 32) {   // trip count is uniform inside a warp
+        int i = c + lane;
+        int key = nk;                          // sentinel for lanes past the end
+        if (i < end) {
+            int s = __ldg(token_slots + i);
+            if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) s = -1;
+            key = s < 0 ? snap.max_slots : s;
+        }
+        unsigned m = __match_any_sync(0xffffffffu, key);
+        int before = __popc(m & ((1u << lane) - 1u));
+        int pos = 0;
+        if (key < nk) {
+            pos = base[key] + hist[warp][key] + before;
+            perm[pos] = i;
+        }
+        __syncwarp();
+        if (key < nk && before == 0) hist[warp][key] += __popc(m);
+        __syncwarp();
+    }
+}
+
+cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
+                                  int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
+                                  cudaStream_t stream)
+{
+    segment_tokens_kernel<<<1, kSegWarps * 32, 0, stream>>>(snap, token_slots, T, perm, seg_offsets,
+                                                           seg_slot_ids, ar.status);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row gather for the perm form of the prefill call: x_grouped[p][:] = x[perm[p]][:].
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) gather_rows_kernel(const uint4* __restrict__ x,
+                                                          const int32_t* __restrict__ perm, int T, int k8,
+                                                          uint4* __restrict__ out, uint32_t* __restrict__ status)
+{
+    const int p = blockIdx.x;
+    int row = __ldg(perm + p);
+    const bool ok = row >= 0 && row < T;
+    if (!ok && threadIdx.x == 0) atomicOr(status, LML_FLAG_BAD_PERM);
+    const uint4* src = x + (size_t)(ok ? row : 0) * k8;
+    uint4* dst = out + (size_t)p * k8;
+    for (int i = threadIdx.x; i < k8; i += blockDim.x) dst[i] = ok ? ldg_nc_v4(src + i) : make_uint4(0, 0, 0, 0);
+}
+
+cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
+                               uint32_t* status, cudaStream_t stream)
+{
+    gather_rows_kernel<<<T, 128, 0, stream>>>((const uint4*)x, perm, T, d_in / 8, (uint4*)x_grouped, status);
+    return cudaGetLastError();
+}
+
+}  // namespace lml

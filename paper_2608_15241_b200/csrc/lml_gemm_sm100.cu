@@ -1,0 +1,414 @@
+// Prefill path: y = bf16( x.W0^T + sum over pieces u_piece.B_slot^T ) on the sm_100a tensor cores.
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0   TMA producer: streams 128x64 tiles of x and BNx64 tiles of W0 (128-byte swizzle) into
+//            a ring of shared-memory stages; after the last k-block of a tile it appends one
+//            stage per LoRA piece of that tile: the piece's 128x64 block of u and the BNx64 block
+//            of the slot's packed B.  So the LoRA expand is just more K for the same accumulator:
+//            [x | u_1 | u_2 ...] . [W0 ; B_s1 ; B_s2 ...].
+//   warp 1   MMA issuer: one lane issues tcgen05.mma (M=128, N=BN, K=16) per 16 columns of a stage
+//            into one of two TMEM accumulators and commits to the stage's "empty" barrier.
+//   warps 2-5 epilogue: tcgen05.ld the accumulator (each warp its 32 TMEM lanes = 32 rows), round to
+//            bf16 once, stage 32x32 chunks in shared memory and write them with TMA stores (or
+//            row-scattered 16-byte stores when a perm is given).  Runs one tile behind the MMA
+//            warp thanks to the second accumulator.
+// Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
+#include "lml_internal.cuh"
+#include "lml_ptx_sm100.cuh"
+
+namespace lml {
+
+using namespace ptx;
+
+constexpr int kBM = kTileM;   // 128
+constexpr int kBK = 64;       // bf16 elements per 128-byte swizzled row
+constexpr int kGemmThreads = 192;
+constexpr int kSegCache = 256;            // segments cached in shared memory
+constexpr int kEpiChunkCols = 32;
+constexpr int kEpiBufBytes = 32 * kEpiChunkCols * 2;   // 2 KB: 32 rows x 64 B
+
+template <int BN> struct GemmCfg {
+    static constexpr int kABytes = kBM * kBK * 2;
+    static constexpr int kBBytes = BN * kBK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = (BN == 256) ? 4 : 6;
+    static constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
+    static constexpr int kTmemCols = 2 * BN;
+    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + kSegCache;   // barriers + segment cache
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiBytes + ((kCtrlBytes + 15) & ~15);
+};
+
+struct GemmCtrl {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    int abort;
+    uint32_t stage_info[8];   // k-steps (1..4) | last-stage-of-tile << 8, written by the producer
+    int32_t pad[6];
+};
+static_assert(sizeof(GemmCtrl) <= 256, "control block");
+
+struct GemmParams {
+    const int32_t* seg_offsets;
+    const int32_t* slot_ids;
+    const int32_t* perm;
+    const PlanWord* plan;
+    __nv_bfloat16* y;
+    uint32_t* status;
+    int T, K, N, G;
+    int num_m, num_n;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
+    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+    const __grid_constant__ CUtensorMap tmap_u, const __grid_constant__ CUtensorMap tmap_b,
+    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ SlotSnapshot snap,
+    const GemmParams p)
+{
+    using Cfg = GemmCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    // 128-byte swizzled tiles need 1024-byte alignment
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+    uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    const uint32_t epi_addr = tiles_addr + Cfg::kStages * Cfg::kStageBytes;
+    uint8_t* epi_ptr = tiles_ptr + Cfg::kStages * Cfg::kStageBytes;
+    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(epi_ptr + Cfg::kEpiBytes);
+    int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
+    int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_tiles = p.num_m * p.num_n;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+    const bool seg_cached = p.G <= kSegCache;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cfg::kStages; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&ctrl->tmem_full[a]), 1);
+            mbar_init(smem_u32(&ctrl->tmem_empty[a]), 4);
+        }
+        ctrl->abort = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u);
+        prefetch_tmap(&tmap_b); prefetch_tmap(&tmap_y);
+    }
+    if (seg_cached) {
+        for (int g = threadIdx.x; g <= p.G; g += kGemmThreads) seg_cache[g] = __ldg(p.seg_offsets + g);
+        for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
+            int s = __ldg(p.slot_ids + g);
+            slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
+        }
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), Cfg::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile int* abort = &ctrl->abort;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const bool lora = p.G > 0 && p.plan->lora_ok != 0;
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            auto acquire = [&]() -> bool {
+                return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
+            };
+            auto advance = [&]() { if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; } };
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m = tile % p.num_m, n = tile / p.num_m;
+                const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+                // pieces of this tile: segments with a live slot that overlap [row0, row1)
+                int g_first = 0, g_end = 0;
+                if (lora) {
+                    if (seg_cached) {
+                        int lo = 0, hi = p.G;
+                        while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+                        g_first = lo;
+                        g_end = g_first;
+                        while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
+                    } else {
+                        g_first = seg_upper(p.seg_offsets, p.G, row0);
+                        g_end = g_first;
+                        while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
+                    }
+                }
+                auto piece_slot = [&](int g) -> int {   // -1 = segment contributes no piece
+                    int s0, s1, s;
+                    if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
+                    else {
+                        s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1); s = __ldg(p.slot_ids + g);
+                        if (slot_rank(snap, s) == 0) s = -1;
+                    }
+                    if (min(s1, row1) <= max(s0, row0)) return -1;
+                    return s;
+                };
+                int last_piece = -1;
+                for (int g = g_first; g < g_end; ++g) if (piece_slot(g) >= 0) last_piece = g;
+
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    ok = acquire();
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                    ctrl->stage_info[stage] = 4u | ((kb == num_kb - 1 && last_piece < 0) ? 0x100u : 0u);
+                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                    tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
+                    tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
+                    advance();
+                }
+                for (int g = g_first; g < g_end && ok; ++g) {
+                    const int s = piece_slot(g);
+                    if (s < 0) continue;
+                    ok = acquire();
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                    const uint32_t ksteps = (uint32_t)((snap.rank[s] + 15) >> 4);
+                    ctrl->stage_info[stage] = ksteps | (g == last_piece ? 0x100u : 0u);
+                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                    tma_load_2d(a_dst, &tmap_u, bar, 0, (m + g) * kBM);
+                    tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
+                    advance();
+                }
+            }
+            // Leave only after every load issued above has landed (its stage was consumed or its
+            // full barrier completed): wait for the ring to drain.
+            for (int i = 0; i < Cfg::kStages && ok; ++i) { ok = acquire(); advance(); }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                ok = mbar_wait(smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1u, abort);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                uint32_t accumulate = 0;
+                for (;;) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t info = ctrl->stage_info[stage];
+                    const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes;
+                    const uint64_t adesc = umma_desc_k128(a_addr);
+                    const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes);
+                    const int ksteps = (int)(info & 0xffu);
+#pragma unroll 4
+                    for (int k = 0; k < ksteps; ++k) {
+                        // 16 bf16 columns = 32 bytes further along the swizzled row: +2 in 16-byte units
+                        umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    umma_commit(smem_u32(&ctrl->empty[stage]));
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                    if (info & 0x100u) break;
+                }
+                if (!ok) break;
+                umma_commit(smem_u32(&ctrl->tmem_full[acc]));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int ew = warp - 2;
+        const uint32_t buf_addr0 = epi_addr + (uint32_t)(ew * 2 * kEpiBufBytes);
+        uint8_t* buf_ptr0 = epi_ptr + ew * 2 * kEpiBufBytes;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        int buf = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int m = tile % p.num_m, n = tile / p.num_m;
+            const int row_base = m * kBM + q * 32;
+            ok = mbar_wait(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN / kEpiChunkCols; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(t_addr + (uint32_t)(c * kEpiChunkCols), r);
+                tmem_ld_wait();
+                if (c == BN / kEpiChunkCols - 1) {
+                    // accumulator fully read: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[acc]));
+                }
+                const int col0 = n * BN + c * kEpiChunkCols;
+                if (col0 >= p.N || row_base >= p.T) continue;   // nothing of this chunk is inside y
+                // the buffer we are about to overwrite must have been read by its earlier store
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
+                uint8_t* bp = buf_ptr0 + buf * kEpiBufBytes;
+                const uint32_t ba = buf_addr0 + (uint32_t)(buf * kEpiBufBytes);
+                // row = lane: 64 bytes, four 16-byte chunks, 64-byte swizzle (chunk ^= (row >> 1) & 3)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 v;
+                    v.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                    v.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                    v.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                    v.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                    const int phys = j ^ ((lane >> 1) & 3);
+                    *reinterpret_cast<uint4*>(bp + lane * 64 + phys * 16) = v;
+                }
+                if (p.perm == nullptr) {
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmap_y, ba, col0, row_base);
+                        tma_store_commit();
+                    }
+                } else {
+                    __syncwarp();
+                    // scatter: 4 lanes write one 64-byte row piece; 8 rows per pass
+#pragma unroll
+                    for (int pass = 0; pass < 4; ++pass) {
+                        const int rr = pass * 8 + (lane >> 2), j = lane & 3;
+                        const int pos = row_base + rr;
+                        if (pos < p.T && col0 + j * 8 < p.N) {
+                            const int row = __ldg(p.perm + pos);
+                            if (row >= 0 && row < p.T) {
+                                const int phys = j ^ ((rr >> 1) & 3);
+                                uint4 v = *reinterpret_cast<const uint4*>(bp + rr * 64 + phys * 16);
+                                *reinterpret_cast<uint4*>(p.y + (size_t)row * p.N + col0 + j * 8) = v;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+                buf ^= 1;
+            }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) tma_store_wait_all();
+    }
+
+    __syncthreads();
+    if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.status, LML_FLAG_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+static CUtensorMapSwizzle swizzle_for(uint32_t box_inner_elems)
+{
+    return box_inner_elems * 2 >= 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : (box_inner_elems * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+bool encode_tmap_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
+                    uint32_t box_inner, uint32_t box_outer)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(box_inner), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool encode_tmap_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                    uint64_t stride2_bytes, uint32_t b0, uint32_t b1, uint32_t b2)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    cuuint32_t box[3] = {b0, b1, b2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(b0), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t gemm_sm100_init(int /*device*/)
+{
+    cudaError_t e = cudaFuncSetAttribute(lora_gemm_sm100_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         GemmCfg<256>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lora_gemm_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                GemmCfg<128>::kSmemBytes);
+}
+
+int gemm_pick_bn(int T, int d_out, int num_sms)
+{
+    const int num_m = (T + kBM - 1) / kBM;
+    const int tiles256 = num_m * ((d_out + 255) / 256);
+    // wide tiles once they fill the machine; otherwise narrower tiles give more CTAs to stream W0
+    return tiles256 >= num_sms ? 256 : 128;
+}
+
+cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B,
+                              const GemmArgs& a, cudaStream_t stream)
+{
+    const int bn = gemm_pick_bn(a.T, a.d_out, a.num_sms);
+    const int num_m = (a.T + kBM - 1) / kBM;
+    const int num_n = (a.d_out + bn - 1) / bn;
+    CUtensorMap tx, tw, tu, ty, tb = tmap_B;
+    if (!encode_tmap_2d(&tx, a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!encode_tmap_2d(&tw, a.W0, (uint64_t)a.d_in, (uint64_t)a.d_out, (uint64_t)a.d_in * 2, kBK, (uint32_t)bn)) return cudaErrorInvalidValue;
+    const uint64_t u_rows = (uint64_t)(num_m + (a.G > 0 ? a.G : 1)) * kBM;
+    if (!encode_tmap_2d(&tu, a.u_blocks, kRankPad, u_rows, kRankPad * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!encode_tmap_2d(&ty, a.y, (uint64_t)a.d_out, (uint64_t)a.T, (uint64_t)a.d_out * 2, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
+    if (bn != 256) {
+        if (!encode_tmap_3d(&tb, ar.B, kRankPad, (uint64_t)a.d_out, (uint64_t)snap.max_slots, kRankPad * 2,
+                            (uint64_t)a.d_out * kRankPad * 2, kBK, (uint32_t)bn, 1)) return cudaErrorInvalidValue;
+    }
+    GemmParams p;
+    p.seg_offsets = a.seg_offsets; p.slot_ids = a.slot_ids; p.perm = a.perm; p.plan = a.plan;
+    p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
+    p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
+    const int grid = min(num_m * num_n, a.num_sms);
+    if (bn == 256)
+        lora_gemm_sm100_kernel<256><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tx, tw, tu, tb, ty, snap, p);
+    else
+        lora_gemm_sm100_kernel<128><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tx, tw, tu, tb, ty, snap, p);
+    return cudaGetLastError();
+}
+
+}  // namespace lml

@@ -1,0 +1,145 @@
+// Internal declarations shared by the sm_100a kernels and the host API of the mixed-adapter
+// LoRA linear library.  Not part of the public ABI.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lora_mixed_linear.h"
+
+namespace lml {
+
+constexpr int kMaxSlots = LML_MAX_SLOTS;
+constexpr int kRankPad = 64;          // adapters are stored zero-padded to this rank
+constexpr int kTileM = 128;           // token rows per GEMM tile and per shrink piece block
+constexpr int kDecodeMaxT = LML_DECODE_MAX_TOKENS;
+
+// Per-call snapshot of the slot table, passed by value as a kernel parameter so that a later
+// register / retire cannot change a call that is already enqueued.
+struct SlotSnapshot {
+    float scale[kMaxSlots];
+    uint8_t rank[kMaxSlots];   // 0 = slot not live
+    int32_t max_slots;
+};
+
+// Device-resident pieces of a table.
+struct Arena {
+    __nv_bfloat16* A;   // [max_slots][kRankPad][d_in]   rows >= rank are zero
+    __nv_bfloat16* B;   // [max_slots][d_out][kRankPad]  columns >= rank are zero
+    uint32_t* status;   // sticky LML_FLAG_* bits
+};
+
+// Workspace header written by the shrink kernels and read by the kernels that follow.
+struct PlanWord {
+    int32_t lora_ok;    // 1 = seg_offsets well formed, expand steps may run
+    int32_t pad[63];
+};
+
+// ---- kernel launchers (each enqueues on `stream` and returns the launch error) ------------
+
+cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const void* B, int rank,
+                                int d_in, int d_out, cudaStream_t stream);
+
+cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
+                                  int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
+                                  cudaStream_t stream);
+
+// u blocks: block b = (tile m) + (segment g) holds the 128 x 64 bf16 values scale*(x.A^T) of
+// the rows of tile m that belong to segment g, zero elsewhere.
+cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
+                                 int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
+                                 const int32_t* perm, PlanWord* plan, __nv_bfloat16* u_blocks,
+                                 cudaStream_t stream);
+
+cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
+                               uint32_t* status, cudaStream_t stream);
+
+struct GemmArgs {
+    const void* x;            // rows in position order (already gathered when perm is used)
+    const void* W0;
+    void* y;
+    const int32_t* perm;      // NULL or position -> output row
+    const int32_t* seg_offsets;
+    const int32_t* slot_ids;
+    const PlanWord* plan;
+    const __nv_bfloat16* u_blocks;
+    int T, d_in, d_out, G;
+    int num_sms;
+};
+// Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
+cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B,
+                              const GemmArgs& a, cudaStream_t stream);
+cudaError_t gemm_sm100_init(int device);   // sets the dynamic shared memory attribute
+bool encode_tmap_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
+                    uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer);
+bool encode_tmap_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                    uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
+                    uint32_t b2);
+
+struct DecodeArgs {
+    const void* x;
+    const void* W0;
+    void* y;
+    const int32_t* perm;
+    const int32_t* seg_offsets;
+    const int32_t* slot_ids;
+    float* u;            // [16][64] fp32, scale folded in
+    int32_t* row_slot;   // [16] slot of each row of x, -1 = none
+    int T, d_in, d_out, G;
+};
+cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
+                          cudaStream_t stream, int* launches);
+
+// ---- small device helpers -------------------------------------------------------------------
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&p);
+}
+
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Segment lookup shared by the kernels.  seg_offsets is assumed monotone (the shrink kernel
+// validates it and clears PlanWord::lora_ok otherwise); all results are clamped so that a
+// malformed array can only produce wrong-but-in-range indices.
+//
+// first segment whose end lies beyond `pos`
+__device__ __forceinline__ int seg_upper(const int32_t* __restrict__ seg_offsets, int G, int pos)
+{
+    int lo = 0, hi = G;   // answer in [0, G]
+    while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(seg_offsets + mid + 1) > pos) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ int slot_rank(const SlotSnapshot& snap, int slot)
+{
+    return (slot >= 0 && slot < snap.max_slots) ? (int)snap.rank[slot] : 0;
+}
+
+}  // namespace lml

@@ -287,7 +287,9 @@ def lattice(seed: int = 0, T: int = 200, d_in: int = 512, d_out: int = 384) -> W
         Af = _rng(seed, _STREAM_ADAPTER_A + e).integers(-1, 2, size=(4, K)).astype(np.float32)
         Bf = _rng(seed, _STREAM_ADAPTER_B + e).integers(-1, 2, size=(N, 4)).astype(np.float32)
         entries.append(AdapterEntry(e % 3, 1 + e // 3, 4, 1.0, f32_to_bf16_bits(Af), f32_to_bf16_bits(Bf)))
-    lens = (T // 3, 0, T // 4, 17, T - T // 3 - T // 4 - 17)
+    l0, l2 = T // 3, T // 4
+    l3 = min(17, T - l0 - l2)
+    lens = (l0, 0, l2, l3, T - l0 - l2 - l3)
     off, seg_entry, tok = segments_from_lengths(lens, (0, 1, 3, -1, 2))
     return Workload("lattice", K, N, T, f32_to_bf16_bits(xf), f32_to_bf16_bits(W0f), entries,
                     off, seg_entry, tok)
