@@ -122,7 +122,7 @@ lml_status lml_slot_info(const lml_table* t, int slot, int* adapter_id, int* ver
                          float* scale);
 
 /*
- * Bytes of device workspace lora_mixed_linear needs for T <= max_tokens and G <= max_segments
+ * Bytes of device workspace (256-byte aligned) lora_mixed_linear needs for T <= max_tokens and G <= max_segments
  * (with or without perm).  Contents need no initialisation and carry nothing between calls.
  * Returns 0 on invalid arguments.
  */

@@ -246,7 +246,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
     const bool decode = T <= kDecodeMaxT;
     const size_t need = decode ? ws.xg_off : (perm ? ws.total : ws.xg_off);
     const bool need_ws = G > 0 || (!decode && perm);
-    if (need_ws && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) || workspace_bytes < need))
+    if (need_ws && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need))
         return LML_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)stream_v;
     SlotSnapshot snap;
@@ -315,7 +315,7 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
     if (!t || T < 0 || G < 0 || T > kMaxTokens || G > kMaxTokens) return LML_ERR_INVALID_ARG;
     if (T == 0) { t->last_launches = 0; return LML_OK; }
     if (!x_host || !W0 || !y_host || (G > 0 && (!seg_offsets_host || !slot_ids_host))) return LML_ERR_INVALID_ARG;
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < lml_host_workspace_bytes(t, T, G))
         return LML_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)stream_v;

@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u);
         prefetch_tmap(&tmap_b); prefetch_tmap(&tmap_y);
     }
-    if (seg_cached) {
+    if (seg_cached && p.G > 0) {
         for (int g = threadIdx.x; g <= p.G; g += kGemmThreads) seg_cache[g] = __ldg(p.seg_offsets + g);
         for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
             int s = __ldg(p.slot_ids + g);
