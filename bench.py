@@ -1,0 +1,482 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-adapter LoRA linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path over one synthetic batch: the token-segmentation pass
+followed by lora_mixed_linear (decode kernels for T <= 16, else shrink + tcgen05 GEMM with the
+fused expand).  The primary workload is the 7B-class q_proj decode batch (8 tokens, 5 resident
+adapter entries); its metric is algorithmic HBM GB/s.  The same line carries, under "prefill",
+the 2048-token post-publish prefill batch in TFLOP/s.  Steps rotate through R distinct
+(W0, adapter table, x) sets so that successive steps never find their weights in L2, and are
+replayed from CUDA graphs so that launch gaps do not dominate microsecond kernels.
+
+Multi-GPU: the layer has no exchange step, so N ranks run N independent replicas (weak scaling);
+`value` is the sum over ranks divided by the slowest rank's time.
+
+--impl reference times the fp64 CPU oracle (test infrastructure, untuned) on the host cores on
+a bounded sample per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2608_15241_b200 import workloads as wl
+
+L2_BYTES = 126e6
+WORKLOADS = {
+    "decode_q_proj": dict(make=wl.decode_q_proj, kind="decode", metric="mixed-LoRA linear HBM GB/s (decode)",
+                          unit="GB/s", dtype="bf16"),
+    "prefill_q_proj": dict(make=wl.prefill_q_proj, kind="prefill", metric="mixed-LoRA linear TFLOP/s (prefill)",
+                           unit="TFLOP/s", dtype="bf16"),
+    "mlp_up_gate": dict(make=wl.mlp_up_gate, kind="prefill", metric="mixed-LoRA linear TFLOP/s (prefill)",
+                        unit="TFLOP/s", dtype="bf16"),
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=p["hbm_gbs"], tensor_burst=p["bf16_tflops"], tensor_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, tensor_burst=1590.0, tensor_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str | None):
+        self.rows = []
+        self.proc = None
+        self.uuid = uuid
+
+    def start(self):
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"]
+        if self.uuid:
+            cmd += ["-i", self.uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        for ts, line in self.rows:
+            if ts < t0 or ts > t1 + 0.06:
+                continue
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------------
+
+class Rotation:
+    """R resident sets of one workload: distinct W0 / x / adapter tables, same shapes and values
+    distribution (set 0 is the seeded workload itself, the others are row-rolled copies)."""
+
+    def __init__(self, w, device, min_bytes):
+        import torch
+        from paper_2608_15241_b200.binding import Table
+        self.w = w
+        self.device = device
+        per_set = w.bytes()
+        self.R = max(2, int(math.ceil(min_bytes / per_set)))
+        dev = lambda b: torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).view(torch.bfloat16).to(device)
+        x0, W00 = dev(w.x), dev(w.W0)
+        A0 = [dev(e.A) for e in w.entries]
+        B0 = [dev(e.B) for e in w.entries]
+        self.sets = []
+        G = len(w.entries) + 1
+        for i in range(self.R):
+            tbl = Table(w.d_in, w.d_out, max_slots=len(w.entries), device=torch.device(device).index or 0)
+            roll = lambda t: t if i == 0 else torch.roll(t, shifts=i, dims=0).contiguous()
+            slots = [tbl.register_adapter(e.adapter_id, e.version, roll(a), roll(b), e.scale)
+                     for e, a, b in zip(w.entries, A0, B0)]
+            tok = np.array([slots[e] if e >= 0 else -1 for e in w.token_entry], np.int32)
+            s = dict(table=tbl, x=x0 if i == 0 else roll(x0), W0=roll(W00),
+                     tok=torch.from_numpy(tok).to(device),
+                     perm=torch.empty(w.T, dtype=torch.int32, device=device),
+                     so=torch.empty(G + 1, dtype=torch.int32, device=device),
+                     ids=torch.empty(G, dtype=torch.int32, device=device),
+                     y=torch.empty((w.T, w.d_out), dtype=torch.bfloat16, device=device),
+                     slots=slots)
+            s["ws"] = torch.empty(tbl.workspace_bytes(w.T, max(G, w.G)), dtype=torch.uint8, device=device)
+            # pre-segmented form (segments as the workload states them) for the layer-only loop
+            s["so_pre"] = torch.from_numpy(w.seg_offsets).to(device)
+            s["ids_pre"] = torch.from_numpy(np.array([slots[e] if e >= 0 else -1 for e in w.seg_entry], np.int32)).to(device)
+            s["perm_pre"] = None if w.perm is None else torch.from_numpy(w.perm).to(device)
+            self.sets.append(s)
+        torch.cuda.synchronize()
+
+    def step(self, i):
+        """Whole hot path: segmentation pass + layer."""
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        t = s["table"]
+        st = b._stream(None)
+        b.lml_segment_tokens(t.handle, s["tok"].data_ptr(), self.w.T, s["perm"].data_ptr(), s["so"].data_ptr(),
+                             s["ids"].data_ptr(), st)
+        b.lora_mixed_linear(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["so"].data_ptr(),
+                            s["ids"].data_ptr(), t.max_slots + 1, s["perm"].data_ptr(), s["y"].data_ptr(),
+                            s["ws"].data_ptr(), s["ws"].numel(), st)
+        return 1 + t.last_launch_count()
+
+    def layer_only(self, i):
+        """lora_mixed_linear on pre-segmented input: the launches the roofline figure refers to."""
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        t = s["table"]
+        b.lora_mixed_linear(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["so_pre"].data_ptr(),
+                            s["ids_pre"].data_ptr(), self.w.G, 0 if s["perm_pre"] is None else s["perm_pre"].data_ptr(),
+                            s["y"].data_ptr(), s["ws"].data_ptr(), s["ws"].numel(), b._stream(None))
+        return t.last_launch_count()
+
+    def close(self):
+        for s in self.sets:
+            s["table"].close()
+
+
+def timed_graph_loop(fn, R, steps, warmup, stream, min_warm_seconds=0.0):
+    """Time exactly `steps` calls fn(i) replayed from CUDA graphs of R consecutive calls.
+    Returns (seconds, kernel launches inside the timed region, (t0, t1) wall clock)."""
+    import torch
+    launches_per = [0] * R
+    with torch.cuda.stream(stream):
+        for i in range(R):          # eager pass: allocations, lazy init
+            launches_per[i] = fn(i)
+        stream.synchronize()
+        g_full = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_full, stream=stream):
+            for i in range(R):
+                fn(i)
+        tail = steps % R
+        g_tail = None
+        if tail:
+            g_tail = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_tail, stream=stream):
+                for i in range(tail):
+                    fn(i)
+        warm_replays = max(1, -(-warmup // R))
+        t_w = time.time()
+        n = 0
+        while n < warm_replays or time.time() - t_w < min_warm_seconds:
+            g_full.replay()
+            n += 1
+            if n % 64 == 0:
+                stream.synchronize()
+        stream.synchronize()
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.time()
+        ev0.record(stream)
+        for _ in range(steps // R):
+            g_full.replay()
+        if g_tail is not None:
+            g_tail.replay()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        barrier()
+    launches = (steps // R) * sum(launches_per) + sum(launches_per[:tail])
+    return ev0.elapsed_time(ev1) / 1e3, launches, (t0, t1)
+
+
+def timed_e2e_loop(rot, steps, warmup, stream):
+    """Host buffers in, host buffer out, through lora_mixed_linear_host; copies inside the timed region."""
+    import torch
+    from paper_2608_15241_b200 import binding as b
+    w = rot.w
+    hosts = []
+    for s in rot.sets[: min(rot.R, 4)]:
+        xh = s["x"].cpu().pin_memory()
+        yh = torch.empty((w.T, w.d_out), dtype=torch.bfloat16).pin_memory()
+        so = s["so_pre"].cpu().pin_memory()
+        ids = s["ids_pre"].cpu().pin_memory()
+        pm = None if s["perm_pre"] is None else s["perm_pre"].cpu().pin_memory()
+        ws = torch.empty(b.lml_host_workspace_bytes(s["table"].handle, w.T, w.G), dtype=torch.uint8, device=rot.device)
+        hosts.append((s, xh, yh, so, ids, pm, ws))
+    h2d = w.T * w.d_in * 2 + (w.G + 1) * 4 + w.G * 4 + (w.T * 4 if w.perm is not None else 0)
+    d2h = w.T * w.d_out * 2
+
+    def call(i):
+        s, xh, yh, so, ids, pm, ws = hosts[i % len(hosts)]
+        b.lora_mixed_linear_host(s["table"].handle, xh.data_ptr(), s["W0"].data_ptr(), w.T, so.data_ptr(),
+                                 ids.data_ptr(), w.G, 0 if pm is None else pm.data_ptr(), yh.data_ptr(),
+                                 ws.data_ptr(), ws.numel(), b._stream(None))
+
+    with torch.cuda.stream(stream):
+        for i in range(max(3, warmup)):
+            call(i)
+        stream.synchronize()
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(steps):
+            call(i)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+    return ev0.elapsed_time(ev1) / 1e3, h2d, d2h
+
+
+_DIST = {"on": False}
+
+
+def barrier():
+    if _DIST["on"]:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(v: float) -> float:
+    if not _DIST["on"]:
+        return v
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([v], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def units_of(w, kind):
+    return w.bytes() / 1e9 if kind == "decode" else w.flops() / 1e12   # GB or TFLOP per step
+
+
+def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e2e_steps):
+    import torch
+    spec = WORKLOADS[name]
+    w = spec["make"]()
+    kind = spec["kind"]
+    rot = Rotation(w, device, 4 * L2_BYTES)
+    stream = torch.cuda.Stream(device=device)
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    t_load0 = time.time()
+    secs, launches, (t0, t1) = timed_graph_loop(rot.step, rot.R, steps, warmup, stream, min_warm_seconds=0.4)
+    clocks = sampler.stop(t_load0, t1)
+    secs = max_over_ranks(secs)
+    unit_per_step = units_of(w, kind)
+    value = world * steps * unit_per_step / secs
+
+    # the layer's own launches (pre-segmented input): what the roofline fraction is computed from
+    ksteps = max(rot.R, min(steps, 2000 if kind == "decode" else 200))
+    ksecs, klaunches, _ = timed_graph_loop(rot.layer_only, rot.R, ksteps, max(3, warmup // 4), stream)
+    per_launch = ksecs / ksteps
+    achieved = unit_per_step / per_launch
+    if kind == "decode":
+        roof = {"bound": "hbm", "kernel": "decode_main_kernel (shrink kernel overlapped by dependent launch)",
+                "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                "peak_source": peaks["source"], "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
+                "us_per_launch": per_launch * 1e6}
+    else:
+        roof = {"bound": "tensor", "kernel": "lora_gemm_sm100_kernel (time includes the shrink kernel before it)",
+                "achieved": achieved, "peak": peaks["tensor_burst"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["tensor_burst"], "peak_source": peaks["source"] + " burst",
+                "frac_of_sustained": achieved / peaks["tensor_sustained"], "frac_of_nominal_2250": achieved / 2250.0,
+                "traffic": None, "us_per_launch": per_launch * 1e6}
+
+    esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
+    esecs = max_over_ranks(esecs)
+    e2e = {"value": world * e2e_steps * unit_per_step / esecs, "unit": spec["unit"], "steps": e2e_steps,
+           "ms_per_step": esecs / e2e_steps * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # quick sampled parity of the last timed step against the oracle (rank 0)
+    out = {"metric": spec["metric"], "value": value, "unit": spec["unit"], "ms_per_step": secs / steps * 1e3,
+           "gpu_launches": launches, "roofline": roof, "e2e": e2e, "clocks": clocks,
+           "config": {"workload": name, "tokens": w.T, "d_in": w.d_in, "d_out": w.d_out,
+                      "resident_entries": len(w.entries), "segments": w.G, "rotation_sets": rot.R,
+                      "l2_policy": f"inputs larger than L2: {rot.R} distinct weight/activation sets "
+                                   f"({rot.R * w.bytes() / 1e6:.0f} MB) visited round-robin",
+                      "timing": "CUDA-graph replay of R-step chunks, CUDA events on the launch stream"}}
+    if want_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w, kind, spec["unit"], budget_s=12.0)
+        out["parity_sample"] = sampled_parity(rot)
+    rot.close()
+    return out
+
+
+def sampled_parity(rot):
+    import torch
+    import oracle
+    w = rot.w
+    s = rot.sets[0]
+    rot.step(0)
+    torch.cuda.synchronize()
+    y = s["y"].view(torch.int16).cpu().numpy().view(np.uint16)
+    rng = np.random.default_rng(0)
+    pos = np.unique(rng.integers(0, w.T, size=min(w.T, 8))).astype(np.int32)
+    ref, _ = oracle.forward_workload(w, positions=pos)
+    rows = pos if w.perm is None else w.perm[pos]
+    r = oracle.compare(y, ref, rows=rows)
+    r["rows"] = int(len(pos))
+    return r
+
+
+def cpu_baseline(w, kind, unit, budget_s):
+    """The oracle as it stands on the host cores, on a bounded row sample of the workload."""
+    import oracle
+    cores = oracle.threads()
+    probe = np.array([0], dtype=np.int32)
+    t = time.time()
+    oracle.forward_workload(w, positions=probe, nthreads=1)
+    per_row = max(time.time() - t, 1e-4)
+    rows = int(min(w.T, max(cores, budget_s * cores / per_row)))
+    pos = np.unique(np.linspace(0, w.T - 1, rows).astype(np.int32))
+    t = time.time()
+    oracle.forward_workload(w, positions=pos)
+    secs = time.time() - t
+    frac = len(pos) / w.T
+    v = units_of(w, kind) * frac / secs
+    return {"value": v, "unit": unit, "cores": cores, "kind": "oracle",
+            "sample": f"{len(pos)} of {w.T} token rows (all output columns), {secs:.2f} s wall on {cores} threads, "
+                      f"scaled by rows"}
+
+
+def run_reference(args):
+    """The reference arm of this tier: the fp64 oracle on host cores, a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    spec = WORKLOADS[args.workload]
+    w = spec["make"]()
+    kind = spec["kind"]
+    cores = oracle.threads()
+    t = time.time()
+    oracle.forward_workload(w, positions=np.array([0], np.int32), nthreads=1)
+    per_row = max(time.time() - t, 1e-4)
+    total = args.steps + args.warmup
+    budget = min(2.0, 150.0 / max(total, 1))                       # seconds of wall clock per step
+    rows = int(max(1, min(w.T, budget * cores / per_row)))
+    # when even one row per step is too slow, shrink the sample along output columns as well
+    col_frac = min(1.0, budget * cores / per_row) if rows == 1 else 1.0
+    n_cols = max(8, int(w.d_out * col_frac) // 8 * 8)
+    W0s = w.W0[:n_cols]
+    ents = [wl.AdapterEntry(e.adapter_id, e.version, e.rank, e.scale, e.A, e.B[:n_cols]) for e in w.entries]
+    pos = np.unique(np.linspace(0, w.T - 1, rows).astype(np.int32))
+
+    def step():
+        oracle.forward(w.x, W0s, ents, w.seg_offsets, w.seg_entry, w.perm, positions=pos)
+
+    for _ in range(args.warmup):
+        step()
+    t = time.time()
+    for _ in range(args.steps):
+        step()
+    secs = time.time() - t
+    frac = (len(pos) / w.T) * (n_cols / w.d_out)
+    value = args.steps * units_of(w, kind) * frac / secs
+    sample = f"{len(pos)} of {w.T} token rows x {n_cols} of {w.d_out} output columns per step, scaled by the fraction"
+    line = {"impl": "reference", "metric": spec["metric"], "value": value, "unit": spec["unit"], "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "tokens": w.T, "d_in": w.d_in, "d_out": w.d_out},
+            "cpu_baseline": {"value": value, "unit": spec["unit"], "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": spec["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=2000)
+    ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-secondary", action="store_true", help="skip the prefill line object")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    import __graft_entry__ as entry
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+        _DIST["on"] = True
+    if rank == 0:
+        entry.build()
+    barrier()
+    peaks = measured_peaks()
+    warmup = max(3, args.warmup)
+    primary = run_workload(args.workload, args.steps, warmup, device, world, peaks, rank == 0,
+                           e2e_steps=max(3, min(args.steps, 200)))
+    line = {"metric": primary.pop("metric"), "value": primary.pop("value"), "unit": primary.pop("unit"),
+            "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": primary.pop("ms_per_step"),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
+    line.update(primary)
+    if not args.no_secondary and args.workload == "decode_q_proj":
+        psteps = max(3, min(args.steps, 400))
+        sec = run_workload("prefill_q_proj", psteps, max(3, min(warmup, 40)), device, world, peaks, rank == 0,
+                           e2e_steps=max(3, min(psteps, 50)))
+        sec["steps"] = psteps
+        line["prefill"] = sec
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if _DIST["on"]:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -93,13 +93,14 @@ int lml_oracle_forward(const uint16_t *x, const uint16_t *W0, int T, int K, int 
         use_lora = 0;
     }
     int count = positions ? npos : T;
+    int nt = 1;
 #ifdef _OPENMP
-    if (nthreads > 0) omp_set_num_threads(nthreads);
+    nt = nthreads > 0 ? nthreads : omp_get_max_threads();
 #else
     (void)nthreads;
 #endif
     uint32_t flag_acc = 0;
-#pragma omp parallel for schedule(dynamic, 1) reduction(| : flag_acc)
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : flag_acc) num_threads(nt)
     for (int i = 0; i < count; ++i) {
         int p = positions ? positions[i] : i;
         int t = perm ? perm[p] : p;
