@@ -61,7 +61,8 @@ typedef enum {
     LML_ERR_UNSUPPORTED = 6, /* device is not sm_100 */
     LML_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed */
     LML_ERR_TIMEOUT = 8,
-    LML_ERR_WORKSPACE = 9    /* workspace missing, misaligned or smaller than lml_workspace_bytes */
+    LML_ERR_WORKSPACE = 9,   /* workspace missing, misaligned or smaller than lml_workspace_bytes */
+    LML_ERR_TOO_LARGE = 10   /* the call is larger than a fixed-capacity entry point can take */
 } lml_status;
 
 /* bits of the device status word (lml_device_status) */
@@ -172,6 +173,37 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
                                   const int32_t* seg_offsets_host, const int32_t* slot_ids_host,
                                   int G, const int32_t* perm_host, void* y_host, void* workspace,
                                   size_t workspace_bytes, void* stream);
+
+/*
+ * lora_mixed_linear_decode_static — the decode form of lora_mixed_linear (T <= 16) for callers
+ * that cannot give the library a workspace.  (The paper has no counterpart; this entry point
+ * exists for integration only.)
+ *
+ * Who needs it: code that runs where device memory cannot be obtained — a plug-in or callback
+ * invoked by a host runtime that owns all allocations and forbids cudaMalloc from inside the
+ * callback, a real-time loop that must not touch the allocator, a process whose memory budget
+ * was handed out completely at start-up.  Such a caller still passes its inputs and the output
+ * (x, W0, seg_offsets, slot_ids, perm, y: same meaning, layout and alignment as in
+ * lora_mixed_linear), but no workspace: the scratch the decode kernels need between their two
+ * passes (the scaled shrink result, 16 x 64 fp32, and the slot of each row) lives in a 4352-byte
+ * array inside the library image.  Every GPU that loads the library holds that array until the
+ * process exits.  The call allocates and frees nothing, and calls no allocating routine.
+ *
+ * Limits and rules
+ *   - T <= LML_DECODE_MAX_TOKENS (16).  A larger T is refused with LML_ERR_TOO_LARGE before
+ *     anything is launched; use lora_mixed_linear with a workspace for it.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.
+ *     The call resets what must not leak from an earlier call (the per-row slots) itself, on
+ *     `stream`, before its kernels run.  Two calls that overlap on the GPU (different streams
+ *     without ordering, or concurrent graph branches) race on the array: order them.
+ *   - Results are identical to lora_mixed_linear on the same inputs.
+ * Errors: INVALID_ARG, TOO_LARGE, CUDA.
+ */
+lml_status lora_mixed_linear_decode_static(lml_table* t, const void* x, const void* W0, int T,
+                                           const int32_t* seg_offsets, const int32_t* slot_ids, int G,
+                                           const int32_t* perm, void* y, void* stream);
 
 /*
  * Read and clear the sticky device status word (LML_FLAG_* bits).  Synchronises `stream`.

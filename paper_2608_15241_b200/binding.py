@@ -20,14 +20,15 @@ LIB_PATH = os.path.join(_HERE, "liblora_mixed_linear.so")
 LML_OK = 0
 STATUS_NAMES = {0: "LML_OK", 1: "LML_ERR_INVALID_ARG", 2: "LML_ERR_BAD_SLOT", 3: "LML_ERR_TABLE_FULL",
                 4: "LML_ERR_DUPLICATE", 5: "LML_ERR_NOT_FOUND", 6: "LML_ERR_UNSUPPORTED",
-                7: "LML_ERR_CUDA", 8: "LML_ERR_TIMEOUT", 9: "LML_ERR_WORKSPACE"}
+                7: "LML_ERR_CUDA", 8: "LML_ERR_TIMEOUT", 9: "LML_ERR_WORKSPACE", 10: "LML_ERR_TOO_LARGE"}
 FLAG_BAD_SLOT, FLAG_BAD_OFFSETS, FLAG_BAD_PERM, FLAG_TIMEOUT = 1, 2, 4, 8
 MAX_SLOTS, MAX_RANK, DECODE_MAX_TOKENS = 64, 64, 16
 
 EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "register_adapter",
            "retire_version", "lml_lookup", "lml_slot_info", "lml_workspace_bytes",
            "lml_segment_tokens", "lora_mixed_linear", "lml_host_workspace_bytes",
-           "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count")
+           "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count",
+           "lora_mixed_linear_decode_static")
 
 
 class LmlError(RuntimeError):
@@ -64,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.lml_segment_tokens.argtypes = [vp, vp, i32, vp, vp, vp, vp]
         L.lora_mixed_linear.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lora_mixed_linear_host.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.lora_mixed_linear_decode_static.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
         L.lml_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
@@ -146,6 +148,14 @@ def lora_mixed_linear_host(table: int, x_host_ptr: int, W0_ptr: int, T: int, seg
     _check(lib().lora_mixed_linear_host(table, x_host_ptr, W0_ptr, T, seg_offsets_host_ptr, slot_ids_host_ptr, G,
                                         perm_host_ptr, y_host_ptr, workspace_ptr, workspace_bytes, stream),
            "lora_mixed_linear_host")
+
+
+def lora_mixed_linear_decode_static(table: int, x_ptr: int, W0_ptr: int, T: int, seg_offsets_ptr: int,
+                                    slot_ids_ptr: int, G: int, perm_ptr: int, y_ptr: int, stream: int = 0) -> None:
+    """Decode form (T <= 16) that takes no workspace: its scratch is a fixed array inside the
+    library, so the call allocates nothing.  For callers that cannot obtain device memory."""
+    _check(lib().lora_mixed_linear_decode_static(table, x_ptr, W0_ptr, T, seg_offsets_ptr, slot_ids_ptr, G,
+                                                 perm_ptr, y_ptr, stream), "lora_mixed_linear_decode_static")
 
 
 def lml_device_status(table: int, stream: int = 0) -> int:

@@ -1,53 +1,14 @@
 // Host side of the C ABI: the adapter slot table, argument validation, workspace layout and
 // dispatch to the decode / prefill kernels.  See include/lora_mixed_linear.h for the contract.
-#include <mutex>
 #include <new>
 
-#include "lml_internal.cuh"
+#include "lml_table.cuh"
 
 using namespace lml;
 
-struct lml_table {
-    int device = 0, d_in = 0, d_out = 0, max_slots = 0, num_sms = 0;
-    struct Entry {
-        bool live = false;
-        int adapter_id = 0, version = 0, rank = 0;
-        float scale = 0.f;
-    } entries[kMaxSlots];
-    Arena arena{};
-    CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
-    int last_launches = 0;
-    mutable std::mutex mu;
-};
-
 namespace {
 
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceGuard(int dev)
-    {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-        if (prev == dev) prev = -1;
-    }
-    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
-};
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
-SlotSnapshot snapshot(const lml_table* t)
-{
-    SlotSnapshot s;
-    for (int i = 0; i < kMaxSlots; ++i) {
-        const bool live = i < t->max_slots && t->entries[i].live;
-        s.rank[i] = live ? (uint8_t)t->entries[i].rank : 0;
-        s.scale[i] = live ? t->entries[i].scale : 0.f;
-    }
-    s.max_slots = t->max_slots;
-    return s;
-}
 
 // Workspace layout of the prefill path: [PlanWord][u blocks][gathered x (perm form only)];
 // the decode path uses [PlanWord][u fp32 16x64][row_slot 16].
@@ -68,8 +29,6 @@ WsLayout ws_layout(const lml_table* t, int T, int G)
     return w;
 }
 
-const int kMaxTokens = kTileM * 32768;   // keeps every grid dimension and int index in range
-
 }  // namespace
 
 extern "C" {
@@ -87,6 +46,7 @@ const char* lml_status_string(lml_status s)
         case LML_ERR_CUDA: return "CUDA call failed";
         case LML_ERR_TIMEOUT: return "device wait timed out";
         case LML_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case LML_ERR_TOO_LARGE: return "call exceeds the fixed capacity of this entry point";
     }
     return "unknown status";
 }
@@ -217,11 +177,7 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
 {
     if (!t || T < 0 || T > kMaxTokens || !seg_offsets || !seg_slot_ids || (T > 0 && (!token_slots || !perm)))
         return LML_ERR_INVALID_ARG;
-    SlotSnapshot snap;
-    {
-        std::lock_guard<std::mutex> lock(t->mu);
-        snap = snapshot(t);
-    }
+    const SlotSnapshot snap = snapshot_locked(t);
     DeviceGuard guard(t->device);
     if (!guard.ok) return LML_ERR_CUDA;
     if (launch_segment_tokens(t->arena, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, (cudaStream_t)stream) !=
@@ -249,11 +205,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
     if (need_ws && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need))
         return LML_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)stream_v;
-    SlotSnapshot snap;
-    {
-        std::lock_guard<std::mutex> lock(t->mu);
-        snap = snapshot(t);
-    }
+    const SlotSnapshot snap = snapshot_locked(t);
     DeviceGuard guard(t->device);
     if (!guard.ok) return LML_ERR_CUDA;
     uint8_t* wsb = static_cast<uint8_t*>(workspace);

@@ -1,0 +1,83 @@
+// lora_mixed_linear_decode_static: the decode form of the layer for callers that cannot hand the
+// library any scratch memory.  See the declaration in include/lora_mixed_linear.h.
+//
+// The decode kernels need a little scratch between the shrink pass and the main pass: the
+// scaled shrink result u[16][64] (fp32) and the slot of each of the 16 rows.  The regular entry
+// point takes it from the caller's workspace.  Here it lives in a file-scope device array that
+// is part of the library image: every GPU context that loads the library carries these 4352
+// bytes until the process exits, and nothing is ever allocated or freed.
+#include "lml_table.cuh"
+
+using namespace lml;
+
+namespace {
+
+constexpr size_t kStaticU = (size_t)kDecodeMaxT * kRankPad * sizeof(float);   // 4096 bytes
+constexpr size_t kStaticRowSlot = kDecodeMaxT * sizeof(int32_t);              // 64 bytes
+constexpr size_t kStaticScratchBytes = 4352;                                   // rounded up to 256
+static_assert(kStaticU + kStaticRowSlot <= kStaticScratchBytes, "static scratch too small");
+
+// In host code this name is only a handle for the runtime, not a device address: the address the
+// kernels get is looked up once per device with cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_setup_mu;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device` (which must be the current device).  The first
+// call on a device asks the runtime for it; later calls reuse the answer.
+cudaError_t scratch_address(int device, void** out)
+{
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (!g_scratch_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_decode_scratch);
+        if (e != cudaSuccess) return e;
+        if (!p) return cudaErrorInvalidSymbol;
+        g_scratch_ptr[device] = p;
+    }
+    *out = g_scratch_ptr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" lml_status lora_mixed_linear_decode_static(lml_table* t, const void* x, const void* W0, int T,
+                                                      const int32_t* seg_offsets, const int32_t* slot_ids, int G,
+                                                      const int32_t* perm, void* y, void* stream_v)
+{
+    if (!t || T < 0 || G < 0 || G > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (T > kDecodeMaxT) return LML_ERR_TOO_LARGE;   // the static scratch holds 16 token rows, no more
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x || !W0 || !y || !aligned16(x) || !aligned16(W0) || !aligned16(y)) return LML_ERR_INVALID_ARG;
+    if (G > 0 && (!seg_offsets || !slot_ids)) return LML_ERR_INVALID_ARG;
+    if (G == 0) perm = nullptr;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    const SlotSnapshot snap = snapshot_locked(t);
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+
+    void* scratch = nullptr;
+    if (scratch_address(t->device, &scratch) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    float* u = static_cast<float*>(scratch);
+    int32_t* row_slot = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(scratch) + kStaticU);
+
+    int launches = 0;
+    if (G > 0) {
+        // The array keeps whatever the previous call left.  u is rewritten for every row the call
+        // addresses, but a row that a malformed perm never names would keep an old slot: start all
+        // rows at "no adapter" (-1 = all bits set).
+        if (cudaMemsetAsync(row_slot, 0xFF, kStaticRowSlot, stream) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    }
+    DecodeArgs a;
+    a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
+    a.u = G > 0 ? u : nullptr;
+    a.row_slot = G > 0 ? row_slot : nullptr;
+    a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G;
+    cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
+    t->last_launches = launches;
+    if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    return LML_OK;
+}

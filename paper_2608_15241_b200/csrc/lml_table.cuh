@@ -1,0 +1,53 @@
+// The adapter slot table object behind the opaque lml_table handle, shared by the files that
+// implement the C ABI.  Not part of the public ABI.
+#pragma once
+#include <mutex>
+
+#include "lml_internal.cuh"
+
+struct lml_table {
+    int device = 0, d_in = 0, d_out = 0, max_slots = 0, num_sms = 0;
+    struct Entry {
+        bool live = false;
+        int adapter_id = 0, version = 0, rank = 0;
+        float scale = 0.f;
+    } entries[lml::kMaxSlots];
+    lml::Arena arena{};
+    CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
+    int last_launches = 0;
+    mutable std::mutex mu;
+};
+
+namespace lml {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Copy of the live slots' rank and scale, taken under the table's lock.
+inline SlotSnapshot snapshot_locked(const lml_table* t)
+{
+    std::lock_guard<std::mutex> lock(t->mu);
+    SlotSnapshot s;
+    for (int i = 0; i < kMaxSlots; ++i) {
+        const bool live = i < t->max_slots && t->entries[i].live;
+        s.rank[i] = live ? (uint8_t)t->entries[i].rank : 0;
+        s.scale[i] = live ? t->entries[i].scale : 0.f;
+    }
+    s.max_slots = t->max_slots;
+    return s;
+}
+
+constexpr int kMaxTokens = kTileM * 32768;   // keeps every grid dimension and int index in range
+
+}  // namespace lml
