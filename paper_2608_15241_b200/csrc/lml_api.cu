@@ -80,6 +80,7 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && cudaMemset(t->arena.B, 0, b_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
     ok = ok && gemm_sm100_init(device) == cudaSuccess;
+    ok = ok && shrink_init() == cudaSuccess;
     ok = ok && encode_tmap_3d(&t->tmap_B256, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -238,6 +239,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
             a.x = xg; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
             a.plan = plan; a.u_blocks = u_blocks ? u_blocks : reinterpret_cast<const __nv_bfloat16*>(x);
             a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
+            a.overlap_with_previous = G > 0;
             if (G == 0) a.u_blocks = reinterpret_cast<const __nv_bfloat16*>(W0);   // never read; map needs a valid base
             e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
             if (e == cudaSuccess) ++launches;

@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            const bool lora = p.G > 0 && p.plan->lora_ok != 0;
+            bool lora = false, lora_known = (p.G == 0);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -129,21 +129,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m = tile % p.num_m, n = tile / p.num_m;
                 const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
-                // pieces of this tile: segments with a live slot that overlap [row0, row1)
-                int g_first = 0, g_end = 0;
-                if (lora) {
-                    if (seg_cached) {
-                        int lo = 0, hi = p.G;
-                        while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
-                        g_first = lo;
-                        g_end = g_first;
-                        while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
-                    } else {
-                        g_first = seg_upper(p.seg_offsets, p.G, row0);
-                        g_end = g_first;
-                        while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
-                    }
-                }
+                int g_first = 0, g_end = 0, last_piece = -1;
                 auto piece_slot = [&](int g) -> int {   // -1 = segment contributes no piece
                     int s0, s1, s;
                     if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
@@ -154,10 +140,31 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                     if (min(s1, row1) <= max(s0, row0)) return -1;
                     return s;
                 };
-                int last_piece = -1;
-                for (int g = g_first; g < g_end; ++g) if (piece_slot(g) >= 0) last_piece = g;
-
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    if (kb == num_kb - 1) {
+                        // Pieces of this tile: segments with a live slot that overlap [row0, row1).
+                        // Everything the shrink kernel wrote (plan word, u blocks) is first touched
+                        // here, after the base k-blocks of the first tile are already in flight.
+                        if (!lora_known) {
+                            grid_dependency_wait();
+                            lora = p.plan->lora_ok != 0;
+                            lora_known = true;
+                        }
+                        if (lora) {
+                            if (seg_cached) {
+                                int lo = 0, hi = p.G;
+                                while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+                                g_first = lo;
+                                g_end = g_first;
+                                while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
+                            } else {
+                                g_first = seg_upper(p.seg_offsets, p.G, row0);
+                                g_end = g_first;
+                                while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
+                            }
+                            for (int g = g_first; g < g_end; ++g) if (piece_slot(g) >= 0) last_piece = g;
+                        }
+                    }
                     ok = acquire();
                     if (!ok) break;
                     const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
@@ -404,11 +411,18 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
     p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
     const int grid = min(num_m * num_n, a.num_sms);
-    if (bn == 256)
-        lora_gemm_sm100_kernel<256><<<grid, kGemmThreads, GemmCfg<256>::kSmemBytes, stream>>>(tx, tw, tu, tb, ty, snap, p);
-    else
-        lora_gemm_sm100_kernel<128><<<grid, kGemmThreads, GemmCfg<128>::kSmemBytes, stream>>>(tx, tw, tu, tb, ty, snap, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.overlap_with_previous ? 1 : 0;   // only ever our own shrink kernel
+    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tw, tu, tb, ty, snap, p);
+    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tw, tu, tb, ty, snap, p);
 }
 
 }  // namespace lml

@@ -67,11 +67,13 @@ struct GemmArgs {
     const __nv_bfloat16* u_blocks;
     int T, d_in, d_out, G;
     int num_sms;
+    bool overlap_with_previous;   // launch as a programmatic dependent of the shrink kernel before it
 };
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
 cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B,
                               const GemmArgs& a, cudaStream_t stream);
-cudaError_t gemm_sm100_init(int device);   // sets the dynamic shared memory attribute
+cudaError_t gemm_sm100_init(int device);
+cudaError_t shrink_init();   // both set the dynamic shared memory attributes of their kernels
 bool encode_tmap_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
                     uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer);
 bool encode_tmap_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,

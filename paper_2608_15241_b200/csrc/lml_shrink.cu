@@ -11,30 +11,53 @@
 // The contraction runs on mma.sync m16n8k16 with operands loaded straight from global memory
 // by 128-bit loads: a dot product does not care about the order of k, so lane (g, t) takes
 // the 8 consecutive k at offset 8t of each 32-wide step for both operands and feeds them to
-// two MMAs.  Each CTA owns 16 rows of one piece; its 4 warps split K and are summed in a
-// fixed order in shared memory (deterministic).
+// two MMAs.  The pass is bound by reading x once, so what matters is bytes in flight: a
+// thread-block cluster of up to 8 CTAs splits K for one 32-row slab of a piece, every warp
+// issues all the loads of four steps before its first MMA, and the partial sums are combined
+// in a fixed order — warps through shared memory, CTAs through distributed shared memory — so
+// the result is deterministic and needs no scratch in global memory.
+#include <cooperative_groups.h>
+
 #include "lml_internal.cuh"
+#include "lml_ptx_sm100.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace lml {
 
-constexpr int kShrinkWarps = 4;
-constexpr int kShrinkRows = 16;
+constexpr int kShrinkWarps = 8;
+constexpr int kShrinkRows = 32;       // rows of one CTA (two 16-row MMA tiles)
+constexpr int kShrinkUnroll = 4;
+constexpr int kShrinkMaxCluster = 8;
 
+template <int NB> struct ShrinkSmem {
+    static constexpr int kCols = NB * 8;
+    static constexpr int kPitch = kCols + 2;
+    static constexpr int kBytes = (kShrinkWarps * kShrinkRows * kPitch + kShrinkRows * kCols) * 4;
+};
+
+// NB = number of 8-column blocks of u that can be non-zero (rank <= 8 * NB).
+template <int NB>
 __global__ void __launch_bounds__(kShrinkWarps * 32) shrink_pieces_kernel(
     const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
     uint32_t* __restrict__ status, const __nv_bfloat16* __restrict__ x, int T, int K,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids, int G,
-    const int32_t* __restrict__ perm, PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks,
-    int num_tiles)
+    PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles)
 {
-    __shared__ float red[kShrinkWarps][kShrinkRows][kRankPad + 2];
+    ptx::grid_launch_dependents();   // the GEMM that follows may start its main loop now
+    extern __shared__ float shrink_smem[];
+    using S = ShrinkSmem<NB>;
+    float* red = shrink_smem;                                           // [warp][row][pitch]
+    float* partial = shrink_smem + kShrinkWarps * kShrinkRows * S::kPitch;   // [row][cols]
     __shared__ int sh_piece[4];   // slot, lo, hi, found
 
+    cg::cluster_group cluster = cg::this_cluster();
+    const int KS = (int)gridDim.z, ks = (int)blockIdx.z;
     const int b = blockIdx.y, sub = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // One CTA validates the segment arrays for the whole call.
-    if (b == 0 && sub == 0) {
+    if (b == 0 && sub == 0 && ks == 0) {
         int bad_off = 0, bad_slot = 0;
         for (int g = tid; g < G; g += blockDim.x) {
             int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
@@ -67,101 +90,163 @@ __global__ void __launch_bounds__(kShrinkWarps * 32) shrink_pieces_kernel(
                 plo = max(max(s0, m * kTileM), 0);
                 phi = min(min(s1, (m + 1) * kTileM), T);
                 slot = __ldg(slot_ids + g);
-                found = (plo < phi) && slot_rank(snap, slot) > 0;
+                const int r = slot_rank(snap, slot);
+                found = (plo < phi) && r > 0 && r <= NB * 8;
             }
         }
         sh_piece[0] = slot; sh_piece[1] = plo; sh_piece[2] = phi; sh_piece[3] = found;
     }
     __syncthreads();
+    // Every CTA of a cluster shares (b, sub) and therefore takes the same exits below.
     if (!sh_piece[3]) return;
     const int slot = sh_piece[0], plo = sh_piece[1], phi = sh_piece[2];
     const int m = plo / kTileM;
-    const int rank = snap.rank[slot];
-    const int nblk = (rank + 7) >> 3;
+    const int nblk = ((int)snap.rank[slot] + 7) >> 3;
     const int p0 = m * kTileM + sub * kShrinkRows;
     uint4* out = reinterpret_cast<uint4*>(u_blocks + ((size_t)b * kTileM + sub * kShrinkRows) * kRankPad);
 
-    if (p0 + kShrinkRows <= plo || p0 >= phi) {   // no row of this sub-block is in the piece
-        out[tid] = make_uint4(0, 0, 0, 0);        // 16 rows x 128 B = 128 x 16 B
+    if (p0 + kShrinkRows <= plo || p0 >= phi) {   // no row of this slab is in the piece
+        if (ks == 0) out[tid] = make_uint4(0, 0, 0, 0);   // 32 rows x 128 B = 256 x 16 B
         return;
     }
 
     const int gq = lane >> 2, tq = lane & 3;
-    int pa = p0 + gq, pb = p0 + gq + 8;
-    bool va = pa >= plo && pa < phi, vb = pb >= plo && pb < phi;
-    if (perm) {
-        bool badp = false;
-        if (va) { pa = __ldg(perm + pa); if (pa < 0 || pa >= T) { va = false; badp = true; } }
-        if (vb) { pb = __ldg(perm + pb); if (pb < 0 || pb >= T) { vb = false; badp = true; } }
-        if (badp) atomicOr(status, LML_FLAG_BAD_PERM);
-    }
-    const __nv_bfloat16* xa = x + (size_t)(va ? pa : 0) * K;
-    const __nv_bfloat16* xb = x + (size_t)(vb ? pb : 0) * K;
-    const __nv_bfloat16* Abase = arenaA + ((size_t)slot * kRankPad + gq) * K;
-
-    float acc[8][4];
+    const __nv_bfloat16* xr[4];
+    bool xv[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
+    for (int i = 0; i < 4; ++i) {
+        const int p = p0 + gq + 8 * i;
+        xv[i] = p >= plo && p < phi;
+        xr[i] = x + (size_t)(xv[i] ? p : 0) * K + tq * 8;
+    }
+    const __nv_bfloat16* Abase = arenaA + ((size_t)slot * kRankPad + gq) * K + tq * 8;
+
+    float acc[2][NB][4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) acc[h][nb][0] = acc[h][nb][1] = acc[h][nb][2] = acc[h][nb][3] = 0.f;
 
     const int steps = (K + 31) >> 5;
+    const int stride = KS * kShrinkWarps;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
-#pragma unroll 2
-    for (int s = warp; s < steps; s += kShrinkWarps) {
-        const int k = s * 32 + tq * 8;
-        const bool kv = k < K;
-        uint4 ra = (va && kv) ? ldg_nc_v4(xa + k) : zero4;
-        uint4 rb = (vb && kv) ? ldg_nc_v4(xb + k) : zero4;
+    for (int s0 = ks * kShrinkWarps + warp; s0 < steps; s0 += stride * kShrinkUnroll) {
+        uint4 xa[kShrinkUnroll][4];
 #pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
+        for (int i = 0; i < kShrinkUnroll; ++i) {
+            const int k = (s0 + i * stride) * 32;
+            const bool kv = k + tq * 8 < K;   // also false for steps past the end
+#pragma unroll
+            for (int r = 0; r < 4; ++r) xa[i][r] = (xv[r] && kv) ? ldg_nc_v4(xr[r] + k) : zero4;
+        }
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
             if (nb < nblk) {
-                uint4 w = kv ? ldg_nc_v4(Abase + (size_t)nb * 8 * K + k) : zero4;
-                mma_bf16_16816(acc[nb], ra.x, rb.x, ra.y, rb.y, w.x, w.y);
-                mma_bf16_16816(acc[nb], ra.z, rb.z, ra.w, rb.w, w.z, w.w);
+                uint4 w[kShrinkUnroll];
+#pragma unroll
+                for (int i = 0; i < kShrinkUnroll; ++i) {
+                    const int k = (s0 + i * stride) * 32;
+                    w[i] = (k + tq * 8 < K) ? ldg_nc_v4(Abase + (size_t)nb * 8 * K + k) : zero4;
+                }
+#pragma unroll
+                for (int i = 0; i < kShrinkUnroll; ++i) {
+                    mma_bf16_16816(acc[0][nb], xa[i][0].x, xa[i][1].x, xa[i][0].y, xa[i][1].y, w[i].x, w[i].y);
+                    mma_bf16_16816(acc[0][nb], xa[i][0].z, xa[i][1].z, xa[i][0].w, xa[i][1].w, w[i].z, w[i].w);
+                    mma_bf16_16816(acc[1][nb], xa[i][2].x, xa[i][3].x, xa[i][2].y, xa[i][3].y, w[i].x, w[i].y);
+                    mma_bf16_16816(acc[1][nb], xa[i][2].z, xa[i][3].z, xa[i][2].w, xa[i][3].w, w[i].z, w[i].w);
+                }
             }
         }
     }
 
+    // warps -> CTA partial, fixed order
+    float* myred = red + warp * kShrinkRows * S::kPitch;
 #pragma unroll
-    for (int nb = 0; nb < 8; ++nb) {
-        if (nb < nblk) {
-            red[warp][gq][nb * 8 + tq * 2] = acc[nb][0];
-            red[warp][gq][nb * 8 + tq * 2 + 1] = acc[nb][1];
-            red[warp][gq + 8][nb * 8 + tq * 2] = acc[nb][2];
-            red[warp][gq + 8][nb * 8 + tq * 2 + 1] = acc[nb][3];
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+            const int c = nb * 8 + tq * 2;
+            myred[(h * 16 + gq) * S::kPitch + c] = acc[h][nb][0];
+            myred[(h * 16 + gq) * S::kPitch + c + 1] = acc[h][nb][1];
+            myred[(h * 16 + gq + 8) * S::kPitch + c] = acc[h][nb][2];
+            myred[(h * 16 + gq + 8) * S::kPitch + c + 1] = acc[h][nb][3];
         }
-    }
     __syncthreads();
-    {
+    for (int e = tid; e < kShrinkRows * S::kCols; e += kShrinkWarps * 32) {
+        const int row = e / S::kCols, col = e % S::kCols;
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kShrinkWarps; ++w) s += red[(w * kShrinkRows + row) * S::kPitch + col];
+        partial[e] = s;
+    }
+    cluster.sync();
+    if (ks == 0) {   // CTAs -> result, fixed order, through distributed shared memory
         const int row = tid >> 3, c0 = (tid & 7) * 8;
         const float sc = snap.scale[slot];
         float v[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float s = 0.f;
-            if (c0 + i < nblk * 8) {
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        if (c0 < S::kCols) {
+            for (int r = 0; r < KS; ++r) {
+                const float* peer = cluster.map_shared_rank(partial, r) + row * S::kCols + c0;
 #pragma unroll
-                for (int w = 0; w < kShrinkWarps; ++w) s += red[w][row][c0 + i];
+                for (int i = 0; i < 8; ++i) v[i] += peer[i];
             }
-            v[i] = s * sc;
         }
         uint4 o;
-        o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]);
-        o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+        o.x = pack_bf16(v[0] * sc, v[1] * sc); o.y = pack_bf16(v[2] * sc, v[3] * sc);
+        o.z = pack_bf16(v[4] * sc, v[5] * sc); o.w = pack_bf16(v[6] * sc, v[7] * sc);
         out[row * 8 + (tid & 7)] = o;
     }
+    cluster.sync();   // peers stay alive until their partials have been read
+}
+
+template <int NB>
+static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
+                                    const int32_t* seg_offsets, const int32_t* slot_ids, int G, PlanWord* plan,
+                                    __nv_bfloat16* u_blocks, cudaStream_t stream)
+{
+    const int num_tiles = (T + kTileM - 1) / kTileM;
+    int ks = (d_in + 1023) / 1024;
+    ks = ks < 1 ? 1 : (ks > kShrinkMaxCluster ? kShrinkMaxCluster : ks);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kTileM / kShrinkRows, num_tiles + G, ks);
+    cfg.blockDim = dim3(kShrinkWarps * 32);
+    cfg.dynamicSmemBytes = ShrinkSmem<NB>::kBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = ks;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const __nv_bfloat16* arenaA = ar.A;
+    uint32_t* status = ar.status;
+    const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
+    return cudaLaunchKernelEx(&cfg, shrink_pieces_kernel<NB>, snap, arenaA, status, xb, T, d_in, seg_offsets,
+                              slot_ids, G, plan, u_blocks, num_tiles);
+}
+
+cudaError_t shrink_init()
+{
+    cudaError_t e = cudaFuncSetAttribute(shrink_pieces_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ShrinkSmem<2>::kBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(shrink_pieces_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                ShrinkSmem<8>::kBytes);
 }
 
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
-                                 const int32_t* perm, PlanWord* plan, __nv_bfloat16* u_blocks,
+                                 const int32_t* /*perm*/, PlanWord* plan, __nv_bfloat16* u_blocks,
                                  cudaStream_t stream)
 {
-    const int num_tiles = (T + kTileM - 1) / kTileM;
-    dim3 grid(kTileM / kShrinkRows, num_tiles + G);
-    shrink_pieces_kernel<<<grid, kShrinkWarps * 32, 0, stream>>>(
-        snap, ar.A, ar.status, (const __nv_bfloat16*)x, T, d_in, seg_offsets, slot_ids, G, perm, plan,
-        u_blocks, num_tiles);
-    return cudaGetLastError();
+    int max_rank = 0;
+    for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
+    if (max_rank <= 16)
+        return launch_shrink_nb<2>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, plan, u_blocks, stream);
+    return launch_shrink_nb<8>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, plan, u_blocks, stream);
 }
 
 }  // namespace lml
