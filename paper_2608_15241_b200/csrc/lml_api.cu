@@ -81,6 +81,7 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
     ok = ok && gemm_sm100_init(device) == cudaSuccess;
     ok = ok && shrink_init() == cudaSuccess;
+    ok = ok && decode_init() == cudaSuccess;
     ok = ok && encode_tmap_3d(&t->tmap_B256, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -219,7 +220,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         a.u = G > 0 ? reinterpret_cast<float*>(wsb + ws.u_off) : nullptr;
         a.row_slot = G > 0 ? reinterpret_cast<int32_t*>(wsb + ws.u_off + (size_t)kDecodeMaxT * kRankPad * sizeof(float))
                            : nullptr;
-        a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G;
+        a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         e = launch_decode(t->arena, snap, a, stream, &launches);
     } else {
         const void* xg = x;

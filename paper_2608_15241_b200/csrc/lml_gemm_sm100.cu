@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int m = tile % p.num_m, n = tile / p.num_m;
             const int row_base = m * kBM + q * 32;
-            ok = mbar_wait(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
+            ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);

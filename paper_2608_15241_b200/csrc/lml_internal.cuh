@@ -90,7 +90,9 @@ struct DecodeArgs {
     float* u;            // [16][64] fp32, scale folded in
     int32_t* row_slot;   // [16] slot of each row of x, -1 = none
     int T, d_in, d_out, G;
+    int num_sms;
 };
+cudaError_t decode_init();   // sets the dynamic shared memory attribute
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
                           cudaStream_t stream, int* launches);
 

@@ -75,7 +75,7 @@ extern "C" lml_status lora_mixed_linear_decode_static(lml_table* t, const void* 
     a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
     a.u = G > 0 ? u : nullptr;
     a.row_slot = G > 0 ? row_slot : nullptr;
-    a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G;
+    a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
     cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
     t->last_launches = launches;
     if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }

@@ -53,6 +53,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Wait on behalf of a whole converged warp: lane 0 polls, the others park at the warp barrier, and
+// everybody gets the same verdict, so the warp never splits around a *.sync / *.aligned instruction
+// after a give-up and the barrier is not polled by 32 threads at once.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+
 // ---- proxy fences -------------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
