@@ -265,7 +265,7 @@ def timed_e2e_loop(rot, steps, warmup, stream):
     return ev0.elapsed_time(ev1) / 1e3, h2d, d2h
 
 
-_DIST = {"on": False}
+_DIST = {"on": False, "device": "cuda"}
 
 
 def barrier():
@@ -275,13 +275,20 @@ def barrier():
 
 
 def max_over_ranks(v: float) -> float:
+    """Slowest rank's time: the job is as fast as its slowest replica."""
     if not _DIST["on"]:
         return v
     import torch
     import torch.distributed as dist
-    t = torch.tensor([v], dtype=torch.float64, device="cuda")
+    t = torch.tensor([v], dtype=torch.float64, device=_DIST["device"])
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def whole_job_value(world: int, steps: int, units_per_step: float, local_seconds: float) -> float:
+    """Replicas only: every rank processes `steps` batches of its own; the job's throughput is all
+    ranks' units over the slowest rank's time."""
+    return world * steps * units_per_step / max_over_ranks(local_seconds)
 
 
 def units_of(w, kind):
@@ -305,9 +312,9 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
     t_load0 = time.time()
     secs, launches, (t0, t1) = timed_graph_loop(rot.step, rot.R, steps, warmup, stream, min_warm_seconds=0.4)
     clocks = sampler.stop(t_load0, t1)
-    secs = max_over_ranks(secs)
     unit_per_step = units_of(w, kind)
-    value = world * steps * unit_per_step / secs
+    value = whole_job_value(world, steps, unit_per_step, secs)
+    secs = max_over_ranks(secs)
 
     # the layer's own launches (pre-segmented input): what the roofline fraction is computed from
     ksteps = max(rot.R, min(steps, 2000 if kind == "decode" else 200))
