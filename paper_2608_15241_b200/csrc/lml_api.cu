@@ -10,17 +10,18 @@ namespace {
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Workspace layout of the prefill path: [PlanWord][u blocks][gathered x (perm form only)];
+// Workspace layout of the prefill path: [PlanWord][tile_identity][u blocks][gathered x (perm form only)];
 // the decode path uses [PlanWord][u fp32 16x64][row_slot 16].
 struct WsLayout {
-    size_t plan_off, u_off, xg_off, total;
+    size_t plan_off, ident_off, u_off, xg_off, total;
 };
 WsLayout ws_layout(const lml_table* t, int T, int G)
 {
     WsLayout w;
     w.plan_off = 0;
-    w.u_off = round_up(sizeof(PlanWord), 1024);
     const size_t num_m = (size_t)(T + kTileM - 1) / kTileM;
+    w.ident_off = round_up(sizeof(PlanWord), 256);
+    w.u_off = round_up(w.ident_off + (num_m + 1) * sizeof(int32_t), 1024);
     size_t u_bytes = (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
     const size_t dec_bytes = (size_t)kDecodeMaxT * kRankPad * sizeof(float) + kDecodeMaxT * sizeof(int32_t);
     if (u_bytes < dec_bytes) u_bytes = dec_bytes;
@@ -224,20 +225,23 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         e = launch_decode(t->arena, snap, a, stream, &launches);
     } else {
         const void* xg = x;
+        int32_t* tile_identity = nullptr;
         if (perm) {
-            e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, t->arena.status, stream);
+            tile_identity = reinterpret_cast<int32_t*>(wsb + ws.ident_off);
+            e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, tile_identity, !gemm_pairs_forced(),
+                                   t->arena.status, stream);
             if (e == cudaSuccess) { ++launches; xg = wsb + ws.xg_off; }
         }
         PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
         __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
         if (e == cudaSuccess && G > 0) {
-            e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids, G, nullptr, plan, u_blocks,
-                                     stream);
+            e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids, G, x, tile_identity, plan,
+                                     u_blocks, stream);
             if (e == cudaSuccess) ++launches;
         }
         if (e == cudaSuccess) {
             GemmArgs a;
-            a.x = xg; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
+            a.x = xg; a.x_in_place = x; a.tile_identity = tile_identity; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
             a.plan = plan; a.u_blocks = u_blocks ? u_blocks : reinterpret_cast<const __nv_bfloat16*>(x);
             a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
             a.overlap_with_previous = G > 0;

@@ -135,24 +135,42 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 
 // ---------------------------------------------------------------------------------------------
 // Row gather for the perm form of the prefill call: x_grouped[p][:] = x[perm[p]][:].
+// Batches usually arrive with each request's tokens together, so the grouping perm is the
+// identity over long stretches.  A 128-row tile whose perm is the identity is not copied: the
+// kernel marks it in tile_identity[] and the kernels that follow read (and write) those rows in
+// place, with TMA, as if no perm had been given.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4* __restrict__ x,
                                                           const int32_t* __restrict__ perm, int T, int k8,
-                                                          uint4* __restrict__ out, uint32_t* __restrict__ status)
+                                                          uint4* __restrict__ out, int32_t* __restrict__ tile_identity,
+                                                          int allow_skip, uint32_t* __restrict__ status)
 {
-    const int p = blockIdx.x;
-    int row = __ldg(perm + p);
-    const bool ok = row >= 0 && row < T;
-    if (!ok && threadIdx.x == 0) atomicOr(status, LML_FLAG_BAD_PERM);
-    const uint4* src = x + (size_t)(ok ? row : 0) * k8;
-    uint4* dst = out + (size_t)p * k8;
-    for (int i = threadIdx.x; i < k8; i += blockDim.x) dst[i] = ok ? ldg_nc_v4(src + i) : make_uint4(0, 0, 0, 0);
+    const int m = blockIdx.y;             // 128-row tile
+    const int p0 = m * kTileM;
+    const int rows = min(kTileM, T - p0);
+    // every CTA of the tile takes the same decision from the same 128 perm entries
+    int mine = (int)threadIdx.x < rows ? __ldg(perm + p0 + threadIdx.x) : p0 + (int)threadIdx.x;
+    const int not_identity = __syncthreads_or(mine != p0 + (int)threadIdx.x);
+    const bool skip = allow_skip && !not_identity;
+    if (blockIdx.x == 0 && threadIdx.x == 0) tile_identity[m] = skip ? 1 : 0;
+    if (skip) return;
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int p = p0 + r;
+        int row = __ldg(perm + p);
+        const bool ok = row >= 0 && row < T;
+        if (!ok && threadIdx.x == 0) atomicOr(status, LML_FLAG_BAD_PERM);
+        const uint4* src = x + (size_t)(ok ? row : 0) * k8;
+        uint4* dst = out + (size_t)p * k8;
+        for (int i = threadIdx.x; i < k8; i += blockDim.x) dst[i] = ok ? ldg_nc_v4(src + i) : make_uint4(0, 0, 0, 0);
+    }
 }
 
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
-                               uint32_t* status, cudaStream_t stream)
+                               int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream)
 {
-    gather_rows_kernel<<<T, 128, 0, stream>>>((const uint4*)x, perm, T, d_in / 8, (uint4*)x_grouped, status);
+    dim3 grid(32, (T + kTileM - 1) / kTileM);   // 32 CTAs share a tile's 128 rows
+    gather_rows_kernel<<<grid, 128, 0, stream>>>((const uint4*)x, perm, T, d_in / 8, (uint4*)x_grouped, tile_identity,
+                                                allow_skip ? 1 : 0, status);
     return cudaGetLastError();
 }
 

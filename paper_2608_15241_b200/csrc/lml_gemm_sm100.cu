@@ -56,6 +56,7 @@ struct GemmParams {
     const int32_t* seg_offsets;
     const int32_t* slot_ids;
     const int32_t* perm;
+    const int32_t* tile_identity;   // perm form: tiles whose rows stayed in place (read tmap_x0, store with TMA)
     const PlanWord* plan;
     __nv_bfloat16* y;
     uint32_t* status;
@@ -65,7 +66,8 @@ struct GemmParams {
 
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
-    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x0,
+    const __grid_constant__ CUtensorMap tmap_w,
     const __grid_constant__ CUtensorMap tmap_u, const __grid_constant__ CUtensorMap tmap_b,
     const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ SlotSnapshot snap,
     const GemmParams p)
@@ -100,6 +102,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         fence_mbar_init();
     }
     if (warp == 0 && lane == 0) {
+        prefetch_tmap(&tmap_x0);
         prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u);
         prefetch_tmap(&tmap_b); prefetch_tmap(&tmap_y);
     }
@@ -125,12 +128,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
             uint32_t phase = 0;
             bool ok = true;
             auto acquire = [&]() -> bool {
-                return mbar_wait_spin(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
+                return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
             };
             auto advance = [&]() { if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; } };
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m = tile % p.num_m, n = tile / p.num_m;
                 const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+                const bool in_place = p.tile_identity && __ldg(p.tile_identity + m);   // rows of x never copied
                 int g_first = 0, g_end = 0, last_piece = -1;
                 auto piece_slot = [&](int g) -> int {   // -1 = segment contributes no piece
                     int s0, s1, s;
@@ -173,7 +177,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                     const uint32_t bar = smem_u32(&ctrl->full[stage]);
                     ctrl->stage_info[stage] = 4u | ((kb == num_kb - 1 && last_piece < 0) ? 0x100u : 0u);
                     mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
-                    tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
+                    // two call sites on purpose: each names its tensor map as a kernel-parameter constant
+                    if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
+                    else tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
                     tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
                     advance();
                 }
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 // stages after it carry a side-band word (how many K-steps, and whether the tile ends).
                 bool more = true;
                 for (int kb = 0; more; ++kb) {
-                    ok = mbar_wait_spin(smem_u32(&ctrl->full[stage]), phase, abort);
+                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
                     if (!ok) break;
                     const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes;
                     const uint64_t adesc = umma_desc_k128(a_addr);
@@ -253,6 +259,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int m = tile % p.num_m, n = tile / p.num_m;
             const int row_base = m * kBM + q * 32;
+            const bool scatter = p.perm != nullptr && !(p.tile_identity && __ldg(p.tile_identity + m));
             ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
             if (!ok) break;
             tc_fence_after();
@@ -286,7 +293,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                     const int phys = j ^ ((lane >> 1) & 3);
                     *reinterpret_cast<uint4*>(bp + lane * 64 + phys * 16) = v;
                 }
-                if (p.perm == nullptr) {
+                if (!scatter) {
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -409,7 +416,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_pair_kernel(
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            auto acquire = [&]() -> bool { return mbar_wait_spin(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort); };
+            auto acquire = [&]() -> bool { return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort); };
             auto advance = [&]() { if (++stage == kPairStages) { stage = 0; phase ^= 1u; } };
             const int u_rows_total = (p.num_m + (p.G > 0 ? p.G : 1)) * kBM;   // first row coordinate that TMA zero-fills
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
@@ -505,7 +512,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_pair_kernel(
                 uint32_t accumulate = 0;
                 bool more = true;
                 for (int kb = 0; more; ++kb) {
-                    ok = mbar_wait_spin(smem_u32(&ctrl->full[stage]), phase, abort);
+                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
                     if (!ok) break;
                     const uint32_t a_addr = tiles_addr + stage * kPairStageBytes;
                     const uint64_t adesc = umma_desc_k128(a_addr);
@@ -698,6 +705,8 @@ static int gemm_forced_mode()
     return mode;
 }
 
+bool gemm_pairs_forced() { return gemm_forced_mode() == 1; }
+
 static bool gemm_use_pairs(int /*T*/, int /*d_out*/, int /*num_sms*/)
 {
     // Measured on B200 (prefill_q_proj / mlp_up_gate, us per call): single-CTA tiles 66 / 314, CTA
@@ -715,8 +724,9 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     const int num_m = (a.T + kBM - 1) / kBM;
     const int num_n = (a.d_out + bn - 1) / bn;
     const uint32_t w_box_rows = pairs ? (uint32_t)(kPairBN / 2) : (uint32_t)bn;
-    CUtensorMap tx, tw, tu, ty, tb = tmap_B;
+    CUtensorMap tx, tx0, tw, tu, ty, tb = tmap_B;
     if (!encode_tmap_2d(&tx, a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!encode_tmap_2d(&tx0, a.x_in_place ? a.x_in_place : a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
     if (!encode_tmap_2d(&tw, a.W0, (uint64_t)a.d_in, (uint64_t)a.d_out, (uint64_t)a.d_in * 2, kBK, w_box_rows)) return cudaErrorInvalidValue;
     const uint64_t u_rows = (uint64_t)(num_m + (a.G > 0 ? a.G : 1)) * kBM;
     if (!encode_tmap_2d(&tu, a.u_blocks, kRankPad, u_rows, kRankPad * 2, kBK, kBM)) return cudaErrorInvalidValue;
@@ -727,6 +737,7 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     }
     GemmParams p;
     p.seg_offsets = a.seg_offsets; p.slot_ids = a.slot_ids; p.perm = a.perm; p.plan = a.plan;
+    p.tile_identity = pairs ? nullptr : a.tile_identity;
     p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
     p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
     cudaLaunchConfig_t cfg = {};
@@ -757,8 +768,8 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
-    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tw, tu, tb, ty, snap, p);
-    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tw, tu, tb, ty, snap, p);
+    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, snap, p);
+    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, snap, p);
 }
 
 }  // namespace lml

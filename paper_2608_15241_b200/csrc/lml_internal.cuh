@@ -48,16 +48,21 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 
 // u blocks: block b = (tile m) + (segment g) holds the 128 x 64 bf16 values scale*(x.A^T) of
 // the rows of tile m that belong to segment g, zero elsewhere.
+// x_in_place / tile_identity: rows of tiles marked identity are read from x_in_place instead of x.
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
-                                 const int32_t* perm, PlanWord* plan, __nv_bfloat16* u_blocks,
-                                 cudaStream_t stream);
+                                 const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream);
 
+// tile_identity[m] = 1: tile m's perm is the identity, its rows were not copied and stay in place.
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
-                               uint32_t* status, cudaStream_t stream);
+                               int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream);
+bool gemm_pairs_forced();   // the CTA-pair kernel does not read tile_identity
 
 struct GemmArgs {
     const void* x;            // rows in position order (already gathered when perm is used)
+    const void* x_in_place;   // perm form: the caller's x, read for tiles whose perm is the identity
+    const int32_t* tile_identity;   // perm form: 1 per 128-row tile that was left in place, else NULL
     const void* W0;
     void* y;
     const int32_t* perm;      // NULL or position -> output row

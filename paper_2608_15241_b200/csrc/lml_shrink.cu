@@ -38,10 +38,11 @@ template <int NB> struct ShrinkSmem {
 
 // NB = number of 8-column blocks of u that can be non-zero (rank <= 8 * NB).
 template <int NB>
-__global__ void __launch_bounds__(kShrinkWarps * 32) shrink_pieces_kernel(
+__global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pieces_kernel(
     const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
     uint32_t* __restrict__ status, const __nv_bfloat16* __restrict__ x, int T, int K,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids, int G,
+    const __nv_bfloat16* __restrict__ x_in_place, const int32_t* __restrict__ tile_identity,
     PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles)
 {
     ptx::grid_launch_dependents();   // the GEMM that follows may start its main loop now
@@ -111,13 +112,14 @@ __global__ void __launch_bounds__(kShrinkWarps * 32) shrink_pieces_kernel(
     }
 
     const int gq = lane >> 2, tq = lane & 3;
+    const __nv_bfloat16* xsrc = (tile_identity && __ldg(tile_identity + m)) ? x_in_place : x;   // in-place tiles were never copied
     const __nv_bfloat16* xr[4];
     bool xv[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int p = p0 + gq + 8 * i;
         xv[i] = p >= plo && p < phi;
-        xr[i] = x + (size_t)(xv[i] ? p : 0) * K + tq * 8;
+        xr[i] = xsrc + (size_t)(xv[i] ? p : 0) * K + tq * 8;
     }
     const __nv_bfloat16* Abase = arenaA + ((size_t)slot * kRankPad + gq) * K + tq * 8;
 
@@ -203,7 +205,8 @@ __global__ void __launch_bounds__(kShrinkWarps * 32) shrink_pieces_kernel(
 
 template <int NB>
 static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
-                                    const int32_t* seg_offsets, const int32_t* slot_ids, int G, PlanWord* plan,
+                                    const int32_t* seg_offsets, const int32_t* slot_ids, int G,
+                                    const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
                                     __nv_bfloat16* u_blocks, cudaStream_t stream)
 {
     const int num_tiles = (T + kTileM - 1) / kTileM;
@@ -224,8 +227,9 @@ static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, c
     const __nv_bfloat16* arenaA = ar.A;
     uint32_t* status = ar.status;
     const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
+    const __nv_bfloat16* xip = (const __nv_bfloat16*)x_in_place;
     return cudaLaunchKernelEx(&cfg, shrink_pieces_kernel<NB>, snap, arenaA, status, xb, T, d_in, seg_offsets,
-                              slot_ids, G, plan, u_blocks, num_tiles);
+                              slot_ids, G, xip, tile_identity, plan, u_blocks, num_tiles);
 }
 
 cudaError_t shrink_init()
@@ -239,14 +243,14 @@ cudaError_t shrink_init()
 
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
-                                 const int32_t* /*perm*/, PlanWord* plan, __nv_bfloat16* u_blocks,
-                                 cudaStream_t stream)
+                                 const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream)
 {
     int max_rank = 0;
     for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
     if (max_rank <= 16)
-        return launch_shrink_nb<2>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, plan, u_blocks, stream);
-    return launch_shrink_nb<8>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, plan, u_blocks, stream);
+        return launch_shrink_nb<2>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream);
+    return launch_shrink_nb<8>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream);
 }
 
 }  // namespace lml

@@ -98,6 +98,26 @@ def test_decode_token_counts(T):
     check_full(w)
 
 
+def test_perm_that_is_the_identity_on_some_tiles():
+    # rows 0..255 already in place (two whole tiles are not copied), the rest shuffled
+    w = wl.ragged(T=400, d_in=264, d_out=328, ranks=(4, 16, 1, 33, 64))
+    rng = np.random.default_rng(5)
+    perm = np.arange(w.T, dtype=np.int32)
+    perm[256:] = 256 + rng.permutation(w.T - 256)
+    w.perm = perm
+    site = Site(w)
+    try:
+        y, flags = site.run()
+        ref, _ = oracle.forward_workload(w)
+        assert flags == 0 and oracle.compare(y, ref)["ok"]
+        # an all-identity perm must give bit for bit what the call without perm gives
+        y_id, _ = site.run(perm=np.arange(w.T, dtype=np.int32))
+        y_none, _ = site.run(perm=None)
+        assert np.array_equal(y_id, y_none)
+    finally:
+        site.close()
+
+
 def test_no_segments_means_base_only():
     for T in (8, 200):
         w = wl.ragged(T=T, d_in=136, d_out=200)
