@@ -47,6 +47,15 @@ WORKLOADS = {
 }
 
 
+def ncu_traffic(workload):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        return json.load(open(path)).get(workload, {}).get("bytes")
+    except (OSError, ValueError):
+        return None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -333,6 +342,8 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                 "frac_of_sustained": achieved / peaks["tensor_sustained"], "frac_of_nominal_2250": achieved / 2250.0,
                 "traffic": None, "us_per_launch": per_launch * 1e6}
 
+    roof["traffic"] = ncu_traffic(name)
+    roof["algorithmic"] = w.bytes() if kind == "decode" else w.flops()
     esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
     esecs = max_over_ranks(esecs)
     e2e = {"value": world * e2e_steps * unit_per_step / esecs, "unit": spec["unit"], "steps": e2e_steps,
