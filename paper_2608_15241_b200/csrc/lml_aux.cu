@@ -1,5 +1,6 @@
 // Small helper kernels: adapter packing (register_adapter), token segmentation, row gather.
 #include "lml_internal.cuh"
+#include "lml_ptx_sm100.cuh"
 
 namespace lml {
 
@@ -65,6 +66,8 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
     const int nk = snap.max_slots + 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < kSegWarps * (kMaxSlots + 1); i += blockDim.x) (&hist[0][0])[i] = 0;
+    ptx::grid_dependency_wait();      // launched as a programmatic dependent: whatever ran before is complete now
+    ptx::grid_launch_dependents();    // the next kernel may get resident; it waits for this one the same way
     __syncthreads();
 
     int per = (T + kSegWarps - 1) / kSegWarps;
@@ -128,9 +131,11 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
                                   int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
                                   cudaStream_t stream)
 {
-    segment_tokens_kernel<<<1, kSegWarps * 32, 0, stream>>>(snap, token_slots, T, perm, seg_offsets,
-                                                           seg_slot_ids, ar.status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3(1), dim3(kSegWarps * 32), 0, stream);
+    uint32_t* status = ar.status;
+    return cudaLaunchKernelEx(&cfg, segment_tokens_kernel, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, status);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -145,6 +150,8 @@ __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4* __restric
                                                           uint4* __restrict__ out, int32_t* __restrict__ tile_identity,
                                                           int allow_skip, uint32_t* __restrict__ status)
 {
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     const int m = blockIdx.y;             // 128-row tile
     const int p0 = m * kTileM;
     const int rows = min(kTileM, T - p0);
@@ -169,9 +176,11 @@ cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_
                                int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream)
 {
     dim3 grid(32, (T + kTileM - 1) / kTileM);   // 32 CTAs share a tile's 128 rows
-    gather_rows_kernel<<<grid, 128, 0, stream>>>((const uint4*)x, perm, T, d_in / 8, (uint4*)x_grouped, tile_identity,
-                                                allow_skip ? 1 : 0, status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, grid, dim3(128), 0, stream);
+    return cudaLaunchKernelEx(&cfg, gather_rows_kernel, (const uint4*)x, perm, T, d_in / 8, (uint4*)x_grouped,
+                              tile_identity, allow_skip ? 1 : 0, status);
 }
 
 }  // namespace lml

@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(256) decode_shrink_kernel(
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids, int G,
     const int32_t* __restrict__ perm, float* __restrict__ u, int32_t* __restrict__ row_slot)
 {
+    grid_dependency_wait();     // work before this call is complete
     grid_launch_dependents();   // the main kernel may start streaming W0 right away
     __shared__ int sh_slot;
     __shared__ float sh_part[8];
@@ -183,6 +184,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         fence_mbar_init();
     }
     if (tid < 16) ctrl->slot_of_row[tid] = -1;
+    if (G == 0) {   // no shrink kernel ran before this one: wait for foreign work here
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
     __syncthreads();
     volatile int* abort = &ctrl->abort;
 
@@ -309,7 +314,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         __syncthreads();   // all partial sums of the round are in the slots
         if (consumer && ok) {
             const bool lora = G > 0 && ctrl->bad_offsets == 0;
-            if (lora) grid_dependency_wait();   // u comes from the shrink kernel
+            if (G > 0) {   // u comes from the shrink kernel
+                grid_dependency_wait();
+                grid_launch_dependents();
+            }
             const int per_token = nunits * kDecUnitRows;
             for (int e = tid; e < T * per_token; e += kDecConsumers * 32) {
                 const int t = e / per_token, j = e % per_token;   // consecutive threads: consecutive n
@@ -367,10 +375,14 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
         int max_rank = 1;
         for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
         dim3 grid(a.T, (max_rank + 7) & ~7);   // one CTA per (position, j); the expand reads u in groups of 8 columns
-        decode_shrink_kernel<<<grid, 256, 0, stream>>>(snap, ar.A, ar.status, (const __nv_bfloat16*)a.x, a.T,
-                                                       a.d_in, a.seg_offsets, a.slot_ids, a.G, a.perm, a.u,
-                                                       a.row_slot);
-        cudaError_t e = cudaGetLastError();
+        cudaLaunchConfig_t scfg = {};
+        cudaLaunchAttribute sattr[1];
+        pdl_config(scfg, sattr, grid, dim3(256), 0, stream);
+        const __nv_bfloat16* arenaA = ar.A;
+        uint32_t* sstatus = ar.status;
+        const __nv_bfloat16* sx = (const __nv_bfloat16*)a.x;
+        cudaError_t e = cudaLaunchKernelEx(&scfg, decode_shrink_kernel, snap, arenaA, sstatus, sx, a.T, a.d_in,
+                                           a.seg_offsets, a.slot_ids, a.G, a.perm, a.u, a.row_slot);
         if (e != cudaSuccess) return e;
         ++*launches;
     }
@@ -384,7 +396,7 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = lora ? 1 : 0;   // only overlap with our own shrink kernel, never with foreign work
+    cfg.numAttrs = 1;   // with adapters the predecessor is the shrink kernel above, else the kernel waits at its top
     const __nv_bfloat16* xb = (const __nv_bfloat16*)a.x;
     const __nv_bfloat16* wb = (const __nv_bfloat16*)a.W0;
     __nv_bfloat16* yb = (__nv_bfloat16*)a.y;

@@ -119,6 +119,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile int* abort = &ctrl->abort;
+    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -153,6 +157,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                         // here, after the base k-blocks of the first tile are already in flight.
                         if (!lora_known) {
                             grid_dependency_wait();
+                            grid_launch_dependents();
                             lora = p.plan->lora_ok != 0;
                             lora_known = true;
                         }
@@ -408,6 +413,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_pair_kernel(
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile int* abort = &ctrl->abort;
+    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -444,6 +453,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_pair_kernel(
                     if (kb == num_kb - 1) {
                         if (!lora_known) {
                             grid_dependency_wait();   // plan word and u blocks come from the shrink kernel
+                            grid_launch_dependents();
                             lora = p.plan->lora_ok != 0;
                             lora_known = true;
                         }
@@ -745,7 +755,7 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     int nattr = 0;
-    if (a.overlap_with_previous) {   // only ever our own shrink kernel
+    {   // with adapters the predecessor is the shrink kernel of this call, else the kernel waits at its top
         attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[nattr].val.programmaticStreamSerializationAllowed = 1;
         ++nattr;

@@ -101,6 +101,24 @@ cudaError_t decode_init();   // sets the dynamic shared memory attribute
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
                           cudaStream_t stream, int* launches);
 
+// Every kernel of the library is launched as a programmatic dependent of whatever precedes it on
+// the stream and executes griddepcontrol.wait before it touches global memory (unless its
+// predecessor is the library's own kernel of the same call, which has already waited).  The wait
+// costs nothing when the predecessor does not trigger early, and otherwise hides launch latency and
+// the prologue behind the predecessor's tail.
+inline void pdl_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream)
+{
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+
 // ---- small device helpers -------------------------------------------------------------------
 
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }

@@ -45,7 +45,9 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     const __nv_bfloat16* __restrict__ x_in_place, const int32_t* __restrict__ tile_identity,
     PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles)
 {
-    ptx::grid_launch_dependents();   // the GEMM that follows may start its main loop now
+    // Launched with a full dependency on the work before it, so nothing to wait for; the GEMM that
+    // follows may start its main loop right away.
+    ptx::grid_launch_dependents();
     extern __shared__ float shrink_smem[];
     using S = ShrinkSmem<NB>;
     float* red = shrink_smem;                                           // [warp][row][pitch]
