@@ -181,6 +181,28 @@ def _stream(stream) -> int:
     return int(stream.cuda_stream)
 
 
+def fuse_projection_adapters(parts):
+    """Adapters of several projections that read the same x (q/k/v, or gate/up) as ONE adapter of
+    the projection with the concatenated weight: parts = [(A_p [r_p, d_in], B_p [d_out_p, r_p]), ...]
+    gives A = cat(A_p) [sum r_p, d_in] and B = blockdiag(B_p) [sum d_out_p, sum r_p], so that
+    x.W0cat + s (x.A^T).B^T equals the per-projection results side by side (same scale for all
+    parts; sum r_p <= 64).  One call then reads x once and launches once instead of once per
+    projection.  Layout plumbing only (torch cat / copy); the arithmetic stays in the kernels."""
+    import torch
+    A = torch.cat([a for a, _ in parts], dim=0).contiguous()
+    rank = int(A.shape[0])
+    assert rank <= MAX_RANK, "fused rank exceeds the table's maximum"
+    n_total = sum(int(b.shape[0]) for _, b in parts)
+    B = torch.zeros((n_total, rank), dtype=parts[0][1].dtype, device=parts[0][1].device)
+    n0 = r0 = 0
+    for a, b in parts:
+        r, n = int(a.shape[0]), int(b.shape[0])
+        B[n0:n0 + n, r0:r0 + r] = b
+        n0 += n
+        r0 += r
+    return A, B
+
+
 class Table:
     """Adapter slot table of one linear site, for torch tensors (bf16 CUDA, contiguous)."""
 
