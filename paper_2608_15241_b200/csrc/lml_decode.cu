@@ -311,7 +311,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 }
             }
         }
-        __syncthreads();   // all partial sums of the round are in the slots
+        // only the consumer warps meet at the round's two barriers: the producer warp keeps filling the
+        // ring with the next round's rows meanwhile
+        if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // partial sums are in the slots
         if (consumer && ok) {
             const bool lora = G > 0 && ctrl->bad_offsets == 0;
             if (G > 0) {   // u comes from the shrink kernel
@@ -346,7 +348,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 y[(size_t)t * N + n] = __float2bfloat16_rn(v);
             }
         }
-        __syncthreads();   // slots are free for the next round
+        if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // slots are free for the next round
     }
     if (ctrl->abort) __nanosleep(50000);   // gave up: let copies still in flight land before the CTA goes away
     if (tid == 0 && ctrl->abort) atomicOr(status, LML_FLAG_TIMEOUT);
