@@ -29,7 +29,7 @@ using namespace ptx;
 constexpr int kDecConsumers = 8;                 // consumer warps
 constexpr int kDecThreads = (kDecConsumers + 1) * 32;
 constexpr int kDecUnitRows = 8;                  // W0 rows per unit = the 8-wide MMA operand
-constexpr int kDecSpan = 4096;                   // columns whose x fragments fit in registers
+constexpr int kDecSpan = 4096;                   // columns whose x fragments fit in registers (half of it for T > 8)
 constexpr int kDecChunk = 2048;                  // columns per stage (one 4 KB bulk copy per row)
 constexpr int kDecChunksPerSpan = kDecSpan / kDecChunk;             // 4
 constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 4 k-steps per warp and stage
@@ -39,7 +39,9 @@ constexpr int kDecStages = 5;
 constexpr int kDecRoundUnits = 6;                // units (= 48 rows) reduced together
 constexpr int kDecSlotFloats = 16 * kDecUnitRows;   // [token][row] partial sums of one warp for one unit
 constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 4;
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + 256;
+constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
+constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256;
+static_assert(kDecSmemBytes <= 232448, "shared memory budget");
 
 struct DecCtrl {
     uint64_t full[kDecStages];
@@ -154,6 +156,7 @@ __global__ void __launch_bounds__(256) decode_shrink_kernel(
     }
 }
 
+template <bool kTwo>   // false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaB,
     const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W0,
@@ -166,13 +169,18 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const uint32_t ring = (raw + 127u) & ~127u;
     uint8_t* base_ptr = dec_smem_raw + (ring - raw);
     float* slots = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes);   // [stage][warp][token][row]
-    DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);
+    float* u_s = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);   // [16][64]
+    DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
     const int row_begin = (int)((long long)blockIdx.x * N / gridDim.x);
     const int row_end = (int)((long long)(blockIdx.x + 1) * N / gridDim.x);
-    const int nspans = (K + kDecSpan - 1) / kDecSpan;
+    // x fragments of a span live in registers; with two 8-token blocks a span is half as wide, so
+    // both variants hold 64 fragment registers and stay clear of spills
+    constexpr int kSpan = kTwo ? kDecSpan / 2 : kDecSpan;
+    constexpr int kChunksPerSpan = kSpan / kDecChunk;
+    const int nspans = (K + kSpan - 1) / kSpan;
 
     if (tid == 0) {
         for (int s = 0; s < kDecStages; ++s) {
@@ -196,6 +204,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
+    bool u_ready = false;
 
     // Consumer warp 0 works out the slot of every row of x (the same rule the shrink kernel
     // applies) and pulls the B rows this CTA will need into L2 while W0 streams.
@@ -227,8 +236,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
         const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
         for (int sp = 0; sp < nspans; ++sp) {
-            const int k_begin = sp * kDecSpan;
-            const int span = min(kDecSpan, K - k_begin);
+            const int k_begin = sp * kSpan;
+            const int span = min(kSpan, K - k_begin);
             const int nchunks = (span + kDecChunk - 1) / kDecChunk;
             if (!consumer) {
                 // ---------------------------------------------------------- producer warp
@@ -254,14 +263,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 // ---------------------------------------------------------- consumer warps
                 // this warp's k-steps of the span: chunk kc, steps warp*4 .. warp*4+3.  The x fragments
                 // live in registers for every row of the round.
-                uint4 xa[kDecChunksPerSpan * kDecStepsPerChunk], xc[kDecChunksPerSpan * kDecStepsPerChunk];
+                uint4 xa[kChunksPerSpan * kDecStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDecStepsPerChunk : 1];
                 const bool ta = gq < T, tb = gq + 8 < T;
 #pragma unroll
-                for (int i = 0; i < kDecChunksPerSpan * kDecStepsPerChunk; ++i) {
+                for (int i = 0; i < kChunksPerSpan * kDecStepsPerChunk; ++i) {
                     const int c = (i / kDecStepsPerChunk) * kDecChunk + (warp * kDecStepsPerChunk + i % kDecStepsPerChunk) * 32 + tq * 8;
                     const bool lv = c < span;
                     xa[i] = (lv && ta) ? ldg_nc_v4(x + (size_t)gq * K + k_begin + c) : make_uint4(0, 0, 0, 0);
-                    xc[i] = (lv && tb) ? ldg_nc_v4(x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
+                    if (kTwo) xc[i] = (lv && tb) ? ldg_nc_v4(x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
                 }
                 for (int un = 0; un < nunits && ok; ++un) {
                     const int rows = min(kDecUnitRows, round_rows - un * kDecUnitRows);
@@ -271,7 +280,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
 #pragma unroll
                     for (int a = 0; a < 4; ++a) acc4[a][0] = acc4[a][1] = acc4[a][2] = acc4[a][3] = 0.f;
 #pragma unroll
-                    for (int kc = 0; kc < kDecChunksPerSpan; ++kc) {
+                    for (int kc = 0; kc < kChunksPerSpan; ++kc) {
                         if (kc < nchunks && ok) {
                             ok = mbar_wait_warp(smem_u32(&ctrl->full[stage]), phase, abort);
                             if (ok) {
@@ -283,7 +292,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                                         const uint4 w = (rv && c0 + tq * 8 < span)
                                                             ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
                                                             : make_uint4(0, 0, 0, 0);
-                                        const uint4 a0 = xa[kc * kDecStepsPerChunk + i], a1 = xc[kc * kDecStepsPerChunk + i];
+                                        const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
+                                        const uint4 a1 = kTwo ? xc[kc * kDecStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
                                         mma_bf16_16816(acc4[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, w.x, w.y);
                                         mma_bf16_16816(acc4[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, w.z, w.w);
                                     }
@@ -314,12 +324,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         // only the consumer warps meet at the round's two barriers: the producer warp keeps filling the
         // ring with the next round's rows meanwhile
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // partial sums are in the slots
+        if (consumer && G > 0 && !u_ready) {   // u comes from the shrink kernel: fetched once into shared memory
+            grid_dependency_wait();
+            grid_launch_dependents();
+            for (int i = tid; i < T * kRankPad / 4; i += kDecConsumers * 32)
+                reinterpret_cast<float4*>(u_s)[i] = reinterpret_cast<const float4*>(u)[i];
+            u_ready = true;
+            asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");
+        }
         if (consumer && ok) {
             const bool lora = G > 0 && ctrl->bad_offsets == 0;
-            if (G > 0) {   // u comes from the shrink kernel
-                grid_dependency_wait();
-                grid_launch_dependents();
-            }
             const int per_token = nunits * kDecUnitRows;
             for (int e = tid; e < T * per_token; e += kDecConsumers * 32) {
                 const int t = e / per_token, j = e % per_token;   // consecutive threads: consecutive n
@@ -333,7 +347,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 if (slot >= 0) {
                     const int r8 = ((int)snap.rank[slot] + 7) >> 3;
                     const uint4* bp = reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
-                    const float4* up = reinterpret_cast<const float4*>(u + t * kRankPad);
+                    const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
                     for (int c = 0; c < r8; ++c) {
                         uint4 b = ldg_nc_v4(bp + c);
@@ -362,10 +376,9 @@ cudaError_t decode_init()
     cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_main_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(decode_main_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(decode_main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
+    return cudaFuncSetAttribute(decode_main_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
 }
 
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a, cudaStream_t stream,
@@ -408,8 +421,10 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const int32_t* so = a.seg_offsets;
     const int32_t* ids = a.slot_ids;
     const int32_t* pm = a.perm;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_main_kernel, snap, arenaB, xb, wb, yb, up, so, ids, pm, status,
-                                       a.T, a.d_in, a.d_out, a.G);
+    cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaB, xb, wb, yb, up, so, ids, pm,
+                                                 status, a.T, a.d_in, a.d_out, a.G)
+                            : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaB, xb, wb, yb, up, so, ids, pm,
+                                                 status, a.T, a.d_in, a.d_out, a.G);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
