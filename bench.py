@@ -331,7 +331,7 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
     per_launch = ksecs / ksteps
     achieved = unit_per_step / per_launch
     if kind == "decode":
-        roof = {"bound": "hbm", "kernel": "decode_main_kernel (shrink kernel overlapped by dependent launch)",
+        roof = {"bound": "hbm", "kernel": "decode_main_kernel (LoRA shrink runs on three of its warps)",
                 "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
                 "peak_source": peaks["source"], "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
                 "us_per_launch": per_launch * 1e6}

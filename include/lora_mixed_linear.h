@@ -73,7 +73,7 @@ typedef enum {
 
 #define LML_MAX_SLOTS 64  /* upper bound for max_slots */
 #define LML_MAX_RANK 64   /* upper bound for an adapter's rank */
-#define LML_DECODE_MAX_TOKENS 16 /* T <= this takes the bandwidth-bound decode kernels */
+#define LML_DECODE_MAX_TOKENS 16 /* T <= this takes the bandwidth-bound decode kernel */
 
 const char* lml_status_string(lml_status s);
 
@@ -151,8 +151,11 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * covers positions [seg_offsets[g], seg_offsets[g+1]); position p is row perm[p] of x and y
  * if perm (device int32[T], a permutation) is given, else row p.  G == 0 means "no adapter
  * anywhere".  T == 0 returns LML_OK without launching.
- * T <= 16 runs the bandwidth-bound decode kernels (W0 read once with 128-bit loads); larger
- * T runs the TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
+ * T <= 16 runs the bandwidth-bound decode kernel (W0 read once through a bulk-copy ring; with
+ * segments it is a cooperative launch whose CTAs hand one another their share of the shrink
+ * result and count themselves in the table's status block, so two decode calls on the SAME table
+ * must not overlap on the GPU: put them on one stream or order them); larger T runs the
+ * TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
  * Errors: INVALID_ARG, WORKSPACE, CUDA.
  */
 lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
@@ -184,9 +187,9 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
  * callback, a real-time loop that must not touch the allocator, a process whose memory budget
  * was handed out completely at start-up.  Such a caller still passes its inputs and the output
  * (x, W0, seg_offsets, slot_ids, perm, y: same meaning, layout and alignment as in
- * lora_mixed_linear), but no workspace: the scratch the decode kernels need between their two
- * passes (the scaled shrink result, 16 x 64 fp32, and the slot of each row) lives in a 4352-byte
- * array inside the library image.  Every GPU that loads the library holds that array until the
+ * lora_mixed_linear), but no workspace: the scratch the decode kernel needs between its two
+ * phases (the scaled shrink result, 16 x 64 fp32) lives in a 4096-byte array inside the library
+ * image.  Every GPU that loads the library holds that array until the
  * process exits.  The call allocates and frees nothing, and calls no allocating routine.
  *
  * Limits and rules
@@ -195,9 +198,9 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.
- *     The call resets what must not leak from an earlier call (the per-row slots) itself, on
- *     `stream`, before its kernels run.  Two calls that overlap on the GPU (different streams
- *     without ordering, or concurrent graph branches) race on the array: order them.
+ *     Nothing in it has to start at zero: the kernel writes every element it later reads.
+ *     Two calls that overlap on the GPU (different streams without ordering, or concurrent
+ *     graph branches) race on the array: order them.
  *   - Results are identical to lora_mixed_linear on the same inputs.
  * Errors: INVALID_ARG, TOO_LARGE, CUDA.
  */
@@ -207,6 +210,8 @@ lml_status lora_mixed_linear_decode_static(lml_table* t, const void* x, const vo
 
 /*
  * Read and clear the sticky device status word (LML_FLAG_* bits).  Synchronises `stream`.
+ * Also puts the decode kernel's grid counters back to zero, which matters only after a call
+ * that reported LML_FLAG_TIMEOUT.
  * Errors: INVALID_ARG, CUDA.
  */
 lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream);

@@ -11,7 +11,7 @@ namespace {
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Workspace layout of the prefill path: [PlanWord][tile_identity][u blocks][gathered x (perm form only)];
-// the decode path uses [PlanWord][u fp32 16x64][row_slot 16].
+// the decode path uses [PlanWord][..][u fp32 16x64].
 struct WsLayout {
     size_t plan_off, ident_off, u_off, xg_off, total;
 };
@@ -219,8 +219,6 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         DecodeArgs a;
         a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
         a.u = G > 0 ? reinterpret_cast<float*>(wsb + ws.u_off) : nullptr;
-        a.row_slot = G > 0 ? reinterpret_cast<int32_t*>(wsb + ws.u_off + (size_t)kDecodeMaxT * kRankPad * sizeof(float))
-                           : nullptr;
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         e = launch_decode(t->arena, snap, a, stream, &launches);
     } else {
@@ -313,7 +311,8 @@ lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
     if (!guard.ok) return LML_ERR_CUDA;
     uint32_t v = 0;
     bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    ok = ok && cudaMemsetAsync(t->arena.status, 0, sizeof v, stream) == cudaSuccess;
+    // also puts the decode kernel's two grid counters (words 1 and 2) back to zero, in case a call gave up
+    ok = ok && cudaMemsetAsync(t->arena.status, 0, 3 * sizeof v, stream) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
     *flags_out = v;

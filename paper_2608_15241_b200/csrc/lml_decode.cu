@@ -1,24 +1,28 @@
 // Decode path (T <= 16 tokens): bandwidth-bound.  W0 is read exactly once.
 //
-// Two kernels, chained with programmatic dependent launch so the second one starts streaming W0
-// while the first (tiny) one is still running:
-//   decode_shrink_kernel  u[row][j] = scale_s * sum_k x[row][k] A_s[j][k]  (fp32, one warp per
-//                         (token, j)).
-//   decode_main_kernel    one persistent CTA per SM, each owning a contiguous, balanced range of
-//                         W0 rows (N/148 of them, +-1), because an SM cannot take in much more than
-//                         its fair share of HBM bandwidth and contiguous addresses stream best.
-//                         A producer warp copies 8 rows x 1024 columns per stage (one 2 KB bulk
-//                         asynchronous copy per row) into a shared-memory ring, unit after unit, so
-//                         the CTA walks its rows front to back.
-//                         Eight consumer warps each own a fixed slice of K: their x fragments are
-//                         loaded once into registers and reused for every row.  y^T += W0.x^T runs on
-//                         mma.sync m16n8k16 with the tokens as the 16-row operand (T <= 16 is exactly
-//                         one tile) and 8 rows of W0 as the 8-wide operand.  The k order inside a
-//                         32-wide step is permuted identically for both operands, which a dot product
-//                         does not see, so operands are plain 16-byte loads.  Per-warp partial sums go
-//                         to per-warp slots and are added in a fixed order; the LoRA expand
-//                         sum_j u[t][j] B_s[n][j] is added in fp32 before the single bf16 rounding.
-//                         d_in > 4096 is walked in spans of 4096 columns.  All waits are bounded.
+// One kernel, decode_main_kernel: one persistent CTA per SM, each owning a contiguous, balanced
+// range of W0 rows (N/148 of them, +-1), because an SM cannot take in much more than its fair share
+// of HBM bandwidth and contiguous addresses stream best.  Twelve warps in three roles:
+//   producer (1 warp)   copies 8 rows x 2048 columns per stage (one 4 KB bulk asynchronous copy per
+//                       row) into a shared-memory ring, unit after unit, so the CTA walks its rows
+//                       front to back; it runs ahead across rounds.
+//   consumers (8 warps) each own a fixed slice of K: their x fragments are loaded once into
+//                       registers and reused for every row.  y^T += W0.x^T runs on mma.sync m16n8k16
+//                       with the tokens as the 16-row operand (T <= 16 is exactly one tile; T <= 8
+//                       uses a variant that feeds zeros for the upper half and keeps twice the span
+//                       of x in registers) and 8 rows of W0 as the 8-wide operand.  The k order
+//                       inside a 32-wide step is permuted identically for both operands, which a dot
+//                       product does not see, so operands are plain 16-byte loads.  Per-warp partial
+//                       sums go to per-warp slots and are added in a fixed order; the LoRA expand
+//                       sum_j u[t][j] B_s[n][j] is added in fp32 before the single bf16 rounding.
+//   shrink (3 warps)    only when the call has segments: look up each row's slot, then compute this
+//                       CTA's share of u[row][j] = scale_s * sum_k x[row][k] A_s[j][k] (fp32, one warp
+//                       per dot product, dealt out round-robin over the whole grid), publish it in
+//                       global memory, wait for the other CTAs' shares on a counter and stage all of u
+//                       in shared memory.  The consumers meet them once, at their first epilogue.
+//                       The hand-over between CTAs needs them all resident, so a call with segments
+//                       is a cooperative launch.
+// d_in wider than a span is walked span by span.  All waits are bounded.
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
 
@@ -27,7 +31,8 @@ namespace lml {
 using namespace ptx;
 
 constexpr int kDecConsumers = 8;                 // consumer warps
-constexpr int kDecThreads = (kDecConsumers + 1) * 32;
+constexpr int kDecShrinkWarps = 3;               // warps after the producer warp: the LoRA shrink
+constexpr int kDecThreads = (kDecConsumers + 1 + kDecShrinkWarps) * 32;
 constexpr int kDecUnitRows = 8;                  // W0 rows per unit = the 8-wide MMA operand
 constexpr int kDecSpan = 4096;                   // columns whose x fragments fit in registers (half of it for T > 8)
 constexpr int kDecChunk = 2048;                  // columns per stage (one 4 KB bulk copy per row)
@@ -68,101 +73,13 @@ __device__ __forceinline__ void prefetch_l2(const void* p)
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
-constexpr int kDecShrinkSegs = 256;   // segments looked up in one parallel pass
-
-// Slot of position `pos` and validity of the segment arrays, found by the whole CTA in one round
-// of loads (every thread looks at one segment) when G is small, else by binary search.
-__device__ __forceinline__ void decode_lookup(const SlotSnapshot& snap, const int32_t* __restrict__ seg_offsets,
-                                              const int32_t* __restrict__ slot_ids, int G, int T, int pos,
-                                              int* sh_slot, int& bad_off, int& bad_slot)
-{
-    bad_off = 0; bad_slot = 0;
-    const int tid = threadIdx.x;
-    if (tid == 0) *sh_slot = -1;
-    __syncthreads();
-    for (int g = tid; g < G; g += blockDim.x) {
-        const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1), s = __ldg(slot_ids + g);
-        if (s1 < s0 || s0 < 0 || s1 > T) bad_off = 1;
-        if (g == 0 && s0 != 0) bad_off = 1;
-        if (g == G - 1 && s1 != T) bad_off = 1;
-        const int r = slot_rank(snap, s);
-        if (s != -1 && r == 0) bad_slot = 1;
-        if (pos >= s0 && pos < s1) *sh_slot = r > 0 ? s : -1;   // at most one segment holds pos when offsets are monotone
-    }
-    bad_off = __syncthreads_or(bad_off);
-    bad_slot = __syncthreads_or(bad_slot);
-}
-
-// One CTA per (position, j): all 256 threads share one dot product, so a thread has only a couple
-// of 16-byte loads of x and of A in flight and the whole kernel is two memory round trips long
-// (segment lookup, then operands).  CTAs whose j is beyond the slot's rank only write a zero.
-__global__ void __launch_bounds__(256) decode_shrink_kernel(
-    const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
-    uint32_t* __restrict__ status, const __nv_bfloat16* __restrict__ x, int T, int K,
-    const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids, int G,
-    const int32_t* __restrict__ perm, float* __restrict__ u, int32_t* __restrict__ row_slot)
-{
-    grid_dependency_wait();     // work before this call is complete
-    grid_launch_dependents();   // the main kernel may start streaming W0 right away
-    __shared__ int sh_slot;
-    __shared__ float sh_part[8];
-    const int pos = blockIdx.x, j = blockIdx.y;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    int row = perm ? __ldg(perm + pos) : pos;   // in flight together with the segment lookup
-    int bad_off, bad_slot;
-    decode_lookup(snap, seg_offsets, slot_ids, G, T, pos, &sh_slot, bad_off, bad_slot);
-    unsigned f = (bad_off ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u);
-    if (row < 0 || row >= T) { row = -1; f |= LML_FLAG_BAD_PERM; }
-    const int slot = (bad_off || row < 0) ? -1 : sh_slot;
-    if (tid == 0 && j == 0) {
-        if (f) atomicOr(status, f);
-        if (row >= 0) row_slot[row] = slot;
-    }
-    if (row < 0) return;
-    if (slot < 0 || j >= (int)snap.rank[slot]) {
-        if (tid == 0) u[row * kRankPad + j] = 0.f;
-        return;
-    }
-    const __nv_bfloat16* xr = x + (size_t)row * K;
-    const __nv_bfloat16* ar = arenaA + ((size_t)slot * kRankPad + j) * K;
-    float dot = 0.f;
-    for (int k0 = tid * 8; k0 < K; k0 += 256 * 8 * 2) {
-        const int k1 = k0 + 256 * 8;
-        const bool v1 = k1 < K;
-        const uint4 a0 = ldg_nc_v4(xr + k0), b0 = ldg_nc_v4(ar + k0);
-        const uint4 a1 = v1 ? ldg_nc_v4(xr + k1) : make_uint4(0, 0, 0, 0);
-        const uint4 b1 = v1 ? ldg_nc_v4(ar + k1) : make_uint4(0, 0, 0, 0);
-        float d0 = 0.f, d1 = 0.f;
-        d0 = fmaf(bf16_lo(a0.x), bf16_lo(b0.x), d0); d0 = fmaf(bf16_hi(a0.x), bf16_hi(b0.x), d0);
-        d0 = fmaf(bf16_lo(a0.y), bf16_lo(b0.y), d0); d0 = fmaf(bf16_hi(a0.y), bf16_hi(b0.y), d0);
-        d0 = fmaf(bf16_lo(a0.z), bf16_lo(b0.z), d0); d0 = fmaf(bf16_hi(a0.z), bf16_hi(b0.z), d0);
-        d0 = fmaf(bf16_lo(a0.w), bf16_lo(b0.w), d0); d0 = fmaf(bf16_hi(a0.w), bf16_hi(b0.w), d0);
-        d1 = fmaf(bf16_lo(a1.x), bf16_lo(b1.x), d1); d1 = fmaf(bf16_hi(a1.x), bf16_hi(b1.x), d1);
-        d1 = fmaf(bf16_lo(a1.y), bf16_lo(b1.y), d1); d1 = fmaf(bf16_hi(a1.y), bf16_hi(b1.y), d1);
-        d1 = fmaf(bf16_lo(a1.z), bf16_lo(b1.z), d1); d1 = fmaf(bf16_hi(a1.z), bf16_hi(b1.z), d1);
-        d1 = fmaf(bf16_lo(a1.w), bf16_lo(b1.w), d1); d1 = fmaf(bf16_hi(a1.w), bf16_hi(b1.w), d1);
-        dot += d0 + d1;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    if (lane == 0) sh_part[warp] = dot;
-    __syncthreads();
-    if (tid == 0) {
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) s += sh_part[w];
-        u[row * kRankPad + j] = s * snap.scale[slot];
-    }
-}
-
 template <bool kTwo>   // false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
-    const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaB,
-    const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ W0,
-    __nv_bfloat16* __restrict__ y, const float* __restrict__ u, const int32_t* __restrict__ seg_offsets,
-    const int32_t* __restrict__ slot_ids, const int32_t* __restrict__ perm, uint32_t* __restrict__ status,
-    int T, int K, int N, int G)
+    const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
+    const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
+    const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
+    const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
+    const int32_t* __restrict__ perm, uint32_t* status, int T, int K, int N, int G)
 {
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
@@ -192,10 +109,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         fence_mbar_init();
     }
     if (tid < 16) ctrl->slot_of_row[tid] = -1;
-    if (G == 0) {   // no shrink kernel ran before this one: wait for foreign work here
-        grid_dependency_wait();
-        grid_launch_dependents();
-    }
+    grid_dependency_wait();     // launched as a programmatic dependent: the work before this call is complete now
+    grid_launch_dependents();
     __syncthreads();
     volatile int* abort = &ctrl->abort;
 
@@ -206,33 +121,144 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     bool ok = true;
     bool u_ready = false;
 
-    // Consumer warp 0 works out the slot of every row of x (the same rule the shrink kernel
-    // applies) and pulls the B rows this CTA will need into L2 while W0 streams.
-    if (warp == 0 && G > 0) {
-        int bad = 0;
-        for (int g = lane; g < G; g += 32) {
-            int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
-            if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
+    // This warp's x fragments (chunk kc, k-steps warp*S .. warp*S+S-1 of a span) stay in registers.
+    uint4 xa[kChunksPerSpan * kDecStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDecStepsPerChunk : 1];
+    auto load_x = [&](int k_begin, int span) {
+        const bool ta = gq < T, tb = gq + 8 < T;
+#pragma unroll
+        for (int i = 0; i < kChunksPerSpan * kDecStepsPerChunk; ++i) {
+            const int c = (i / kDecStepsPerChunk) * kDecChunk + (warp * kDecStepsPerChunk + i % kDecStepsPerChunk) * 32 + tq * 8;
+            const bool lv = c < span;
+            xa[i] = (lv && ta) ? ldg_nc_v4(x + (size_t)gq * K + k_begin + c) : make_uint4(0, 0, 0, 0);
+            if (kTwo) xc[i] = (lv && tb) ? ldg_nc_v4(x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
         }
-        if (lane == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
-        bad = __any_sync(0xffffffffu, bad);
-        if (lane == 0) ctrl->bad_offsets = bad;
-        if (!bad && lane < T) {
-            int row = perm ? __ldg(perm + lane) : lane;
-            if (row >= 0 && row < T) {
-                int g = seg_upper(seg_offsets, G, lane);
-                int slot = -1;
-                if (g < G) { int s = __ldg(slot_ids + g); if (slot_rank(snap, s) > 0) slot = s; }
-                ctrl->slot_of_row[row] = slot;
-                if (slot >= 0) {
-                    const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                    for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+    };
+
+    // ---- LoRA shrink, part of this kernel ---------------------------------------------------------------
+    // Three extra warps do it while the other nine stream W0, so the base path never waits for it.
+    // The first of them works out the slot of every row of x, raises the status flags and pulls the B
+    // rows this CTA will need into L2.  Then the (token, j) dot products u = scale * x.A_j are dealt
+    // out round-robin to the CTAs of the grid and, inside a CTA, to its three shrink warps: one warp per
+    // dot product, sixteen 16-byte loads in flight per lane.  The results go to u in global memory; a
+    // counter in the table's status block tells every CTA when all of u is there (the launch is
+    // cooperative, so all CTAs are resident).  The consumers look at it only in their first epilogue.
+    unsigned int* sync_words = status + 1;   // [0] CTAs whose share of u is written, [1] CTAs that have left
+    const bool shrinker = warp > kDecConsumers;
+    if (shrinker && G > 0) {
+        const int sw = warp - kDecConsumers - 1;
+        if (sw == 0) {
+            int bad = 0, bad_slot = 0;
+            for (int g = lane; g < G; g += 32) {
+                const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1), sl = __ldg(slot_ids + g);
+                if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
+                if (sl != -1 && slot_rank(snap, sl) == 0) bad_slot = 1;
+            }
+            if (lane == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
+            bad = __any_sync(0xffffffffu, bad);
+            bad_slot = __any_sync(0xffffffffu, bad_slot);
+            int bad_perm = 0;
+            if (!bad && lane < T) {
+                const int row = perm ? __ldg(perm + lane) : lane;
+                if (row >= 0 && row < T) {
+                    const int g = seg_upper(seg_offsets, G, lane);
+                    int slot = -1;
+                    if (g < G) { const int sl = __ldg(slot_ids + g); if (slot_rank(snap, sl) > 0) slot = sl; }
+                    ctrl->slot_of_row[row] = slot;
+                } else bad_perm = 1;
+            }
+            bad_perm = __any_sync(0xffffffffu, bad_perm);
+            if (lane == 0) {
+                ctrl->bad_offsets = bad;
+                const unsigned f = (bad ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u) |
+                                   (bad_perm ? LML_FLAG_BAD_PERM : 0u);
+                if (f && blockIdx.x == 0) atomicOr(status, f);
+            }
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
+        // Dot product d (rows of x in order, j ascending inside a row, each row padded to a multiple of
+        // eight columns because the expand reads u in groups of eight) belongs to CTA d mod grid.
+        int total = 0;
+        for (int t = 0; t < T; ++t) {
+            const int slot = ctrl->slot_of_row[t];
+            total += slot >= 0 ? (((int)snap.rank[slot] + 7) & ~7) : 0;
+        }
+        for (int d = (int)blockIdx.x + sw * (int)gridDim.x; d < total; d += kDecShrinkWarps * (int)gridDim.x) {
+            int t = 0, j = d, slot = -1, rank = 0;
+            for (; t < T; ++t) {   // which row does d fall into
+                slot = ctrl->slot_of_row[t];
+                rank = slot >= 0 ? (int)snap.rank[slot] : 0;
+                const int rank8 = (rank + 7) & ~7;
+                if (j < rank8) break;
+                j -= rank8;
+            }
+            if (j >= rank) {   // padding column: B is zero there, u must at least be finite
+                if (lane == 0) u[t * kRankPad + j] = 0.f;
+                continue;
+            }
+            const __nv_bfloat16* xr = x + (size_t)t * K;
+            const __nv_bfloat16* ar = arenaA + ((size_t)slot * kRankPad + j) * K;
+            float dot = 0.f;
+            for (int kb = lane * 8; kb < K; kb += 8 * 256) {
+                uint4 xv[8], av[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int k0 = kb + i * 256;
+                    const bool v = k0 < K;
+                    xv[i] = v ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
+                    av[i] = v ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
                 }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float p = 0.f;
+                    p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
+                    p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
+                    p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
+                    p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
+                    dot += p;
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (lane == 0) u[t * kRankPad + j] = dot * snap.scale[slot];
+        }
+        if (lane == 0) __threadfence();
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // this CTA's share of u is written
+        if (sw == 0 && lane == 0) {
+            __threadfence();
+            atomicAdd(sync_words, 1u);
+        }
+        if (sw == 0 && lane < T) {   // the expand's B rows for this CTA's output columns, towards L2
+            const int slot = ctrl->slot_of_row[lane];
+            if (slot >= 0) {
+                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
+                for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+            }
+        }
+        // Wait (bounded) until every CTA has reported its dot products, then stage u in shared memory
+        // for the consumers' epilogue, off their critical path.
+        if (sw == 0 && lane == 0) {
+            const long long t0 = clock64();
+            while (*reinterpret_cast<volatile unsigned int*>(sync_words) < gridDim.x) {
+                if (clock64() - t0 > (1ll << 31)) { ctrl->abort = 1; break; }
+            }
+            __threadfence();
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+        for (int i = tid - (kDecConsumers + 1) * 32; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
+            reinterpret_cast<float4*>(u_s)[i] = __ldcg(reinterpret_cast<const float4*>(u) + i);
+        // tell the consumers that u_s, slot_of_row and bad_offsets are final
+        asm volatile("bar.arrive 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
+        // Every CTA that gets here has seen the full count, so nobody reads the counters any more once
+        // all have: the last one puts both back to zero for the next call on this table.
+        if (sw == 0 && lane == 0 && ctrl->abort == 0) {
+            if (atomicAdd(sync_words + 1, 1u) == gridDim.x - 1) {
+                sync_words[0] = 0u;
+                sync_words[1] = 0u;
             }
         }
     }
 
-    for (int round_begin = row_begin; round_begin < row_end; round_begin += kDecRoundUnits * kDecUnitRows) {
+    for (int round_begin = shrinker ? row_end : row_begin; round_begin < row_end; round_begin += kDecRoundUnits * kDecUnitRows) {
         const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
         const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
         for (int sp = 0; sp < nspans; ++sp) {
@@ -263,15 +289,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 // ---------------------------------------------------------- consumer warps
                 // this warp's k-steps of the span: chunk kc, steps warp*4 .. warp*4+3.  The x fragments
                 // live in registers for every row of the round.
-                uint4 xa[kChunksPerSpan * kDecStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDecStepsPerChunk : 1];
-                const bool ta = gq < T, tb = gq + 8 < T;
-#pragma unroll
-                for (int i = 0; i < kChunksPerSpan * kDecStepsPerChunk; ++i) {
-                    const int c = (i / kDecStepsPerChunk) * kDecChunk + (warp * kDecStepsPerChunk + i % kDecStepsPerChunk) * 32 + tq * 8;
-                    const bool lv = c < span;
-                    xa[i] = (lv && ta) ? ldg_nc_v4(x + (size_t)gq * K + k_begin + c) : make_uint4(0, 0, 0, 0);
-                    if (kTwo) xc[i] = (lv && tb) ? ldg_nc_v4(x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
-                }
+                load_x(k_begin, span);
                 for (int un = 0; un < nunits && ok; ++un) {
                     const int rows = min(kDecUnitRows, round_rows - un * kDecUnitRows);
                     const bool rv = gq < rows;   // lanes whose row of the 8-wide operand is real
@@ -324,13 +342,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         // only the consumer warps meet at the round's two barriers: the producer warp keeps filling the
         // ring with the next round's rows meanwhile
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // partial sums are in the slots
-        if (consumer && G > 0 && !u_ready) {   // u comes from the shrink kernel: fetched once into shared memory
-            grid_dependency_wait();
-            grid_launch_dependents();
-            for (int i = tid; i < T * kRankPad / 4; i += kDecConsumers * 32)
-                reinterpret_cast<float4*>(u_s)[i] = reinterpret_cast<const float4*>(u)[i];
+        if (consumer && G > 0 && !u_ready) {   // first epilogue: the shrink warps have staged u in shared memory
+            asm volatile("bar.sync 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
             u_ready = true;
-            asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");
         }
         if (consumer && ok) {
             const bool lora = G > 0 && ctrl->bad_offsets == 0;
@@ -370,13 +384,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
 
 cudaError_t decode_init()
 {
-    // The shrink kernel asks for the same (maximal) shared-memory carve-out as the main kernel: an SM
-    // cannot host CTAs of two kernels that want different L1 / shared-memory splits, and the main
-    // kernel's CTAs must be able to start beside the shrink CTAs that are still running.
-    cudaError_t e = cudaFuncSetAttribute(decode_shrink_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                         cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_main_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(decode_main_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(decode_main_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
 }
@@ -384,47 +392,38 @@ cudaError_t decode_init()
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a, cudaStream_t stream,
                           int* launches)
 {
-    const bool lora = a.G > 0;
     *launches = 0;
-    if (lora) {
-        int max_rank = 1;
-        for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
-        dim3 grid(a.T, (max_rank + 7) & ~7);   // one CTA per (position, j); the expand reads u in groups of 8 columns
-        cudaLaunchConfig_t scfg = {};
-        cudaLaunchAttribute sattr[1];
-        pdl_config(scfg, sattr, grid, dim3(256), 0, stream);
-        const __nv_bfloat16* arenaA = ar.A;
-        uint32_t* sstatus = ar.status;
-        const __nv_bfloat16* sx = (const __nv_bfloat16*)a.x;
-        cudaError_t e = cudaLaunchKernelEx(&scfg, decode_shrink_kernel, snap, arenaA, sstatus, sx, a.T, a.d_in,
-                                           a.seg_offsets, a.slot_ids, a.G, a.perm, a.u, a.row_slot);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-    }
     const int row_pairs = (a.d_out + 1) / 2;   // at least two rows per CTA
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(row_pairs < a.num_sms ? row_pairs : a.num_sms);
     cfg.blockDim = dim3(kDecThreads);
     cfg.dynamicSmemBytes = kDecSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    // With adapters the CTAs hand one another their share of u through global memory and wait for it
+    // in the epilogue, so they must all be resident: a cooperative launch guarantees that (the grid
+    // never exceeds one CTA per SM).  Without adapters the kernel is launched as a programmatic
+    // dependent of whatever precedes it (it waits at its top).
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;   // with adapters the predecessor is the shrink kernel above, else the kernel waits at its top
+    cfg.numAttrs = a.G > 0 ? 2 : 1;
     const __nv_bfloat16* xb = (const __nv_bfloat16*)a.x;
     const __nv_bfloat16* wb = (const __nv_bfloat16*)a.W0;
     __nv_bfloat16* yb = (__nv_bfloat16*)a.y;
-    const float* up = a.u;
+    float* up = a.u;
+    const __nv_bfloat16* arenaA = ar.A;
     const __nv_bfloat16* arenaB = ar.B;
     uint32_t* status = ar.status;
     const int32_t* so = a.seg_offsets;
     const int32_t* ids = a.slot_ids;
     const int32_t* pm = a.perm;
-    cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaB, xb, wb, yb, up, so, ids, pm,
-                                                 status, a.T, a.d_in, a.d_out, a.G)
-                            : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaB, xb, wb, yb, up, so, ids, pm,
-                                                 status, a.T, a.d_in, a.d_out, a.G);
+    cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaA, arenaB, xb, wb, yb, up, so,
+                                                 ids, pm, status, a.T, a.d_in, a.d_out, a.G)
+                            : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaA, arenaB, xb, wb, yb, up, so,
+                                                 ids, pm, status, a.T, a.d_in, a.d_out, a.G);
     if (e == cudaSuccess) ++*launches;
     return e;
 }

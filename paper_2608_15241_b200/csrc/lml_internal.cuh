@@ -92,8 +92,7 @@ struct DecodeArgs {
     const int32_t* perm;
     const int32_t* seg_offsets;
     const int32_t* slot_ids;
-    float* u;            // [16][64] fp32, scale folded in
-    int32_t* row_slot;   // [16] slot of each row of x, -1 = none
+    float* u;            // [16][64] fp32 scratch: scale * x.A^T, written and read by the decode kernel
     int T, d_in, d_out, G;
     int num_sms;
 };

@@ -1,10 +1,10 @@
 // lora_mixed_linear_decode_static: the decode form of the layer for callers that cannot hand the
 // library any scratch memory.  See the declaration in include/lora_mixed_linear.h.
 //
-// The decode kernels need a little scratch between the shrink pass and the main pass: the
-// scaled shrink result u[16][64] (fp32) and the slot of each of the 16 rows.  The regular entry
-// point takes it from the caller's workspace.  Here it lives in a file-scope device array that
-// is part of the library image: every GPU context that loads the library carries these 4352
+// The decode kernel needs a little scratch between its shrink phase and its epilogue: the scaled
+// shrink result u[16][64] (fp32), which the CTAs of the grid write for one another.  The regular
+// entry point takes it from the caller's workspace.  Here it lives in a file-scope device array
+// that is part of the library image: every GPU context that loads the library carries these 4096
 // bytes until the process exits, and nothing is ever allocated or freed.
 #include "lml_table.cuh"
 
@@ -13,9 +13,8 @@ using namespace lml;
 namespace {
 
 constexpr size_t kStaticU = (size_t)kDecodeMaxT * kRankPad * sizeof(float);   // 4096 bytes
-constexpr size_t kStaticRowSlot = kDecodeMaxT * sizeof(int32_t);              // 64 bytes
-constexpr size_t kStaticScratchBytes = 4352;                                   // rounded up to 256
-static_assert(kStaticU + kStaticRowSlot <= kStaticScratchBytes, "static scratch too small");
+constexpr size_t kStaticScratchBytes = 4096;
+static_assert(kStaticU <= kStaticScratchBytes, "static scratch too small");
 
 // In host code this name is only a handle for the runtime, not a device address: the address the
 // kernels get is looked up once per device with cudaGetSymbolAddress below.
@@ -62,19 +61,14 @@ extern "C" lml_status lora_mixed_linear_decode_static(lml_table* t, const void* 
     void* scratch = nullptr;
     if (scratch_address(t->device, &scratch) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
     float* u = static_cast<float*>(scratch);
-    int32_t* row_slot = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(scratch) + kStaticU);
 
+    // The array keeps whatever the previous call left.  Nothing has to start at zero: the kernel
+    // writes every element of u that it later reads (all columns of a row's slot up to the next
+    // multiple of eight) before the grid-wide counter lets any CTA read it.
     int launches = 0;
-    if (G > 0) {
-        // The array keeps whatever the previous call left.  u is rewritten for every row the call
-        // addresses, but a row that a malformed perm never names would keep an old slot: start all
-        // rows at "no adapter" (-1 = all bits set).
-        if (cudaMemsetAsync(row_slot, 0xFF, kStaticRowSlot, stream) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
-    }
     DecodeArgs a;
     a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
     a.u = G > 0 ? u : nullptr;
-    a.row_slot = G > 0 ? row_slot : nullptr;
     a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
     cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
     t->last_launches = launches;
