@@ -156,6 +156,9 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * result and count themselves in the table's status block, so two decode calls on the SAME table
  * must not overlap on the GPU: put them on one stream or order them); larger T runs the
  * TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
+ * W0 is the frozen base weight: it must not be written by the operation that immediately precedes
+ * the call on `stream` (the decode kernel starts fetching W0 while the kernel before it is still
+ * draining; x, the segment arrays and the adapters are read only after that kernel has finished).
  * Errors: INVALID_ARG, WORKSPACE, CUDA.
  */
 lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,

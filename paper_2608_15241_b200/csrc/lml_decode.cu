@@ -5,7 +5,9 @@
 // of HBM bandwidth and contiguous addresses stream best.  Twelve warps in three roles:
 //   producer (1 warp)   copies 8 rows x 2048 columns per stage (one 4 KB bulk asynchronous copy per
 //                       row) into a shared-memory ring, unit after unit, so the CTA walks its rows
-//                       front to back; it runs ahead across rounds.
+//                       front to back; it runs ahead across rounds.  It starts right at kernel entry,
+//                       before the wait for the preceding work on the stream (W0 does not depend on
+//                       it), so HBM already streams this call's weights while that work drains.
 //   consumers (8 warps) each own a fixed slice of K: their x fragments are loaded once into
 //                       registers and reused for every row.  y^T += W0.x^T runs on mma.sync m16n8k16
 //                       with the tokens as the 16-row operand (T <= 16 is exactly one tile; T <= 8
@@ -45,7 +47,9 @@ constexpr int kDecRoundUnits = 6;                // units (= 48 rows) reduced to
 constexpr int kDecSlotFloats = 16 * kDecUnitRows;   // [token][row] partial sums of one warp for one unit
 constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 4;
 constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256;
+constexpr int kDecSegCache = 128;                 // segments whose offsets and slots are looked up in shared memory
+constexpr int kDecSegBytes = (2 * kDecSegCache + 2) * 4;
+constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes;
 static_assert(kDecSmemBytes <= 232448, "shared memory budget");
 
 struct DecCtrl {
@@ -88,6 +92,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     float* slots = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes);   // [stage][warp][token][row]
     float* u_s = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);   // [16][64]
     DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
+    int* ctrl_seg = reinterpret_cast<int*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
@@ -99,26 +104,64 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     constexpr int kChunksPerSpan = kSpan / kDecChunk;
     const int nspans = (K + kSpan - 1) / kSpan;
 
-    if (tid == 0) {
-        for (int s = 0; s < kDecStages; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
-        }
-        ctrl->abort = 0;
-        ctrl->bad_offsets = 0;
-        fence_mbar_init();
-    }
-    if (tid < 16) ctrl->slot_of_row[tid] = -1;
-    grid_dependency_wait();     // launched as a programmatic dependent: the work before this call is complete now
-    grid_launch_dependents();
-    __syncthreads();
     volatile int* abort = &ctrl->abort;
-
-    const int gq = lane >> 2, tq = lane & 3;
     const bool consumer = warp < kDecConsumers;
+    const bool producer = warp == kDecConsumers;
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
+
+    // ---- producer warp ----------------------------------------------------------------------------------
+    // It sets up the ring's barriers, meets the other warps once so that they see them, and starts
+    // copying at once: W0 is the frozen base weight and does not depend on the work that precedes this
+    // call on the stream, so only the other warps (which read x, the segments and the adapters) wait
+    // for that work.  Lane r < 8 copies this stage's 4 KB of row r; a unit's chunks follow each other,
+    // so the CTA walks its rows front to back, and the warp never waits for a round's epilogue, only
+    // for free stages.
+    if (producer) {
+        if (lane == 0) {
+            for (int s = 0; s < kDecStages; ++s) {
+                mbar_init(smem_u32(&ctrl->full[s]), 1);
+                mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
+            }
+            ctrl->abort = 0;
+            ctrl->bad_offsets = 0;
+            fence_mbar_init();
+        }
+        if (lane < 16) ctrl->slot_of_row[lane] = -1;
+        asm volatile("bar.sync 4, %0;" ::"n"(kDecThreads) : "memory");   // the barriers are set up
+        grid_launch_dependents();
+        for (int round_begin = row_begin; round_begin < row_end && ok; round_begin += kDecRoundUnits * kDecUnitRows) {
+            const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
+            const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
+            for (int sp = 0; sp < nspans && ok; ++sp) {
+                const int k_begin = sp * kSpan;
+                const int span = min(kSpan, K - k_begin);
+                const int nchunks = (span + kDecChunk - 1) / kDecChunk;
+                for (int un = 0; un < nunits && ok; ++un) {
+                    const int r0 = round_begin + un * kDecUnitRows;
+                    const int rows = min(kDecUnitRows, round_begin + round_rows - r0);
+                    for (int kc = 0; kc < nchunks && ok; ++kc) {
+                        const int cols = min(kDecChunk, span - kc * kDecChunk);
+                        ok = mbar_wait_warp(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
+                        if (!ok) break;
+                        if (lane == 0) mbar_arrive_expect_tx(smem_u32(&ctrl->full[stage]), (uint32_t)(rows * cols * 2));
+                        __syncwarp();
+                        if (lane < rows)
+                            bulk_copy_g2s(ring + stage * kDecStageBytes + lane * kDecRowPitch,
+                                          W0 + (size_t)(r0 + lane) * K + k_begin + kc * kDecChunk,
+                                          (uint32_t)(cols * 2), smem_u32(&ctrl->full[stage]));
+                        if (++stage == kDecStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else {
+        asm volatile("bar.sync 4, %0;" ::"n"(kDecThreads) : "memory");
+        grid_dependency_wait();     // launched as a programmatic dependent: the work before this call is complete now
+    }
+
+    const int gq = lane >> 2, tq = lane & 3;
     bool u_ready = false;
 
     // This warp's x fragments (chunk kc, k-steps warp*S .. warp*S+S-1 of a span) stay in registers.
@@ -147,22 +190,59 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     if (shrinker && G > 0) {
         const int sw = warp - kDecConsumers - 1;
         if (sw == 0) {
+            // One memory round trip for everything the lookup needs: the segment arrays go to shared
+            // memory (all loads issued before the first is used), the search then runs there.  Calls
+            // with more segments than the cache holds search in global memory instead.
+            const bool cached = G <= kDecSegCache;
+            int* seg_s = ctrl_seg;                       // [G + 1]
+            int* ids_s = ctrl_seg + kDecSegCache + 1;    // [G]
+            int my_row = lane;
+            if (cached) {
+                int so[kDecSegCache / 32 + 1], si[kDecSegCache / 32 + 1];
+#pragma unroll
+                for (int i = 0; i <= kDecSegCache / 32; ++i) {
+                    const int g = lane + 32 * i;
+                    so[i] = g <= G ? __ldg(seg_offsets + g) : 0;
+                    si[i] = g < G ? __ldg(slot_ids + g) : -1;
+                }
+                if (perm && lane < T) my_row = __ldg(perm + lane);
+#pragma unroll
+                for (int i = 0; i <= kDecSegCache / 32; ++i) {
+                    const int g = lane + 32 * i;
+                    if (g <= G) seg_s[g] = so[i];
+                    if (g < G) ids_s[g] = si[i];
+                }
+                __syncwarp();
+            } else if (perm && lane < T) {
+                my_row = __ldg(perm + lane);
+            }
             int bad = 0, bad_slot = 0;
             for (int g = lane; g < G; g += 32) {
-                const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1), sl = __ldg(slot_ids + g);
+                const int s0 = cached ? seg_s[g] : __ldg(seg_offsets + g), s1 = cached ? seg_s[g + 1] : __ldg(seg_offsets + g + 1);
+                const int sl = cached ? ids_s[g] : __ldg(slot_ids + g);
                 if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
                 if (sl != -1 && slot_rank(snap, sl) == 0) bad_slot = 1;
             }
-            if (lane == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
+            if (lane == 0 && ((cached ? seg_s[0] : __ldg(seg_offsets)) != 0 || (cached ? seg_s[G] : __ldg(seg_offsets + G)) != T)) bad = 1;
             bad = __any_sync(0xffffffffu, bad);
             bad_slot = __any_sync(0xffffffffu, bad_slot);
             int bad_perm = 0;
             if (!bad && lane < T) {
-                const int row = perm ? __ldg(perm + lane) : lane;
+                const int row = my_row;
                 if (row >= 0 && row < T) {
-                    const int g = seg_upper(seg_offsets, G, lane);
+                    int g;
+                    if (cached) {   // first segment whose end lies beyond this position
+                        int lo = 0, hi = G;
+                        while (lo < hi) {
+                            const int mid = (lo + hi) >> 1;
+                            if (seg_s[mid + 1] > lane) hi = mid; else lo = mid + 1;
+                        }
+                        g = lo;
+                    } else {
+                        g = seg_upper(seg_offsets, G, lane);
+                    }
                     int slot = -1;
-                    if (g < G) { const int sl = __ldg(slot_ids + g); if (slot_rank(snap, sl) > 0) slot = sl; }
+                    if (g < G) { const int sl = cached ? ids_s[g] : __ldg(slot_ids + g); if (slot_rank(snap, sl) > 0) slot = sl; }
                     ctrl->slot_of_row[row] = slot;
                 } else bad_perm = 1;
             }
@@ -175,6 +255,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
+        if (sw == kDecShrinkWarps - 1 && lane < T) {   // the expand's B rows for this CTA's output columns, towards L2
+            const int slot = ctrl->slot_of_row[lane];
+            if (slot >= 0) {
+                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
+                for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+            }
+        }
         // Dot product d (rows of x in order, j ascending inside a row, each row padded to a multiple of
         // eight columns because the expand reads u in groups of eight) belongs to CTA d mod grid.
         int total = 0;
@@ -198,17 +285,17 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             const __nv_bfloat16* xr = x + (size_t)t * K;
             const __nv_bfloat16* ar = arenaA + ((size_t)slot * kRankPad + j) * K;
             float dot = 0.f;
-            for (int kb = lane * 8; kb < K; kb += 8 * 256) {
-                uint4 xv[8], av[8];
+            for (int kb = lane * 8; kb < K; kb += 16 * 256) {   // 32 loads in flight per lane: one round trip for K <= 4096
+                uint4 xv[16], av[16];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 16; ++i) {
                     const int k0 = kb + i * 256;
                     const bool v = k0 < K;
                     xv[i] = v ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
                     av[i] = v ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 16; ++i) {
                     float p = 0.f;
                     p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
                     p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
@@ -226,13 +313,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         if (sw == 0 && lane == 0) {
             __threadfence();
             atomicAdd(sync_words, 1u);
-        }
-        if (sw == 0 && lane < T) {   // the expand's B rows for this CTA's output columns, towards L2
-            const int slot = ctrl->slot_of_row[lane];
-            if (slot >= 0) {
-                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
-            }
         }
         // Wait (bounded) until every CTA has reported its dot products, then stage u in shared memory
         // for the consumers' epilogue, off their critical path.
@@ -258,34 +338,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         }
     }
 
-    for (int round_begin = shrinker ? row_end : row_begin; round_begin < row_end; round_begin += kDecRoundUnits * kDecUnitRows) {
+    for (int round_begin = consumer ? row_begin : row_end; round_begin < row_end; round_begin += kDecRoundUnits * kDecUnitRows) {
         const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
         const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
         for (int sp = 0; sp < nspans; ++sp) {
             const int k_begin = sp * kSpan;
             const int span = min(kSpan, K - k_begin);
             const int nchunks = (span + kDecChunk - 1) / kDecChunk;
-            if (!consumer) {
-                // ---------------------------------------------------------- producer warp
-                // lane r < 8 copies this stage's 2 KB of row r; a unit's chunks follow each other, so the
-                // CTA walks its rows front to back
-                for (int un = 0; un < nunits && ok; ++un) {
-                    const int r0 = round_begin + un * kDecUnitRows;
-                    const int rows = min(kDecUnitRows, round_begin + round_rows - r0);
-                    for (int kc = 0; kc < nchunks && ok; ++kc) {
-                        const int cols = min(kDecChunk, span - kc * kDecChunk);
-                        ok = mbar_wait_warp(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
-                        if (!ok) break;
-                        if (lane == 0) mbar_arrive_expect_tx(smem_u32(&ctrl->full[stage]), (uint32_t)(rows * cols * 2));
-                        __syncwarp();
-                        if (lane < rows)
-                            bulk_copy_g2s(ring + stage * kDecStageBytes + lane * kDecRowPitch,
-                                          W0 + (size_t)(r0 + lane) * K + k_begin + kc * kDecChunk,
-                                          (uint32_t)(cols * 2), smem_u32(&ctrl->full[stage]));
-                        if (++stage == kDecStages) { stage = 0; phase ^= 1u; }
-                    }
-                }
-            } else {
+            {
                 // ---------------------------------------------------------- consumer warps
                 // this warp's k-steps of the span: chunk kc, steps warp*4 .. warp*4+3.  The x fragments
                 // live in registers for every row of the round.
@@ -303,17 +363,23 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                             ok = mbar_wait_warp(smem_u32(&ctrl->full[stage]), phase, abort);
                             if (ok) {
                                 const uint32_t wbase = ring + stage * kDecStageBytes + gq * kDecRowPitch + tq * 16;
+                                // all of the stage's operand reads first, then the stage can go back to the producer
+                                // before the MMAs run
+                                uint4 w[kDecStepsPerChunk];
+#pragma unroll
+                                for (int i = 0; i < kDecStepsPerChunk; ++i) {
+                                    const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
+                                    w[i] = (rv && c0 + tq * 8 < span) ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
+                                                                      : make_uint4(0, 0, 0, 0);
+                                }
 #pragma unroll
                                 for (int i = 0; i < kDecStepsPerChunk; ++i) {
                                     const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
                                     if (c0 < span) {   // uniform across the warp: all lanes issue the MMAs or none
-                                        const uint4 w = (rv && c0 + tq * 8 < span)
-                                                            ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
-                                                            : make_uint4(0, 0, 0, 0);
                                         const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
                                         const uint4 a1 = kTwo ? xc[kc * kDecStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
-                                        mma_bf16_16816(acc4[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, w.x, w.y);
-                                        mma_bf16_16816(acc4[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, w.z, w.w);
+                                        mma_bf16_16816(acc4[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, w[i].x, w[i].y);
+                                        mma_bf16_16816(acc4[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, w[i].z, w[i].w);
                                     }
                                 }
                                 __syncwarp();
