@@ -17,11 +17,14 @@
 //                       product does not see, so operands are plain 16-byte loads.  Per-warp partial
 //                       sums go to per-warp slots and are added in a fixed order; the LoRA expand
 //                       sum_j u[t][j] B_s[n][j] is added in fp32 before the single bf16 rounding.
-//   shrink (3 warps)    only when the call has segments: look up each row's slot, then compute this
-//                       CTA's share of u[row][j] = scale_s * sum_k x[row][k] A_s[j][k] (fp32, one warp
-//                       per dot product, dealt out round-robin over the whole grid), publish it in
-//                       global memory, wait for the other CTAs' shares on a counter and stage all of u
-//                       in shared memory.  The consumers meet them once, at their first epilogue.
+//   shrink (3 warps)    only when the call has segments: look up each row's slot (segment arrays cached in
+//                       shared memory), then compute this CTA's share of u[row][j] = scale_s * sum_k
+//                       x[row][k] A_s[j][k] (fp32; dot products dealt out round-robin over the whole
+//                       grid; all three warps on one when the CTA has only one), publish each result in
+//                       global memory with a release-add on a grid-wide counter, wait for the counter
+//                       and stage all of u in shared memory.  When the table's live adapters are few,
+//                       their rows of A are asked into L2 at kernel entry, ahead of the weight stream.
+//                       The consumers meet the shrink warps once, at their first epilogue.
 //                       The hand-over between CTAs needs them all resident, so a call with segments
 //                       is a cooperative launch.
 // d_in wider than a span is walked span by span.  All waits are bounded.
@@ -42,14 +45,26 @@ constexpr int kDecChunksPerSpan = kDecSpan / kDecChunk;             // 4
 constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 4 k-steps per warp and stage
 constexpr int kDecRowPitch = kDecChunk * 2 + 64; // bytes; a multiple of 16 that is 4 mod 8 in 16-byte chunks: rows land on different banks
 constexpr int kDecStageBytes = kDecUnitRows * kDecRowPitch;
-constexpr int kDecStages = 5;
+constexpr int kDecStages = 4;
 constexpr int kDecRoundUnits = 6;                // units (= 48 rows) reduced together
 constexpr int kDecSlotFloats = 16 * kDecUnitRows;   // [token][row] partial sums of one warp for one unit
 constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 4;
 constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
 constexpr int kDecSegCache = 128;                 // segments whose offsets and slots are looked up in shared memory
-constexpr int kDecSegBytes = (2 * kDecSegCache + 2) * 4;
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes;
+struct DecLookup {   // what the shrink warps work out about the call, in shared memory
+    int seg[kDecSegCache + 1];
+    int ids[kDecSegCache];
+    float scale_s[kMaxSlots];
+    uint8_t rank_s[kMaxSlots];
+    int dot_end[16];        // running total of dot products up to and including each row of x
+    int rank_of_row[16];
+    float scale_of_row[16];
+    float dot_part[2][4];
+    int pad[1];
+};
+constexpr int kDecSegBytes = (int)sizeof(DecLookup);
+constexpr int kDecBBytes = 32768;                  // shared-memory copy of the B rows this CTA's epilogue needs
+constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecBBytes;
 static_assert(kDecSmemBytes <= 232448, "shared memory budget");
 
 struct DecCtrl {
@@ -58,8 +73,11 @@ struct DecCtrl {
     int abort;
     int bad_offsets;
     int slot_of_row[16];
+    int b_of_row[16];    // which block of the B copy in shared memory serves this row of x, -1: read B from global memory
+    int b_staged;        // blocks on their way into shared memory
+    uint64_t bfull;
 };
-static_assert(sizeof(DecCtrl) <= 256, "control block");
+static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control block");
 
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
@@ -71,6 +89,20 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)   // 16-byte aligned, multiple of 16
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
@@ -92,7 +124,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     float* slots = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes);   // [stage][warp][token][row]
     float* u_s = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);   // [16][64]
     DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
-    int* ctrl_seg = reinterpret_cast<int*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
+    DecLookup* lk = reinterpret_cast<DecLookup*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
+    uint8_t* b_s = base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8;   // 16-byte aligned
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
@@ -124,11 +157,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 mbar_init(smem_u32(&ctrl->full[s]), 1);
                 mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
             }
+            mbar_init(smem_u32(&ctrl->bfull), 1);
             ctrl->abort = 0;
             ctrl->bad_offsets = 0;
+            ctrl->b_staged = 0;
             fence_mbar_init();
         }
-        if (lane < 16) ctrl->slot_of_row[lane] = -1;
+        if (lane < 16) { ctrl->slot_of_row[lane] = -1; ctrl->b_of_row[lane] = -1; }
         asm volatile("bar.sync 4, %0;" ::"n"(kDecThreads) : "memory");   // the barriers are set up
         grid_launch_dependents();
         for (int round_begin = row_begin; round_begin < row_end && ok; round_begin += kDecRoundUnits * kDecUnitRows) {
@@ -185,66 +220,121 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     // dot product, sixteen 16-byte loads in flight per lane.  The results go to u in global memory; a
     // counter in the table's status block tells every CTA when all of u is there (the launch is
     // cooperative, so all CTAs are resident).  The consumers look at it only in their first epilogue.
-    unsigned int* sync_words = status + 1;   // [0] CTAs whose share of u is written, [1] CTAs that have left
+    unsigned int* sync_words = status + 1;   // [0] elements of u that are written, [1] CTAs that have left
     const bool shrinker = warp > kDecConsumers;
+    if (consumer && G > 0)   // let the lookup's loads go first through the load/store path (see below)
+        asm volatile("bar.sync 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
     if (shrinker && G > 0) {
         const int sw = warp - kDecConsumers - 1;
+        if (sw == 1) {
+            // Which adapters this call names is known only after the lookup below, a memory round trip
+            // from now, and their rows of A are cold: with W0 streaming at full rate a read from HBM
+            // then takes several microseconds.  So when the table's live adapters are few (their rows
+            // of A together at most a sixteenth of W0), all of them are asked into L2 right now,
+            // ahead of the weight stream, a row or two per CTA; the dot products below find them there.
+            int rows_before = 0, my_rank[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int sl = lane + 32 * h;
+                my_rank[h] = sl < snap.max_slots && sl < kMaxSlots ? (int)snap.rank[sl] : 0;
+            }
+            // running count of live rows in slot order: slots 0..31 first, then 32..63
+            int incl0 = my_rank[0], incl1 = my_rank[1];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v0 = __shfl_up_sync(0xffffffffu, incl0, o), v1 = __shfl_up_sync(0xffffffffu, incl1, o);
+                if (lane >= o) { incl0 += v0; incl1 += v1; }
+            }
+            const int total0 = __shfl_sync(0xffffffffu, incl0, 31);
+            const int live_rows = total0 + __shfl_sync(0xffffffffu, incl1, 31);
+            if ((long long)live_rows * K * 16 <= (long long)N * K) {
+                // lane L of this CTA takes live row blockIdx + L * grid
+                const int i = (int)blockIdx.x + lane * (int)gridDim.x;
+                // find the slot holding live row i: the first whose inclusive count exceeds i
+                const unsigned m0 = __ballot_sync(0xffffffffu, incl0 > 0);   // (dummy use keeps the shuffles converged)
+                (void)m0;
+                int slot = -1, j = 0;
+                for (int src = 0; src < 32; ++src) {   // uniform loop: every lane reads every lane's counts
+                    const int e0 = __shfl_sync(0xffffffffu, incl0, src), r0 = __shfl_sync(0xffffffffu, my_rank[0], src);
+                    const int e1 = __shfl_sync(0xffffffffu, incl1, src) + total0, r1 = __shfl_sync(0xffffffffu, my_rank[1], src);
+                    if (slot < 0 && i < e0 && i >= e0 - r0) { slot = src; j = i - (e0 - r0); }
+                    if (slot < 0 && i < e1 && i >= e1 - r1) { slot = src + 32; j = i - (e1 - r1); }
+                }
+                if (i < live_rows && slot >= 0)
+                    bulk_prefetch_l2(arenaA + ((size_t)slot * kRankPad + j) * K, (uint32_t)(K * 2));
+                (void)rows_before;
+            }
+        }
         if (sw == 0) {
             // One memory round trip for everything the lookup needs: the segment arrays go to shared
             // memory (all loads issued before the first is used), the search then runs there.  Calls
-            // with more segments than the cache holds search in global memory instead.
+            // with more segments than the cache holds search in global memory instead.  The consumer
+            // warps hold their (many) loads of x back until these few are on their way, and while they
+            // are, the slots' ranks and scales move from the kernel parameters to shared memory:
+            // indexed reads of parameters are slow the first time, and everything later reads the copy.
             const bool cached = G <= kDecSegCache;
-            int* seg_s = ctrl_seg;                       // [G + 1]
-            int* ids_s = ctrl_seg + kDecSegCache + 1;    // [G]
             int my_row = lane;
+            int so[kDecSegCache / 32 + 1], si[kDecSegCache / 32 + 1];
             if (cached) {
-                int so[kDecSegCache / 32 + 1], si[kDecSegCache / 32 + 1];
 #pragma unroll
                 for (int i = 0; i <= kDecSegCache / 32; ++i) {
                     const int g = lane + 32 * i;
                     so[i] = g <= G ? __ldg(seg_offsets + g) : 0;
                     si[i] = g < G ? __ldg(slot_ids + g) : -1;
                 }
-                if (perm && lane < T) my_row = __ldg(perm + lane);
+            }
+            if (perm && lane < T) my_row = __ldg(perm + lane);
+            asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
+            for (int sl = lane; sl < kMaxSlots; sl += 32) {
+                lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
+                lk->scale_s[sl] = snap.scale[sl];
+            }
+            if (cached) {
 #pragma unroll
                 for (int i = 0; i <= kDecSegCache / 32; ++i) {
                     const int g = lane + 32 * i;
-                    if (g <= G) seg_s[g] = so[i];
-                    if (g < G) ids_s[g] = si[i];
+                    if (g <= G) lk->seg[g] = so[i];
+                    if (g < G) lk->ids[g] = si[i];
                 }
-                __syncwarp();
-            } else if (perm && lane < T) {
-                my_row = __ldg(perm + lane);
             }
-            int bad = 0, bad_slot = 0;
-            for (int g = lane; g < G; g += 32) {
-                const int s0 = cached ? seg_s[g] : __ldg(seg_offsets + g), s1 = cached ? seg_s[g + 1] : __ldg(seg_offsets + g + 1);
-                const int sl = cached ? ids_s[g] : __ldg(slot_ids + g);
-                if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
-                if (sl != -1 && slot_rank(snap, sl) == 0) bad_slot = 1;
+            __syncwarp();
+            auto rank_of = [&](int sl) { return (sl >= 0 && sl < kMaxSlots) ? (int)lk->rank_s[sl] : 0; };
+            // (two separate code paths: written as one with selects, the compiler issues the global loads
+            // of the uncached path unconditionally, a memory round trip on the critical path)
+            int bad = 0, bad_slot = 0, bad_perm = 0, slot = -1;
+            const int row = my_row;
+            const bool row_ok = lane < T && row >= 0 && row < T;
+            if (cached) {
+                for (int g = lane; g < G; g += 32) {
+                    const int s0 = lk->seg[g], s1 = lk->seg[g + 1], sl = lk->ids[g];
+                    if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
+                    if (sl != -1 && rank_of(sl) == 0) bad_slot = 1;
+                }
+                if (lane == 0 && (lk->seg[0] != 0 || lk->seg[G] != T)) bad = 1;
+                if (row_ok) {   // first segment whose end lies beyond this position
+                    int lo = 0, hi = G;
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        if (lk->seg[mid + 1] > lane) hi = mid; else lo = mid + 1;
+                    }
+                    if (lo < G && rank_of(lk->ids[lo]) > 0) slot = lk->ids[lo];
+                }
+            } else {
+                for (int g = lane; g < G; g += 32) {
+                    const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1), sl = __ldg(slot_ids + g);
+                    if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
+                    if (sl != -1 && rank_of(sl) == 0) bad_slot = 1;
+                }
+                if (lane == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
+                if (row_ok) {
+                    const int g = seg_upper(seg_offsets, G, lane);
+                    if (g < G) { const int sl = __ldg(slot_ids + g); if (rank_of(sl) > 0) slot = sl; }
+                }
             }
-            if (lane == 0 && ((cached ? seg_s[0] : __ldg(seg_offsets)) != 0 || (cached ? seg_s[G] : __ldg(seg_offsets + G)) != T)) bad = 1;
             bad = __any_sync(0xffffffffu, bad);
             bad_slot = __any_sync(0xffffffffu, bad_slot);
-            int bad_perm = 0;
             if (!bad && lane < T) {
-                const int row = my_row;
-                if (row >= 0 && row < T) {
-                    int g;
-                    if (cached) {   // first segment whose end lies beyond this position
-                        int lo = 0, hi = G;
-                        while (lo < hi) {
-                            const int mid = (lo + hi) >> 1;
-                            if (seg_s[mid + 1] > lane) hi = mid; else lo = mid + 1;
-                        }
-                        g = lo;
-                    } else {
-                        g = seg_upper(seg_offsets, G, lane);
-                    }
-                    int slot = -1;
-                    if (g < G) { const int sl = cached ? ids_s[g] : __ldg(slot_ids + g); if (slot_rank(snap, sl) > 0) slot = sl; }
-                    ctrl->slot_of_row[row] = slot;
-                } else bad_perm = 1;
+                if (row_ok) ctrl->slot_of_row[row] = slot; else bad_perm = 1;
             }
             bad_perm = __any_sync(0xffffffffu, bad_perm);
             if (lane == 0) {
@@ -253,75 +343,124 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                                    (bad_perm ? LML_FLAG_BAD_PERM : 0u);
                 if (f && blockIdx.x == 0) atomicOr(status, f);
             }
+            __syncwarp();
+            // Per row of x: rank, scale, and where its dot products end in the grid-wide numbering (rows
+            // in order, j ascending inside a row, each row padded to a multiple of eight columns because
+            // the expand reads u in groups of eight).
+            {
+                const int slot = lane < T ? ctrl->slot_of_row[lane] : -1;
+                const int rank = slot >= 0 ? (int)lk->rank_s[slot] : 0;
+                int end = (rank + 7) & ~7;
+#pragma unroll
+                for (int o = 1; o < 16; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, end, o);
+                    if (lane >= o) end += v;
+                }
+                if (lane < 16) {
+                    lk->dot_end[lane] = end;
+                    lk->rank_of_row[lane] = rank;
+                    lk->scale_of_row[lane] = slot >= 0 ? lk->scale_s[slot] : 0.f;
+                }
+            }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
-        if (sw == kDecShrinkWarps - 1 && lane < T) {   // the expand's B rows for this CTA's output columns, towards L2
-            const int slot = ctrl->slot_of_row[lane];
-            if (slot >= 0) {
+        if (sw == kDecShrinkWarps - 1) {
+            // The expand's B rows for this CTA's output columns: one contiguous block per distinct slot,
+            // copied into shared memory now so that the epilogue has no memory round trip left.  Slots
+            // that do not fit (many adapters in one call, or many rows per CTA) are prefetched into L2
+            // and read from there.
+            const int slot = lane < T ? ctrl->slot_of_row[lane] : -1;
+            const unsigned same = __match_any_sync(0xffffffffu, slot);
+            const bool leader = slot >= 0 && (same & ((1u << lane) - 1u)) == 0u;
+            const unsigned leaders = __ballot_sync(0xffffffffu, leader);
+            const int block_bytes = (row_end - row_begin) * kRankPad * 2;
+            const int fit = block_bytes > 0 ? kDecBBytes / block_bytes : 0;
+            const int my_block = __popc(leaders & ((1u << (__ffs(same) - 1)) - 1u));   // rank of this lane's slot among the distinct ones
+            const bool staged = slot >= 0 && my_block < fit;
+            const int nblocks = min(__popc(leaders), fit);
+            if (lane < T) ctrl->b_of_row[lane] = staged ? my_block : -1;
+            if (lane == 0) {
+                ctrl->b_staged = nblocks;
+                if (nblocks > 0) mbar_arrive_expect_tx(smem_u32(&ctrl->bfull), (uint32_t)(nblocks * block_bytes));
+            }
+            __syncwarp();
+            if (leader) {
                 const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+                if (staged) bulk_copy_g2s(smem_u32(b_s) + my_block * block_bytes, b, (uint32_t)block_bytes, smem_u32(&ctrl->bfull));
+                else for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
             }
         }
-        // Dot product d (rows of x in order, j ascending inside a row, each row padded to a multiple of
-        // eight columns because the expand reads u in groups of eight) belongs to CTA d mod grid.
-        int total = 0;
-        for (int t = 0; t < T; ++t) {
-            const int slot = ctrl->slot_of_row[t];
-            total += slot >= 0 ? (((int)snap.rank[slot] + 7) & ~7) : 0;
-        }
-        for (int d = (int)blockIdx.x + sw * (int)gridDim.x; d < total; d += kDecShrinkWarps * (int)gridDim.x) {
-            int t = 0, j = d, slot = -1, rank = 0;
-            for (; t < T; ++t) {   // which row does d fall into
-                slot = ctrl->slot_of_row[t];
-                rank = slot >= 0 ? (int)snap.rank[slot] : 0;
-                const int rank8 = (rank + 7) & ~7;
-                if (j < rank8) break;
-                j -= rank8;
-            }
-            if (j >= rank) {   // padding column: B is zero there, u must at least be finite
-                if (lane == 0) u[t * kRankPad + j] = 0.f;
-                continue;
-            }
-            const __nv_bfloat16* xr = x + (size_t)t * K;
-            const __nv_bfloat16* ar = arenaA + ((size_t)slot * kRankPad + j) * K;
+        // Dot product d belongs to CTA d mod grid.  A lane keeps twelve 16-byte loads in flight (six of x,
+        // six of A: what the register budget allows), so a warp alone needs several memory round trips per
+        // dot product.  A CTA with a single dot product (the usual case: a few tokens, rank 16) therefore
+        // puts all three shrink warps on it, one round trip in all; with more, each warp takes its own.
+        // Each result is published by its own release-add on the grid-wide counter: nobody waits for a fence.
+        const int total = lk->dot_end[15];
+        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+        const int mine = total > (int)blockIdx.x ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+        auto partial_dot = [&](int d, int first, int nthreads, int& t, int& j, bool& real) {
+            t = 0;
+            while (lk->dot_end[t] <= d) ++t;   // which row does d fall into
+            j = d - (t > 0 ? lk->dot_end[t - 1] : 0);
+            real = j < lk->rank_of_row[t];     // else a padding column: B is zero there, u must at least be finite
             float dot = 0.f;
-            for (int kb = lane * 8; kb < K; kb += 16 * 256) {   // 32 loads in flight per lane: one round trip for K <= 4096
-                uint4 xv[16], av[16];
+            if (real) {
+                const __nv_bfloat16* xr = x + (size_t)t * K;
+                const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
+                constexpr int kPer = 6;
+                const int stride = nthreads * 8;
+                for (int kb = first * 8; kb < K; kb += kPer * stride) {
+                    uint4 xv[kPer], av[kPer];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int k0 = kb + i * 256;
-                    const bool v = k0 < K;
-                    xv[i] = v ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
-                    av[i] = v ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
+                    for (int i = 0; i < kPer; ++i) {
+                        const int k0 = kb + i * stride;
+                        const bool v = k0 < K;
+                        xv[i] = v ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
+                        av[i] = v ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        float p = 0.f;
+                        p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
+                        p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
+                        p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
+                        p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
+                        dot += p;
+                    }
                 }
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float p = 0.f;
-                    p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
-                    p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
-                    p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
-                    p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
-                    dot += p;
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            }
+            return dot;
+        };
+        if (mine == 1) {
+            int t, j;
+            bool real;
+            const float dot = partial_dot((int)blockIdx.x, me, kDecShrinkWarps * 32, t, j, real);
+            if (lane == 0) lk->dot_part[0][sw] = dot;
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+            if (me == 0) {
+                u[t * kRankPad + j] = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_of_row[t] : 0.f;
+                red_release_gpu_add(sync_words, 1u);
+            }
+        } else {
+            for (int d = (int)blockIdx.x + sw * (int)gridDim.x; d < total; d += kDecShrinkWarps * (int)gridDim.x) {
+                int t, j;
+                bool real;
+                const float dot = partial_dot(d, lane, 32, t, j, real);
+                if (lane == 0) {
+                    u[t * kRankPad + j] = real ? dot * lk->scale_of_row[t] : 0.f;
+                    red_release_gpu_add(sync_words, 1u);
                 }
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            if (lane == 0) u[t * kRankPad + j] = dot * snap.scale[slot];
         }
-        if (lane == 0) __threadfence();
-        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // this CTA's share of u is written
-        if (sw == 0 && lane == 0) {
-            __threadfence();
-            atomicAdd(sync_words, 1u);
-        }
-        // Wait (bounded) until every CTA has reported its dot products, then stage u in shared memory
-        // for the consumers' epilogue, off their critical path.
+        // Wait (bounded) until all of u is written, then stage it in shared memory for the consumers'
+        // epilogue, off their critical path.
         if (sw == 0 && lane == 0) {
             const long long t0 = clock64();
-            while (*reinterpret_cast<volatile unsigned int*>(sync_words) < gridDim.x) {
+            while (ld_acquire_gpu(sync_words) < (unsigned)total) {
                 if (clock64() - t0 > (1ll << 31)) { ctrl->abort = 1; break; }
             }
-            __threadfence();
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
         for (int i = tid - (kDecConsumers + 1) * 32; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
@@ -410,6 +549,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // partial sums are in the slots
         if (consumer && G > 0 && !u_ready) {   // first epilogue: the shrink warps have staged u in shared memory
             asm volatile("bar.sync 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
+            if (ctrl->b_staged > 0 && ok) ok = mbar_wait_warp(smem_u32(&ctrl->bfull), 0u, abort);   // long since there
             u_ready = true;
         }
         if (consumer && ok) {
@@ -425,12 +565,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
                 const int slot = lora ? ctrl->slot_of_row[t] : -1;
                 if (slot >= 0) {
-                    const int r8 = ((int)snap.rank[slot] + 7) >> 3;
+                    const int r8 = (lk->rank_of_row[t] + 7) >> 3;
                     const uint4* bp = reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
+                    const int bb = ctrl->b_of_row[t];
+                    const uint4* bs = reinterpret_cast<const uint4*>(b_s + ((size_t)bb * (row_end - row_begin) + (n - row_begin)) * kRankPad * 2);
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
                     for (int c = 0; c < r8; ++c) {
-                        uint4 b = ldg_nc_v4(bp + c);
+                        uint4 b = bb >= 0 ? bs[c] : ldg_nc_v4(bp + c);
                         float4 u0 = up[2 * c], u1 = up[2 * c + 1];
                         d = fmaf(u0.x, bf16_lo(b.x), d); d = fmaf(u0.y, bf16_hi(b.x), d);
                         d = fmaf(u0.z, bf16_lo(b.y), d); d = fmaf(u0.w, bf16_hi(b.y), d);
