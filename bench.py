@@ -130,7 +130,7 @@ class Rotation:
 
     def __init__(self, w, device, min_bytes):
         import torch
-        from paper_2608_15241_b200.binding import Table
+        from paper_2608_15241_b200.binding import Table, lml_tokens_workspace_bytes as b_tokens_ws
         self.w = w
         self.device = device
         per_set = w.bytes()
@@ -154,7 +154,8 @@ class Rotation:
                      ids=torch.empty(G, dtype=torch.int32, device=device),
                      y=torch.empty((w.T, w.d_out), dtype=torch.bfloat16, device=device),
                      slots=slots)
-            s["ws"] = torch.empty(tbl.workspace_bytes(w.T, max(G, w.G)), dtype=torch.uint8, device=device)
+            s["ws"] = torch.empty(max(tbl.workspace_bytes(w.T, max(G, w.G)), b_tokens_ws(tbl.handle, w.T)), dtype=torch.uint8,
+                                  device=device)
             # pre-segmented form (segments as the workload states them) for the layer-only loop
             s["so_pre"] = torch.from_numpy(w.seg_offsets).to(device)
             s["ids_pre"] = torch.from_numpy(np.array([slots[e] if e >= 0 else -1 for e in w.seg_entry], np.int32)).to(device)
@@ -163,17 +164,16 @@ class Rotation:
         torch.cuda.synchronize()
 
     def step(self, i):
-        """Whole hot path: segmentation pass + layer."""
+        """Whole hot path from one slot id per token: token segmentation + layer, through the call a
+        serving loop makes (lora_mixed_linear_tokens).  Up to 16 tokens that is one launch (the decode
+        kernel binds every row to its slot itself); above, the segmentation kernel, the row gather, the
+        shrink kernel and the GEMM."""
         from paper_2608_15241_b200 import binding as b
         s = self.sets[i % self.R]
         t = s["table"]
-        st = b._stream(None)
-        b.lml_segment_tokens(t.handle, s["tok"].data_ptr(), self.w.T, s["perm"].data_ptr(), s["so"].data_ptr(),
-                             s["ids"].data_ptr(), st)
-        b.lora_mixed_linear(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["so"].data_ptr(),
-                            s["ids"].data_ptr(), t.max_slots + 1, s["perm"].data_ptr(), s["y"].data_ptr(),
-                            s["ws"].data_ptr(), s["ws"].numel(), st)
-        return 1 + t.last_launch_count()
+        b.lora_mixed_linear_tokens(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["tok"].data_ptr(),
+                                   s["y"].data_ptr(), s["ws"].data_ptr(), s["ws"].numel(), b._stream(None))
+        return t.last_launch_count()
 
     def layer_only(self, i):
         """lora_mixed_linear on pre-segmented input: the launches the roofline figure refers to."""

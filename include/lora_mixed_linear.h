@@ -147,7 +147,8 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * lora_mixed_linear — the layer.  x: device bf16 [T][d_in]; W0: device bf16 [d_out][d_in];
  * y: device bf16 [T][d_out], overwritten.  seg_offsets: device int32[G+1] with
  * seg_offsets[0] = 0 <= ... <= seg_offsets[G] = T; slot_ids: device int32[G], physical slot
- * or -1 per segment (repeated slots, empty segments and any order are fine).  Segment g
+ * or -1 per segment (repeated slots, empty segments and any order are fine; a non-empty
+ * segment whose slot holds no live adapter gets base output and sets LML_FLAG_BAD_SLOT).  Segment g
  * covers positions [seg_offsets[g], seg_offsets[g+1]); position p is row perm[p] of x and y
  * if perm (device int32[T], a permutation) is given, else row p.  G == 0 means "no adapter
  * anywhere".  T == 0 returns LML_OK without launching.
@@ -165,6 +166,22 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
                              const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                              const int32_t* perm, void* y, void* workspace, size_t workspace_bytes,
                              void* stream);
+
+/*
+ * lora_mixed_linear_tokens — segmentation and layer in one call, for callers that hold one slot id
+ * per token (what a scheduler hands a decode step).  token_slots: device int32[T], physical slot
+ * per row of x or -1; ids outside [-1, max_slots) or naming a free slot count as -1 and set
+ * LML_FLAG_BAD_SLOT, exactly as in lml_segment_tokens.  x, W0, y as in lora_mixed_linear.
+ * T <= 16: one launch; the decode kernel treats every row on its own and reads the ids itself, no
+ * grouping is computed.  Larger T: the segmentation pass runs into the tail of the workspace and
+ * the perm form of lora_mixed_linear follows on the same stream.  Results are identical to
+ * lml_segment_tokens followed by lora_mixed_linear.  workspace: device, 256-byte aligned, at least
+ * lml_tokens_workspace_bytes(t, T) bytes.  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens);
+lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T,
+                                    const int32_t* token_slots, void* y, void* workspace,
+                                    size_t workspace_bytes, void* stream);
 
 /*
  * Host-buffer form of the same call, for callers whose activations live in host memory.

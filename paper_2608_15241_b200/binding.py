@@ -28,7 +28,7 @@ EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "regist
            "retire_version", "lml_lookup", "lml_slot_info", "lml_workspace_bytes",
            "lml_segment_tokens", "lora_mixed_linear", "lml_host_workspace_bytes",
            "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count",
-           "lora_mixed_linear_decode_static")
+           "lora_mixed_linear_decode_static", "lml_tokens_workspace_bytes", "lora_mixed_linear_tokens")
 
 
 class LmlError(RuntimeError):
@@ -66,10 +66,14 @@ def lib() -> ctypes.CDLL:
         L.lora_mixed_linear.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lora_mixed_linear_host.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lora_mixed_linear_decode_static.argtypes = [vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
+        L.lml_tokens_workspace_bytes.restype = sz
+        L.lml_tokens_workspace_bytes.argtypes = [vp, i32]
+        L.lora_mixed_linear_tokens.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lml_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
-            if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes"):
+            if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes",
+                            "lml_tokens_workspace_bytes"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -148,6 +152,17 @@ def lora_mixed_linear_host(table: int, x_host_ptr: int, W0_ptr: int, T: int, seg
     _check(lib().lora_mixed_linear_host(table, x_host_ptr, W0_ptr, T, seg_offsets_host_ptr, slot_ids_host_ptr, G,
                                         perm_host_ptr, y_host_ptr, workspace_ptr, workspace_bytes, stream),
            "lora_mixed_linear_host")
+
+
+def lml_tokens_workspace_bytes(table: int, max_tokens: int) -> int:
+    return int(lib().lml_tokens_workspace_bytes(table, max_tokens))
+
+
+def lora_mixed_linear_tokens(table: int, x_ptr: int, W0_ptr: int, T: int, token_slots_ptr: int, y_ptr: int,
+                             workspace_ptr: int, workspace_bytes: int, stream: int = 0) -> None:
+    """Segmentation and layer in one call: one slot id per token instead of segments."""
+    _check(lib().lora_mixed_linear_tokens(table, x_ptr, W0_ptr, T, token_slots_ptr, y_ptr, workspace_ptr,
+                                          workspace_bytes, stream), "lora_mixed_linear_tokens")
 
 
 def lora_mixed_linear_decode_static(table: int, x_ptr: int, W0_ptr: int, T: int, seg_offsets_ptr: int,
@@ -284,6 +299,22 @@ class Table:
         lora_mixed_linear(self.handle, _ptr(x), _ptr(W0), T, _ptr(seg_offsets) if G else 0,
                           _ptr(slot_ids) if G else 0, G, _ptr(perm), _ptr(y), _ptr(workspace),
                           int(workspace.numel()), _stream(stream))
+        return y
+
+    def lora_mixed_linear_tokens(self, x, W0, token_slots, y=None, workspace=None, stream=None):
+        """x bf16 [T][d_in], W0 bf16 [d_out][d_in], token_slots int32[T] (all cuda) -> y bf16 [T][d_out]."""
+        import torch
+        assert x.dtype == torch.bfloat16 and W0.dtype == torch.bfloat16 and token_slots.dtype == torch.int32
+        assert x.is_cuda and W0.is_cuda and token_slots.is_cuda and x.is_contiguous() and W0.is_contiguous()
+        T = int(x.shape[0])
+        assert token_slots.shape[0] == T and x.shape[1] == self.d_in and W0.shape == (self.d_out, self.d_in)
+        if y is None:
+            y = torch.empty((T, self.d_out), dtype=torch.bfloat16, device=x.device)
+        if workspace is None:
+            workspace = torch.empty(max(lml_tokens_workspace_bytes(self.handle, T), 256), dtype=torch.uint8,
+                                    device=x.device)
+        lora_mixed_linear_tokens(self.handle, _ptr(x), _ptr(W0), T, _ptr(token_slots), _ptr(y), _ptr(workspace),
+                                 int(workspace.numel()), _stream(stream))
         return y
 
     def lora_mixed_linear_host(self, x_host, W0, seg_offsets_host, slot_ids_host, y_host, perm_host=None,

@@ -253,6 +253,57 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
     return LML_OK;
 }
 
+size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens)
+{
+    if (!t || max_tokens < 0 || max_tokens > kMaxTokens) return 0;
+    size_t n = ws_layout(t, max_tokens, t->max_slots + 1).total;
+    n += round_up((size_t)max_tokens * 4 + 4, 1024);               // perm
+    n += 2 * round_up((size_t)(t->max_slots + 2) * 4, 1024);       // seg_offsets, seg_slot_ids
+    return n;
+}
+
+lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T, const int32_t* token_slots,
+                                    void* y, void* workspace, size_t workspace_bytes, void* stream_v)
+{
+    if (!t || T < 0 || T > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x || !W0 || !y || !token_slots || !aligned16(x) || !aligned16(W0) || !aligned16(y)) return LML_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < lml_tokens_workspace_bytes(t, T))
+        return LML_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    uint8_t* wsb = static_cast<uint8_t*>(workspace);
+    if (T <= kDecodeMaxT) {
+        // Up to 16 tokens need no grouping: the decode kernel handles every row of x on its own, so it reads
+        // the slot ids directly.  One launch.
+        const SlotSnapshot snap = snapshot_locked(t);
+        DeviceGuard guard(t->device);
+        if (!guard.ok) return LML_ERR_CUDA;
+        const WsLayout ws = ws_layout(t, T, 1);
+        DecodeArgs a;
+        a.x = x; a.W0 = W0; a.y = y; a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
+        a.token_slots = token_slots;
+        a.u = reinterpret_cast<float*>(wsb + ws.u_off);
+        a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = 1; a.num_sms = t->num_sms;
+        int launches = 0;
+        const cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
+        t->last_launches = launches;
+        if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+        return LML_OK;
+    }
+    // Prefill: the segmentation pass writes perm and the segment arrays behind the layer's own workspace,
+    // and the layer call follows on the same stream.
+    const int G = t->max_slots + 1;
+    const size_t base = ws_layout(t, T, G).total;
+    int32_t* perm = reinterpret_cast<int32_t*>(wsb + base);
+    int32_t* seg_offsets = reinterpret_cast<int32_t*>(wsb + base + round_up((size_t)T * 4 + 4, 1024));
+    int32_t* seg_ids = seg_offsets + round_up((size_t)(t->max_slots + 2) * 4, 1024) / 4;
+    lml_status st = lml_segment_tokens(t, token_slots, T, perm, seg_offsets, seg_ids, stream_v);
+    if (st != LML_OK) return st;
+    st = lora_mixed_linear(t, x, W0, T, seg_offsets, seg_ids, G, perm, y, workspace, base, stream_v);
+    if (st == LML_OK) t->last_launches += 1;
+    return st;
+}
+
 size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
 {
     if (!t || max_tokens < 0 || max_segments < 0 || max_tokens > kMaxTokens) return 0;

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
     const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
-    const int32_t* __restrict__ perm, uint32_t* status, int T, int K, int N, int G)
+    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, uint32_t* status, int T, int K, int N, int G)
 {
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
@@ -272,7 +272,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             // warps hold their (many) loads of x back until these few are on their way, and while they
             // are, the slots' ranks and scales move from the kernel parameters to shared memory:
             // indexed reads of parameters are slow the first time, and everything later reads the copy.
-            const bool cached = G <= kDecSegCache;
+            const bool by_token = token_slots != nullptr;   // one slot id per row of x instead of segments
+            const bool cached = !by_token && G <= kDecSegCache;
             int my_row = lane;
             int so[kDecSegCache / 32 + 1], si[kDecSegCache / 32 + 1];
             if (cached) {
@@ -284,6 +285,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 }
             }
             if (perm && lane < T) my_row = __ldg(perm + lane);
+            int my_token_slot = -1;
+            if (by_token && lane < T) my_token_slot = __ldg(token_slots + lane);
             asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32) {
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
@@ -304,11 +307,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             int bad = 0, bad_slot = 0, bad_perm = 0, slot = -1;
             const int row = my_row;
             const bool row_ok = lane < T && row >= 0 && row < T;
-            if (cached) {
+            if (by_token) {   // same rule as the segmentation pass: an id that names no live adapter means none, and raises the flag
+                if (lane < T) {
+                    if (my_token_slot >= 0 && rank_of(my_token_slot) > 0) slot = my_token_slot;
+                    else if (my_token_slot != -1) bad_slot = 1;
+                }
+            } else if (cached) {
                 for (int g = lane; g < G; g += 32) {
                     const int s0 = lk->seg[g], s1 = lk->seg[g + 1], sl = lk->ids[g];
                     if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
-                    if (sl != -1 && rank_of(sl) == 0) bad_slot = 1;
+                    if (sl != -1 && s1 > s0 && rank_of(sl) == 0) bad_slot = 1;   // an empty segment may name anything
                 }
                 if (lane == 0 && (lk->seg[0] != 0 || lk->seg[G] != T)) bad = 1;
                 if (row_ok) {   // first segment whose end lies beyond this position
@@ -323,7 +331,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 for (int g = lane; g < G; g += 32) {
                     const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1), sl = __ldg(slot_ids + g);
                     if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
-                    if (sl != -1 && rank_of(sl) == 0) bad_slot = 1;
+                    if (sl != -1 && s1 > s0 && rank_of(sl) == 0) bad_slot = 1;   // an empty segment may name anything
                 }
                 if (lane == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
                 if (row_ok) {
@@ -628,10 +636,11 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const int32_t* so = a.seg_offsets;
     const int32_t* ids = a.slot_ids;
     const int32_t* pm = a.perm;
+    const int32_t* ts = a.token_slots;
     cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, status, a.T, a.d_in, a.d_out, a.G)
+                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G)
                             : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, status, a.T, a.d_in, a.d_out, a.G);
+                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G);
     if (e == cudaSuccess) ++*launches;
     return e;
 }

@@ -92,6 +92,7 @@ struct DecodeArgs {
     const int32_t* perm;
     const int32_t* seg_offsets;
     const int32_t* slot_ids;
+    const int32_t* token_slots = nullptr;   // instead of segments: one slot id per row of x (then G is 1 and perm is null)
     float* u;            // [16][64] fp32 scratch: scale * x.A^T, written and read by the decode kernel
     int T, d_in, d_out, G;
     int num_sms;

@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
             int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
             if (s1 < s0 || s0 < 0 || s1 > T) bad_off = 1;
             int s = __ldg(slot_ids + g);
-            if (s != -1 && slot_rank(snap, s) == 0) bad_slot = 1;
+            if (s != -1 && s1 > s0 && slot_rank(snap, s) == 0) bad_slot = 1;   // an empty segment may name anything
         }
         if (tid == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad_off = 1;
         bad_off = __syncthreads_or(bad_off);

@@ -1,0 +1,89 @@
+"""lora_mixed_linear_tokens (one slot id per token) against the two-call form it replaces:
+lml_segment_tokens followed by lora_mixed_linear with the perm it produced.  Both forms run the
+same arithmetic per output element, so the results must agree bit for bit; the oracle is checked
+on top.  Covers the one-launch decode form (T <= 16), the prefill form, ids that name no live
+adapter (flagged, treated as -1) and the all-base case."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_15241_b200 import workloads as wl
+
+from gpu_util import to_bits, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _table(K, N, ranks, seed):
+    from paper_2608_15241_b200.binding import Table
+    tbl = Table(K, N, len(ranks) + 2)
+    entries = []
+    for s, r in enumerate(ranks):
+        A = wl.normal_bf16(seed, 100 + s, (r, K), 0.05)
+        B = wl.normal_bf16(seed, 200 + s, (N, r), 0.05)
+        slot = tbl.register_adapter(s, 1, to_dev(A), to_dev(B), 1.5)
+        entries.append((slot, wl.AdapterEntry(s, 1, r, 1.5, A, B)))
+    return tbl, entries
+
+
+@pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384)])
+def test_tokens_call_equals_segment_then_layer(T, K, N):
+    import torch
+    tbl, entries = _table(K, N, (4, 16, 33), seed=21)
+    rng = np.random.default_rng(T * 7 + 1)
+    slots = np.array([e[0] for e in entries] + [-1], np.int32)
+    token_slots = slots[rng.integers(0, len(slots), size=T)].astype(np.int32)
+    x_bits = wl.normal_bf16(21, 1, (T, K), 1.0)
+    W_bits = wl.normal_bf16(21, 2, (N, K), 0.05)
+    x, W, ts = to_dev(x_bits), to_dev(W_bits), torch.from_numpy(token_slots).cuda()
+
+    y_tok = to_bits(tbl.lora_mixed_linear_tokens(x, W, ts))
+    launches_tok = tbl.last_launch_count()
+    perm, so, ids = tbl.segment_tokens(ts)
+    y_two = to_bits(tbl.lora_mixed_linear(x, W, so, ids, perm=perm))
+    torch.cuda.synchronize()
+    assert tbl.device_status() == 0
+    assert np.array_equal(y_tok, y_two)
+    if T <= 16:
+        assert launches_tok == 1
+
+    # oracle on the same problem: one segment per token, rows in their original order
+    slot_to_entry = {slot: i for i, (slot, _) in enumerate(entries)}
+    seg_entry = np.array([slot_to_entry.get(int(s), -1) for s in token_slots], np.int32)
+    ref, _ = oracle.forward(x_bits, W_bits, [e for _, e in entries], np.arange(T + 1, dtype=np.int32), seg_entry)
+    cmp = oracle.compare(y_tok, ref)
+    assert cmp["ok"], cmp
+    tbl.close()
+
+
+def test_tokens_call_flags_ids_without_adapter():
+    import torch
+    K, N, T = 264, 136, 8
+    tbl, entries = _table(K, N, (8,), seed=5)
+    good = entries[0][0]
+    free = [s for s in range(tbl.max_slots) if s != good][0]
+    token_slots = np.array([good, free, -1, 99, good, -7, good, -1], np.int32)
+    x, W = to_dev(wl.normal_bf16(5, 1, (T, K), 1.0)), to_dev(wl.normal_bf16(5, 2, (N, K), 0.05))
+    y = to_bits(tbl.lora_mixed_linear_tokens(x, W, torch.from_numpy(token_slots).cuda()))
+    torch.cuda.synchronize()
+    from paper_2608_15241_b200.binding import FLAG_BAD_SLOT
+    assert tbl.device_status() == FLAG_BAD_SLOT
+    cleaned = np.where(token_slots == good, good, -1).astype(np.int32)
+    y_ref = to_bits(tbl.lora_mixed_linear_tokens(x, W, torch.from_numpy(cleaned).cuda()))
+    torch.cuda.synchronize()
+    assert tbl.device_status() == 0
+    assert np.array_equal(y, y_ref)
+    tbl.close()
+
+
+def test_tokens_call_all_base_equals_no_segments():
+    import torch
+    K, N, T = 520, 264, 16
+    tbl, _ = _table(K, N, (8,), seed=9)
+    x, W = to_dev(wl.normal_bf16(9, 1, (T, K), 1.0)), to_dev(wl.normal_bf16(9, 2, (N, K), 0.05))
+    ts = torch.full((T,), -1, dtype=torch.int32, device="cuda")
+    y = to_bits(tbl.lora_mixed_linear_tokens(x, W, ts))
+    y0 = to_bits(tbl.lora_mixed_linear(x, W, None, None))
+    torch.cuda.synchronize()
+    assert np.array_equal(y, y0)
+    tbl.close()
