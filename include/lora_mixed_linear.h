@@ -153,9 +153,10 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * if perm (device int32[T], a permutation) is given, else row p.  G == 0 means "no adapter
  * anywhere".  T == 0 returns LML_OK without launching.
  * T <= 16 runs the bandwidth-bound decode kernel (W0 read once through a bulk-copy ring; with
- * segments it is a cooperative launch whose CTAs hand one another their share of the shrink
- * result and count themselves in the table's status block, so two decode calls on the SAME table
- * must not overlap on the GPU: put them on one stream or order them); larger T runs the
+ * segments its CTAs hand one another their share of the shrink result and count themselves in
+ * the table's status block, so two decode calls on the SAME table must not overlap on the GPU:
+ * put them on one stream or order them; a CTA whose peers are late computes their share itself,
+ * so the call completes even when the grid cannot be resident all at once); larger T runs the
  * TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
  * W0 is the frozen base weight: it must not be written by the operation that immediately precedes
  * the call on `stream` (the decode kernel starts fetching W0 while the kernel before it is still

@@ -25,9 +25,11 @@
 //                       and stage all of u in shared memory.  When the table's live adapters are few,
 //                       their rows of A are asked into L2 at kernel entry, ahead of the weight stream.
 //                       The consumers meet the shrink warps once, at their first epilogue.
-//                       The hand-over between CTAs needs them all resident, so a call with segments
-//                       is a cooperative launch.
+//                       No CTA depends on the others being resident: after a bounded wait for their
+//                       shares it computes all of u itself (same arithmetic, same bits).  So the
+//                       launch is an ordinary one and needs no co-residency guarantee.
 // d_in wider than a span is walked span by span.  All waits are bounded.
+#include <cstdlib>
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
 
@@ -60,7 +62,7 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     int rank_of_row[16];
     float scale_of_row[16];
     float dot_part[2][4];
-    int pad[1];
+    int u_complete;
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
 constexpr int kDecBBytes = 32768;                  // shared-memory copy of the B rows this CTA's epilogue needs
@@ -115,7 +117,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
     const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
-    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, uint32_t* status, int T, int K, int N, int G)
+    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, uint32_t* status, int T, int K, int N, int G, int patience)
 {
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
@@ -218,8 +220,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     // rows this CTA will need into L2.  Then the (token, j) dot products u = scale * x.A_j are dealt
     // out round-robin to the CTAs of the grid and, inside a CTA, to its three shrink warps: one warp per
     // dot product, sixteen 16-byte loads in flight per lane.  The results go to u in global memory; a
-    // counter in the table's status block tells every CTA when all of u is there (the launch is
-    // cooperative, so all CTAs are resident).  The consumers look at it only in their first epilogue.
+    // counter in the table's status block tells every CTA when all of u is there.  The consumers look at
+    // it only in their first epilogue.
     unsigned int* sync_words = status + 1;   // [0] elements of u that are written, [1] CTAs that have left
     const bool shrinker = warp > kDecConsumers;
     if (consumer && G > 0)   // let the lookup's loads go first through the load/store path (see below)
@@ -398,86 +400,111 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 else for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
             }
         }
-        // Dot product d belongs to CTA d mod grid.  A lane keeps twelve 16-byte loads in flight (six of x,
-        // six of A: what the register budget allows), so a warp alone needs several memory round trips per
-        // dot product.  A CTA with a single dot product (the usual case: a few tokens, rank 16) therefore
-        // puts all three shrink warps on it, one round trip in all; with more, each warp takes its own.
+        // Dot product d belongs to CTA d mod grid.  Its arithmetic is fixed, whoever computes it: 96 "virtual
+        // threads" each sum the 8-column groups m, m + 96, m + 192, ... of the row in order, each virtual
+        // warp of 32 adds its threads' sums up with the butterfly, and the result is (w0 + w1) + w2 times
+        // the scale.  A lane keeps twelve 16-byte loads in flight (six of x, six of A: what the register
+        // budget allows).  A CTA with a single dot product (the usual case: a few tokens, rank 16) puts its
+        // three shrink warps on it as the three virtual warps, one memory round trip in all; with more,
+        // each warp takes its own dot products and plays the three virtual warps one after the other.
         // Each result is published by its own release-add on the grid-wide counter: nobody waits for a fence.
         const int total = lk->dot_end[15];
-        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
         const int mine = total > (int)blockIdx.x ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-        auto partial_dot = [&](int d, int first, int nthreads, int& t, int& j, bool& real) {
+        auto locate = [&](int d, int& t, int& j) {
             t = 0;
             while (lk->dot_end[t] <= d) ++t;   // which row does d fall into
             j = d - (t > 0 ? lk->dot_end[t - 1] : 0);
-            real = j < lk->rank_of_row[t];     // else a padding column: B is zero there, u must at least be finite
+            return j < lk->rank_of_row[t];     // else a padding column: B is zero there, u must at least be finite
+        };
+        auto virtual_warp = [&](int t, int j, int v) {   // sum of virtual warp v, in every lane
+            const __nv_bfloat16* xr = x + (size_t)t * K;
+            const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
+            constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
             float dot = 0.f;
-            if (real) {
-                const __nv_bfloat16* xr = x + (size_t)t * K;
-                const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
-                constexpr int kPer = 6;
-                const int stride = nthreads * 8;
-                for (int kb = first * 8; kb < K; kb += kPer * stride) {
-                    uint4 xv[kPer], av[kPer];
+            for (int kb = (v * 32 + lane) * 8; kb < K; kb += kPer * kStride) {
+                uint4 xv[kPer], av[kPer];
 #pragma unroll
-                    for (int i = 0; i < kPer; ++i) {
-                        const int k0 = kb + i * stride;
-                        const bool v = k0 < K;
-                        xv[i] = v ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
-                        av[i] = v ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
-                    }
-#pragma unroll
-                    for (int i = 0; i < kPer; ++i) {
-                        float p = 0.f;
-                        p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
-                        p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
-                        p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
-                        p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
-                        dot += p;
-                    }
+                for (int i = 0; i < kPer; ++i) {
+                    const int k0 = kb + i * kStride;
+                    const bool ok_k = k0 < K;
+                    xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
+                    av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                for (int i = 0; i < kPer; ++i) {
+                    float p = 0.f;
+                    p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
+                    p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
+                    p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
+                    p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
+                    dot += p;
+                }
             }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
             return dot;
         };
+        auto whole_dot = [&](int d, int& t, int& j) {   // one warp, all three virtual warps
+            float val = 0.f;
+            if (locate(d, t, j)) {
+                const float w0 = virtual_warp(t, j, 0), w1 = virtual_warp(t, j, 1), w2 = virtual_warp(t, j, 2);
+                val = ((w0 + w1) + w2) * lk->scale_of_row[t];
+            }
+            return val;
+        };
+        const long long t_shrink = clock64();
         if (mine == 1) {
             int t, j;
-            bool real;
-            const float dot = partial_dot((int)blockIdx.x, me, kDecShrinkWarps * 32, t, j, real);
-            if (lane == 0) lk->dot_part[0][sw] = dot;
+            const bool real = locate((int)blockIdx.x, t, j);
+            if (real) {
+                const float w = virtual_warp(t, j, sw);
+                if (lane == 0) lk->dot_part[0][sw] = w;
+            }
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
-            if (me == 0) {
+            if (sw == 0 && lane == 0) {
                 u[t * kRankPad + j] = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_of_row[t] : 0.f;
                 red_release_gpu_add(sync_words, 1u);
             }
         } else {
             for (int d = (int)blockIdx.x + sw * (int)gridDim.x; d < total; d += kDecShrinkWarps * (int)gridDim.x) {
                 int t, j;
-                bool real;
-                const float dot = partial_dot(d, lane, 32, t, j, real);
+                const float val = whole_dot(d, t, j);
                 if (lane == 0) {
-                    u[t * kRankPad + j] = real ? dot * lk->scale_of_row[t] : 0.f;
+                    u[t * kRankPad + j] = val;
                     red_release_gpu_add(sync_words, 1u);
                 }
             }
         }
-        // Wait (bounded) until all of u is written, then stage it in shared memory for the consumers'
-        // epilogue, off their critical path.
+        // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
+        // other CTAs' shares normally arrive within microseconds and are then read from global memory.
+        // But this CTA never depends on them: nothing guarantees that the whole grid is resident at once
+        // (the launch is an ordinary one, so that it can start while its predecessor drains), so after a
+        // bounded wait it simply computes every dot product itself, with the same arithmetic and hence the
+        // same bits, finishes and makes room for whichever CTAs have not started yet.
         if (sw == 0 && lane == 0) {
-            const long long t0 = clock64();
+            int complete = 1;
             while (ld_acquire_gpu(sync_words) < (unsigned)total) {
-                if (clock64() - t0 > (1ll << 31)) { ctrl->abort = 1; break; }
+                if (clock64() - t_shrink > (long long)patience) { complete = 0; break; }
             }
+            lk->u_complete = complete;
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
-        for (int i = tid - (kDecConsumers + 1) * 32; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
-            reinterpret_cast<float4*>(u_s)[i] = __ldcg(reinterpret_cast<const float4*>(u) + i);
+        if (lk->u_complete) {
+            for (int i = tid - (kDecConsumers + 1) * 32; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
+                reinterpret_cast<float4*>(u_s)[i] = __ldcg(reinterpret_cast<const float4*>(u) + i);
+        } else {
+            for (int d = sw; d < total; d += kDecShrinkWarps) {
+                int t, j;
+                const float val = whole_dot(d, t, j);
+                if (lane == 0) u_s[t * kRankPad + j] = val;
+            }
+        }
         // tell the consumers that u_s, slot_of_row and bad_offsets are final
         asm volatile("bar.arrive 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
-        // Every CTA that gets here has seen the full count, so nobody reads the counters any more once
-        // all have: the last one puts both back to zero for the next call on this table.
-        if (sw == 0 && lane == 0 && ctrl->abort == 0) {
+        // Every CTA signs off once it has its copy of u and has published its own share; the last one puts
+        // both counters back to zero for the next call on this table.
+        if (sw == 0 && lane == 0) {
+            __threadfence();
             if (atomicAdd(sync_words + 1, 1u) == gridDim.x - 1) {
                 sync_words[0] = 0u;
                 sync_words[1] = 0u;
@@ -598,8 +625,17 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     if (tid == 0 && ctrl->abort) atomicOr(status, LML_FLAG_TIMEOUT);
 }
 
+namespace {
+// How long (SM clock cycles) a CTA waits for the other CTAs' share of u before it computes all of it
+// itself: far longer than the normal hand-over takes (a few microseconds), short enough that a grid
+// that cannot be resident all at once still finishes promptly.  LML_DECODE_PATIENCE overrides it (the
+// tests set 0 to run the self-sufficient path on purpose).
+int g_dec_patience = 100000;
+}  // namespace
+
 cudaError_t decode_init()
 {
+    if (const char* e = getenv("LML_DECODE_PATIENCE")) g_dec_patience = atoi(e) < 0 ? 0 : atoi(e);
     cudaError_t e = cudaFuncSetAttribute(decode_main_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(decode_main_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
@@ -615,17 +651,15 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     cfg.blockDim = dim3(kDecThreads);
     cfg.dynamicSmemBytes = kDecSmemBytes;
     cfg.stream = stream;
-    // With adapters the CTAs hand one another their share of u through global memory and wait for it
-    // in the epilogue, so they must all be resident: a cooperative launch guarantees that (the grid
-    // never exceeds one CTA per SM).  Without adapters the kernel is launched as a programmatic
-    // dependent of whatever precedes it (it waits at its top).
-    cudaLaunchAttribute attr[2];
+    // An ordinary launch, as a programmatic dependent of whatever precedes it on the stream (the kernel
+    // waits for that work itself, after it has started on W0).  The CTAs hand one another their share of
+    // u, but none of them depends on the others being resident (see the kernel), so no cooperative
+    // launch is needed, and the kernel can start while its predecessor drains.
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeCooperative;
-    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = a.G > 0 ? 2 : 1;
+    cfg.numAttrs = 1;
     const __nv_bfloat16* xb = (const __nv_bfloat16*)a.x;
     const __nv_bfloat16* wb = (const __nv_bfloat16*)a.W0;
     __nv_bfloat16* yb = (__nv_bfloat16*)a.y;
@@ -638,9 +672,9 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const int32_t* pm = a.perm;
     const int32_t* ts = a.token_slots;
     cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G)
+                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience)
                             : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G);
+                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
