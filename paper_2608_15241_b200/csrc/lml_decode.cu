@@ -17,17 +17,19 @@
 //                       product does not see, so operands are plain 16-byte loads.  Per-warp partial
 //                       sums go to per-warp slots and are added in a fixed order; the LoRA expand
 //                       sum_j u[t][j] B_s[n][j] is added in fp32 before the single bf16 rounding.
-//   shrink (3 warps)    only when the call has segments: look up each row's slot (segment arrays cached in
-//                       shared memory), then compute this CTA's share of u[row][j] = scale_s * sum_k
-//                       x[row][k] A_s[j][k] (fp32; dot products dealt out round-robin over the whole
-//                       grid; all three warps on one when the CTA has only one), publish each result in
-//                       global memory with a release-add on a grid-wide counter, wait for the counter
-//                       and stage all of u in shared memory.  When the table's live adapters are few,
-//                       their rows of A are asked into L2 at kernel entry, ahead of the weight stream.
-//                       The consumers meet the shrink warps once, at their first epilogue.
-//                       No CTA depends on the others being resident: after a bounded wait for their
-//                       shares it computes all of u itself (same arithmetic, same bits).  So the
-//                       launch is an ordinary one and needs no co-residency guarantee.
+//   shrink (3 warps)    only when the call has adapters: look up each row's slot (from segments, cached in
+//                       shared memory, or from one slot id per row), then compute this CTA's share of
+//                       u[row][j] = scale_s * sum_k x[row][k] A_s[j][k] (fp32).  The dot products are dealt
+//                       out over the whole grid in groups of 1, 2 or 4 columns of one row; a group's
+//                       operands are staged in shared memory by asynchronous copies (one memory round
+//                       trip per group; single dot products stay in registers).  Each result is
+//                       published in global memory with a release-add on a grid-wide counter; the warps
+//                       wait for the counter and stage all of u in shared memory.  When the table's live
+//                       adapters are few, their rows of A are asked into L2 at kernel entry, ahead of
+//                       the weight stream.  The consumers meet the shrink warps once, at their first
+//                       epilogue.  No CTA depends on the others being resident: after a bounded wait
+//                       for their shares it computes all of u itself (same arithmetic, same bits).  So
+//                       the launch is an ordinary one and needs no co-residency guarantee.
 // d_in wider than a span is walked span by span.  All waits are bounded.
 #include <cstdlib>
 #include "lml_internal.cuh"
@@ -48,11 +50,14 @@ constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 4 k-steps
 constexpr int kDecRowPitch = kDecChunk * 2 + 64; // bytes; a multiple of 16 that is 4 mod 8 in 16-byte chunks: rows land on different banks
 constexpr int kDecStageBytes = kDecUnitRows * kDecRowPitch;
 constexpr int kDecStages = 4;
-constexpr int kDecRoundUnits = 6;                // units (= 48 rows) reduced together
+constexpr int kDecRoundUnits = 4;                // units (= 32 rows) reduced together
 constexpr int kDecSlotFloats = 16 * kDecUnitRows;   // [token][row] partial sums of one warp for one unit
 constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 4;
 constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
 constexpr int kDecSegCache = 128;                 // segments whose offsets and slots are looked up in shared memory
+constexpr int kDecDotGroup = 4;                    // dot products of one row of x that a CTA takes together
+constexpr int kDecDotCols = 4096;                  // columns of a pass over the rows that a dot-product group needs
+constexpr int kDecDotBytes = (1 + kDecDotGroup) * kDecDotCols * 2;   // staging: one row of x, four rows of A
 struct DecLookup {   // what the shrink warps work out about the call, in shared memory
     int seg[kDecSegCache + 1];
     int ids[kDecSegCache];
@@ -61,13 +66,14 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     int dot_end[16];        // running total of dot products up to and including each row of x
     int rank_of_row[16];
     float scale_of_row[16];
-    float dot_part[2][4];
+    float dot_part[kDecDotGroup][4];
     int u_complete;
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
-constexpr int kDecBBytes = 32768;                  // shared-memory copy of the B rows this CTA's epilogue needs
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecBBytes;
-static_assert(kDecSmemBytes <= 232448, "shared memory budget");
+constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecDotBytes;
+// 196 KB is also the largest shared-memory carve-out that leaves the SM a useful L1 for the loads of x:
+// one step more and the base-only call is 0.8 us slower.
+static_assert(kDecSmemBytes + 1024 <= 200704, "shared memory budget");   // the system keeps 1 KB per CTA for itself
 
 struct DecCtrl {
     uint64_t full[kDecStages];
@@ -106,6 +112,14 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)   // global -> shared, past L1, no registers
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
@@ -127,7 +141,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     float* u_s = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);   // [16][64]
     DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
     DecLookup* lk = reinterpret_cast<DecLookup*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
-    uint8_t* b_s = base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8;   // 16-byte aligned
+    uint8_t* dot_s = base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8;   // 16-byte aligned
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
@@ -374,17 +388,38 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
-        if (sw == kDecShrinkWarps - 1) {
-            // The expand's B rows for this CTA's output columns: one contiguous block per distinct slot,
-            // copied into shared memory now so that the epilogue has no memory round trip left.  Slots
-            // that do not fit (many adapters in one call, or many rows per CTA) are prefetched into L2
-            // and read from there.
+        // The dot products are dealt out in groups of one, two or four columns j of one row of x (a group
+        // shares the row of x): group g belongs to CTA g mod grid.  A dot product's arithmetic is fixed, whoever
+        // computes it: 96 "virtual threads" (the three shrink warps) each sum the 8-column chunks m, m + 96,
+        // m + 192, ... of the row in order, each warp adds its threads' sums up with the butterfly, and the
+        // result is (w0 + w1) + w2 times the scale.  The operands of a whole group are brought into shared
+        // memory with asynchronous 16-byte copies, all in flight at once (registers would hold a fraction of
+        // them), so a group costs one memory round trip.  A group's results are published with one
+        // release-add on the grid-wide counter: nobody waits for a fence.
+        const int total = lk->dot_end[15];
+        // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
+        // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
+        const int gsize = total <= (int)gridDim.x ? 1 : (total <= 2 * (int)gridDim.x ? 2 : kDecDotGroup);
+        const int ngroups = total / gsize;
+        if (sw == kDecShrinkWarps - 1 && gsize > 1) {   // the staging buffer is needed for the dot products: B goes to L2 only
+            if (lane < T) {
+                const int slot = ctrl->slot_of_row[lane];
+                if (slot >= 0) {
+                    const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
+                    for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+                }
+            }
+        } else if (sw == kDecShrinkWarps - 1) {
+            // The expand's B rows for this CTA's output columns.  When the staging buffer below is not
+            // needed (single dot products), they are copied into it now, one contiguous block per distinct
+            // slot, so that the epilogue has no memory round trip left; otherwise, and for slots that do
+            // not fit, they are asked into L2 and read from there.
             const int slot = lane < T ? ctrl->slot_of_row[lane] : -1;
             const unsigned same = __match_any_sync(0xffffffffu, slot);
             const bool leader = slot >= 0 && (same & ((1u << lane) - 1u)) == 0u;
             const unsigned leaders = __ballot_sync(0xffffffffu, leader);
             const int block_bytes = (row_end - row_begin) * kRankPad * 2;
-            const int fit = block_bytes > 0 ? kDecBBytes / block_bytes : 0;
+            const int fit = (gsize == 1 && block_bytes > 0) ? kDecDotBytes / block_bytes : 0;
             const int my_block = __popc(leaders & ((1u << (__ffs(same) - 1)) - 1u));   // rank of this lane's slot among the distinct ones
             const bool staged = slot >= 0 && my_block < fit;
             const int nblocks = min(__popc(leaders), fit);
@@ -396,83 +431,120 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             __syncwarp();
             if (leader) {
                 const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                if (staged) bulk_copy_g2s(smem_u32(b_s) + my_block * block_bytes, b, (uint32_t)block_bytes, smem_u32(&ctrl->bfull));
+                if (staged) bulk_copy_g2s(smem_u32(dot_s) + my_block * block_bytes, b, (uint32_t)block_bytes, smem_u32(&ctrl->bfull));
                 else for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
             }
         }
-        // Dot product d belongs to CTA d mod grid.  Its arithmetic is fixed, whoever computes it: 96 "virtual
-        // threads" each sum the 8-column groups m, m + 96, m + 192, ... of the row in order, each virtual
-        // warp of 32 adds its threads' sums up with the butterfly, and the result is (w0 + w1) + w2 times
-        // the scale.  A lane keeps twelve 16-byte loads in flight (six of x, six of A: what the register
-        // budget allows).  A CTA with a single dot product (the usual case: a few tokens, rank 16) puts its
-        // three shrink warps on it as the three virtual warps, one memory round trip in all; with more,
-        // each warp takes its own dot products and plays the three virtual warps one after the other.
-        // Each result is published by its own release-add on the grid-wide counter: nobody waits for a fence.
-        const int total = lk->dot_end[15];
-        const int mine = total > (int)blockIdx.x ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-        auto locate = [&](int d, int& t, int& j) {
+        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+        auto group = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
+            const int d0 = g * gsize;
             t = 0;
-            while (lk->dot_end[t] <= d) ++t;   // which row does d fall into
-            j = d - (t > 0 ? lk->dot_end[t - 1] : 0);
-            return j < lk->rank_of_row[t];     // else a padding column: B is zero there, u must at least be finite
-        };
-        auto virtual_warp = [&](int t, int j, int v) {   // sum of virtual warp v, in every lane
+            while (lk->dot_end[t] <= d0) ++t;   // which row do the group's dot products fall into
+            j0 = d0 - (t > 0 ? lk->dot_end[t - 1] : 0);
+            const int nreal = max(0, min(gsize, lk->rank_of_row[t] - j0));   // the rest are padding columns: zero
+            float acc[kDecDotGroup];
+#pragma unroll
+            for (int i = 0; i < kDecDotGroup; ++i) acc[i] = 0.f;
             const __nv_bfloat16* xr = x + (size_t)t * K;
-            const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
-            constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
-            float dot = 0.f;
-            for (int kb = (v * 32 + lane) * 8; kb < K; kb += kPer * kStride) {
-                uint4 xv[kPer], av[kPer];
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    const int k0 = kb + i * kStride;
-                    const bool ok_k = k0 < K;
-                    xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
-                    av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
+            const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j0) * K;
+            for (int k_pass = 0; k_pass < K && nreal > 0; k_pass += kDecDotCols) {
+                const int chunks = min(kDecDotCols, K - k_pass) / 8;
+                for (int c = me; c < chunks; c += kDecShrinkWarps * 32) {
+                    cp_async_16(smem_u32(dot_s) + c * 16, xr + k_pass + c * 8);
+                    for (int i = 0; i < nreal; ++i)
+                        cp_async_16(smem_u32(dot_s) + (1 + i) * kDecDotCols * 2 + c * 16, ar + (size_t)i * K + k_pass + c * 8);
                 }
+                cp_async_wait_all();
+                asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // everybody's copies have landed
+                for (int c = me; c < chunks; c += kDecShrinkWarps * 32) {
+                    const uint4 xv = *reinterpret_cast<const uint4*>(dot_s + c * 16);
 #pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    float p = 0.f;
-                    p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
-                    p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
-                    p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
-                    p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
-                    dot += p;
+                    for (int i = 0; i < kDecDotGroup; ++i) {
+                        if (i < nreal) {
+                            const uint4 av = *reinterpret_cast<const uint4*>(dot_s + (1 + i) * kDecDotCols * 2 + c * 16);
+                            float p = 0.f;
+                            p = fmaf(bf16_lo(xv.x), bf16_lo(av.x), p); p = fmaf(bf16_hi(xv.x), bf16_hi(av.x), p);
+                            p = fmaf(bf16_lo(xv.y), bf16_lo(av.y), p); p = fmaf(bf16_hi(xv.y), bf16_hi(av.y), p);
+                            p = fmaf(bf16_lo(xv.z), bf16_lo(av.z), p); p = fmaf(bf16_hi(xv.z), bf16_hi(av.z), p);
+                            p = fmaf(bf16_lo(xv.w), bf16_lo(av.w), p); p = fmaf(bf16_hi(xv.w), bf16_hi(av.w), p);
+                            acc[i] += p;
+                        }
+                    }
                 }
+                asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the staging buffer is free again
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            return dot;
+            for (int i = 0; i < kDecDotGroup; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
+                if (lane == 0) lk->dot_part[i][sw] = acc[i];
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+#pragma unroll
+            for (int i = 0; i < kDecDotGroup; ++i)
+                val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_of_row[t] : 0.f;
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
         };
-        auto whole_dot = [&](int d, int& t, int& j) {   // one warp, all three virtual warps
-            float val = 0.f;
-            if (locate(d, t, j)) {
-                const float w0 = virtual_warp(t, j, 0), w1 = virtual_warp(t, j, 1), w2 = virtual_warp(t, j, 2);
-                val = ((w0 + w1) + w2) * lk->scale_of_row[t];
+        // A single dot product per CTA (few tokens, rank 16: the usual decode call) skips the staging: each
+        // virtual thread keeps its six chunks of x and of A in registers, same order, same sums.
+        auto single = [&](int d, int& t, int& j) {
+            t = 0;
+            while (lk->dot_end[t] <= d) ++t;
+            j = d - (t > 0 ? lk->dot_end[t - 1] : 0);
+            const bool real = j < lk->rank_of_row[t];
+            if (real) {
+                const __nv_bfloat16* xr = x + (size_t)t * K;
+                const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
+                constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
+                float dot = 0.f;
+                for (int kb = me * 8; kb < K; kb += kPer * kStride) {
+                    uint4 xv[kPer], av[kPer];
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        const int k0 = kb + i * kStride;
+                        const bool ok_k = k0 < K;
+                        xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
+                        av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        if (kb + i * kStride < K) {
+                            float p = 0.f;
+                            p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
+                            p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
+                            p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
+                            p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
+                            dot += p;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                if (lane == 0) lk->dot_part[0][sw] = dot;
             }
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+            const float val = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_of_row[t] : 0.f;
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
             return val;
         };
         const long long t_shrink = clock64();
-        if (mine == 1) {
-            int t, j;
-            const bool real = locate((int)blockIdx.x, t, j);
-            if (real) {
-                const float w = virtual_warp(t, j, sw);
-                if (lane == 0) lk->dot_part[0][sw] = w;
-            }
-            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
-            if (sw == 0 && lane == 0) {
-                u[t * kRankPad + j] = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_of_row[t] : 0.f;
-                red_release_gpu_add(sync_words, 1u);
-            }
-        } else {
-            for (int d = (int)blockIdx.x + sw * (int)gridDim.x; d < total; d += kDecShrinkWarps * (int)gridDim.x) {
+        if (gsize == 1) {
+            if ((int)blockIdx.x < total) {
                 int t, j;
-                const float val = whole_dot(d, t, j);
-                if (lane == 0) {
+                const float val = single((int)blockIdx.x, t, j);
+                if (me == 0) {
                     u[t * kRankPad + j] = val;
                     red_release_gpu_add(sync_words, 1u);
                 }
+            }
+        } else
+        for (int g = (int)blockIdx.x; g < ngroups; g += (int)gridDim.x) {
+            float val[kDecDotGroup];
+            int t, j0;
+            group(g, val, t, j0);
+            if (me == 0) {
+                for (int i = 0; i < gsize; ++i) u[t * kRankPad + j0 + i] = val[i];
+                red_release_gpu_add(sync_words, (unsigned)gsize);
             }
         }
         // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
@@ -490,13 +562,20 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
         if (lk->u_complete) {
-            for (int i = tid - (kDecConsumers + 1) * 32; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
+            for (int i = me; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
                 reinterpret_cast<float4*>(u_s)[i] = __ldcg(reinterpret_cast<const float4*>(u) + i);
-        } else {
-            for (int d = sw; d < total; d += kDecShrinkWarps) {
+        } else if (gsize == 1) {   // (the staging buffer may hold B rows: stay in registers)
+            for (int d = 0; d < total; ++d) {
                 int t, j;
-                const float val = whole_dot(d, t, j);
-                if (lane == 0) u_s[t * kRankPad + j] = val;
+                const float val = single(d, t, j);
+                if (me == 0) u_s[t * kRankPad + j] = val;
+            }
+        } else {
+            for (int g = 0; g < ngroups; ++g) {
+                float val[kDecDotGroup];
+                int t, j0;
+                group(g, val, t, j0);
+                if (me == 0) for (int i = 0; i < gsize; ++i) u_s[t * kRankPad + j0 + i] = val[i];
             }
         }
         // tell the consumers that u_s, slot_of_row and bad_offsets are final
@@ -603,16 +682,20 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                     const int r8 = (lk->rank_of_row[t] + 7) >> 3;
                     const uint4* bp = reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
                     const int bb = ctrl->b_of_row[t];
-                    const uint4* bs = reinterpret_cast<const uint4*>(b_s + ((size_t)bb * (row_end - row_begin) + (n - row_begin)) * kRankPad * 2);
+                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + ((size_t)bb * (row_end - row_begin) + (n - row_begin)) * kRankPad * 2);
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
-                    for (int c = 0; c < r8; ++c) {
-                        uint4 b = bb >= 0 ? bs[c] : ldg_nc_v4(bp + c);
-                        float4 u0 = up[2 * c], u1 = up[2 * c + 1];
+                    auto fma8 = [&](const uint4& b, int c) {
+                        const float4 u0 = up[2 * c], u1 = up[2 * c + 1];
                         d = fmaf(u0.x, bf16_lo(b.x), d); d = fmaf(u0.y, bf16_hi(b.x), d);
                         d = fmaf(u0.z, bf16_lo(b.y), d); d = fmaf(u0.w, bf16_hi(b.y), d);
                         d = fmaf(u1.x, bf16_lo(b.z), d); d = fmaf(u1.y, bf16_hi(b.z), d);
                         d = fmaf(u1.z, bf16_lo(b.w), d); d = fmaf(u1.w, bf16_hi(b.w), d);
+                    };
+                    if (bb >= 0) {   // (two loops: with a select inside one loop the global loads no longer overlap)
+                        for (int c = 0; c < r8; ++c) fma8(bs[c], c);
+                    } else {
+                        for (int c = 0; c < r8; ++c) fma8(ldg_nc_v4(bp + c), c);
                     }
                     v += d;
                 }
