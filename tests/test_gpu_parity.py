@@ -363,3 +363,20 @@ def test_host_buffer_entry_point():
             assert np.array_equal(to_bits(yh), ref_y)
         finally:
             site.close()
+
+
+@pytest.mark.parametrize("T,G", [(16, 200), (7, 129), (16, 128)])
+def test_decode_with_many_mostly_empty_segments(T, G):
+    """More segments than the decode kernel caches in shared memory (128): the lookup then searches
+    the arrays in global memory.  Most segments are empty and may repeat slots."""
+    w = wl.ragged(T=T, d_in=520, d_out=264, ranks=(4, 16, 1, 33, 64))
+    rng = np.random.default_rng(G * 31 + T)
+    cuts = np.sort(rng.integers(0, T + 1, size=G - 1))
+    so = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    se = rng.integers(-1, len(w.entries), size=G).astype(np.int32)
+    site = Site(w)
+    y, flags = site.run(seg_offsets=so, seg_entry=se, perm=None)
+    ref, _ = oracle.forward(w.x, w.W0, w.entries, so, se)
+    r = oracle.compare(y, ref)
+    assert flags == 0 and r["ok"], r
+    site.close()
