@@ -65,7 +65,6 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     uint8_t rank_s[kMaxSlots];
     int dot_end[16];        // running total of dot products up to and including each row of x
     int rank_of_row[16];
-    float scale_of_row[16];
     float dot_part[kDecDotGroup][4];
     int u_complete;
 };
@@ -281,6 +280,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 (void)rows_before;
             }
         }
+        if (sw == kDecShrinkWarps - 1)
+            for (int sl = lane; sl < kMaxSlots; sl += 32) lk->scale_s[sl] = snap.scale[sl];
         if (sw == 0) {
             // One memory round trip for everything the lookup needs: the segment arrays go to shared
             // memory (all loads issued before the first is used), the search then runs there.  Calls
@@ -304,10 +305,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             int my_token_slot = -1;
             if (by_token && lane < T) my_token_slot = __ldg(token_slots + lane);
             asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
-            for (int sl = lane; sl < kMaxSlots; sl += 32) {
+            for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
-                lk->scale_s[sl] = snap.scale[sl];
-            }
             if (cached) {
 #pragma unroll
                 for (int i = 0; i <= kDecSegCache / 32; ++i) {
@@ -383,7 +382,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 if (lane < 16) {
                     lk->dot_end[lane] = end;
                     lk->rank_of_row[lane] = rank;
-                    lk->scale_of_row[lane] = slot >= 0 ? lk->scale_s[slot] : 0.f;
                 }
             }
         }
@@ -482,7 +480,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
 #pragma unroll
             for (int i = 0; i < kDecDotGroup; ++i)
-                val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_of_row[t] : 0.f;
+                val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_s[ctrl->slot_of_row[t]] : 0.f;
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
         };
         // A single dot product per CTA (few tokens, rank 16: the usual decode call) skips the staging: each
@@ -523,7 +521,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 if (lane == 0) lk->dot_part[0][sw] = dot;
             }
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
-            const float val = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_of_row[t] : 0.f;
+            const float val = real ? ((lk->dot_part[0][0] + lk->dot_part[0][1]) + lk->dot_part[0][2]) * lk->scale_s[ctrl->slot_of_row[t]] : 0.f;
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
             return val;
         };
@@ -619,20 +617,34 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                                 // all of the stage's operand reads first, then the stage can go back to the producer
                                 // before the MMAs run
                                 uint4 w[kDecStepsPerChunk];
+                                if (rows == kDecUnitRows && span - kc * kDecChunk >= kDecChunk) {
+                                    // a full stage (all but the ragged edges): no predicates
 #pragma unroll
-                                for (int i = 0; i < kDecStepsPerChunk; ++i) {
-                                    const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
-                                    w[i] = (rv && c0 + tq * 8 < span) ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
-                                                                      : make_uint4(0, 0, 0, 0);
-                                }
+                                    for (int i = 0; i < kDecStepsPerChunk; ++i)
+                                        w[i] = lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64));
 #pragma unroll
-                                for (int i = 0; i < kDecStepsPerChunk; ++i) {
-                                    const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
-                                    if (c0 < span) {   // uniform across the warp: all lanes issue the MMAs or none
+                                    for (int i = 0; i < kDecStepsPerChunk; ++i) {
                                         const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
                                         const uint4 a1 = kTwo ? xc[kc * kDecStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
                                         mma_bf16_16816(acc4[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, w[i].x, w[i].y);
                                         mma_bf16_16816(acc4[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, w[i].z, w[i].w);
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int i = 0; i < kDecStepsPerChunk; ++i) {
+                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
+                                        w[i] = (rv && c0 + tq * 8 < span) ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
+                                                                          : make_uint4(0, 0, 0, 0);
+                                    }
+#pragma unroll
+                                    for (int i = 0; i < kDecStepsPerChunk; ++i) {
+                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
+                                        if (c0 < span) {   // uniform across the warp: all lanes issue the MMAs or none
+                                            const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
+                                            const uint4 a1 = kTwo ? xc[kc * kDecStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
+                                            mma_bf16_16816(acc4[(2 * i) & 3], a0.x, a1.x, a0.y, a1.y, w[i].x, w[i].y);
+                                            mma_bf16_16816(acc4[(2 * i + 1) & 3], a0.z, a1.z, a0.w, a1.w, w[i].z, w[i].w);
+                                        }
                                     }
                                 }
                                 __syncwarp();

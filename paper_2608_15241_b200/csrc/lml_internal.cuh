@@ -19,9 +19,9 @@ constexpr int kDecodeMaxT = LML_DECODE_MAX_TOKENS;
 // Per-call snapshot of the slot table, passed by value as a kernel parameter so that a later
 // register / retire cannot change a call that is already enqueued.
 struct SlotSnapshot {
-    float scale[kMaxSlots];
-    uint8_t rank[kMaxSlots];   // 0 = slot not live
-    int32_t max_slots;
+    uint8_t rank[kMaxSlots];   // 0 = slot not live.  First, with max_slots right behind: what a kernel needs
+    int32_t max_slots;         // first sits in one or two lines of the parameter cache (a miss there costs
+    float scale[kMaxSlots];    // as much as a trip to L2)
 };
 
 // Device-resident pieces of a table.
