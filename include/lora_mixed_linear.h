@@ -73,6 +73,7 @@ typedef enum {
 
 #define LML_MAX_SLOTS 64  /* upper bound for max_slots */
 #define LML_MAX_RANK 64   /* upper bound for an adapter's rank */
+#define LML_MAX_ADAPTER_IDS 4096 /* adapter ids 0 .. this-1 can be published and resolved on the device */
 #define LML_DECODE_MAX_TOKENS 16 /* T <= this takes the bandwidth-bound decode kernel */
 
 const char* lml_status_string(lml_status s);
@@ -130,6 +131,37 @@ lml_status lml_slot_info(const lml_table* t, int slot, int* adapter_id, int* ver
 size_t lml_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
 
 /*
+ * Publication (Section 4.2: requests bind to the last committed adapter; Section 5.3: a staged
+ * version runs privately while the old one serves, and becomes visible at one controlled point).
+ *
+ * An entry made by register_adapter is RESIDENT: usable by whoever names its slot (that is how a
+ * staged version is exercised before it is published), invisible to calls that name adapters.
+ * lml_publish makes (adapter_id, version), which must be resident, the SERVING version of the
+ * adapter: from that point of `stream` on, calls that name the adapter (the *_adapters forms
+ * below) resolve to its slot; calls enqueued on `stream` earlier still resolve to the version
+ * that served before.  The switch is a single 4-byte store on the device, so no call sees a
+ * mixture.  The version that served before becomes RETIRING: it stays resident while work is
+ * pinned to it and is retired (slot free again) by the unpin that brings its count to zero, or at
+ * once if nothing is pinned.  previous_version_out (may be NULL) receives that version, or -1.
+ * 0 <= adapter_id < LML_MAX_ADAPTER_IDS.  Errors: INVALID_ARG, NOT_FOUND, CUDA.
+ *
+ * lml_pin / lml_unpin count work in flight that is bound to a slot (a request that started under
+ * a version keeps it until it ends).  retire_version on a pinned entry likewise only marks it
+ * RETIRING.  Errors: INVALID_ARG, BAD_SLOT (slot free), and for unpin INVALID_ARG if not pinned.
+ *
+ * lml_resolve: serving slot and version of an adapter on the host (NOT_FOUND if none).
+ * lml_slot_state: state (LML_STATE_*) and pin count of a live slot; out pointers may be NULL.
+ */
+#define LML_STATE_RESIDENT 0
+#define LML_STATE_SERVING 1
+#define LML_STATE_RETIRING 2
+lml_status lml_publish(lml_table* t, int adapter_id, int version, void* stream, int* previous_version_out);
+lml_status lml_pin(lml_table* t, int slot);
+lml_status lml_unpin(lml_table* t, int slot);
+lml_status lml_resolve(const lml_table* t, int adapter_id, int* slot_out, int* version_out);
+lml_status lml_slot_state(const lml_table* t, int slot, int* state_out, int* pins_out);
+
+/*
  * lml_segment_tokens — the token-segmentation pass: group T tokens by slot.
  * token_slots: device int32[T], physical slot per token or -1 (no adapter).
  * Outputs (device): perm int32[T] (position -> token row); seg_offsets int32[max_slots + 2];
@@ -183,6 +215,18 @@ size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens);
 lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T,
                                     const int32_t* token_slots, void* y, void* workspace,
                                     size_t workspace_bytes, void* stream);
+
+/*
+ * The same two calls for callers that hold ADAPTER ids per token instead of slots: every id is
+ * resolved on the device to the adapter's serving slot at the moment the call runs in stream
+ * order (see lml_publish).  -1 means no adapter; an id without a serving version counts as -1 and
+ * sets LML_FLAG_BAD_SLOT.  Otherwise identical to lml_segment_tokens / lora_mixed_linear_tokens.
+ */
+lml_status lml_segment_tokens_adapters(lml_table* t, const int32_t* token_adapter_ids, int T, int32_t* perm,
+                                       int32_t* seg_offsets, int32_t* seg_slot_ids, void* stream);
+lml_status lora_mixed_linear_adapters(lml_table* t, const void* x, const void* W0, int T,
+                                      const int32_t* token_adapter_ids, void* y, void* workspace,
+                                      size_t workspace_bytes, void* stream);
 
 /*
  * Host-buffer form of the same call, for callers whose activations live in host memory.

@@ -22,13 +22,16 @@ STATUS_NAMES = {0: "LML_OK", 1: "LML_ERR_INVALID_ARG", 2: "LML_ERR_BAD_SLOT", 3:
                 4: "LML_ERR_DUPLICATE", 5: "LML_ERR_NOT_FOUND", 6: "LML_ERR_UNSUPPORTED",
                 7: "LML_ERR_CUDA", 8: "LML_ERR_TIMEOUT", 9: "LML_ERR_WORKSPACE", 10: "LML_ERR_TOO_LARGE"}
 FLAG_BAD_SLOT, FLAG_BAD_OFFSETS, FLAG_BAD_PERM, FLAG_TIMEOUT = 1, 2, 4, 8
-MAX_SLOTS, MAX_RANK, DECODE_MAX_TOKENS = 64, 64, 16
+MAX_SLOTS, MAX_RANK, DECODE_MAX_TOKENS, MAX_ADAPTER_IDS = 64, 64, 16, 4096
+ERR_INVALID_ARG, ERR_BAD_SLOT, ERR_NOT_FOUND = 1, 2, 5
 
 EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "register_adapter",
            "retire_version", "lml_lookup", "lml_slot_info", "lml_workspace_bytes",
            "lml_segment_tokens", "lora_mixed_linear", "lml_host_workspace_bytes",
            "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count",
-           "lora_mixed_linear_decode_static", "lml_tokens_workspace_bytes", "lora_mixed_linear_tokens")
+           "lora_mixed_linear_decode_static", "lml_tokens_workspace_bytes", "lora_mixed_linear_tokens",
+           "lml_publish", "lml_pin", "lml_unpin", "lml_resolve", "lml_slot_state",
+           "lml_segment_tokens_adapters", "lora_mixed_linear_adapters")
 
 
 class LmlError(RuntimeError):
@@ -69,6 +72,13 @@ def lib() -> ctypes.CDLL:
         L.lml_tokens_workspace_bytes.restype = sz
         L.lml_tokens_workspace_bytes.argtypes = [vp, i32]
         L.lora_mixed_linear_tokens.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.lora_mixed_linear_adapters.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.lml_segment_tokens_adapters.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.lml_publish.argtypes = [vp, i32, i32, vp, ctypes.POINTER(i32)]
+        L.lml_pin.argtypes = [vp, i32]
+        L.lml_unpin.argtypes = [vp, i32]
+        L.lml_resolve.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.lml_slot_state.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.lml_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
@@ -163,6 +173,52 @@ def lora_mixed_linear_tokens(table: int, x_ptr: int, W0_ptr: int, T: int, token_
     """Segmentation and layer in one call: one slot id per token instead of segments."""
     _check(lib().lora_mixed_linear_tokens(table, x_ptr, W0_ptr, T, token_slots_ptr, y_ptr, workspace_ptr,
                                           workspace_bytes, stream), "lora_mixed_linear_tokens")
+
+
+STATE_RESIDENT, STATE_SERVING, STATE_RETIRING = 0, 1, 2
+
+
+def lml_publish(table: int, adapter_id: int, version: int, stream: int = 0) -> int:
+    """Make (adapter_id, version) the adapter's serving version from this point of the stream on.
+    Returns the version that served before, or -1."""
+    prev = ctypes.c_int32(-1)
+    _check(lib().lml_publish(table, adapter_id, version, stream, ctypes.byref(prev)), "lml_publish")
+    return int(prev.value)
+
+
+def lml_pin(table: int, slot: int) -> None:
+    _check(lib().lml_pin(table, slot), "lml_pin")
+
+
+def lml_unpin(table: int, slot: int) -> None:
+    _check(lib().lml_unpin(table, slot), "lml_unpin")
+
+
+def lml_resolve(table: int, adapter_id: int):
+    """(slot, version) of the adapter's serving entry; raises LmlError(NOT_FOUND) if none."""
+    slot, ver = ctypes.c_int32(-1), ctypes.c_int32(-1)
+    _check(lib().lml_resolve(table, adapter_id, ctypes.byref(slot), ctypes.byref(ver)), "lml_resolve")
+    return int(slot.value), int(ver.value)
+
+
+def lml_slot_state(table: int, slot: int):
+    """(state, pins) of a live slot."""
+    st, pins = ctypes.c_int32(-1), ctypes.c_int32(-1)
+    _check(lib().lml_slot_state(table, slot, ctypes.byref(st), ctypes.byref(pins)), "lml_slot_state")
+    return int(st.value), int(pins.value)
+
+
+def lml_segment_tokens_adapters(table: int, token_adapter_ids_ptr: int, T: int, perm_ptr: int, seg_offsets_ptr: int,
+                                seg_slot_ids_ptr: int, stream: int = 0) -> None:
+    _check(lib().lml_segment_tokens_adapters(table, token_adapter_ids_ptr, T, perm_ptr, seg_offsets_ptr,
+                                             seg_slot_ids_ptr, stream), "lml_segment_tokens_adapters")
+
+
+def lora_mixed_linear_adapters(table: int, x_ptr: int, W0_ptr: int, T: int, token_adapter_ids_ptr: int, y_ptr: int,
+                               workspace_ptr: int, workspace_bytes: int, stream: int = 0) -> None:
+    """lora_mixed_linear_tokens with adapter ids, resolved on the device to each adapter's serving slot."""
+    _check(lib().lora_mixed_linear_adapters(table, x_ptr, W0_ptr, T, token_adapter_ids_ptr, y_ptr, workspace_ptr,
+                                            workspace_bytes, stream), "lora_mixed_linear_adapters")
 
 
 def lora_mixed_linear_decode_static(table: int, x_ptr: int, W0_ptr: int, T: int, seg_offsets_ptr: int,
@@ -301,7 +357,26 @@ class Table:
                           int(workspace.numel()), _stream(stream))
         return y
 
-    def lora_mixed_linear_tokens(self, x, W0, token_slots, y=None, workspace=None, stream=None):
+    def publish(self, adapter_id: int, version: int, stream=None) -> int:
+        return lml_publish(self.handle, adapter_id, version, _stream(stream))
+
+    def pin(self, slot: int) -> None:
+        lml_pin(self.handle, slot)
+
+    def unpin(self, slot: int) -> None:
+        lml_unpin(self.handle, slot)
+
+    def resolve(self, adapter_id: int):
+        return lml_resolve(self.handle, adapter_id)
+
+    def slot_state(self, slot: int):
+        return lml_slot_state(self.handle, slot)
+
+    def lora_mixed_linear_adapters(self, x, W0, token_adapter_ids, y=None, workspace=None, stream=None):
+        """As lora_mixed_linear_tokens, with one ADAPTER id per token (resolved on the device)."""
+        return self.lora_mixed_linear_tokens(x, W0, token_adapter_ids, y, workspace, stream, by_adapter=True)
+
+    def lora_mixed_linear_tokens(self, x, W0, token_slots, y=None, workspace=None, stream=None, by_adapter=False):
         """x bf16 [T][d_in], W0 bf16 [d_out][d_in], token_slots int32[T] (all cuda) -> y bf16 [T][d_out]."""
         import torch
         assert x.dtype == torch.bfloat16 and W0.dtype == torch.bfloat16 and token_slots.dtype == torch.int32
@@ -313,8 +388,9 @@ class Table:
         if workspace is None:
             workspace = torch.empty(max(lml_tokens_workspace_bytes(self.handle, T), 256), dtype=torch.uint8,
                                     device=x.device)
-        lora_mixed_linear_tokens(self.handle, _ptr(x), _ptr(W0), T, _ptr(token_slots), _ptr(y), _ptr(workspace),
-                                 int(workspace.numel()), _stream(stream))
+        fn = lora_mixed_linear_adapters if by_adapter else lora_mixed_linear_tokens
+        fn(self.handle, _ptr(x), _ptr(W0), T, _ptr(token_slots), _ptr(y), _ptr(workspace), int(workspace.numel()),
+           _stream(stream))
         return y
 
     def lora_mixed_linear_host(self, x_host, W0, seg_offsets_host, slot_ids_host, y_host, perm_host=None,

@@ -77,9 +77,11 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     bool ok = cudaMalloc(&t->arena.A, a_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&t->arena.B, b_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&t->arena.status, 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&t->arena.adapter_map, kMaxAdapterIds * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.A, 0, a_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.B, 0, b_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.adapter_map, 0xff, kMaxAdapterIds * sizeof(int32_t)) == cudaSuccess;   // -1: no serving version
     ok = ok && gemm_sm100_init(device) == cudaSuccess;
     ok = ok && shrink_init() == cudaSuccess;
     ok = ok && decode_init() == cudaSuccess;
@@ -88,7 +90,7 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status);
+        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
         delete t;
         return LML_ERR_CUDA;
     }
@@ -101,7 +103,7 @@ lml_status lml_table_destroy(lml_table* t)
     if (!t) return LML_ERR_INVALID_ARG;
     {
         DeviceGuard guard(t->device);
-        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status);
+        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
     }
     delete t;
     return LML_OK;
@@ -129,6 +131,7 @@ lml_status register_adapter(lml_table* t, int adapter_id, int version, const voi
     }
     auto& e = t->entries[free_slot];
     e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
+    e.state = LML_STATE_RESIDENT; e.pins = 0;
     e.live = true;   // published last: the entry is complete before it becomes visible
     *slot_out = free_slot;
     return LML_OK;
@@ -140,9 +143,97 @@ lml_status retire_version(lml_table* t, int adapter_id, int version)
     std::lock_guard<std::mutex> lock(t->mu);
     for (int i = 0; i < t->max_slots; ++i) {
         auto& e = t->entries[i];
-        if (e.live && e.adapter_id == adapter_id && e.version == version) { e.live = false; return LML_OK; }
+        if (e.live && e.adapter_id == adapter_id && e.version == version) {
+            if (e.state == LML_STATE_SERVING) {
+                // no longer the adapter's serving version: calls that name the adapter must stop resolving to it
+                DeviceGuard guard(t->device);
+                const int32_t none = -1;
+                if (!guard.ok || cudaMemcpy(t->arena.adapter_map + adapter_id, &none, sizeof none, cudaMemcpyHostToDevice) != cudaSuccess) {
+                    cudaGetLastError();
+                    return LML_ERR_CUDA;
+                }
+            }
+            if (e.pins > 0) e.state = LML_STATE_RETIRING;   // freed by the last unpin
+            else e.live = false;
+            return LML_OK;
+        }
     }
     return LML_ERR_NOT_FOUND;
+}
+
+lml_status lml_publish(lml_table* t, int adapter_id, int version, void* stream, int* previous_version_out)
+{
+    if (!t || adapter_id < 0 || adapter_id >= kMaxAdapterIds) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    int slot = -1, prev = -1;
+    for (int i = 0; i < t->max_slots; ++i) {
+        const auto& e = t->entries[i];
+        if (!e.live || e.adapter_id != adapter_id) continue;
+        if (e.version == version && e.state != LML_STATE_RETIRING) slot = i;
+        else if (e.state == LML_STATE_SERVING) prev = i;
+    }
+    if (slot < 0) return LML_ERR_NOT_FOUND;
+    if (previous_version_out) *previous_version_out = prev >= 0 ? t->entries[prev].version : -1;
+    if (t->entries[slot].state == LML_STATE_SERVING) return LML_OK;   // already the serving version
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    // the controlled publication point: one 4-byte store, in stream order
+    if (launch_set_word(t->arena.adapter_map + adapter_id, slot, (cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
+    t->entries[slot].state = LML_STATE_SERVING;
+    if (prev >= 0) {
+        auto& o = t->entries[prev];
+        if (o.pins > 0) o.state = LML_STATE_RETIRING;
+        else o.live = false;
+    }
+    return LML_OK;
+}
+
+lml_status lml_pin(lml_table* t, int slot)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (slot < 0 || slot >= t->max_slots || !t->entries[slot].live) return LML_ERR_BAD_SLOT;
+    ++t->entries[slot].pins;
+    return LML_OK;
+}
+
+lml_status lml_unpin(lml_table* t, int slot)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (slot < 0 || slot >= t->max_slots || !t->entries[slot].live) return LML_ERR_BAD_SLOT;
+    auto& e = t->entries[slot];
+    if (e.pins <= 0) return LML_ERR_INVALID_ARG;
+    if (--e.pins == 0 && e.state == LML_STATE_RETIRING) e.live = false;   // the last work bound to a replaced version has ended
+    return LML_OK;
+}
+
+lml_status lml_resolve(const lml_table* t, int adapter_id, int* slot_out, int* version_out)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    for (int i = 0; i < t->max_slots; ++i) {
+        const auto& e = t->entries[i];
+        if (e.live && e.adapter_id == adapter_id && e.state == LML_STATE_SERVING) {
+            if (slot_out) *slot_out = i;
+            if (version_out) *version_out = e.version;
+            return LML_OK;
+        }
+    }
+    return LML_ERR_NOT_FOUND;
+}
+
+lml_status lml_slot_state(const lml_table* t, int slot, int* state_out, int* pins_out)
+{
+    if (!t) return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t->mu);
+    if (slot < 0 || slot >= t->max_slots || !t->entries[slot].live) return LML_ERR_BAD_SLOT;
+    if (state_out) *state_out = t->entries[slot].state;
+    if (pins_out) *pins_out = t->entries[slot].pins;
+    return LML_OK;
 }
 
 lml_status lml_lookup(const lml_table* t, int adapter_id, int version, int* slot_out)
@@ -175,21 +266,33 @@ size_t lml_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
     return ws_layout(t, max_tokens, max_segments).total;
 }
 
-lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, int32_t* perm, int32_t* seg_offsets,
-                              int32_t* seg_slot_ids, void* stream)
+static lml_status segment_tokens_impl(lml_table* t, const int32_t* ids, int T, int32_t* perm, int32_t* seg_offsets,
+                                      int32_t* seg_slot_ids, void* stream, bool by_adapter)
 {
-    if (!t || T < 0 || T > kMaxTokens || !seg_offsets || !seg_slot_ids || (T > 0 && (!token_slots || !perm)))
+    if (!t || T < 0 || T > kMaxTokens || !seg_offsets || !seg_slot_ids || (T > 0 && (!ids || !perm)))
         return LML_ERR_INVALID_ARG;
     const SlotSnapshot snap = snapshot_locked(t);
     DeviceGuard guard(t->device);
     if (!guard.ok) return LML_ERR_CUDA;
-    if (launch_segment_tokens(t->arena, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, (cudaStream_t)stream) !=
+    if (launch_segment_tokens(t->arena, snap, ids, T, perm, seg_offsets, seg_slot_ids, (cudaStream_t)stream, by_adapter) !=
         cudaSuccess) {
         cudaGetLastError();
         return LML_ERR_CUDA;
     }
     t->last_launches = 1;
     return LML_OK;
+}
+
+lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, int32_t* perm, int32_t* seg_offsets,
+                              int32_t* seg_slot_ids, void* stream)
+{
+    return segment_tokens_impl(t, token_slots, T, perm, seg_offsets, seg_slot_ids, stream, false);
+}
+
+lml_status lml_segment_tokens_adapters(lml_table* t, const int32_t* token_adapter_ids, int T, int32_t* perm,
+                                       int32_t* seg_offsets, int32_t* seg_slot_ids, void* stream)
+{
+    return segment_tokens_impl(t, token_adapter_ids, T, perm, seg_offsets, seg_slot_ids, stream, true);
 }
 
 lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T, const int32_t* seg_offsets,
@@ -262,8 +365,8 @@ size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens)
     return n;
 }
 
-lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T, const int32_t* token_slots,
-                                    void* y, void* workspace, size_t workspace_bytes, void* stream_v)
+static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T, const int32_t* token_slots, void* y,
+                              void* workspace, size_t workspace_bytes, void* stream_v, bool by_adapter)
 {
     if (!t || T < 0 || T > kMaxTokens) return LML_ERR_INVALID_ARG;
     if (T == 0) { t->last_launches = 0; return LML_OK; }
@@ -282,6 +385,7 @@ lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0,
         DecodeArgs a;
         a.x = x; a.W0 = W0; a.y = y; a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
         a.token_slots = token_slots;
+        a.by_adapter = by_adapter;
         a.u = reinterpret_cast<float*>(wsb + ws.u_off);
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = 1; a.num_sms = t->num_sms;
         int launches = 0;
@@ -297,11 +401,24 @@ lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0,
     int32_t* perm = reinterpret_cast<int32_t*>(wsb + base);
     int32_t* seg_offsets = reinterpret_cast<int32_t*>(wsb + base + round_up((size_t)T * 4 + 4, 1024));
     int32_t* seg_ids = seg_offsets + round_up((size_t)(t->max_slots + 2) * 4, 1024) / 4;
-    lml_status st = lml_segment_tokens(t, token_slots, T, perm, seg_offsets, seg_ids, stream_v);
+    lml_status st = segment_tokens_impl(t, token_slots, T, perm, seg_offsets, seg_ids, stream_v, by_adapter);
     if (st != LML_OK) return st;
     st = lora_mixed_linear(t, x, W0, T, seg_offsets, seg_ids, G, perm, y, workspace, base, stream_v);
     if (st == LML_OK) t->last_launches += 1;
     return st;
+}
+
+lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T, const int32_t* token_slots,
+                                    void* y, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return tokens_impl(t, x, W0, T, token_slots, y, workspace, workspace_bytes, stream, false);
+}
+
+lml_status lora_mixed_linear_adapters(lml_table* t, const void* x, const void* W0, int T,
+                                      const int32_t* token_adapter_ids, void* y, void* workspace,
+                                      size_t workspace_bytes, void* stream)
+{
+    return tokens_impl(t, x, W0, T, token_adapter_ids, y, workspace, workspace_bytes, stream, true);
 }
 
 size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)

@@ -56,10 +56,27 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
 // ---------------------------------------------------------------------------------------------
 constexpr int kSegWarps = 32;
 
+// adapter id -> serving slot through the table's device map; -1 stays -1, anything else unknown is -2 (flagged)
+__device__ __forceinline__ int resolve_adapter(const int32_t* __restrict__ adapter_map, int id)
+{
+    if (id == -1) return -1;
+    if (id < 0 || id >= kMaxAdapterIds) return -2;
+    const int s = __ldg(adapter_map + id);
+    return s < 0 ? -2 : s;
+}
+
+__global__ void set_word_kernel(int32_t* dst, int32_t value) { *dst = value; }
+
+cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream)
+{
+    set_word_kernel<<<1, 1, 0, stream>>>(dst, value);
+    return cudaGetLastError();
+}
+
 __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
     const __grid_constant__ SlotSnapshot snap, const int32_t* __restrict__ token_slots, int T,
     int32_t* __restrict__ perm, int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_slot_ids,
-    uint32_t* __restrict__ status)
+    uint32_t* __restrict__ status, const int32_t* __restrict__ adapter_map)
 {
     __shared__ int hist[kSegWarps][kMaxSlots + 1];
     __shared__ int base[kMaxSlots + 2];
@@ -80,6 +97,7 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
         int i = c + lane;
         if (i < end) {
             int s = __ldg(token_slots + i);
+            if (adapter_map) s = resolve_adapter(adapter_map, s);
             if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) { bad = true; s = -1; }
             int key = s < 0 ? snap.max_slots : s;
             atomicAdd(&hist[warp][key], 1);
@@ -111,6 +129,7 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
         int key = nk;                          // sentinel for lanes past the end
         if (i < end) {
             int s = __ldg(token_slots + i);
+            if (adapter_map) s = resolve_adapter(adapter_map, s);
             if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) s = -1;
             key = s < 0 ? snap.max_slots : s;
         }
@@ -129,13 +148,14 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
 
 cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
                                   int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
-                                  cudaStream_t stream)
+                                  cudaStream_t stream, bool by_adapter)
 {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     pdl_config(cfg, attr, dim3(1), dim3(kSegWarps * 32), 0, stream);
     uint32_t* status = ar.status;
-    return cudaLaunchKernelEx(&cfg, segment_tokens_kernel, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, status);
+    const int32_t* map = by_adapter ? ar.adapter_map : nullptr;
+    return cudaLaunchKernelEx(&cfg, segment_tokens_kernel, snap, token_slots, T, perm, seg_offsets, seg_slot_ids, status, map);
 }
 
 // ---------------------------------------------------------------------------------------------

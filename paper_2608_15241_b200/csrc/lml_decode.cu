@@ -130,7 +130,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
     const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
-    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, uint32_t* status, int T, int K, int N, int G, int patience)
+    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, const int32_t* __restrict__ adapter_map, uint32_t* status, int T, int K, int N,
+    int G, int patience)
 {
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
@@ -303,7 +304,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             }
             if (perm && lane < T) my_row = __ldg(perm + lane);
             int my_token_slot = -1;
-            if (by_token && lane < T) my_token_slot = __ldg(token_slots + lane);
+            if (by_token && lane < T) {
+                my_token_slot = __ldg(token_slots + lane);
+                if (adapter_map) {   // the ids are adapter ids: the table's device map names the serving slot (-2: none, flagged below)
+                    const int id = my_token_slot;
+                    my_token_slot = id == -1 ? -1 : ((id < 0 || id >= kMaxAdapterIds) ? -2 : __ldg(adapter_map + id));
+                    if (id != -1 && my_token_slot < 0) my_token_slot = -2;
+                }
+            }
             asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
@@ -766,10 +774,11 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const int32_t* ids = a.slot_ids;
     const int32_t* pm = a.perm;
     const int32_t* ts = a.token_slots;
+    const int32_t* amap = a.by_adapter ? ar.adapter_map : nullptr;
     cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience)
+                                                 ids, pm, ts, amap, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience)
                             : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience);
+                                                 ids, pm, ts, amap, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience);
     if (e == cudaSuccess) ++*launches;
     return e;
 }

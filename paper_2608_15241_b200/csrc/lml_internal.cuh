@@ -15,6 +15,7 @@ constexpr int kMaxSlots = LML_MAX_SLOTS;
 constexpr int kRankPad = 64;          // adapters are stored zero-padded to this rank
 constexpr int kTileM = 128;           // token rows per GEMM tile and per shrink piece block
 constexpr int kDecodeMaxT = LML_DECODE_MAX_TOKENS;
+constexpr int kMaxAdapterIds = LML_MAX_ADAPTER_IDS;   // adapter ids that can be resolved on the device
 
 // Per-call snapshot of the slot table, passed by value as a kernel parameter so that a later
 // register / retire cannot change a call that is already enqueued.
@@ -29,6 +30,7 @@ struct Arena {
     __nv_bfloat16* A;   // [max_slots][kRankPad][d_in]   rows >= rank are zero
     __nv_bfloat16* B;   // [max_slots][d_out][kRankPad]  columns >= rank are zero
     uint32_t* status;   // sticky LML_FLAG_* bits
+    int32_t* adapter_map;   // [kMaxAdapterIds] serving slot of each adapter id, -1 = none; written by lml_publish
 };
 
 // Workspace header written by the shrink kernels and read by the kernels that follow.
@@ -42,9 +44,10 @@ struct PlanWord {
 cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const void* B, int rank,
                                 int d_in, int d_out, cudaStream_t stream);
 
+cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream);
 cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
                                   int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, bool by_adapter = false);   // by_adapter: the ids are adapter ids, resolved through ar.adapter_map
 
 // u blocks: block b = (tile m) + (segment g) holds the 128 x 64 bf16 values scale*(x.A^T) of
 // the rows of tile m that belong to segment g, zero elsewhere.
@@ -93,6 +96,7 @@ struct DecodeArgs {
     const int32_t* seg_offsets;
     const int32_t* slot_ids;
     const int32_t* token_slots = nullptr;   // instead of segments: one slot id per row of x (then G is 1 and perm is null)
+    bool by_adapter = false;                // the ids in token_slots are adapter ids, resolved through the table's device map
     float* u;            // [16][64] fp32 scratch: scale * x.A^T, written and read by the decode kernel
     int T, d_in, d_out, G;
     int num_sms;

@@ -11,6 +11,8 @@ struct lml_table {
         bool live = false;
         int adapter_id = 0, version = 0, rank = 0;
         float scale = 0.f;
+        int state = 0;   // LML_STATE_*: resident (staged or plain), serving, retiring
+        int pins = 0;    // work in flight that is bound to this entry
     } entries[lml::kMaxSlots];
     lml::Arena arena{};
     CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
