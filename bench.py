@@ -185,6 +185,43 @@ class Rotation:
                             s["y"].data_ptr(), s["ws"].data_ptr(), s["ws"].numel(), b._stream(None))
         return t.last_launch_count()
 
+    def prepare_dual(self):
+        """Second binding for the dual-version call: every segment takes its neighbour's entry."""
+        import torch
+        from paper_2608_15241_b200.binding import lml_dual_workspace_bytes
+        w = self.w
+        for s in self.sets:
+            other = np.roll(w.seg_entry, 1)
+            s["ids_b"] = torch.from_numpy(np.array([s["slots"][e] if e >= 0 else -1 for e in other], np.int32)).to(self.device)
+            s["y_b"] = torch.empty_like(s["y"])
+            s["ws_dual"] = torch.empty(lml_dual_workspace_bytes(s["table"].handle, w.T, w.G), dtype=torch.uint8,
+                                       device=self.device)
+        torch.cuda.synchronize()
+
+    def dual_only(self, i):
+        """Both bindings in one call (shared base product)."""
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        t = s["table"]
+        b.lora_mixed_linear_dual(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["so_pre"].data_ptr(),
+                                 s["ids_pre"].data_ptr(), s["ids_b"].data_ptr(), self.w.G,
+                                 0 if s["perm_pre"] is None else s["perm_pre"].data_ptr(), s["y"].data_ptr(),
+                                 s["y_b"].data_ptr(), s["ws_dual"].data_ptr(), s["ws_dual"].numel(), b._stream(None))
+        return t.last_launch_count()
+
+    def two_singles(self, i):
+        """The same two outputs by two ordinary calls."""
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        t = s["table"]
+        n = 0
+        for ids, y in ((s["ids_pre"], s["y"]), (s["ids_b"], s["y_b"])):
+            b.lora_mixed_linear(t.handle, s["x"].data_ptr(), s["W0"].data_ptr(), self.w.T, s["so_pre"].data_ptr(),
+                                ids.data_ptr(), self.w.G, 0 if s["perm_pre"] is None else s["perm_pre"].data_ptr(),
+                                y.data_ptr(), s["ws"].data_ptr(), s["ws"].numel(), b._stream(None))
+            n += t.last_launch_count()
+        return n
+
     def close(self):
         for s in self.sets:
             s["table"].close()
@@ -342,6 +379,14 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                 "frac_of_sustained": achieved / peaks["tensor_sustained"], "frac_of_nominal_2250": achieved / 2250.0,
                 "traffic": None, "us_per_launch": per_launch * 1e6}
 
+    dual = None
+    if kind != "decode" and w.G >= 1:
+        # the same tokens under two bindings: one call with a shared base product against two ordinary calls
+        rot.prepare_dual()
+        dsteps = max(rot.R, min(steps, 100))
+        d_secs, _, _ = timed_graph_loop(rot.dual_only, rot.R, dsteps, 3, stream)
+        t_secs, _, _ = timed_graph_loop(rot.two_singles, rot.R, dsteps, 3, stream)
+        dual = {"us_per_call": d_secs / dsteps * 1e6, "two_single_calls_us": t_secs / dsteps * 1e6}
     roof["traffic"] = ncu_traffic(name)
     roof["algorithmic"] = w.bytes() if kind == "decode" else w.flops()
     esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
@@ -357,6 +402,8 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                       "l2_policy": f"inputs larger than L2: {rot.R} distinct weight/activation sets "
                                    f"({rot.R * w.bytes() / 1e6:.0f} MB) visited round-robin",
                       "timing": "CUDA-graph replay of R-step chunks, CUDA events on the launch stream"}}
+    if dual:
+        out["dual_version_call"] = dual
     if want_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, kind, spec["unit"], budget_s=6.0)
         out["parity_sample"] = sampled_parity(rot)

@@ -201,6 +201,24 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
                              void* stream);
 
 /*
+ * lora_mixed_linear_dual — the same tokens under two bindings in one call (Section 5.3: hot prefixes
+ * are recomputed under the staged version while the old one still serves).  slot_ids_a / slot_ids_b:
+ * device int32[G], the slot of every segment under the first and under the second binding (-1 = no
+ * adapter, either side).  y_a = x.W0 + delta_a, y_b = x.W0 + delta_b, both device bf16 [T][d_out],
+ * distinct buffers.  For T > 16 the base product x.W0 is computed once: y_a is read out of the
+ * accumulator, then (delta_b - delta_a) is added to it with a few more tensor-core steps and y_b is
+ * read out, so y_a is bit-identical to lora_mixed_linear with slot_ids_a and y_b agrees with
+ * lora_mixed_linear with slot_ids_b to fp32 rounding of the accumulator.  For T <= 16 the call is two
+ * decode calls.  G >= 1.  workspace: at least lml_dual_workspace_bytes(t, T, G).  Other arguments,
+ * flags and errors as lora_mixed_linear.
+ */
+size_t lml_dual_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
+lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, int T,
+                                  const int32_t* seg_offsets, const int32_t* slot_ids_a,
+                                  const int32_t* slot_ids_b, int G, const int32_t* perm, void* y_a, void* y_b,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * lora_mixed_linear_tokens — segmentation and layer in one call, for callers that hold one slot id
  * per token (what a scheduler hands a decode step).  token_slots: device int32[T], physical slot
  * per row of x or -1; ids outside [-1, max_slots) or naming a free slot count as -1 and set

@@ -31,7 +31,8 @@ EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "regist
            "lora_mixed_linear_host", "lml_device_status", "lml_last_launch_count",
            "lora_mixed_linear_decode_static", "lml_tokens_workspace_bytes", "lora_mixed_linear_tokens",
            "lml_publish", "lml_pin", "lml_unpin", "lml_resolve", "lml_slot_state",
-           "lml_segment_tokens_adapters", "lora_mixed_linear_adapters")
+           "lml_segment_tokens_adapters", "lora_mixed_linear_adapters",
+           "lml_dual_workspace_bytes", "lora_mixed_linear_dual")
 
 
 class LmlError(RuntimeError):
@@ -74,6 +75,9 @@ def lib() -> ctypes.CDLL:
         L.lora_mixed_linear_tokens.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lora_mixed_linear_adapters.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lml_segment_tokens_adapters.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.lml_dual_workspace_bytes.restype = sz
+        L.lml_dual_workspace_bytes.argtypes = [vp, i32, i32]
+        L.lora_mixed_linear_dual.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.lml_publish.argtypes = [vp, i32, i32, vp, ctypes.POINTER(i32)]
         L.lml_pin.argtypes = [vp, i32]
         L.lml_unpin.argtypes = [vp, i32]
@@ -83,7 +87,7 @@ def lib() -> ctypes.CDLL:
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
             if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes",
-                            "lml_tokens_workspace_bytes"):
+                            "lml_tokens_workspace_bytes", "lml_dual_workspace_bytes"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -173,6 +177,19 @@ def lora_mixed_linear_tokens(table: int, x_ptr: int, W0_ptr: int, T: int, token_
     """Segmentation and layer in one call: one slot id per token instead of segments."""
     _check(lib().lora_mixed_linear_tokens(table, x_ptr, W0_ptr, T, token_slots_ptr, y_ptr, workspace_ptr,
                                           workspace_bytes, stream), "lora_mixed_linear_tokens")
+
+
+def lml_dual_workspace_bytes(table: int, max_tokens: int, max_segments: int) -> int:
+    return int(lib().lml_dual_workspace_bytes(table, max_tokens, max_segments))
+
+
+def lora_mixed_linear_dual(table: int, x_ptr: int, W0_ptr: int, T: int, seg_offsets_ptr: int, slot_ids_a_ptr: int,
+                           slot_ids_b_ptr: int, G: int, perm_ptr: int, y_a_ptr: int, y_b_ptr: int, workspace_ptr: int,
+                           workspace_bytes: int, stream: int = 0) -> None:
+    """The same tokens under two slot bindings in one call; the base product is shared for T > 16."""
+    _check(lib().lora_mixed_linear_dual(table, x_ptr, W0_ptr, T, seg_offsets_ptr, slot_ids_a_ptr, slot_ids_b_ptr, G,
+                                        perm_ptr, y_a_ptr, y_b_ptr, workspace_ptr, workspace_bytes, stream),
+           "lora_mixed_linear_dual")
 
 
 STATE_RESIDENT, STATE_SERVING, STATE_RETIRING = 0, 1, 2
@@ -371,6 +388,18 @@ class Table:
 
     def slot_state(self, slot: int):
         return lml_slot_state(self.handle, slot)
+
+    def lora_mixed_linear_dual(self, x, W0, seg_offsets, slot_ids_a, slot_ids_b, perm=None, stream=None):
+        """-> (y_a, y_b): the layer under two slot bindings of the same segments."""
+        import torch
+        T, G = int(x.shape[0]), int(slot_ids_a.shape[0])
+        assert slot_ids_b.shape[0] == G and seg_offsets.shape[0] == G + 1
+        y_a = torch.empty((T, self.d_out), dtype=torch.bfloat16, device=x.device)
+        y_b = torch.empty_like(y_a)
+        ws = torch.empty(max(lml_dual_workspace_bytes(self.handle, T, G), 256), dtype=torch.uint8, device=x.device)
+        lora_mixed_linear_dual(self.handle, _ptr(x), _ptr(W0), T, _ptr(seg_offsets), _ptr(slot_ids_a), _ptr(slot_ids_b),
+                               G, _ptr(perm), _ptr(y_a), _ptr(y_b), _ptr(ws), int(ws.numel()), _stream(stream))
+        return y_a, y_b
 
     def lora_mixed_linear_adapters(self, x, W0, token_adapter_ids, y=None, workspace=None, stream=None):
         """As lora_mixed_linear_tokens, with one ADAPTER id per token (resolved on the device)."""

@@ -15,14 +15,14 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct WsLayout {
     size_t plan_off, ident_off, u_off, xg_off, total;
 };
-WsLayout ws_layout(const lml_table* t, int T, int G)
+WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
 {
     WsLayout w;
     w.plan_off = 0;
     const size_t num_m = (size_t)(T + kTileM - 1) / kTileM;
     w.ident_off = round_up(sizeof(PlanWord), 256);
     w.u_off = round_up(w.ident_off + (num_m + 1) * sizeof(int32_t), 1024);
-    size_t u_bytes = (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
+    size_t u_bytes = (size_t)u_sets * (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
     const size_t dec_bytes = (size_t)kDecodeMaxT * kRankPad * sizeof(float) + kDecodeMaxT * sizeof(int32_t);
     if (u_bytes < dec_bytes) u_bytes = dec_bytes;
     w.xg_off = w.u_off + round_up(u_bytes, 1024);
@@ -363,6 +363,77 @@ size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens)
     n += round_up((size_t)max_tokens * 4 + 4, 1024);               // perm
     n += 2 * round_up((size_t)(t->max_slots + 2) * 4, 1024);       // seg_offsets, seg_slot_ids
     return n;
+}
+
+size_t lml_dual_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
+{
+    if (!t || max_tokens < 0 || max_segments < 0 || max_tokens > kMaxTokens) return 0;
+    return ws_layout(t, max_tokens, max_segments, 3).total;
+}
+
+lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, int T, const int32_t* seg_offsets,
+                                  const int32_t* slot_ids_a, const int32_t* slot_ids_b, int G, const int32_t* perm,
+                                  void* y_a, void* y_b, void* workspace, size_t workspace_bytes, void* stream_v)
+{
+    if (!t || T < 0 || G < 1 || T > kMaxTokens || G > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x || !W0 || !y_a || !y_b || y_a == y_b || !seg_offsets || !slot_ids_a || !slot_ids_b || !aligned16(x) ||
+        !aligned16(W0) || !aligned16(y_a) || !aligned16(y_b))
+        return LML_ERR_INVALID_ARG;
+    if (T <= kDecodeMaxT) {
+        // The decode kernel has no two-output form: two calls, W0 streamed twice.
+        lml_status st = lora_mixed_linear(t, x, W0, T, seg_offsets, slot_ids_a, G, perm, y_a, workspace, workspace_bytes, stream_v);
+        if (st != LML_OK) return st;
+        const int first = t->last_launches;
+        st = lora_mixed_linear(t, x, W0, T, seg_offsets, slot_ids_b, G, perm, y_b, workspace, workspace_bytes, stream_v);
+        if (st == LML_OK) t->last_launches += first;
+        return st;
+    }
+    const WsLayout ws = ws_layout(t, T, G, 3);
+    const size_t need = perm ? ws.total : ws.xg_off;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return LML_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    const SlotSnapshot snap = snapshot_locked(t);
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    uint8_t* wsb = static_cast<uint8_t*>(workspace);
+    int launches = 0;
+    cudaError_t e = cudaSuccess;
+    const void* xg = x;
+    int32_t* tile_identity = nullptr;
+    if (perm) {
+        tile_identity = reinterpret_cast<int32_t*>(wsb + ws.ident_off);
+        e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, tile_identity, true, t->arena.status, stream);
+        if (e == cudaSuccess) { ++launches; xg = wsb + ws.xg_off; }
+    }
+    PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
+    __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
+    const size_t num_m = (size_t)(T + kTileM - 1) / kTileM;
+    const size_t set_elems = (num_m + (size_t)G) * kTileM * kRankPad;
+    // three sets of u blocks: scale.x.A^T under the first slots (set 0) and its negation (set 2), written by
+    // one shrink pass, and under the second slots (set 1), by a second pass that runs beside the first:
+    // the second output is the first accumulator plus (second delta - first delta)
+    e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids_a, G, x, tile_identity, plan, u_blocks,
+                             stream, false, u_blocks + 2 * set_elems);
+    if (e == cudaSuccess) {
+        ++launches;
+        e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids_b, G, x, tile_identity, plan,
+                                 u_blocks + set_elems, stream, true);
+        if (e == cudaSuccess) ++launches;
+    }
+    if (e == cudaSuccess) {
+        GemmArgs a;
+        a.x = xg; a.x_in_place = x; a.tile_identity = tile_identity; a.W0 = W0; a.y = y_a; a.perm = perm;
+        a.seg_offsets = seg_offsets; a.slot_ids = slot_ids_a; a.slot_ids2 = slot_ids_b; a.y2 = y_b;
+        a.plan = plan; a.u_blocks = u_blocks;
+        a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
+        a.overlap_with_previous = true;
+        e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
+        if (e == cudaSuccess) ++launches;
+    }
+    t->last_launches = launches;
+    if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    return LML_OK;
 }
 
 static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T, const int32_t* token_slots, void* y,

@@ -12,6 +12,12 @@
 //            bf16 once, stage 32x32 chunks in shared memory and write them with TMA stores (or
 //            row-scattered 16-byte stores when a perm is given).  Runs one tile behind the MMA
 //            warp thanks to the second accumulator.
+// Dual form (two slot bindings of the same segments, two outputs): the base product is computed once.
+// The epilogue reads the first output out of the accumulator and tells the MMA thread; that thread
+// then adds (second binding's delta - first binding's delta) on top, as further K-steps whose u
+// operands come from two more sets of u blocks (second slots; first slots negated), and the epilogue
+// reads the second output.  The producer slips those stages into the middle of the next tile's
+// k-blocks, by when the first read is long done.
 // Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
 #include <cstdlib>
 
@@ -36,7 +42,7 @@ template <int BN> struct GemmCfg {
     static constexpr int kStages = (BN == 256) ? 4 : 6;
     static constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
     static constexpr int kTmemCols = 2 * BN;
-    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + kSegCache;   // barriers + segment cache
+    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache;   // barriers + segment cache (two slot arrays)
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiBytes + ((kCtrlBytes + 15) & ~15);
 };
 
@@ -45,11 +51,18 @@ struct GemmCtrl {
     uint64_t empty[8];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t tmem_read1[2];   // dual form: the first output of the tile has been read out of the accumulator
     uint32_t tmem_base;
     int abort;
-    uint32_t stage_info[8];   // k-steps (1..4) | last-stage-of-tile << 8, written by the producer
-    int32_t pad[6];
+    uint32_t stage_info[8];   // written by the producer: k-steps (0..4) | kStage* flags
+    int32_t pad[2];
 };
+// stage_info flags
+constexpr uint32_t kStageCommit = 0x100u;   // after this stage the accumulator holds an output: commit it to the epilogue
+constexpr uint32_t kStageAcc1 = 0x200u;     // the stage belongs to accumulator 1 (else 0)
+constexpr uint32_t kStageFresh = 0x400u;    // first stage of a tile: wait for the accumulator to be free, overwrite it
+constexpr uint32_t kStageDelta = 0x800u;    // dual form: first stage of a tile's second output: wait until the first was read
+
 static_assert(sizeof(GemmCtrl) <= 256, "control block");
 
 struct GemmParams {
@@ -58,6 +71,9 @@ struct GemmParams {
     const int32_t* perm;
     const int32_t* tile_identity;   // perm form: tiles whose rows stayed in place (read tmap_x0, store with TMA)
     const PlanWord* plan;
+    const int32_t* slot_ids2;   // dual form: the second slot per segment (else null)
+    __nv_bfloat16* y2;          // dual form: the second output
+    int u_set_rows;             // dual form: rows between the three sets of u blocks (first slots, second slots, minus first)
     __nv_bfloat16* y;
     uint32_t* status;
     int T, K, N, G;
@@ -69,10 +85,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x0,
     const __grid_constant__ CUtensorMap tmap_w,
     const __grid_constant__ CUtensorMap tmap_u, const __grid_constant__ CUtensorMap tmap_b,
-    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ SlotSnapshot snap,
-    const GemmParams p)
+    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_y2,
+    const __grid_constant__ SlotSnapshot snap, const GemmParams p)
 {
     using Cfg = GemmCfg<BN>;
+    const bool dual = p.slot_ids2 != nullptr;
     extern __shared__ uint8_t smem_raw[];
     // 128-byte swizzled tiles need 1024-byte alignment
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -83,6 +100,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(epi_ptr + Cfg::kEpiBytes);
     int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
     int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
+    int8_t* slot_cache2 = slot_cache + kSegCache;   // dual form: the second slot per segment
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = p.num_m * p.num_n;
@@ -97,6 +115,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctrl->tmem_full[a]), 1);
             mbar_init(smem_u32(&ctrl->tmem_empty[a]), 4);
+            mbar_init(smem_u32(&ctrl->tmem_read1[a]), 4);
         }
         ctrl->abort = 0;
         fence_mbar_init();
@@ -105,12 +124,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         prefetch_tmap(&tmap_x0);
         prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u);
         prefetch_tmap(&tmap_b); prefetch_tmap(&tmap_y);
+        if (dual) prefetch_tmap(&tmap_y2);
     }
     if (seg_cached && p.G > 0) {
         for (int g = threadIdx.x; g <= p.G; g += kGemmThreads) seg_cache[g] = __ldg(p.seg_offsets + g);
         for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
             int s = __ldg(p.slot_ids + g);
             slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
+            if (dual) {
+                const int s2 = __ldg(p.slot_ids2 + g);
+                slot_cache2[g] = (int8_t)((s2 >= 0 && s2 < snap.max_slots && snap.rank[s2] > 0) ? s2 : -1);
+            }
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), Cfg::kTmemCols);
@@ -126,6 +150,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
+        // Stage order.  A tile is its base k-blocks followed by one stage per LoRA piece; the last of
+        // these carries kStageCommit.  In the dual form every tile has a second output, the same
+        // accumulator plus (second slots' delta minus first slots' delta): its stages ("delta
+        // stages": one per piece of the second slot array, one per piece of the first with the
+        // negated u) can only run once the epilogue has read the first output, so they are slipped
+        // into the middle of the NEXT tile's k-blocks (or follow the last tile), where the MMA thread
+        // does not have to wait for that.
         if (lane == 0) {
             bool lora = false, lora_known = (p.G == 0);
             int stage = 0;
@@ -135,52 +166,109 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort);
             };
             auto advance = [&]() { if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; } };
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m = tile % p.num_m, n = tile / p.num_m;
+            auto learn_lora = [&]() {
+                // Everything the shrink kernel wrote (plan word, u blocks) is first touched after the
+                // base k-blocks of the first tile are already in flight.
+                if (!lora_known) {
+                    grid_dependency_wait();
+                    grid_launch_dependents();
+                    lora = p.plan->lora_ok != 0;
+                    lora_known = true;
+                }
+            };
+            // slot of segment g as far as tile rows [row0, row1) are concerned; -1 = no piece
+            auto piece_slot = [&](int g, int row0, int row1, bool second) -> int {
+                int s0, s1, s;
+                if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = second ? slot_cache2[g] : slot_cache[g]; }
+                else {
+                    s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1);
+                    s = __ldg((second ? p.slot_ids2 : p.slot_ids) + g);
+                    if (slot_rank(snap, s) == 0) s = -1;
+                }
+                if (min(s1, row1) <= max(s0, row0)) return -1;
+                return s;
+            };
+            auto segment_range = [&](int row0, int row1, int& g_first, int& g_end) {
+                if (seg_cached) {
+                    int lo = 0, hi = p.G;
+                    while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+                    g_first = lo;
+                    g_end = g_first;
+                    while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
+                } else {
+                    g_first = seg_upper(p.seg_offsets, p.G, row0);
+                    g_end = g_first;
+                    while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
+                }
+            };
+            // one stage per piece of a tile from one of the three sets of u blocks; `flags_first` go on the
+            // first stage emitted, `flags_last` on the last; returns how many stages went out
+            auto emit_pieces = [&](int m, int n, int set, bool second, uint32_t acc_flag, uint32_t flags_first,
+                                   uint32_t flags_last, bool count_only) -> int {
                 const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+                int g_first = 0, g_end = 0, count = 0, last_piece = -1;
+                if (lora) {
+                    segment_range(row0, row1, g_first, g_end);
+                    for (int g = g_first; g < g_end; ++g) if (piece_slot(g, row0, row1, second) >= 0) { last_piece = g; ++count; }
+                }
+                if (count_only) return count;
+                bool first = true;
+                for (int g = g_first; g < g_end && ok; ++g) {
+                    const int s = piece_slot(g, row0, row1, second);
+                    if (s < 0) continue;
+                    ok = acquire();
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                    const uint32_t ksteps = (uint32_t)((snap.rank[s] + 15) >> 4);
+                    ctrl->stage_info[stage] = ksteps | acc_flag | (first ? flags_first : 0u) | (g == last_piece ? flags_last : 0u);
+                    first = false;
+                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                    tma_load_2d(a_dst, &tmap_u, bar, 0, set * p.u_set_rows + (m + g) * kBM);
+                    tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
+                    advance();
+                }
+                return count;
+            };
+            // a stage without operands: only its flags matter to the MMA thread
+            auto emit_marker = [&](uint32_t info) {
+                ok = acquire();
+                if (!ok) return;
+                ctrl->stage_info[stage] = info;
+                mbar_arrive(smem_u32(&ctrl->full[stage]));
+                advance();
+            };
+            // the delta stages of tile (m, n) on accumulator flag acc_flag
+            auto emit_delta = [&](int m, int n, uint32_t acc_flag) {
+                const int n_new = emit_pieces(m, n, 1, true, acc_flag, 0u, 0u, true);
+                const int n_old = emit_pieces(m, n, 2, false, acc_flag, 0u, 0u, true);
+                if (n_new + n_old == 0) { emit_marker(acc_flag | kStageDelta | kStageCommit); return; }
+                emit_pieces(m, n, 1, true, acc_flag, kStageDelta, n_old == 0 ? kStageCommit : 0u, false);
+                if (ok && n_old > 0) emit_pieces(m, n, 2, false, acc_flag, n_new == 0 ? kStageDelta : 0u, kStageCommit, false);
+            };
+            int ordinal = 0, prev_m = -1, prev_n = -1;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ordinal) {
+                const int m = tile % p.num_m, n = tile / p.num_m;
+                const int row0 = m * kBM;
+                const uint32_t acc_flag = (ordinal & 1) ? kStageAcc1 : 0u;
                 const bool in_place = p.tile_identity && __ldg(p.tile_identity + m);   // rows of x never copied
-                int g_first = 0, g_end = 0, last_piece = -1;
-                auto piece_slot = [&](int g) -> int {   // -1 = segment contributes no piece
-                    int s0, s1, s;
-                    if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
-                    else {
-                        s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1); s = __ldg(p.slot_ids + g);
-                        if (slot_rank(snap, s) == 0) s = -1;
-                    }
-                    if (min(s1, row1) <= max(s0, row0)) return -1;
-                    return s;
-                };
+                int pieces = 0;
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
                     if (kb == num_kb - 1) {
-                        // Pieces of this tile: segments with a live slot that overlap [row0, row1).
-                        // Everything the shrink kernel wrote (plan word, u blocks) is first touched
-                        // here, after the base k-blocks of the first tile are already in flight.
-                        if (!lora_known) {
-                            grid_dependency_wait();
-                            grid_launch_dependents();
-                            lora = p.plan->lora_ok != 0;
-                            lora_known = true;
-                        }
-                        if (lora) {
-                            if (seg_cached) {
-                                int lo = 0, hi = p.G;
-                                while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
-                                g_first = lo;
-                                g_end = g_first;
-                                while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
-                            } else {
-                                g_first = seg_upper(p.seg_offsets, p.G, row0);
-                                g_end = g_first;
-                                while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
-                            }
-                            for (int g = g_first; g < g_end; ++g) if (piece_slot(g) >= 0) last_piece = g;
-                        }
+                        learn_lora();
+                        pieces = emit_pieces(m, n, 0, false, acc_flag, 0u, 0u, true);
+                    }
+                    if (dual && prev_m >= 0 && kb == min((num_kb + 1) / 2, num_kb - 1)) {
+                        learn_lora();
+                        emit_delta(prev_m, prev_n, acc_flag ^ kStageAcc1);
+                        if (!ok) break;
                     }
                     ok = acquire();
                     if (!ok) break;
                     const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
                     const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                    ctrl->stage_info[stage] = 4u | ((kb == num_kb - 1 && last_piece < 0) ? 0x100u : 0u);
+                    ctrl->stage_info[stage] = 4u | acc_flag | (kb == 0 ? kStageFresh : 0u) |
+                                              ((kb == num_kb - 1 && pieces == 0) ? kStageCommit : 0u);
                     mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                     // two call sites on purpose: each names its tensor map as a kernel-parameter constant
                     if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
@@ -188,20 +276,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                     tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
                     advance();
                 }
-                for (int g = g_first; g < g_end && ok; ++g) {
-                    const int s = piece_slot(g);
-                    if (s < 0) continue;
-                    ok = acquire();
-                    if (!ok) break;
-                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
-                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                    const uint32_t ksteps = (uint32_t)((snap.rank[s] + 15) >> 4);
-                    ctrl->stage_info[stage] = ksteps | (g == last_piece ? 0x100u : 0u);
-                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
-                    tma_load_2d(a_dst, &tmap_u, bar, 0, (m + g) * kBM);
-                    tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
-                    advance();
-                }
+                if (ok && pieces > 0) emit_pieces(m, n, 0, false, acc_flag, 0u, kStageCommit, false);
+                prev_m = m; prev_n = n;
+            }
+            if (ok && dual && prev_m >= 0) {
+                learn_lora();
+                emit_delta(prev_m, prev_n, ((ordinal - 1) & 1) ? kStageAcc1 : 0u);
             }
             // Leave only after every load issued above has landed (its stage was consumed or its
             // full barrier completed): wait for the ring to drain.
@@ -209,47 +289,74 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // Walks the same schedule as the producer.  The base k-blocks are always four K-steps and need no
+        // side-band word; the last one, the LoRA stages after it and the delta stages carry one (how
+        // many K-steps, and whether an output is complete after the stage).
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN);
             int stage = 0;
             uint32_t phase = 0;
-            int acc = 0;
-            uint32_t acc_phase = 0;
+            uint32_t empty_ph0 = 0, empty_ph1 = 0, read1_ph0 = 0, read1_ph1 = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                ok = mbar_wait(smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1u, abort);
+            // one stage: ksteps MMAs into d_tmem, then the stage goes back to the producer
+            auto issue = [&](uint32_t d_tmem, int ksteps, uint32_t& accumulate) {
+                const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes;
+                const uint64_t adesc = umma_desc_k128(a_addr);
+                const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes);
+#pragma unroll 4
+                for (int k = 0; k < ksteps; ++k) {
+                    // 16 bf16 columns = 32 bytes further along the swizzled row: +2 in 16-byte units
+                    umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
+                    accumulate = 1;
+                }
+                umma_commit(smem_u32(&ctrl->empty[stage]));
+                if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+            };
+            // stages with a side-band word, up to and including the one that completes an output
+            auto flagged_stages = [&](int acc, uint32_t& accumulate) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (bool more = true; more && ok;) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
+                    if (!ok) break;
+                    const uint32_t info = ctrl->stage_info[stage];
+                    more = (info & kStageCommit) == 0;
+                    issue(d_tmem, (int)(info & 0xffu), accumulate);
+                }
+                if (ok) umma_commit(smem_u32(&ctrl->tmem_full[acc]));
+            };
+            // the second output of the tile that sits in accumulator acc: once the epilogue has read the
+            // first, add (second slots' delta - first slots' delta) on top
+            auto delta_stages = [&](int acc) {
+                uint32_t& ph = acc ? read1_ph1 : read1_ph0;
+                ok = mbar_wait(smem_u32(&ctrl->tmem_read1[acc]), ph, abort);
+                if (!ok) return;
+                ph ^= 1u;
+                tc_fence_after();
+                uint32_t accumulate = 1;
+                flagged_stages(acc, accumulate);
+            };
+            int ordinal = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ordinal) {
+                const int acc = ordinal & 1;
+                uint32_t& eph = acc ? empty_ph1 : empty_ph0;
+                ok = mbar_wait(smem_u32(&ctrl->tmem_empty[acc]), eph ^ 1u, abort);
                 if (!ok) break;
+                eph ^= 1u;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 uint32_t accumulate = 0;
-                // The num_kb base k-blocks are always four K-steps; only the last one and the LoRA
-                // stages after it carry a side-band word (how many K-steps, and whether the tile ends).
-                bool more = true;
-                for (int kb = 0; more; ++kb) {
+                const int mid = min((num_kb + 1) / 2, num_kb - 1);
+                for (int kb = 0; kb < num_kb - 1 && ok; ++kb) {
+                    if (dual && ordinal > 0 && kb == mid) { delta_stages(acc ^ 1); if (!ok) break; }
                     ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
                     if (!ok) break;
-                    const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes;
-                    const uint64_t adesc = umma_desc_k128(a_addr);
-                    const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes);
-                    int ksteps = 4;
-                    if (kb >= num_kb - 1) {
-                        const uint32_t info = ctrl->stage_info[stage];
-                        ksteps = (int)(info & 0xffu);
-                        more = (info & 0x100u) == 0;
-                    }
-#pragma unroll 4
-                    for (int k = 0; k < ksteps; ++k) {
-                        // 16 bf16 columns = 32 bytes further along the swizzled row: +2 in 16-byte units
-                        umma_bf16(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
-                        accumulate = 1;
-                    }
-                    umma_commit(smem_u32(&ctrl->empty[stage]));
-                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                    issue(d_tmem, 4, accumulate);
                 }
                 if (!ok) break;
-                umma_commit(smem_u32(&ctrl->tmem_full[acc]));
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                if (dual && ordinal > 0 && mid == num_kb - 1) { delta_stages(acc ^ 1); if (!ok) break; }
+                flagged_stages(acc, accumulate);   // the last k-block and the tile's LoRA pieces
             }
+            if (ok && dual && ordinal > 0) delta_stages((ordinal - 1) & 1);
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -258,74 +365,83 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         const uint32_t buf_addr0 = epi_addr + (uint32_t)(ew * 2 * kEpiBufBytes);
         uint8_t* buf_ptr0 = epi_ptr + ew * 2 * kEpiBufBytes;
         int acc = 0;
-        uint32_t acc_phase = 0;
+        uint32_t full_ph0 = 0, full_ph1 = 0;
         int buf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int m = tile % p.num_m, n = tile / p.num_m;
             const int row_base = m * kBM + q * 32;
             const bool scatter = p.perm != nullptr && !(p.tile_identity && __ldg(p.tile_identity + m));
-            ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+            for (int pass = 0; pass < (dual ? 2 : 1) && ok; ++pass) {
+                uint32_t& fph = acc ? full_ph1 : full_ph0;
+                ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), fph, abort);
+                if (!ok) break;
+                fph ^= 1u;
+                tc_fence_after();
+                const bool last_pass = pass == (dual ? 1 : 0);
+                __nv_bfloat16* yout = pass == 0 ? p.y : p.y2;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
-            for (int c = 0; c < BN / kEpiChunkCols; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(t_addr + (uint32_t)(c * kEpiChunkCols), r);
-                tmem_ld_wait();
-                if (c == BN / kEpiChunkCols - 1) {
-                    // accumulator fully read: hand it back to the MMA warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[acc]));
-                }
-                const int col0 = n * BN + c * kEpiChunkCols;
-                if (col0 >= p.N || row_base >= p.T) continue;   // nothing of this chunk is inside y
-                // the buffer we are about to overwrite must have been read by its earlier store
-                if (lane == 0) tma_store_wait_read<1>();
-                __syncwarp();
-                uint8_t* bp = buf_ptr0 + buf * kEpiBufBytes;
-                const uint32_t ba = buf_addr0 + (uint32_t)(buf * kEpiBufBytes);
-                // row = lane: 64 bytes, four 16-byte chunks, 64-byte swizzle (chunk ^= (row >> 1) & 3)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                    v.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                    v.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                    v.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                    const int phys = j ^ ((lane >> 1) & 3);
-                    *reinterpret_cast<uint4*>(bp + lane * 64 + phys * 16) = v;
-                }
-                if (!scatter) {
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmap_y, ba, col0, row_base);
-                        tma_store_commit();
+                for (int c = 0; c < BN / kEpiChunkCols; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_addr + (uint32_t)(c * kEpiChunkCols), r);
+                    tmem_ld_wait();
+                    if (c == BN / kEpiChunkCols - 1) {
+                        // accumulator fully read: hand it back to the MMA warp (for the tile's second
+                        // output, or for the next tile)
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(last_pass ? &ctrl->tmem_empty[acc] : &ctrl->tmem_read1[acc]));
                     }
-                } else {
+                    const int col0 = n * BN + c * kEpiChunkCols;
+                    if (col0 >= p.N || row_base >= p.T) continue;   // nothing of this chunk is inside y
+                    // the buffer we are about to overwrite must have been read by its earlier store
+                    if (lane == 0) tma_store_wait_read<1>();
                     __syncwarp();
-                    // scatter: 4 lanes write one 64-byte row piece; 8 rows per pass
+                    uint8_t* bp = buf_ptr0 + buf * kEpiBufBytes;
+                    const uint32_t ba = buf_addr0 + (uint32_t)(buf * kEpiBufBytes);
+                    // row = lane: 64 bytes, four 16-byte chunks, 64-byte swizzle (chunk ^= (row >> 1) & 3)
 #pragma unroll
-                    for (int pass = 0; pass < 4; ++pass) {
-                        const int rr = pass * 8 + (lane >> 2), j = lane & 3;
-                        const int pos = row_base + rr;
-                        if (pos < p.T && col0 + j * 8 < p.N) {
-                            const int row = __ldg(p.perm + pos);
-                            if (row >= 0 && row < p.T) {
-                                const int phys = j ^ ((rr >> 1) & 3);
-                                uint4 v = *reinterpret_cast<const uint4*>(bp + rr * 64 + phys * 16);
-                                *reinterpret_cast<uint4*>(p.y + (size_t)row * p.N + col0 + j * 8) = v;
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
+                        v.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                        v.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                        v.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                        const int phys = j ^ ((lane >> 1) & 3);
+                        *reinterpret_cast<uint4*>(bp + lane * 64 + phys * 16) = v;
+                    }
+                    if (!scatter) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            // two call sites on purpose: each names its tensor map as a kernel-parameter constant
+                            if (pass == 0) tma_store_2d(&tmap_y, ba, col0, row_base);
+                            else tma_store_2d(&tmap_y2, ba, col0, row_base);
+                            tma_store_commit();
+                        }
+                    } else {
+                        __syncwarp();
+                        // scatter: 4 lanes write one 64-byte row piece; 8 rows per pass
+#pragma unroll
+                        for (int sp = 0; sp < 4; ++sp) {
+                            const int rr = sp * 8 + (lane >> 2), j = lane & 3;
+                            const int pos = row_base + rr;
+                            if (pos < p.T && col0 + j * 8 < p.N) {
+                                const int row = __ldg(p.perm + pos);
+                                if (row >= 0 && row < p.T) {
+                                    const int phys = j ^ ((rr >> 1) & 3);
+                                    uint4 v = *reinterpret_cast<const uint4*>(bp + rr * 64 + phys * 16);
+                                    *reinterpret_cast<uint4*>(yout + (size_t)row * p.N + col0 + j * 8) = v;
+                                }
                             }
                         }
+                        __syncwarp();
                     }
-                    __syncwarp();
+                    buf ^= 1;
                 }
-                buf ^= 1;
             }
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            acc ^= 1;
         }
         if (lane == 0) tma_store_wait_all();
     }
@@ -734,13 +850,17 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     const int num_m = (a.T + kBM - 1) / kBM;
     const int num_n = (a.d_out + bn - 1) / bn;
     const uint32_t w_box_rows = pairs ? (uint32_t)(kPairBN / 2) : (uint32_t)bn;
-    CUtensorMap tx, tx0, tw, tu, ty, tb = tmap_B;
+    const bool dual = a.slot_ids2 != nullptr;
+    if (dual && (pairs || a.G <= 0 || !a.y2)) return cudaErrorInvalidValue;
+    CUtensorMap tx, tx0, tw, tu, ty, ty2, tb = tmap_B;
     if (!encode_tmap_2d(&tx, a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
     if (!encode_tmap_2d(&tx0, a.x_in_place ? a.x_in_place : a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
     if (!encode_tmap_2d(&tw, a.W0, (uint64_t)a.d_in, (uint64_t)a.d_out, (uint64_t)a.d_in * 2, kBK, w_box_rows)) return cudaErrorInvalidValue;
-    const uint64_t u_rows = (uint64_t)(num_m + (a.G > 0 ? a.G : 1)) * kBM;
+    const uint64_t u_set_rows = (uint64_t)(num_m + (a.G > 0 ? a.G : 1)) * kBM;
+    const uint64_t u_rows = u_set_rows * (dual ? 3 : 1);
     if (!encode_tmap_2d(&tu, a.u_blocks, kRankPad, u_rows, kRankPad * 2, kBK, kBM)) return cudaErrorInvalidValue;
     if (!encode_tmap_2d(&ty, a.y, (uint64_t)a.d_out, (uint64_t)a.T, (uint64_t)a.d_out * 2, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
+    if (!encode_tmap_2d(&ty2, dual ? a.y2 : a.y, (uint64_t)a.d_out, (uint64_t)a.T, (uint64_t)a.d_out * 2, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
     if (pairs || bn != 256) {
         if (!encode_tmap_3d(&tb, ar.B, kRankPad, (uint64_t)a.d_out, (uint64_t)snap.max_slots, kRankPad * 2,
                             (uint64_t)a.d_out * kRankPad * 2, kBK, w_box_rows, 1)) return cudaErrorInvalidValue;
@@ -749,6 +869,7 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     p.seg_offsets = a.seg_offsets; p.slot_ids = a.slot_ids; p.perm = a.perm; p.plan = a.plan;
     p.tile_identity = pairs ? nullptr : a.tile_identity;
     p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
+    p.slot_ids2 = a.slot_ids2; p.y2 = (__nv_bfloat16*)a.y2; p.u_set_rows = (int)u_set_rows;
     p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kGemmThreads);
@@ -778,8 +899,8 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
-    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, snap, p);
-    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, snap, p);
+    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
+    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
 }
 
 }  // namespace lml

@@ -55,7 +55,8 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                  const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                 __nv_bfloat16* u_blocks, cudaStream_t stream);
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained = false,   // chained: a further pass of the same call, may run beside the one before
+                                 __nv_bfloat16* u_blocks_neg = nullptr);                              // optional second copy of the blocks, negated
 
 // tile_identity[m] = 1: tile m's perm is the identity, its rows were not copied and stay in place.
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
@@ -73,6 +74,8 @@ struct GemmArgs {
     const int32_t* slot_ids;
     const PlanWord* plan;
     const __nv_bfloat16* u_blocks;
+    const int32_t* slot_ids2 = nullptr;   // dual form: second slot per segment; u_blocks then holds three sets of
+    void* y2 = nullptr;                   // (num_m + G) blocks: first slots, second slots, first slots negated
     int T, d_in, d_out, G;
     int num_sms;
     bool overlap_with_previous;   // launch as a programmatic dependent of the shrink kernel before it

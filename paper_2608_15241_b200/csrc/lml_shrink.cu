@@ -43,10 +43,14 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     uint32_t* __restrict__ status, const __nv_bfloat16* __restrict__ x, int T, int K,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids, int G,
     const __nv_bfloat16* __restrict__ x_in_place, const int32_t* __restrict__ tile_identity,
-    PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles)
+    PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles, int chained,
+    __nv_bfloat16* __restrict__ u_blocks_neg)   // optional second copy of the blocks with the sign flipped
 {
     // Launched with a full dependency on the work before it, so nothing to wait for; the GEMM that
-    // follows may start its main loop right away.
+    // follows may start its main loop right away.  (chained: this is a further shrink pass of the same
+    // call, launched as a programmatic dependent of the first, which had that full dependency: the
+    // passes run side by side.  One CTA then stays until the pass before is complete, so that whoever
+    // waits for this grid has waited for all of them.)
     ptx::grid_launch_dependents();
     extern __shared__ float shrink_smem[];
     using S = ShrinkSmem<NB>;
@@ -61,6 +65,7 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
 
     // One CTA validates the segment arrays for the whole call.
     if (b == 0 && sub == 0 && ks == 0) {
+        if (chained && tid == 0) ptx::grid_dependency_wait();
         int bad_off = 0, bad_slot = 0;
         for (int g = tid; g < G; g += blockDim.x) {
             int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
@@ -107,9 +112,13 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     const int nblk = ((int)snap.rank[slot] + 7) >> 3;
     const int p0 = m * kTileM + sub * kShrinkRows;
     uint4* out = reinterpret_cast<uint4*>(u_blocks + ((size_t)b * kTileM + sub * kShrinkRows) * kRankPad);
+    uint4* out_neg = u_blocks_neg ? reinterpret_cast<uint4*>(u_blocks_neg + ((size_t)b * kTileM + sub * kShrinkRows) * kRankPad) : nullptr;
 
     if (p0 + kShrinkRows <= plo || p0 >= phi) {   // no row of this slab is in the piece
-        if (ks == 0) out[tid] = make_uint4(0, 0, 0, 0);   // 32 rows x 128 B = 256 x 16 B
+        if (ks == 0) {   // 32 rows x 128 B = 256 x 16 B
+            out[tid] = make_uint4(0, 0, 0, 0);
+            if (out_neg) out_neg[tid] = make_uint4(0, 0, 0, 0);
+        }
         return;
     }
 
@@ -201,6 +210,7 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
         o.x = pack_bf16(v[0] * sc, v[1] * sc); o.y = pack_bf16(v[2] * sc, v[3] * sc);
         o.z = pack_bf16(v[4] * sc, v[5] * sc); o.w = pack_bf16(v[6] * sc, v[7] * sc);
         out[row * 8 + (tid & 7)] = o;
+        if (out_neg) out_neg[row * 8 + (tid & 7)] = make_uint4(o.x ^ 0x80008000u, o.y ^ 0x80008000u, o.z ^ 0x80008000u, o.w ^ 0x80008000u);
     }
     cluster.sync();   // peers stay alive until their partials have been read
 }
@@ -209,7 +219,7 @@ template <int NB>
 static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
                                     const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                     const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                    __nv_bfloat16* u_blocks, cudaStream_t stream)
+                                    __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
 {
     const int num_tiles = (T + kTileM - 1) / kTileM;
     int ks = (d_in + 1023) / 1024;
@@ -219,19 +229,21 @@ static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, c
     cfg.blockDim = dim3(kShrinkWarps * 32);
     cfg.dynamicSmemBytes = ShrinkSmem<NB>::kBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = ks;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = chained ? 2 : 1;
     const __nv_bfloat16* arenaA = ar.A;
     uint32_t* status = ar.status;
     const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
     const __nv_bfloat16* xip = (const __nv_bfloat16*)x_in_place;
     return cudaLaunchKernelEx(&cfg, shrink_pieces_kernel<NB>, snap, arenaA, status, xb, T, d_in, seg_offsets,
-                              slot_ids, G, xip, tile_identity, plan, u_blocks, num_tiles);
+                              slot_ids, G, xip, tile_identity, plan, u_blocks, num_tiles, chained ? 1 : 0, u_blocks_neg);
 }
 
 cudaError_t shrink_init()
@@ -246,13 +258,13 @@ cudaError_t shrink_init()
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                  const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                 __nv_bfloat16* u_blocks, cudaStream_t stream)
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
 {
     int max_rank = 0;
     for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
     if (max_rank <= 16)
-        return launch_shrink_nb<2>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream);
-    return launch_shrink_nb<8>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream);
+        return launch_shrink_nb<2>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream, chained, u_blocks_neg);
+    return launch_shrink_nb<8>(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan, u_blocks, stream, chained, u_blocks_neg);
 }
 
 }  // namespace lml
