@@ -39,6 +39,7 @@ def _load():
         _lib = ctypes.CDLL(_LIB)
         _lib.lml_oracle_forward.restype = ctypes.c_int
         _lib.lml_oracle_forward_brute.restype = ctypes.c_int
+        _lib.lml_oracle_backward.restype = ctypes.c_int
         _lib.lml_oracle_segment.restype = ctypes.c_int
         _lib.lml_oracle_threads.restype = ctypes.c_int
     return _lib
@@ -115,6 +116,33 @@ def forward(x, W0, entries, seg_offsets, seg_entry, perm=None, positions=None, l
 def forward_workload(w, positions=None, nthreads: int = 0):
     return forward(w.x, w.W0, w.entries, w.seg_offsets, w.seg_entry, w.perm, positions,
                    nthreads=nthreads)
+
+
+def backward(x, dy, W0, entries, seg_offsets, seg_entry, perm=None, live=None):
+    """fp64 reference gradients of the layer.  Returns (dx [T, K], [dA_e [rank_e, K]], [dB_e [N, rank_e]], flags)."""
+    lib = _load()
+    x, dy, W0 = _u16(x), _u16(dy), _u16(W0)
+    T, K = x.shape
+    N = W0.shape[0]
+    assert W0.shape == (N, K) and dy.shape == (T, N)
+    Ap, Bp, rank, scale, keep = _entry_arrays(entries, K, N)
+    ne = len(entries)
+    live_a = np.ones(max(ne, 1), dtype=np.int32) if live is None else _i32(live)
+    so, se = _i32(seg_offsets), _i32(seg_entry)
+    pm = None if perm is None else _i32(perm)
+    dx = np.zeros((T, K), dtype=np.float64)
+    dA = [np.zeros((e.rank, K), dtype=np.float64) for e in entries]
+    dB = [np.zeros((N, e.rank), dtype=np.float64) for e in entries]
+    PP = ctypes.c_void_p * max(ne, 1)
+    dAp = PP(*[a.ctypes.data for a in dA]) if ne else PP()
+    dBp = PP(*[b.ctypes.data for b in dB]) if ne else PP()
+    flags = ctypes.c_uint32(0)
+    rc = lib.lml_oracle_backward(_p(x), _p(dy), _p(W0), T, K, N, ne, Ap, Bp, _p(rank), _p(scale), _p(live_a),
+                                 int(se.shape[0]), _p(so), _p(se), _p(pm), _p(dx), dAp, dBp, ctypes.byref(flags))
+    del keep
+    if rc != 0:
+        raise ValueError("lml_oracle_backward: bad argument")
+    return dx, dA, dB, int(flags.value)
 
 
 def forward_brute(x, W0, entries, seg_offsets, seg_entry, perm=None):

@@ -22,6 +22,10 @@
  * agreement with the merged weight W0 + s*A*B formed by numpy in float64, exact row
  * permutation under segment permutation, closed forms for constant inputs, one-hot inputs,
  * a hand-worked 2x2 example, an integer-lattice case, and the brute-force twin below.
+ * The backward pass (lml_oracle_backward, the gradients of the training task) is pinned in
+ * tests/test_oracle_backward_pins.py: central differences of the forward oracle in every
+ * coordinate of x, A and B, a hand-worked rank-one example, the matrix identities formed by
+ * numpy in float64, and structural cases (unbound rows, unused and repeated entries).
  */
 #include <stdint.h>
 #include <stddef.h>
@@ -211,6 +215,84 @@ int lml_oracle_segment(const int32_t *token_entry, int T, int num_entries, int32
         }
     }
     *num_segs = segs;
+    if (flags_out) *flags_out = flags;
+    return 0;
+}
+
+/*
+ * Backward pass of the layer for the training task (Section 3.1: adapters are trained in the
+ * background; Section 4.1: the training step is one of the tasks that share the GPU).  With
+ *     y[t] = x[t].W0^T + s_e (x[t].A_e^T).B_e^T          (e = entry of the position of row t)
+ * and an upstream gradient dy [T][N] (bf16 like every activation), the definitions are
+ *     dx[t]     = dy[t].W0 + s_e (dy[t].B_e).A_e
+ *     dA_e[j][k] = s_e sum_{t bound to e} (dy[t].B_e)[j] x[t][k]
+ *     dB_e[n][j] = s_e sum_{t bound to e} dy[t][n] (x[t].A_e^T)[j]
+ * written out as plain loops in double precision.  dx64 is [T][K]; dA64[e] is [rank_e][K] and
+ * dB64[e] is [N][rank_e], both overwritten (zero for entries no token is bound to).  Any of the
+ * three output arguments may be NULL.  Rows are addressed as in the forward pass (perm).
+ * Positions bound to a dead or out-of-range entry count as unbound (flag); malformed offsets:
+ * flag set, every row unbound.  Returns 0, or -1 on a null / negative argument.
+ */
+int lml_oracle_backward(const uint16_t *x, const uint16_t *dy, const uint16_t *W0, int T, int K, int N,
+                        int num_entries, const uint16_t *const *A, const uint16_t *const *B,
+                        const int32_t *rank, const float *scale, const int32_t *live,
+                        int G, const int32_t *seg_offsets, const int32_t *seg_entry,
+                        const int32_t *perm, double *dx64, double *const *dA64, double *const *dB64,
+                        uint32_t *flags_out)
+{
+    if (T < 0 || K < 0 || N < 0 || G < 0 || num_entries < 0) return -1;
+    if (T > 0 && (!x || !dy || !W0)) return -1;
+    uint32_t flags = 0;
+    int use_lora = 1;
+    if (!offsets_ok(T, G, seg_offsets)) {
+        flags |= ORC_FLAG_BAD_OFFSETS;
+        use_lora = 0;
+    }
+    for (int e = 0; e < num_entries; ++e) {
+        if (dA64 && dA64[e]) for (size_t i = 0; i < (size_t)rank[e] * K; ++i) dA64[e][i] = 0.0;
+        if (dB64 && dB64[e]) for (size_t i = 0; i < (size_t)N * rank[e]; ++i) dB64[e][i] = 0.0;
+    }
+    for (int p = 0; p < T; ++p) {
+        int t = perm ? perm[p] : p;
+        const uint16_t *xr = x + (size_t)t * K;
+        const uint16_t *gr = dy + (size_t)t * N;
+        int e = use_lora ? entry_of_position(p, G, seg_offsets, seg_entry, num_entries, live, &flags) : -1;
+        if (dx64) {
+            double *dxr = dx64 + (size_t)t * K;
+            for (int k = 0; k < K; ++k) {
+                double acc = 0.0;
+                for (int n = 0; n < N; ++n) acc += bf16_to_f64(gr[n]) * bf16_to_f64(W0[(size_t)n * K + k]);
+                dxr[k] = acc;
+            }
+        }
+        if (e < 0) continue;
+        int r = rank[e];
+        if (r > 256) r = 256;
+        double s = (double)scale[e];
+        double g[256], h[256];
+        for (int j = 0; j < r; ++j) {
+            double acc = 0.0;
+            for (int n = 0; n < N; ++n) acc += bf16_to_f64(gr[n]) * bf16_to_f64(B[e][(size_t)n * rank[e] + j]);
+            g[j] = acc;                       /* (dy.B)[j] */
+            acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += bf16_to_f64(xr[k]) * bf16_to_f64(A[e][(size_t)j * K + k]);
+            h[j] = acc;                       /* (x.A^T)[j] */
+        }
+        if (dx64) {
+            double *dxr = dx64 + (size_t)t * K;
+            for (int k = 0; k < K; ++k) {
+                double acc = 0.0;
+                for (int j = 0; j < r; ++j) acc += g[j] * bf16_to_f64(A[e][(size_t)j * K + k]);
+                dxr[k] += s * acc;
+            }
+        }
+        if (dA64 && dA64[e])
+            for (int j = 0; j < r; ++j)
+                for (int k = 0; k < K; ++k) dA64[e][(size_t)j * K + k] += s * g[j] * bf16_to_f64(xr[k]);
+        if (dB64 && dB64[e])
+            for (int n = 0; n < N; ++n)
+                for (int j = 0; j < r; ++j) dB64[e][(size_t)n * rank[e] + j] += s * bf16_to_f64(gr[n]) * h[j];
+    }
     if (flags_out) *flags_out = flags;
     return 0;
 }
