@@ -222,9 +222,56 @@ class Rotation:
             n += t.last_launch_count()
         return n
 
+    def prepare_backward(self):
+        """Transposed tables (for dx), an upstream gradient and gradient buffers for the backward pass."""
+        import torch
+        from paper_2608_15241_b200.binding import Table, lml_backward_workspace_bytes
+        w = self.w
+        dev = lambda b: torch.from_numpy(np.ascontiguousarray(b).view(np.int16)).view(torch.bfloat16).to(self.device)
+        from paper_2608_15241_b200 import workloads as wl
+        dy0 = dev(wl.normal_bf16(4242, 1, (w.T, w.d_out), 1.0))
+        A0 = [dev(e.A) for e in w.entries]
+        B0 = [dev(e.B) for e in w.entries]
+        for i, s in enumerate(self.sets):
+            tT = Table(w.d_out, w.d_in, max_slots=len(w.entries), device=torch.device(self.device).index or 0)
+            roll = lambda t: t if i == 0 else torch.roll(t, shifts=i, dims=0).contiguous()
+            slots_T = [tT.register_adapter_transposed(e.adapter_id, e.version, roll(a), roll(b), e.scale)
+                       for e, a, b in zip(w.entries, A0, B0)]
+            s["table_T"] = tT
+            s["ids_T"] = torch.from_numpy(np.array([slots_T[e] if e >= 0 else -1 for e in w.seg_entry], np.int32)).to(self.device)
+            s["W0T"] = s["W0"].t().contiguous()
+            s["dy"] = roll(dy0)
+            s["dx"] = torch.empty((w.T, w.d_in), dtype=torch.bfloat16, device=self.device)
+            s["dA"] = torch.zeros((tT.max_slots, 64, w.d_in), dtype=torch.float32, device=self.device)
+            s["dB"] = torch.zeros((tT.max_slots, w.d_out, 64), dtype=torch.float32, device=self.device)
+            s["ws_bwd"] = torch.empty(max(lml_backward_workspace_bytes(s["table"].handle, w.T, w.G),
+                                          tT.workspace_bytes(w.T, w.G)), dtype=torch.uint8, device=self.device)
+        torch.cuda.synchronize()
+
+    def backward_dx(self, i):
+        """dx = dy.W0 + s (dy.B).A: the layer on the transposed table."""
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        t = s["table_T"]
+        b.lora_mixed_linear(t.handle, s["dy"].data_ptr(), s["W0T"].data_ptr(), self.w.T, s["so_pre"].data_ptr(),
+                            s["ids_T"].data_ptr(), self.w.G, 0, s["dx"].data_ptr(), s["ws_bwd"].data_ptr(),
+                            s["ws_bwd"].numel(), b._stream(None))
+        return t.last_launch_count()
+
+    def backward_adapters(self, i):
+        from paper_2608_15241_b200 import binding as b
+        s = self.sets[i % self.R]
+        b.lora_mixed_linear_backward_adapters(s["table"].handle, s["table_T"].handle, s["x"].data_ptr(), s["dy"].data_ptr(),
+                                              self.w.T, s["so_pre"].data_ptr(), s["ids_pre"].data_ptr(),
+                                              s["ids_T"].data_ptr(), self.w.G, s["dA"].data_ptr(), s["dB"].data_ptr(),
+                                              s["ws_bwd"].data_ptr(), s["ws_bwd"].numel(), b._stream(None))
+        return s["table"].last_launch_count()
+
     def close(self):
         for s in self.sets:
             s["table"].close()
+            if "table_T" in s:
+                s["table_T"].close()
 
 
 def timed_graph_loop(fn, R, steps, warmup, stream, min_warm_seconds=0.0):
@@ -387,6 +434,14 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
         d_secs, _, _ = timed_graph_loop(rot.dual_only, rot.R, dsteps, 3, stream)
         t_secs, _, _ = timed_graph_loop(rot.two_singles, rot.R, dsteps, 3, stream)
         dual = {"us_per_call": d_secs / dsteps * 1e6, "two_single_calls_us": t_secs / dsteps * 1e6}
+    backward = None
+    if kind != "decode" and w.G >= 1 and w.perm is None:
+        # the training task's pass through the layer: dx (the layer on the transposed table) and the adapter gradients
+        rot.prepare_backward()
+        bsteps = max(rot.R, min(steps, 100))
+        x_secs, _, _ = timed_graph_loop(rot.backward_dx, rot.R, bsteps, 3, stream)
+        a_secs, _, _ = timed_graph_loop(rot.backward_adapters, rot.R, bsteps, 3, stream)
+        backward = {"dx_us": x_secs / bsteps * 1e6, "adapter_gradients_us": a_secs / bsteps * 1e6}
     roof["traffic"] = ncu_traffic(name)
     roof["algorithmic"] = w.bytes() if kind == "decode" else w.flops()
     esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
@@ -404,6 +459,8 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                       "timing": "CUDA-graph replay of R-step chunks, CUDA events on the launch stream"}}
     if dual:
         out["dual_version_call"] = dual
+    if backward:
+        out["backward"] = backward
     if want_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(w, kind, spec["unit"], budget_s=6.0)
         out["parity_sample"] = sampled_parity(rot)

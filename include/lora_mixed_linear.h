@@ -219,6 +219,33 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
                                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Backward pass of the layer, for the training task that shares the GPU with inference (Section 3.1,
+ * Section 4.1).  With y = x.W0^T + s (x.A^T).B^T per segment and an upstream gradient dy [T][d_out]:
+ *
+ *   dx = dy.W0 + s (dy.B).A  is the layer itself on the transposed problem: a second table t_T with
+ *   d_in = d_out(t), d_out = d_in(t), the caller's W0^T [d_in][d_out] as base weight and every adapter
+ *   registered with register_adapter_transposed (which stores B^T as "A" and A^T as "B").  Call
+ *   lora_mixed_linear(t_T, dy, W0T, ...) with the slots of t_T: same kernels, same accuracy.
+ *
+ *   lora_mixed_linear_backward_adapters adds the adapter gradients of one batch onto dA and dB:
+ *     dA[slot][j][k] += s sum_t (dy.B)[t][j] x[t][k],  float32 [max_slots(t)][64][d_in], rows j >= rank untouched
+ *     dB[slot][n][j] += s sum_t dy[t][n] (x.A^T)[t][j], float32 [max_slots(t)][d_out][64], columns j >= rank untouched
+ *   over the tokens t of the segments bound to the slot (slot numbering of t).  The two small
+ *   products (x.A^T and dy.B) go through the shrink kernels and are rounded to bf16 before the
+ *   sums, which run in fp32 in a fixed order.  x, dy: device bf16, rows in segment order (no perm).
+ *   slot_ids / slot_ids_T: device int32[G], the slot of every segment in t and in t_T (-1 = none,
+ *   both).  The caller zeroes dA and dB at the start of a step; several calls accumulate.
+ *   workspace: lml_backward_workspace_bytes(t, T, G).  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+lml_status register_adapter_transposed(lml_table* t_T, int adapter_id, int version, const void* A, const void* B,
+                                       int rank, float scale, void* stream, int* slot_out);
+size_t lml_backward_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
+lml_status lora_mixed_linear_backward_adapters(lml_table* t, lml_table* t_T, const void* x, const void* dy, int T,
+                                               const int32_t* seg_offsets, const int32_t* slot_ids,
+                                               const int32_t* slot_ids_T, int G, float* dA, float* dB,
+                                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * lora_mixed_linear_tokens — segmentation and layer in one call, for callers that hold one slot id
  * per token (what a scheduler hands a decode step).  token_slots: device int32[T], physical slot
  * per row of x or -1; ids outside [-1, max_slots) or naming a free slot count as -1 and set

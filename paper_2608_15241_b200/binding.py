@@ -32,7 +32,8 @@ EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "regist
            "lora_mixed_linear_decode_static", "lml_tokens_workspace_bytes", "lora_mixed_linear_tokens",
            "lml_publish", "lml_pin", "lml_unpin", "lml_resolve", "lml_slot_state",
            "lml_segment_tokens_adapters", "lora_mixed_linear_adapters",
-           "lml_dual_workspace_bytes", "lora_mixed_linear_dual")
+           "lml_dual_workspace_bytes", "lora_mixed_linear_dual", "register_adapter_transposed",
+           "lml_backward_workspace_bytes", "lora_mixed_linear_backward_adapters")
 
 
 class LmlError(RuntimeError):
@@ -75,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.lora_mixed_linear_tokens.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lora_mixed_linear_adapters.argtypes = [vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lml_segment_tokens_adapters.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.register_adapter_transposed.argtypes = [vp, i32, i32, vp, vp, i32, ctypes.c_float, vp, ctypes.POINTER(i32)]
+        L.lml_backward_workspace_bytes.restype = sz
+        L.lml_backward_workspace_bytes.argtypes = [vp, i32, i32]
+        L.lora_mixed_linear_backward_adapters.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.lml_dual_workspace_bytes.restype = sz
         L.lml_dual_workspace_bytes.argtypes = [vp, i32, i32]
         L.lora_mixed_linear_dual.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
@@ -87,7 +92,7 @@ def lib() -> ctypes.CDLL:
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
             if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes",
-                            "lml_tokens_workspace_bytes", "lml_dual_workspace_bytes"):
+                            "lml_tokens_workspace_bytes", "lml_dual_workspace_bytes", "lml_backward_workspace_bytes"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -177,6 +182,28 @@ def lora_mixed_linear_tokens(table: int, x_ptr: int, W0_ptr: int, T: int, token_
     """Segmentation and layer in one call: one slot id per token instead of segments."""
     _check(lib().lora_mixed_linear_tokens(table, x_ptr, W0_ptr, T, token_slots_ptr, y_ptr, workspace_ptr,
                                           workspace_bytes, stream), "lora_mixed_linear_tokens")
+
+
+def register_adapter_transposed(table_T: int, adapter_id: int, version: int, A_ptr: int, B_ptr: int, rank: int,
+                                scale: float, stream: int = 0) -> int:
+    """Register the forward adapter (A [rank][K], B [N][rank]) in the transposed table (d_in = N, d_out = K)."""
+    slot = ctypes.c_int32(-1)
+    _check(lib().register_adapter_transposed(table_T, adapter_id, version, A_ptr, B_ptr, rank, scale, stream,
+                                             ctypes.byref(slot)), "register_adapter_transposed")
+    return int(slot.value)
+
+
+def lml_backward_workspace_bytes(table: int, max_tokens: int, max_segments: int) -> int:
+    return int(lib().lml_backward_workspace_bytes(table, max_tokens, max_segments))
+
+
+def lora_mixed_linear_backward_adapters(table: int, table_T: int, x_ptr: int, dy_ptr: int, T: int, seg_offsets_ptr: int,
+                                        slot_ids_ptr: int, slot_ids_T_ptr: int, G: int, dA_ptr: int, dB_ptr: int,
+                                        workspace_ptr: int, workspace_bytes: int, stream: int = 0) -> None:
+    """dA, dB (fp32, packed like the arena) += this batch's adapter gradients."""
+    _check(lib().lora_mixed_linear_backward_adapters(table, table_T, x_ptr, dy_ptr, T, seg_offsets_ptr, slot_ids_ptr,
+                                                     slot_ids_T_ptr, G, dA_ptr, dB_ptr, workspace_ptr, workspace_bytes,
+                                                     stream), "lora_mixed_linear_backward_adapters")
 
 
 def lml_dual_workspace_bytes(table: int, max_tokens: int, max_segments: int) -> int:
@@ -388,6 +415,24 @@ class Table:
 
     def slot_state(self, slot: int):
         return lml_slot_state(self.handle, slot)
+
+    def register_adapter_transposed(self, adapter_id: int, version: int, A, B, scale: float, stream=None) -> int:
+        """On the TRANSPOSED table (d_in = N, d_out = K): A [rank][K], B [N][rank] of the forward layer."""
+        rank = int(A.shape[0])
+        assert A.shape[1] == self.d_out and B.shape == (self.d_in, rank)
+        return register_adapter_transposed(self.handle, adapter_id, version, _ptr(A), _ptr(B), rank, float(scale),
+                                           _stream(stream))
+
+    def backward_adapters(self, table_T, x, dy, seg_offsets, slot_ids, slot_ids_T, dA, dB, stream=None):
+        """dA fp32 [max_slots][64][d_in], dB fp32 [max_slots][d_out][64] += gradients of this batch."""
+        import torch
+        T, G = int(x.shape[0]), int(slot_ids.shape[0])
+        assert dA.dtype == torch.float32 and dB.dtype == torch.float32
+        assert tuple(dA.shape) == (self.max_slots, 64, self.d_in) and tuple(dB.shape) == (self.max_slots, self.d_out, 64)
+        ws = torch.empty(max(lml_backward_workspace_bytes(self.handle, T, G), 256), dtype=torch.uint8, device=x.device)
+        lora_mixed_linear_backward_adapters(self.handle, table_T.handle, _ptr(x), _ptr(dy), T, _ptr(seg_offsets),
+                                            _ptr(slot_ids), _ptr(slot_ids_T), G, _ptr(dA), _ptr(dB), _ptr(ws),
+                                            int(ws.numel()), _stream(stream))
 
     def lora_mixed_linear_dual(self, x, W0, seg_offsets, slot_ids_a, slot_ids_b, perm=None, stream=None):
         """-> (y_a, y_b): the layer under two slot bindings of the same segments."""

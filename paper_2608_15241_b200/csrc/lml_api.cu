@@ -137,6 +137,35 @@ lml_status register_adapter(lml_table* t, int adapter_id, int version, const voi
     return LML_OK;
 }
 
+lml_status register_adapter_transposed(lml_table* t_T, int adapter_id, int version, const void* A, const void* B, int rank,
+                                       float scale, void* stream, int* slot_out)
+{
+    // A [rank][K], B [N][rank] are the FORWARD layer's matrices; t_T has d_in = N and d_out = K
+    if (!t_T || !A || !B || !slot_out || rank < 1 || rank > LML_MAX_RANK || !aligned16(A) || !aligned16(B) || !(scale == scale))
+        return LML_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(t_T->mu);
+    int free_slot = -1;
+    for (int i = 0; i < t_T->max_slots; ++i) {
+        const auto& e = t_T->entries[i];
+        if (e.live && e.adapter_id == adapter_id && e.version == version) return LML_ERR_DUPLICATE;
+        if (!e.live && free_slot < 0) free_slot = i;
+    }
+    if (free_slot < 0) return LML_ERR_TABLE_FULL;
+    DeviceGuard guard(t_T->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    if (launch_pack_adapter_transposed(t_T->arena, free_slot, A, B, rank, /*K=*/t_T->d_out, /*N=*/t_T->d_in,
+                                       (cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
+    auto& e = t_T->entries[free_slot];
+    e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
+    e.state = LML_STATE_RESIDENT; e.pins = 0;
+    e.live = true;
+    *slot_out = free_slot;
+    return LML_OK;
+}
+
 lml_status retire_version(lml_table* t, int adapter_id, int version)
 {
     if (!t) return LML_ERR_INVALID_ARG;
@@ -431,6 +460,59 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
         e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
         if (e == cudaSuccess) ++launches;
     }
+    t->last_launches = launches;
+    if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    return LML_OK;
+}
+
+size_t lml_backward_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
+{
+    if (!t || max_tokens < 0 || max_segments < 0 || max_tokens > kMaxTokens) return 0;
+    return ws_layout(t, max_tokens, max_segments, 2).xg_off;
+}
+
+lml_status lora_mixed_linear_backward_adapters(lml_table* t, lml_table* t_T, const void* x, const void* dy, int T,
+                                               const int32_t* seg_offsets, const int32_t* slot_ids,
+                                               const int32_t* slot_ids_T, int G, float* dA, float* dB, void* workspace,
+                                               size_t workspace_bytes, void* stream_v)
+{
+    if (!t || !t_T || T < 0 || G < 1 || T > kMaxTokens || G > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (t_T->d_in != t->d_out || t_T->d_out != t->d_in || t_T->device != t->device) return LML_ERR_INVALID_ARG;
+    if (T == 0) { t->last_launches = 0; return LML_OK; }
+    if (!x || !dy || !seg_offsets || !slot_ids || !slot_ids_T || !dA || !dB || !aligned16(x) || !aligned16(dy) ||
+        !aligned16(dA) || !aligned16(dB))
+        return LML_ERR_INVALID_ARG;
+    const WsLayout ws = ws_layout(t, T, G, 2);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < ws.xg_off) return LML_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    const SlotSnapshot snap = snapshot_locked(t);
+    const SlotSnapshot snap_T = snapshot_locked(t_T);
+    DeviceGuard guard(t->device);
+    if (!guard.ok) return LML_ERR_CUDA;
+    uint8_t* wsb = static_cast<uint8_t*>(workspace);
+    PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
+    __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
+    const size_t num_m = (size_t)(T + kTileM - 1) / kTileM;
+    const size_t set_elems = (num_m + (size_t)G) * kTileM * kRankPad;
+    int launches = 0;
+    // set 0: scale.(x.A^T) per position (the forward shrink); set 1: scale.(dy.B), the same pass on the
+    // transposed table, whose "A" is B^T
+    cudaError_t e = launch_shrink_pieces(t->arena, snap, x, T, t->d_in, seg_offsets, slot_ids, G, x, nullptr, plan, u_blocks, stream);
+    if (e == cudaSuccess) {
+        ++launches;
+        e = launch_shrink_pieces(t_T->arena, snap_T, dy, T, t_T->d_in, seg_offsets, slot_ids_T, G, dy, nullptr, plan,
+                                 u_blocks + set_elems, stream);
+    }
+    if (e == cudaSuccess) {
+        ++launches;
+        // dA_s[j][k] += sum_t scale.(dy.B)[t][j] x[t][k];   dB_s[n][j] += sum_t dy[t][n] scale.(x.A^T)[t][j]
+        e = launch_weight_grad(snap, u_blocks + set_elems, x, T, t->d_in, seg_offsets, slot_ids, G, dA, 0, stream);
+    }
+    if (e == cudaSuccess) {
+        ++launches;
+        e = launch_weight_grad(snap, u_blocks, dy, T, t->d_out, seg_offsets, slot_ids, G, dB, 1, stream);
+    }
+    if (e == cudaSuccess) ++launches;
     t->last_launches = launches;
     if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
     return LML_OK;

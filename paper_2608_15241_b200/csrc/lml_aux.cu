@@ -203,4 +203,211 @@ cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_
                               tile_identity, allow_skip ? 1 : 0, status);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Transposed registration for the backward pass: the gradient with respect to x of the layer
+// (d_in = K, d_out = N, adapter A [r][K], B [N][r]) is the layer itself on the transposed problem
+// (d_in = N, d_out = K, base weight W0^T, adapter A' = B^T [r][N], B' = A^T [K][r]).  This kernel
+// packs (A', B') into the arena of the transposed table straight from the caller's A and B.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pack_adapter_transposed_kernel(__nv_bfloat16* __restrict__ dstA,
+                                                                      __nv_bfloat16* __restrict__ dstB,
+                                                                      const __nv_bfloat16* __restrict__ A,
+                                                                      const __nv_bfloat16* __restrict__ B,
+                                                                      int rank, int K, int N)
+{
+    const unsigned short* As = reinterpret_cast<const unsigned short*>(A);
+    const unsigned short* Bs = reinterpret_cast<const unsigned short*>(B);
+    unsigned short* Ad = reinterpret_cast<unsigned short*>(dstA);   // [64][N]: A'[j][n] = B[n][j]
+    unsigned short* Bd = reinterpret_cast<unsigned short*>(dstB);   // [K][64]: B'[k][j] = A[j][k]
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    for (long long i = tid; i < (long long)kRankPad * N; i += stride) {
+        const int j = (int)(i / N);
+        const long long n = i % N;
+        Ad[i] = j < rank ? Bs[n * rank + j] : (unsigned short)0;
+    }
+    for (long long i = tid; i < (long long)K * kRankPad; i += stride) {
+        const int j = (int)(i % kRankPad);
+        const long long k = i / kRankPad;
+        Bd[i] = j < rank ? As[(long long)j * K + k] : (unsigned short)0;
+    }
+}
+
+cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const void* A, const void* B, int rank,
+                                           int K, int N, cudaStream_t stream)
+{
+    __nv_bfloat16* dstA = arT.A + (size_t)slot * kRankPad * N;   // the transposed table has d_in = N ...
+    __nv_bfloat16* dstB = arT.B + (size_t)slot * K * kRankPad;   // ... and d_out = K
+    long long work = (long long)(K > N ? K : N) * kRankPad;
+    int blocks = (int)((work + 255) / 256);
+    if (blocks > 1184) blocks = 1184;
+    pack_adapter_transposed_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, (const __nv_bfloat16*)A,
+                                                               (const __nv_bfloat16*)B, rank, K, N);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Adapter gradients: out_s += P_s^T . Q_s over the tokens bound to slot s, where P holds one
+// 64-wide row per position (the piece blocks a shrink pass wrote: scale.(dy.B) for dA, scale.(x.A^T)
+// for dB) and Q is x (for dA, C = d_in) or dy (for dB, C = d_out).  One CTA per (256 columns, slot);
+// a thread owns one column and all 64 rows j of the output, walks the slot's positions in order and
+// keeps the sums in registers, so the result does not depend on scheduling.  fp32 accumulation, added
+// onto what out holds.  mode 0: out[slot][j][c] (dA);  mode 1: out[slot][c][j] (dB).
+// ---------------------------------------------------------------------------------------------
+constexpr int kGradCols = 256;                                  // columns of Q (and of the output) per CTA
+constexpr int kGradQPitch = kGradCols * 2 + 16;                 // bytes per row of the staged Q tile (16 more: no bank conflicts in ldmatrix)
+constexpr int kGradPPitch = kRankPad * 2 + 16;                  // bytes per row of the staged piece block
+constexpr int kGradQBytes = kTileM * kGradQPitch;
+constexpr int kGradPBytes = kTileM * kGradPPitch;
+constexpr int kGradSmemBytes = 2 * (kGradQBytes + kGradPBytes); // two work items in flight
+
+__device__ __forceinline__ void grad_cp_async_16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+
+// out_s (64 x C) += P_s^T (64 x positions) . Q_s (positions x C) on mma.sync m16n8k16: the contraction
+// runs over positions, 16 at a time.  P is staged as [position][j] and Q as [position][column], so both
+// operands are read with ldmatrix .trans.  Warp w owns columns 32w .. 32w+31 (four 8-wide tiles) and all
+// 16-row groups of j that the slot's rank needs.
+__global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant__ SlotSnapshot snap,
+                                                          const __nv_bfloat16* __restrict__ pieces,
+                                                          const __nv_bfloat16* __restrict__ Q, int T, int C,
+                                                          const int32_t* __restrict__ seg_offsets,
+                                                          const int32_t* __restrict__ slot_ids, int G,
+                                                          float* __restrict__ out, int mode)
+{
+    extern __shared__ __align__(16) unsigned char grad_smem[];
+    ptx::grid_dependency_wait();     // the shrink passes before this kernel are complete now
+    ptx::grid_launch_dependents();
+    const int slot = blockIdx.y;
+    const int rank = slot < snap.max_slots ? (int)snap.rank[slot] : 0;
+    if (rank == 0) return;
+    const int mtiles = (rank + 15) >> 4;   // 16-row groups of j
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c0 = blockIdx.x * kGradCols;
+    const int ncols = min(kGradCols, C - c0);
+    float acc[4][4][4];   // [16-row group of j][8-column tile][fragment]
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int n = 0; n < 4; ++n) acc[a][n][0] = acc[a][n][1] = acc[a][n][2] = acc[a][n][3] = 0.f;
+    const uint32_t smem = (uint32_t)__cvta_generic_to_shared(grad_smem);
+    auto q_off = [](int buf) { return (uint32_t)(buf * (kGradQBytes + kGradPBytes)); };
+    auto p_off = [](int buf) { return (uint32_t)(buf * (kGradQBytes + kGradPBytes) + kGradQBytes); };
+
+    // Work items of this CTA: the slot's segments in order, each tile of a segment in order.  A piece block
+    // (tile m, segment g) holds the rows of tile m that belong to g and zeros elsewhere, so the whole tile
+    // of Q is multiplied (rows past T are zero-filled here).  Block and tile are brought into shared memory
+    // by asynchronous copies, one item ahead of the arithmetic.
+    int g = -1, m = 0, m_last = -1;
+    auto advance = [&]() -> bool {   // next (g, m); false when the slot has no more
+        if (m < m_last) { ++m; return true; }
+        for (++g; g < G; ++g) {
+            if (__ldg(slot_ids + g) != slot) continue;
+            const int s0 = max(__ldg(seg_offsets + g), 0), s1 = min(__ldg(seg_offsets + g + 1), T);
+            if (s1 <= s0) continue;
+            m = s0 / kTileM;
+            m_last = (s1 - 1) / kTileM;
+            return true;
+        }
+        return false;
+    };
+    auto issue = [&](int buf) {
+        const char* blk = reinterpret_cast<const char*>(pieces + (size_t)(m + g) * kTileM * kRankPad);
+        for (int i = tid; i < kTileM * (kRankPad / 8); i += 256) {
+            const int r = i / (kRankPad / 8), ch = i % (kRankPad / 8);
+            grad_cp_async_16(smem + p_off(buf) + r * kGradPPitch + ch * 16, blk + (size_t)i * 16);
+        }
+        const int rows = min(kTileM, T - m * kTileM);
+        const int chunks = ncols / 8;   // 16-byte chunks per row
+        for (int i = tid; i < kTileM * chunks; i += 256) {
+            const int r = i / chunks, ch = i % chunks;
+            const uint32_t dst = smem + q_off(buf) + r * kGradQPitch + ch * 16;
+            if (r < rows) grad_cp_async_16(dst, Q + (size_t)(m * kTileM + r) * C + c0 + ch * 8);
+            else asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(dst), "r"(0u) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    bool have = advance();
+    int buf = 0;
+    if (have) issue(0);
+    while (have) {
+        const bool more = advance();
+        if (more) issue(buf ^ 1);
+        if (more) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();   // everybody's copies of the current item have landed
+        const uint32_t qb = smem + q_off(buf), pb = smem + p_off(buf);
+        // ldmatrix x4: lanes 0-7 address the rows of matrix 0, 8-15 of matrix 1, 16-23 of matrix 2, 24-31 of 3
+        const int mi = lane >> 3, rr = lane & 7;
+#pragma unroll 2
+        for (int ks = 0; ks < kTileM / 16; ++ks) {
+            const int p0 = ks * 16;
+            // B operand for the warp's four column tiles: matrices (p 0-7 | 8-15) x (tile 2h | tile 2h+1)
+            uint32_t bq[4][2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t addr = qb + (uint32_t)((p0 + (mi & 1) * 8 + rr) * kGradQPitch + (warp * 32 + h * 16 + (mi >> 1) * 8) * 2);
+                ldmatrix_x4_trans(addr, bq[2 * h][0], bq[2 * h][1], bq[2 * h + 1][0], bq[2 * h + 1][1]);
+            }
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                if (a < mtiles) {
+                    // A operand (j x p) from the block stored [p][j]: matrices (p 0-7, j 0-7), (p 0-7, j 8-15),
+                    // (p 8-15, j 0-7), (p 8-15, j 8-15) give a0..a3
+                    uint32_t a0, a1, a2, a3;
+                    const uint32_t addr = pb + (uint32_t)((p0 + (mi >> 1) * 8 + rr) * kGradPPitch + (a * 16 + (mi & 1) * 8) * 2);
+                    ldmatrix_x4_trans(addr, a0, a1, a2, a3);
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) mma_bf16_16816(acc[a][n], a0, a1, a2, a3, bq[n][0], bq[n][1]);
+                }
+            }
+        }
+        __syncthreads();   // the buffer may be refilled two items from now
+        have = more;
+        buf ^= 1;
+    }
+    // fragment: c0,c1 = (j = gq, columns 2tq, 2tq+1), c2,c3 = (j = gq + 8, same columns)
+    const int gq = lane >> 2, tq = lane & 3;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        if (a >= mtiles) continue;
+#pragma unroll
+        for (int n = 0; n < 4; ++n) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = a * 16 + gq + (e >> 1) * 8;
+                const int c = c0 + warp * 32 + n * 8 + tq * 2 + (e & 1);
+                if (j < rank && c < C) {
+                    float* o = mode == 0 ? out + ((size_t)slot * kRankPad + j) * C + c : out + ((size_t)slot * C + c) * kRankPad + j;
+                    *o += acc[a][n][e];
+                }
+            }
+        }
+    }
+}
+
+cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pieces, const void* Q, int T, int C,
+                               const int32_t* seg_offsets, const int32_t* slot_ids, int G, float* out, int mode,
+                               cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(weight_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGradSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    pdl_config(cfg, attr, dim3((C + kGradCols - 1) / kGradCols, snap.max_slots), dim3(256), kGradSmemBytes, stream);
+    return cudaLaunchKernelEx(&cfg, weight_grad_kernel, snap, pieces, (const __nv_bfloat16*)Q, T, C, seg_offsets, slot_ids, G,
+                              out, mode);
+}
+
 }  // namespace lml

@@ -45,6 +45,13 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
                                 int d_in, int d_out, cudaStream_t stream);
 
 cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream);
+// (A', B') = (B^T, A^T) of a forward adapter A [rank][K], B [N][rank] into slot `slot` of the transposed table's arena
+cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const void* A, const void* B, int rank,
+                                           int K, int N, cudaStream_t stream);
+// out_s += P_s^T . Q_s per slot (adapter gradients); mode 0: out[slot][j][c], mode 1: out[slot][c][j]
+cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pieces, const void* Q, int T, int C,
+                               const int32_t* seg_offsets, const int32_t* slot_ids, int G, float* out, int mode,
+                               cudaStream_t stream);
 cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
                                   int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
                                   cudaStream_t stream, bool by_adapter = false);   // by_adapter: the ids are adapter ids, resolved through ar.adapter_map
