@@ -509,6 +509,32 @@ def cpu_baseline(w, kind, unit, budget_s):
                       f"{secs * repeats:.1f} s wall on {cores} threads, scaled by rows"}
 
 
+def run_layer_sweep(device, peaks, steps):
+    """The decoder-layer sweep (three distinct projection shapes x five token counts), one cell after
+    the other: microseconds per call of lora_mixed_linear_tokens and the fraction of the bound that
+    holds for the cell (the slower of bytes / HBM peak and flops / tensor peak)."""
+    import torch
+    stream = torch.cuda.Stream(device=device)
+    cells = []
+    for proj, same_as in (("q", "q k v o"), ("gate", "gate up"), ("down", "down")):
+        for T in wl.SWEEP_TOKENS:
+            w = wl.layer_sweep(proj, T)
+            rot = Rotation(w, device, 3 * L2_BYTES)
+            n = max(rot.R, min(steps, 400 if T <= 16 else (100 if T <= 1024 else 30)))
+            secs, launches, _ = timed_graph_loop(rot.step, rot.R, n, 3 * rot.R, stream)
+            us = secs / n * 1e6
+            t_hbm = w.bytes() / (peaks["hbm"] * 1e9)
+            t_tensor = w.flops() / (peaks["tensor_burst"] * 1e12)
+            cells.append({"projections": same_as, "d_in": w.d_in, "d_out": w.d_out, "tokens": T, "segments": w.G,
+                          "us_per_call": us, "launches_per_call": launches // n, "GB/s": w.bytes() / secs * n / 1e9,
+                          "TFLOP/s": w.flops() / secs * n / 1e12, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
+                          "frac_of_bound": max(t_hbm, t_tensor) / (secs / n)})
+            rot.close()
+            del rot
+            torch.cuda.empty_cache()
+    return cells
+
+
 def run_reference(args):
     """The reference arm of this tier: the fp64 oracle on host cores, a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -559,7 +585,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=2000)
-    ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS) + ["layer_sweep"],
+                    help="layer_sweep: per-cell timings of the decoder-layer sweep (1 GPU, its own JSON line)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-secondary", action="store_true", help="skip the prefill line object")
     args = ap.parse_args()
@@ -585,6 +612,13 @@ def main():
     barrier()
     peaks = measured_peaks()
     warmup = max(3, args.warmup)
+    if args.workload == "layer_sweep":
+        if rank == 0:
+            print(json.dumps({"metric": "decoder-layer sweep, per-cell time of lora_mixed_linear_tokens", "unit": "us",
+                              "n_gpus": 1, "dtype": "bf16", "data": "synthetic", "peak_source": peaks["source"],
+                              "cells": run_layer_sweep(device, peaks, args.steps)}), flush=True)
+        barrier()
+        return
     primary = run_workload(args.workload, args.steps, warmup, device, world, peaks, rank == 0,
                            e2e_steps=max(3, min(args.steps, 200)))
     line = {"metric": primary.pop("metric"), "value": primary.pop("value"), "unit": primary.pop("unit"),

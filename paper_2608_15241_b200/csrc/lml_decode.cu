@@ -69,7 +69,8 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     int u_complete;
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecDotBytes;
+constexpr int kDecDeferBytes = 2048;   // base sums of rounds whose expand is put off: 16 x 32 or 2 x (8 x 32) fp32
+constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecDotBytes + kDecDeferBytes;
 // 196 KB is also the largest shared-memory carve-out that leaves the SM a useful L1 for the loads of x:
 // one step more and the base-only call is 0.8 us slower.
 static_assert(kDecSmemBytes + 1024 <= 200704, "shared memory budget");   // the system keeps 1 KB per CTA for itself
@@ -77,12 +78,12 @@ static_assert(kDecSmemBytes + 1024 <= 200704, "shared memory budget");   // the 
 struct DecCtrl {
     uint64_t full[kDecStages];
     uint64_t empty[kDecStages];
+    uint64_t ufull;      // the shrink warps' results (u, the slots, the copies of B) are in shared memory
     int abort;
     int bad_offsets;
     int slot_of_row[16];
-    int b_of_row[16];    // which block of the B copy in shared memory serves this row of x, -1: read B from global memory
-    int b_staged;        // blocks on their way into shared memory
-    uint64_t bfull;
+    int b_of_row[16];    // byte offset, in the staging buffer, of the B copy that serves this row of x; -1: read B from global memory
+    uint8_t b_lead[16];  // 1: this row of x is the first with its slot (it stands for the slot's block of B)
 };
 static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control block");
 
@@ -124,7 +125,10 @@ __device__ __forceinline__ void prefetch_l2(const void* p)
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
-template <bool kTwo>   // false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers
+// kTwo false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers.
+// kMulti: the CTAs have more than one round of rows; compiled with the code that saves reloads of x between rounds.
+// kPutOff: compiled with the code that puts the expand of early rounds off (kMulti calls with adapters).
+template <bool kTwo, bool kMulti, bool kPutOff>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
     const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
@@ -142,6 +146,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
     DecLookup* lk = reinterpret_cast<DecLookup*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
     uint8_t* dot_s = base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8;   // 16-byte aligned
+    float* defer_s = reinterpret_cast<float*>(dot_s + kDecDotBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
@@ -173,19 +178,20 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 mbar_init(smem_u32(&ctrl->full[s]), 1);
                 mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
             }
-            mbar_init(smem_u32(&ctrl->bfull), 1);
+            mbar_init(smem_u32(&ctrl->ufull), kDecShrinkWarps * 32);
             ctrl->abort = 0;
             ctrl->bad_offsets = 0;
-            ctrl->b_staged = 0;
             fence_mbar_init();
         }
-        if (lane < 16) { ctrl->slot_of_row[lane] = -1; ctrl->b_of_row[lane] = -1; }
+        if (lane < 16) { ctrl->slot_of_row[lane] = -1; ctrl->b_of_row[lane] = -1; ctrl->b_lead[lane] = 0; }
         asm volatile("bar.sync 4, %0;" ::"n"(kDecThreads) : "memory");   // the barriers are set up
         grid_launch_dependents();
         for (int round_begin = row_begin; round_begin < row_end && ok; round_begin += kDecRoundUnits * kDecUnitRows) {
             const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
             const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
-            for (int sp = 0; sp < nspans && ok; ++sp) {
+            const bool backwards = kMulti && (((round_begin - row_begin) / (kDecRoundUnits * kDecUnitRows)) & 1) != 0;
+            for (int si = 0; si < nspans && ok; ++si) {
+                const int sp = backwards ? nspans - 1 - si : si;   // (the consumers' order: see there)
                 const int k_begin = sp * kSpan;
                 const int span = min(kSpan, K - k_begin);
                 const int nchunks = (span + kDecChunk - 1) / kDecChunk;
@@ -214,6 +220,11 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
 
     const int gq = lane >> 2, tq = lane & 3;
     bool u_ready = false;
+    constexpr int kDecPerThread = kTwo ? 2 : 1;      // elements of y per consumer thread and round (16 x 32 or 8 x 32 over 256 threads)
+    constexpr int kDecDefer = kDecDeferBytes / (kDecPerThread * kDecConsumers * 32 * 4);   // rounds whose expand can be put off
+    static_assert(kDecRoundUnits * kDecUnitRows * (kTwo ? 16 : 8) <= kDecConsumers * 32 * kDecPerThread && kDecDefer >= 1, "elements per thread");
+    int ndefer = 0;
+    int span_loaded = -1;   // whose x fragments the registers hold
 
     // This warp's x fragments (chunk kc, k-steps warp*S .. warp*S+S-1 of a span) stay in registers.
     uint4 xa[kChunksPerSpan * kDecStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDecStepsPerChunk : 1];
@@ -391,6 +402,26 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                     lk->dot_end[lane] = end;
                     lk->rank_of_row[lane] = rank;
                 }
+                // The expand reads, per distinct slot, the first ceil(rank / 8) 16-byte chunks of this CTA's
+                // rows of B.  Those go into the staging buffer, chunk-major ([chunk][row]: consecutive
+                // threads of the epilogue read consecutive 16 bytes), one block per distinct slot as long
+                // as they fit; the first row of x with a slot stands for the slot's block.
+                const unsigned same = __match_any_sync(0xffffffffu, slot);
+                const int first = __ffs(same) - 1;
+                const bool leader = rank > 0 && first == lane;
+                const int chunks = leader ? (row_end - row_begin) * ((rank + 7) >> 3) : 0;
+                int base = chunks;
+#pragma unroll
+                for (int o = 1; o < 16; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, base, o);
+                    if (lane >= o) base += v;
+                }
+                const int fits = base * 16 <= kDecDotBytes;   // (inclusive end of this block)
+                const int my_off = __shfl_sync(0xffffffffu, fits ? (base - chunks) * 16 : -1, first);
+                if (lane < 16) {
+                    ctrl->b_of_row[lane] = rank > 0 ? my_off : -1;
+                    ctrl->b_lead[lane] = leader ? 1 : 0;
+                }
             }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
@@ -407,41 +438,28 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
         const int gsize = total <= (int)gridDim.x ? 1 : (total <= 2 * (int)gridDim.x ? 2 : kDecDotGroup);
         const int ngroups = total / gsize;
-        if (sw == kDecShrinkWarps - 1 && gsize > 1) {   // the staging buffer is needed for the dot products: B goes to L2 only
-            if (lane < T) {
-                const int slot = ctrl->slot_of_row[lane];
-                if (slot >= 0) {
-                    const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                    for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
+        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+        // Brings the blocks of B into the staging buffer (16-byte asynchronous copies, all in flight at
+        // once); blocks that did not fit are asked into L2 and read from there by the epilogue.
+        auto stage_b = [&]() {
+            const int rows_cta = row_end - row_begin;
+            for (int t = 0; t < T; ++t) {
+                if (!ctrl->b_lead[t]) continue;
+                const int r8 = (lk->rank_of_row[t] + 7) >> 3;
+                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)ctrl->slot_of_row[t] * N + row_begin) * kRankPad);
+                const int off = ctrl->b_of_row[t];
+                if (off >= 0) {
+                    for (int i = me; i < rows_cta * r8; i += kDecShrinkWarps * 32) {
+                        const int c = i / rows_cta, r = i - c * rows_cta;
+                        cp_async_16(smem_u32(dot_s) + off + i * 16, b + (size_t)r * kRankPad * 2 + c * 16);
+                    }
+                } else {
+                    for (int r = me; r < rows_cta; r += kDecShrinkWarps * 32) prefetch_l2(b + (size_t)r * kRankPad * 2);
                 }
             }
-        } else if (sw == kDecShrinkWarps - 1) {
-            // The expand's B rows for this CTA's output columns.  When the staging buffer below is not
-            // needed (single dot products), they are copied into it now, one contiguous block per distinct
-            // slot, so that the epilogue has no memory round trip left; otherwise, and for slots that do
-            // not fit, they are asked into L2 and read from there.
-            const int slot = lane < T ? ctrl->slot_of_row[lane] : -1;
-            const unsigned same = __match_any_sync(0xffffffffu, slot);
-            const bool leader = slot >= 0 && (same & ((1u << lane) - 1u)) == 0u;
-            const unsigned leaders = __ballot_sync(0xffffffffu, leader);
-            const int block_bytes = (row_end - row_begin) * kRankPad * 2;
-            const int fit = (gsize == 1 && block_bytes > 0) ? kDecDotBytes / block_bytes : 0;
-            const int my_block = __popc(leaders & ((1u << (__ffs(same) - 1)) - 1u));   // rank of this lane's slot among the distinct ones
-            const bool staged = slot >= 0 && my_block < fit;
-            const int nblocks = min(__popc(leaders), fit);
-            if (lane < T) ctrl->b_of_row[lane] = staged ? my_block : -1;
-            if (lane == 0) {
-                ctrl->b_staged = nblocks;
-                if (nblocks > 0) mbar_arrive_expect_tx(smem_u32(&ctrl->bfull), (uint32_t)(nblocks * block_bytes));
-            }
-            __syncwarp();
-            if (leader) {
-                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)slot * N + row_begin) * kRankPad);
-                if (staged) bulk_copy_g2s(smem_u32(dot_s) + my_block * block_bytes, b, (uint32_t)block_bytes, smem_u32(&ctrl->bfull));
-                else for (int r = 0; r < row_end - row_begin; ++r) prefetch_l2(b + (size_t)r * kRankPad * 2);
-            }
-        }
-        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+        };
+        // With single dot products the staging buffer is not needed for them: B can come in right away.
+        if (gsize == 1) stage_b();
         auto group = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
             const int d0 = g * gsize;
             t = 0;
@@ -553,6 +571,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 red_release_gpu_add(sync_words, (unsigned)gsize);
             }
         }
+        if (gsize > 1) stage_b();   // the staging buffer is free now (the groups end with a barrier of these warps)
         // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
         // other CTAs' shares normally arrive within microseconds and are then read from global memory.
         // But this CTA never depends on them: nothing guarantees that the whole grid is resident at once
@@ -577,15 +596,21 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 if (me == 0) u_s[t * kRankPad + j] = val;
             }
         } else {
+            cp_async_wait_all();   // the copies of B must not land on top of the groups' operands
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
             for (int g = 0; g < ngroups; ++g) {
                 float val[kDecDotGroup];
                 int t, j0;
                 group(g, val, t, j0);
                 if (me == 0) for (int i = 0; i < gsize; ++i) u_s[t * kRankPad + j0 + i] = val[i];
             }
+            stage_b();   // the groups went through the staging buffer: bring B in once more
         }
-        // tell the consumers that u_s, slot_of_row and bad_offsets are final
-        asm volatile("bar.arrive 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
+        cp_async_wait_all();   // this thread's chunks of B have landed
+        // tell the consumers that u_s, slot_of_row, bad_offsets and the copies of B are final (each thread
+        // releases what it wrote)
+        if (kPutOff) mbar_arrive(smem_u32(&ctrl->ufull));   // (the consumers can test this one without waiting)
+        else asm volatile("bar.arrive 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
         // Every CTA signs off once it has its copy of u and has published its own share; the last one puts
         // both counters back to zero for the next call on this table.
         if (sw == 0 && lane == 0) {
@@ -600,7 +625,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     for (int round_begin = consumer ? row_begin : row_end; round_begin < row_end; round_begin += kDecRoundUnits * kDecUnitRows) {
         const int round_rows = min(kDecRoundUnits * kDecUnitRows, row_end - round_begin);
         const int nunits = (round_rows + kDecUnitRows - 1) / kDecUnitRows;
-        for (int sp = 0; sp < nspans; ++sp) {
+        // The spans are walked forwards in even rounds and backwards in odd ones: the x fragments of the
+        // span a round ends with are the ones the next round starts with and need no reload (with a
+        // single span, x is loaded once per CTA).
+        const bool backwards = kMulti && (((round_begin - row_begin) / (kDecRoundUnits * kDecUnitRows)) & 1) != 0;
+        for (int si = 0; si < nspans; ++si) {
+            const int sp = backwards ? nspans - 1 - si : si;
             const int k_begin = sp * kSpan;
             const int span = min(kSpan, K - k_begin);
             const int nchunks = (span + kDecChunk - 1) / kDecChunk;
@@ -608,7 +638,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 // ---------------------------------------------------------- consumer warps
                 // this warp's k-steps of the span: chunk kc, steps warp*4 .. warp*4+3.  The x fragments
                 // live in registers for every row of the round.
-                load_x(k_begin, span);
+                if (!kMulti) load_x(k_begin, span);
+                else if (sp != span_loaded) { load_x(k_begin, span); span_loaded = sp; }
                 for (int un = 0; un < nunits && ok; ++un) {
                     const int rows = min(kDecUnitRows, round_rows - un * kDecUnitRows);
                     const bool rv = gq < rows;   // lanes whose row of the 8-wide operand is real
@@ -668,7 +699,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                     for (int a = 0; a < 4; ++a)
                         vs[a] = (acc4[0][a] + acc4[1][a]) + (acc4[2][a] + acc4[3][a]);
                     const float v0 = vs[0], v1 = vs[1], v2 = vs[2], v3 = vs[3];
-                    if (sp == 0) {
+                    if (si == 0) {
                         sl[gq * 8 + tq * 2] = v0;       sl[gq * 8 + tq * 2 + 1] = v1;
                         sl[(gq + 8) * 8 + tq * 2] = v2; sl[(gq + 8) * 8 + tq * 2 + 1] = v3;
                     } else {
@@ -681,28 +712,38 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         // only the consumer warps meet at the round's two barriers: the producer warp keeps filling the
         // ring with the next round's rows meanwhile
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // partial sums are in the slots
-        if (consumer && G > 0 && !u_ready) {   // first epilogue: the shrink warps have staged u in shared memory
-            asm volatile("bar.sync 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
-            if (ctrl->b_staged > 0 && ok) ok = mbar_wait_warp(smem_u32(&ctrl->bfull), 0u, abort);   // long since there
-            u_ready = true;
+        // The expand needs u, which the whole grid computes: it is there a few microseconds after the call
+        // before this one has ended everywhere.  A CTA with several rounds does not wait for it: until u
+        // has arrived, each thread keeps the base sums of its elements of up to kDecDefer rounds in
+        // shared memory (the same thread finishes them later), and only then, or in its last round, it waits.
+        if (!kPutOff) {
+            if (consumer && G > 0 && !u_ready) {   // first epilogue: the shrink warps have staged u in shared memory
+                asm volatile("bar.sync 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
+                u_ready = true;
+            }
+        } else if (consumer && ok && G > 0 && !u_ready) {
+            const bool last_round = round_begin + kDecRoundUnits * kDecUnitRows >= row_end;
+            if (last_round || ndefer == kDecDefer) {
+                int there = 1;   // (polling: the flip is seen within a few cycles, no wake-up)
+                if (lane == 0) there = mbar_wait_spin(smem_u32(&ctrl->ufull), 0u, abort) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, there, 0) != 0;
+                u_ready = ok;
+            } else {
+                int there = lane == 0 ? (mbar_test_wait(smem_u32(&ctrl->ufull), 0u) ? 1 : 0) : 0;
+                u_ready = __shfl_sync(0xffffffffu, there, 0) != 0;
+            }
         }
         if (consumer && ok) {
-            const bool lora = G > 0 && ctrl->bad_offsets == 0;
-            const int per_token = nunits * kDecUnitRows;
-            for (int e = tid; e < T * per_token; e += kDecConsumers * 32) {
-                const int t = e / per_token, j = e % per_token;   // consecutive threads: consecutive n
-                if (j >= round_rows) continue;
-                const int un = j / kDecUnitRows, r = j % kDecUnitRows;
-                const int n = round_begin + j;
-                float v = 0.f;
-#pragma unroll
-                for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
+            const bool lora = G > 0 && u_ready && ctrl->bad_offsets == 0;
+            const int rows_cta = row_end - row_begin;
+            // y[t][n] = base sum + u_t . B_slot[n] (the first ceil(rank / 8) chunks of the row), rounded once
+            auto finish = [&](int t, int n, float v) {
                 const int slot = lora ? ctrl->slot_of_row[t] : -1;
                 if (slot >= 0) {
                     const int r8 = (lk->rank_of_row[t] + 7) >> 3;
                     const uint4* bp = reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
                     const int bb = ctrl->b_of_row[t];
-                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + ((size_t)bb * (row_end - row_begin) + (n - row_begin)) * kRankPad * 2);
+                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + bb) + (n - row_begin);
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
                     auto fma8 = [&](const uint4& b, int c) {
@@ -713,13 +754,47 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                         d = fmaf(u1.z, bf16_lo(b.w), d); d = fmaf(u1.w, bf16_hi(b.w), d);
                     };
                     if (bb >= 0) {   // (two loops: with a select inside one loop the global loads no longer overlap)
-                        for (int c = 0; c < r8; ++c) fma8(bs[c], c);
+                        for (int c = 0; c < r8; ++c) fma8(bs[c * rows_cta], c);
                     } else {
                         for (int c = 0; c < r8; ++c) fma8(ldg_nc_v4(bp + c), c);
                     }
                     v += d;
                 }
                 y[(size_t)t * N + n] = __float2bfloat16_rn(v);
+            };
+            const int per_token = nunits * kDecUnitRows;
+            if (kPutOff && G > 0 && !u_ready) {   // put this round off (a full round: the last one waits)
+#pragma unroll
+                for (int i = 0; i < kDecPerThread; ++i) {
+                    const int e = tid + i * kDecConsumers * 32;
+                    if (e < T * per_token) {
+                        const int t = e / per_token, j = e % per_token;
+                        const int un = j / kDecUnitRows, r = j % kDecUnitRows;
+                        float v = 0.f;
+#pragma unroll
+                        for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
+                        defer_s[ndefer * (kDecPerThread * kDecConsumers * 32) + e] = v;   // read back by this very thread
+                    }
+                }
+                ++ndefer;
+            } else {
+                if (kPutOff && ndefer > 0) {   // the rounds that were put off
+                    constexpr int kFull = kDecRoundUnits * kDecUnitRows;
+                    for (int dd = 0; dd < ndefer; ++dd)
+                        for (int e = tid; e < T * kFull; e += kDecConsumers * 32)
+                            finish(e / kFull, round_begin - (ndefer - dd) * kFull + e % kFull,
+                                   defer_s[dd * (kDecPerThread * kDecConsumers * 32) + e]);
+                    ndefer = 0;
+                }
+                for (int e = tid; e < T * per_token; e += kDecConsumers * 32) {
+                    const int t = e / per_token, j = e % per_token;   // consecutive threads: consecutive n
+                    if (j >= round_rows) continue;
+                    const int un = j / kDecUnitRows, r = j % kDecUnitRows;
+                    float v = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
+                    finish(t, round_begin + j, v);
+                }
             }
         }
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // slots are free for the next round
@@ -739,9 +814,13 @@ int g_dec_patience = 100000;
 cudaError_t decode_init()
 {
     if (const char* e = getenv("LML_DECODE_PATIENCE")) g_dec_patience = atoi(e) < 0 ? 0 : atoi(e);
-    cudaError_t e = cudaFuncSetAttribute(decode_main_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(decode_main_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
+    cudaError_t e = cudaSuccess;
+    auto set = [&](auto kernel) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
+    };
+    set(decode_main_kernel<false, false, false>); set(decode_main_kernel<false, true, false>); set(decode_main_kernel<false, true, true>);
+    set(decode_main_kernel<true, false, false>);  set(decode_main_kernel<true, true, false>);  set(decode_main_kernel<true, true, true>);
+    return e;
 }
 
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a, cudaStream_t stream,
@@ -775,10 +854,23 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const int32_t* pm = a.perm;
     const int32_t* ts = a.token_slots;
     const int32_t* amap = a.by_adapter ? ar.adapter_map : nullptr;
-    cudaError_t e = a.T > 8 ? cudaLaunchKernelEx(&cfg, decode_main_kernel<true>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, amap, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience)
-                            : cudaLaunchKernelEx(&cfg, decode_main_kernel<false>, snap, arenaA, arenaB, xb, wb, yb, up, so,
-                                                 ids, pm, ts, amap, status, a.T, a.d_in, a.d_out, a.G, g_dec_patience);
+    // Three builds of the kernel per token count: CTAs with one round of rows (the plain loop), with
+    // several rounds (x is kept between rounds), and with several rounds and adapters (the expand of
+    // early rounds is put off until u has arrived).
+    const int rows_per_cta = (a.d_out + (int)cfg.gridDim.x - 1) / (int)cfg.gridDim.x;
+    const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
+    const bool put_off = multi && a.G > 0;
+    auto launch = [&](auto kernel) {
+        return cudaLaunchKernelEx(&cfg, kernel, snap, arenaA, arenaB, xb, wb, yb, up, so, ids, pm, ts, amap, status, a.T,
+                                  a.d_in, a.d_out, a.G, g_dec_patience);
+    };
+    cudaError_t e;
+    if (a.T > 8)
+        e = put_off ? launch(decode_main_kernel<true, true, true>)
+                    : (multi ? launch(decode_main_kernel<true, true, false>) : launch(decode_main_kernel<true, false, false>));
+    else
+        e = put_off ? launch(decode_main_kernel<false, true, true>)
+                    : (multi ? launch(decode_main_kernel<false, true, false>) : launch(decode_main_kernel<false, false, false>));
     if (e == cudaSuccess) ++*launches;
     return e;
 }

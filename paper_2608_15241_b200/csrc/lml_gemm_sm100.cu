@@ -19,6 +19,7 @@
 // reads the second output.  The producer slips those stages into the middle of the next tile's
 // k-blocks, by when the first read is long done.
 // Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
+#include <cstdio>
 #include <cstdlib>
 
 #include "lml_internal.cuh"
@@ -454,6 +455,267 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     }
 }
 
+// ---- split-K variant for few tokens ---------------------------------------------------------------------
+// With a few hundred tokens or fewer the layer is bound by the read of W0, and 128 x 256 tiles give far
+// fewer CTAs than the machine has SMs.  Here a cluster of S CTAs shares one tile: CTA r multiplies its
+// share of the k-blocks (and of the tile's LoRA pieces, which are just more K) into its own TMEM
+// accumulator, so S times as many SMs stream W0.  The partial sums are then exchanged through
+// distributed shared memory: the tile's eight 32-column chunks are dealt out to the CTAs, every CTA
+// writes each chunk of its partial sums into the owner's (by then idle) stage memory, and the owner adds
+// the S contributions in rank order, rounds once and writes its columns of y.  Two cluster barriers
+// frame the exchange: nobody writes into a CTA that is still multiplying, nobody adds before all
+// have written.  Warp roles and the stage ring are those of the kernel above; every stage carries its
+// side-band word.
+constexpr int kSplitMaxS = 8;
+
+__device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel(
+    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x0,
+    const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_u,
+    const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ SlotSnapshot snap, const GemmParams p)
+{
+    using Cfg = GemmCfg<BN>;
+    constexpr int kSplitChunks = BN / kEpiChunkCols;   // 32-column chunks of the tile: 4 or 8
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+    uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    uint8_t* epi_ptr = tiles_ptr + Cfg::kStages * Cfg::kStageBytes;
+    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(epi_ptr + Cfg::kEpiBytes);
+    int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
+    int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = (int)gridDim.x, rank = (int)blockIdx.x;   // the cluster spans the grid's x dimension
+    const int n = (int)blockIdx.y, m = (int)blockIdx.z;
+    const int num_kb = (p.K + kBK - 1) / kBK;
+    const bool seg_cached = p.G <= kSegCache;
+    // chunks of the tile's 256 columns that CTA r reduces: [first(r), first(r + 1))
+    auto first_chunk = [&](int r) { return r * kSplitChunks / S; };
+    const int cpr = (kSplitChunks + S - 1) / S;   // most chunks any CTA owns
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cfg::kStages; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctrl->tmem_full[0]), 1);
+        ctrl->abort = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0 && lane == 0) {
+        prefetch_tmap(&tmap_x0); prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u); prefetch_tmap(&tmap_b);
+    }
+    if (seg_cached && p.G > 0) {
+        for (int g = threadIdx.x; g <= p.G; g += kGemmThreads) seg_cache[g] = __ldg(p.seg_offsets + g);
+        for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
+            int s = __ldg(p.slot_ids + g);
+            slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
+        }
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile int* abort = &ctrl->abort;
+    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            auto acquire = [&]() -> bool { return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort); };
+            auto advance = [&]() { if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; } };
+            const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+            const bool in_place = p.tile_identity && __ldg(p.tile_identity + m);
+            const int kb0 = rank * num_kb / S, kb1 = (rank + 1) * num_kb / S;
+            auto piece_slot = [&](int g) -> int {
+                int s0, s1, s;
+                if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
+                else {
+                    s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1); s = __ldg(p.slot_ids + g);
+                    if (slot_rank(snap, s) == 0) s = -1;
+                }
+                return min(s1, row1) <= max(s0, row0) ? -1 : s;
+            };
+            // base k-blocks first: they do not depend on the shrink kernel that precedes this one
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                ok = acquire();
+                if (!ok) break;
+                const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                ctrl->stage_info[stage] = 4u;
+                mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
+                else tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
+                tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
+                advance();
+            }
+            // this CTA's share of the tile's LoRA pieces
+            bool lora = false;
+            if (p.G > 0) {
+                grid_dependency_wait();
+                grid_launch_dependents();
+                lora = p.plan->lora_ok != 0;
+            }
+            if (lora && ok) {
+                int g_first, g_end;
+                if (seg_cached) {
+                    int lo = 0, hi = p.G;
+                    while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+                    g_first = lo;
+                    g_end = g_first;
+                    while (g_end < p.G && seg_cache[g_end] < row1) ++g_end;
+                } else {
+                    g_first = seg_upper(p.seg_offsets, p.G, row0);
+                    g_end = g_first;
+                    while (g_end < p.G && __ldg(p.seg_offsets + g_end) < row1) ++g_end;
+                }
+                // segment g's piece goes to CTA g mod S: which CTA adds a row's LoRA term depends only on the
+                // row's own segment, so a row's bits do not change with what other segments are bound to
+                for (int g = g_first; g < g_end && ok; ++g) {
+                    if (g % S != rank) continue;
+                    const int s = piece_slot(g);
+                    if (s < 0) continue;
+                    ok = acquire();
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                    ctrl->stage_info[stage] = (uint32_t)((snap.rank[s] + 15) >> 4);
+                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                    tma_load_2d(a_dst, &tmap_u, bar, 0, (m + g) * kBM);
+                    tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
+                    advance();
+                }
+            }
+            if (ok) {   // end of this CTA's K: a stage without operands
+                ok = acquire();
+                if (ok) {
+                    ctrl->stage_info[stage] = kStageCommit;
+                    mbar_arrive(smem_u32(&ctrl->full[stage]));
+                    advance();
+                }
+            }
+            // leave the role only after every load has landed and been consumed
+            for (int i = 0; i < Cfg::kStages && ok; ++i) { ok = acquire(); advance(); }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN);
+            int stage = 0;
+            uint32_t phase = 0, accumulate = 0;
+            bool ok = true;
+            for (bool more = true; more && ok;) {
+                ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
+                if (!ok) break;
+                const uint32_t info = ctrl->stage_info[stage];
+                more = (info & kStageCommit) == 0;
+                const int ksteps = (int)(info & 0xffu);
+                const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes;
+                const uint64_t adesc = umma_desc_k128(a_addr);
+                const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes);
+                tc_fence_after();
+#pragma unroll 4
+                for (int k = 0; k < ksteps; ++k) {
+                    umma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
+                    accumulate = 1;
+                }
+                umma_commit(smem_u32(&ctrl->empty[stage]));
+                if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) umma_commit(smem_u32(&ctrl->tmem_full[0]));
+            ctrl->stage_info[7] = accumulate;   // 0: this CTA had no K at all, its accumulator holds nothing
+        }
+    }
+    // ---------------------------------------------------------------------- exchange and reduction
+    __syncwarp();   // (the producer's and the MMA issuer's other lanes waited here: the cluster barrier wants whole warps)
+    bool ok = true;
+    if (warp >= 2) {
+        ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[0]), 0u, abort);   // this CTA's MMAs are complete: so are its loads
+        tc_fence_after();
+    }
+    cluster_sync_all();   // every CTA of the cluster is done with its stage memory
+    const int q = warp & 3;   // TMEM lane quarter an epilogue warp may read
+    const int row = q * 32 + lane;
+    if (warp >= 2 && ok) {
+        const bool have = ctrl->stage_info[7] != 0u;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        int owner = 0;
+#pragma unroll 1
+        for (int c = 0; c < kSplitChunks; ++c) {
+            while (first_chunk(owner + 1) <= c) ++owner;
+            uint32_t r[32];
+            tmem_ld_32x32(t_addr + (uint32_t)(c * kEpiChunkCols), r);
+            tmem_ld_wait();
+            if (!have) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = 0u;
+            }
+            // slot (this CTA's rank, chunk within the owner's share) of the owner's receive area, 16 KB: the
+            // 16-byte pieces of the 128 rows, piece-major, so that a warp's store is 512 contiguous bytes
+            const uint32_t local = tiles_addr + (uint32_t)((rank * cpr + (c - first_chunk(owner))) * (kBM * 128) + row * 16);
+            const uint32_t remote = mapa_shared(local, (uint32_t)owner);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                st_shared_cluster_v4(remote + (uint32_t)(j * kBM * 16), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        }
+        tc_fence_before();
+    }
+    cluster_sync_all();   // all contributions have arrived
+    if (warp >= 2 && ok) {
+        const int pos = m * kBM + row;
+        const bool scatter = p.perm != nullptr && !(p.tile_identity && __ldg(p.tile_identity + m));
+        int out_row = pos;
+        if (pos < p.T && scatter) out_row = __ldg(p.perm + pos);
+        const bool row_ok = pos < p.T && out_row >= 0 && out_row < p.T;
+        const int c_first = first_chunk(rank), c_end = first_chunk(rank + 1);
+#pragma unroll 1
+        for (int c = c_first; c < c_end; ++c) {
+            float acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+            for (int src = 0; src < S; ++src) {   // rank order: the sum does not depend on timing
+                const uint8_t* rp = tiles_ptr + (size_t)(src * cpr + (c - c_first)) * (kBM * 128) + row * 16;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 v = *reinterpret_cast<const float4*>(rp + j * kBM * 16);
+                    acc[4 * j] += v.x; acc[4 * j + 1] += v.y; acc[4 * j + 2] += v.z; acc[4 * j + 3] += v.w;
+                }
+            }
+            const int col0 = n * BN + c * kEpiChunkCols;
+            if (!row_ok) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (col0 + j * 8 >= p.N) continue;
+                uint4 v;
+                v.x = pack_bf16(acc[8 * j + 0], acc[8 * j + 1]);
+                v.y = pack_bf16(acc[8 * j + 2], acc[8 * j + 3]);
+                v.z = pack_bf16(acc[8 * j + 4], acc[8 * j + 5]);
+                v.w = pack_bf16(acc[8 * j + 6], acc[8 * j + 7]);
+                *reinterpret_cast<uint4*>(p.y + (size_t)out_row * p.N + col0 + j * 8) = v;
+            }
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.status, LML_FLAG_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, BN);
+    }
+}
+
 // ---- CTA-pair variant ---------------------------------------------------------------------------------
 // Two CTAs of a cluster share a 256 x 256 tile (cta_group::2).  CTA r of the pair owns rows
 // [256 m2 + 128 r, +128): it stages its own 128 x 64 block of x and HALF of the W0 block (rows
@@ -807,6 +1069,12 @@ cudaError_t gemm_sm100_init(int /*device*/)
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lora_gemm_sm100_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             GemmCfg<256>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             GemmCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(lora_gemm_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 GemmCfg<128>::kSmemBytes);
 }
@@ -814,9 +1082,63 @@ cudaError_t gemm_sm100_init(int /*device*/)
 int gemm_pick_bn(int T, int d_out, int num_sms)
 {
     const int num_m = (T + kBM - 1) / kBM;
-    const int tiles256 = num_m * ((d_out + 255) / 256);
-    // wide tiles once they fill the machine; otherwise narrower tiles give more CTAs to stream W0
-    return tiles256 >= num_sms ? 256 : 128;
+    const int tiles256 = num_m * ((d_out + 255) / 256), tiles128 = num_m * ((d_out + 127) / 128);
+    // Rounds of tiles over the SMs times the cost of a tile: a 128-column tile takes about 0.82 of the
+    // time of a 256-column one (measured: the narrow kernel needs 1.64 times as long for the same work).
+    const float t256 = (float)((tiles256 + num_sms - 1) / num_sms);
+    const float t128 = 0.82f * (float)((tiles128 + num_sms - 1) / num_sms);
+    return t256 <= t128 ? 256 : 128;
+}
+
+// Split-K choice for few tokens: tile width and how many CTAs share a tile (split 0: do not use it).
+// It pays while the 128-column tiles are too few to keep most SMs busy.  Of the shapes whose clusters all
+// fit the machine at once, take the one with the most CTAs, and among equals the smaller cluster (less
+// to exchange); every CTA keeps at least two k-blocks, and the exchange area must fit the stage memory.
+struct SplitChoice { int bn, split; };
+static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
+{
+    static int max_clusters[2][kSplitMaxS + 1];
+    static bool probed = false;
+    if (const char* e = getenv("LML_GEMM_SPLIT")) {   // test knob: "<bn>x<split>", or 0 for no split
+        int bn = 0, sp = 0;
+        if (sscanf(e, "%dx%d", &bn, &sp) == 2 && (bn == 128 || bn == 256) && sp >= 2 && sp <= kSplitMaxS &&
+            sp * ((bn / 32 + sp - 1) / sp) * 16384 <= GemmCfg<128>::kStages * GemmCfg<128>::kStageBytes)
+            return {bn, sp};
+        return {0, 0};
+    }
+    if (!probed) {   // clusters of each size that can be resident together
+        for (int w = 0; w < 2; ++w)
+            for (int S = 2; S <= kSplitMaxS; ++S) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(S, num_sms / S, 1);
+                cfg.blockDim = dim3(kGemmThreads);
+                cfg.dynamicSmemBytes = w ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr; cfg.numAttrs = 1;
+                int n = 0;
+                cudaError_t e = w ? cudaOccupancyMaxActiveClusters(&n, lora_gemm_sm100_splitk_kernel<256>, &cfg)
+                                  : cudaOccupancyMaxActiveClusters(&n, lora_gemm_sm100_splitk_kernel<128>, &cfg);
+                if (e != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
+                max_clusters[w][S] = n;
+            }
+        probed = true;
+    }
+    const int num_m = (T + kBM - 1) / kBM, num_kb = (d_in + kBK - 1) / kBK;
+    if (num_m * ((d_out + 127) / 128) * 4 > num_sms * 3) return {0, 0};   // enough tiles without splitting
+    SplitChoice best = {0, 0};
+    int best_ctas = 0;
+    for (int S = 2; S <= kSplitMaxS; ++S)
+        for (int w = 0; w < 2; ++w) {
+            const int bn = w ? 256 : 128;
+            const int tiles = num_m * ((d_out + bn - 1) / bn);
+            const int cpr = (bn / 32 + S - 1) / S;
+            if (tiles > max_clusters[w][S] || num_kb < 2 * S) continue;
+            if (S * cpr * 16384 > GemmCfg<128>::kStages * GemmCfg<128>::kStageBytes) continue;
+            if (tiles * S > best_ctas) { best_ctas = tiles * S; best = {bn, S}; }
+        }
+    return best;
 }
 
 // LML_FORCE_GEMM=pair|single overrides the choice below (a test knob: small problems would
@@ -846,7 +1168,9 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
                               const GemmArgs& a, cudaStream_t stream)
 {
     const bool pairs = gemm_use_pairs(a.T, a.d_out, a.num_sms);
-    const int bn = pairs ? kPairBN : gemm_pick_bn(a.T, a.d_out, a.num_sms);
+    const SplitChoice sc = (pairs || a.slot_ids2 != nullptr) ? SplitChoice{0, 0} : gemm_pick_split(a.T, a.d_in, a.d_out, a.num_sms);
+    const int split = sc.split;
+    const int bn = pairs ? kPairBN : (split ? sc.bn : gemm_pick_bn(a.T, a.d_out, a.num_sms));
     const int num_m = (a.T + kBM - 1) / kBM;
     const int num_n = (a.d_out + bn - 1) / bn;
     const uint32_t w_box_rows = pairs ? (uint32_t)(kPairBN / 2) : (uint32_t)bn;
@@ -894,6 +1218,19 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
         cfg.attrs = attr;
         cfg.numAttrs = nattr;
         return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_pair_kernel, tx, tw, tu, tb, ty, snap, p);
+    }
+    if (split) {
+        cfg.gridDim = dim3(split, num_n, num_m);
+        cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = split;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+        cfg.attrs = attr;
+        cfg.numAttrs = nattr;
+        if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_splitk_kernel<256>, tx, tx0, tw, tu, tb, snap, p);
+        return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_splitk_kernel<128>, tx, tx0, tw, tu, tb, snap, p);
     }
     cfg.gridDim = dim3(min(num_m * num_n, a.num_sms));
     cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
