@@ -40,7 +40,7 @@ template <int BN> struct GemmCfg {
     static constexpr int kABytes = kBM * kBK * 2;
     static constexpr int kBBytes = BN * kBK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = (BN == 256) ? 4 : 6;
+    static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
     static constexpr int kTmemCols = 2 * BN;
     static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache;   // barriers + segment cache (two slot arrays)
@@ -56,6 +56,7 @@ struct GemmCtrl {
     uint32_t tmem_base;
     int abort;
     uint32_t stage_info[8];   // written by the producer: k-steps (0..4) | kStage* flags
+    int32_t piece[4];         // shrink form of the split-K kernel: found, slot, first row, end row of the CTA's piece
     int32_t pad[2];
 };
 // stage_info flags
@@ -473,7 +474,11 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-template <int BN>
+// kShrink: the same machinery computes the LoRA shrink.  A work item is a piece (block index b = tile m +
+// segment g, see the shrink kernel): u = scale * x_tile . A_slot^T, a 128 x 64 product over all of K with
+// the slot's 64 (zero-padded) rows of A in the place of W0; rows outside the segment are zeroed and the
+// result is written as a bf16 u block.  Launched with a full dependency on the work before it.
+template <int BN, bool kShrink = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel(
     const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x0,
     const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_u,
@@ -492,7 +497,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = (int)gridDim.x, rank = (int)blockIdx.x;   // the cluster spans the grid's x dimension
-    const int n = (int)blockIdx.y, m = (int)blockIdx.z;
+    const int n = (int)blockIdx.y;
+    int m = (int)blockIdx.z;   // (shrink: the block index b; the tile follows from the lookup below)
     const int num_kb = (p.K + kBK - 1) / kBK;
     const bool seg_cached = p.G <= kSegCache;
     // chunks of the tile's 256 columns that CTA r reduces: [first(r), first(r + 1))
@@ -518,13 +524,60 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
             slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
         }
     }
+    int piece_slot_id = -1, piece_lo = 0, piece_hi = 0;
+    if (kShrink) {
+        grid_launch_dependents();   // the GEMM behind this kernel may start on its base k-blocks
+        const int b = (int)blockIdx.z;
+        if (b == 0 && rank == 0) {   // one CTA validates the segment arrays for the whole call
+            if (p.u_set_rows && threadIdx.x == 0) grid_dependency_wait();   // (a chained pass: see the launcher)
+            int bad_off = 0, bad_slot = 0;
+            for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
+                const int s0 = __ldg(p.seg_offsets + g), s1 = __ldg(p.seg_offsets + g + 1);
+                if (s1 < s0 || s0 < 0 || s1 > p.T) bad_off = 1;
+                const int sl = __ldg(p.slot_ids + g);
+                if (sl != -1 && s1 > s0 && slot_rank(snap, sl) == 0) bad_slot = 1;   // an empty segment may name anything
+            }
+            if (threadIdx.x == 0 && (__ldg(p.seg_offsets) != 0 || __ldg(p.seg_offsets + p.G) != p.T)) bad_off = 1;
+            bad_off = __syncthreads_or(bad_off);
+            bad_slot = __syncthreads_or(bad_slot);
+            if (threadIdx.x == 0) {
+                const_cast<PlanWord*>(p.plan)->lora_ok = bad_off ? 0 : 1;
+                const unsigned f = (bad_off ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u);
+                if (f) atomicOr(p.status, f);
+            }
+        }
+        __syncthreads();   // the segment cache is loaded
+        if (threadIdx.x == 0) {   // which piece has block index b: the largest g with g + first tile of g <= b
+            int lo = 0, hi = p.G;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                const int off = seg_cached ? seg_cache[mid] : __ldg(p.seg_offsets + mid);
+                if (mid + off / kBM <= b) lo = mid; else hi = mid;
+            }
+            const int g = lo, mm = b - g;
+            int found = 0, sl = -1, plo = 0, phi = 0;
+            if (p.G > 0 && mm >= 0 && mm < p.num_m) {
+                const int s0 = seg_cached ? seg_cache[g] : __ldg(p.seg_offsets + g);
+                const int s1 = seg_cached ? seg_cache[g + 1] : __ldg(p.seg_offsets + g + 1);
+                plo = max(max(s0, mm * kBM), 0);
+                phi = min(min(s1, (mm + 1) * kBM), p.T);
+                sl = __ldg(p.slot_ids + g);
+                found = plo < phi && slot_rank(snap, sl) > 0;
+            }
+            ctrl->piece[0] = found; ctrl->piece[1] = sl; ctrl->piece[2] = plo; ctrl->piece[3] = phi;
+        }
+        __syncthreads();
+        if (!ctrl->piece[0]) return;   // every CTA of the cluster shares b and leaves together; nothing reads this block
+        piece_slot_id = ctrl->piece[1]; piece_lo = ctrl->piece[2]; piece_hi = ctrl->piece[3];
+        m = piece_lo / kBM;
+    }
     if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), BN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile int* abort = &ctrl->abort;
-    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+    if (!kShrink && p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
         grid_dependency_wait();
         grid_launch_dependents();
     }
@@ -559,12 +612,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                 if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
                 else tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
-                tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
+                if (kShrink) tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, kb * kBK, 0, piece_slot_id);   // (tmap_b: the arena of A here)
+                else tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
                 advance();
             }
             // this CTA's share of the tile's LoRA pieces
             bool lora = false;
-            if (p.G > 0) {
+            if (!kShrink && p.G > 0) {
                 grid_dependency_wait();
                 grid_launch_dependents();
                 lora = p.plan->lora_ok != 0;
@@ -636,7 +690,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
             }
             if (ok) umma_commit(smem_u32(&ctrl->tmem_full[0]));
-            ctrl->stage_info[7] = accumulate;   // 0: this CTA had no K at all, its accumulator holds nothing
+            ctrl->pad[0] = (int32_t)accumulate;   // 0: this CTA had no K at all, its accumulator holds nothing
         }
     }
     // ---------------------------------------------------------------------- exchange and reduction
@@ -650,7 +704,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
     const int q = warp & 3;   // TMEM lane quarter an epilogue warp may read
     const int row = q * 32 + lane;
     if (warp >= 2 && ok) {
-        const bool have = ctrl->stage_info[7] != 0u;
+        const bool have = ctrl->pad[0] != 0;
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         int owner = 0;
 #pragma unroll 1
@@ -695,6 +749,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 }
             }
             const int col0 = n * BN + c * kEpiChunkCols;
+            if (kShrink) {
+                // the piece's u block: scale, zero outside the segment's rows, round; all 128 rows are written
+                const bool mine = pos >= piece_lo && pos < piece_hi;
+                const float sc = mine ? snap.scale[piece_slot_id] : 0.f;
+                __nv_bfloat16* out = p.y + ((size_t)blockIdx.z * kBM + row) * kRankPad + col0;
+                __nv_bfloat16* out_neg = p.y2 ? p.y2 + ((size_t)blockIdx.z * kBM + row) * kRankPad + col0 : nullptr;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 v;
+                    v.x = pack_bf16(acc[8 * j + 0] * sc, acc[8 * j + 1] * sc);
+                    v.y = pack_bf16(acc[8 * j + 2] * sc, acc[8 * j + 3] * sc);
+                    v.z = pack_bf16(acc[8 * j + 4] * sc, acc[8 * j + 5] * sc);
+                    v.w = pack_bf16(acc[8 * j + 6] * sc, acc[8 * j + 7] * sc);
+                    if (!mine) v = make_uint4(0, 0, 0, 0);   // (0 * garbage may be a NaN)
+                    *reinterpret_cast<uint4*>(out + j * 8) = v;
+                    if (out_neg) *reinterpret_cast<uint4*>(out_neg + j * 8) = make_uint4(v.x ^ 0x80008000u, v.y ^ 0x80008000u, v.z ^ 0x80008000u, v.w ^ 0x80008000u);
+                }
+                continue;
+            }
             if (!row_ok) continue;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -1075,6 +1148,9 @@ cudaError_t gemm_sm100_init(int /*device*/)
     e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              GemmCfg<128>::kSmemBytes);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             GemmCfg<64>::kSmemBytes);
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(lora_gemm_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 GemmCfg<128>::kSmemBytes);
 }
@@ -1238,6 +1314,66 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.numAttrs = nattr;
     if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
     return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
+}
+
+
+// The LoRA shrink on the tensor cores: the shrink form of the split-K kernel, one cluster per block index.
+// Returns cudaErrorNotSupported when the caller should use the mma.sync kernel instead.
+cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
+                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, const void* x_in_place,
+                                const int32_t* tile_identity, PlanWord* plan, __nv_bfloat16* u_blocks,
+                                cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
+{
+    static int max_clusters[kSplitMaxS + 1];
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return cudaErrorNotSupported;
+        for (int S = 1; S <= kSplitMaxS; ++S) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(S, 1, num_sms / S);
+            cfg.blockDim = dim3(kGemmThreads);
+            cfg.dynamicSmemBytes = GemmCfg<64>::kSmemBytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, lora_gemm_sm100_splitk_kernel<64, true>, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
+            max_clusters[S] = n;
+        }
+    }
+    const int num_m = (T + kBM - 1) / kBM, num_kb = (d_in + kBK - 1) / kBK;
+    const int blocks = num_m + (G > 0 ? G : 1);
+    // as many CTAs per piece as still leaves every block index a cluster that is resident at once
+    int split = 1;
+    for (int S = 2; S <= kSplitMaxS; ++S)
+        if (blocks <= max_clusters[S] && num_kb >= 2 * S) split = S;
+    CUtensorMap tx, tx0, ta;
+    if (!encode_tmap_2d(&tx, x, (uint64_t)d_in, (uint64_t)T, (uint64_t)d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!encode_tmap_2d(&tx0, x_in_place ? x_in_place : x, (uint64_t)d_in, (uint64_t)T, (uint64_t)d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!encode_tmap_3d(&ta, ar.A, (uint64_t)d_in, kRankPad, (uint64_t)snap.max_slots, (uint64_t)d_in * 2,
+                        (uint64_t)d_in * kRankPad * 2, kBK, kRankPad, 1)) return cudaErrorInvalidValue;
+    GemmParams p = {};
+    p.seg_offsets = seg_offsets; p.slot_ids = slot_ids; p.perm = nullptr; p.plan = plan;
+    p.tile_identity = tile_identity;
+    p.y = u_blocks; p.y2 = u_blocks_neg; p.status = ar.status; p.slot_ids2 = nullptr;
+    p.u_set_rows = chained ? 1 : 0;
+    p.T = T; p.K = d_in; p.N = kRankPad; p.G = G; p.num_m = num_m; p.num_n = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(split, 1, blocks);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = GemmCfg<64>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // only a chained pass starts before its predecessor ends
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_splitk_kernel<64, true>, tx, tx0, tx, tx, ta, snap, p);
 }
 
 }  // namespace lml

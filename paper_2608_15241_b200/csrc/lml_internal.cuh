@@ -65,6 +65,12 @@ cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, cons
                                  __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained = false,   // chained: a further pass of the same call, may run beside the one before
                                  __nv_bfloat16* u_blocks_neg = nullptr);                              // optional second copy of the blocks, negated
 
+// The same pass on the tcgen05 tensor cores (the split-K kernel's shrink form); same arguments.
+cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
+                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, const void* x_in_place,
+                                const int32_t* tile_identity, PlanWord* plan, __nv_bfloat16* u_blocks,
+                                cudaStream_t stream, bool chained = false, __nv_bfloat16* u_blocks_neg = nullptr);
+
 // tile_identity[m] = 1: tile m's perm is the identity, its rows were not copied and stay in place.
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
                                int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream);
