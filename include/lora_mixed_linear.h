@@ -280,6 +280,10 @@ lml_status lora_mixed_linear_adapters(lml_table* t, const void* x, const void* W
  * weight).  The call enqueues on `stream`: copies in, the layer, the copy of y out.  The
  * device staging lives in `workspace`, which must hold lml_host_workspace_bytes().  y_host
  * is valid once the stream has been synchronised.  Errors as lora_mixed_linear.
+ * Up to LML_DECODE_MAX_TOKENS tokens, when every host buffer is pinned (cudaHostAlloc /
+ * cudaHostRegister; x_host and y_host 16-byte aligned), no copy is enqueued at all: one kernel
+ * reads the inputs out of host memory into the staging and the decode kernel writes y straight
+ * into y_host (two launches).  Pageable buffers, and larger calls, take the copies.
  */
 size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
 lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* W0, int T,

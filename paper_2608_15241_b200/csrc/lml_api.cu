@@ -606,6 +606,35 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
     uint8_t* so = ys + round_up((size_t)T * t->d_out * 2, 1024);
     uint8_t* si = so + round_up((size_t)(G + 1) * 4, 1024);
     uint8_t* pm = si + round_up((size_t)G * 4 + 4, 1024);
+    // Decode calls on pinned buffers: no DMA copies.  One kernel pulls the inputs out of host memory, and
+    // the decode kernel writes y straight into the caller's buffer.  (Anything else: copies, below.)
+    if (T <= kDecodeMaxT) {
+        auto device_view = [](const void* h, size_t align) -> void* {
+            if (!h) return nullptr;
+            cudaPointerAttributes a;
+            if (cudaPointerGetAttributes(&a, h) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+            if (a.type != cudaMemoryTypeHost || !a.devicePointer) return nullptr;
+            return (reinterpret_cast<uintptr_t>(a.devicePointer) & (align - 1)) ? nullptr : a.devicePointer;
+        };
+        void* xd = device_view(x_host, 16);
+        void* yd = device_view(y_host, 16);
+        void* sod = G > 0 ? device_view(seg_offsets_host, 4) : nullptr;
+        void* sid = G > 0 ? device_view(slot_ids_host, 4) : nullptr;
+        void* pmd = perm_host ? device_view(perm_host, 4) : nullptr;
+        if (xd && yd && (G == 0 || (sod && sid)) && (!perm_host || pmd)) {
+            if (launch_stage_host_inputs(xd, xs, (size_t)T * t->d_in * 2, (const int32_t*)sod, reinterpret_cast<int32_t*>(so),
+                                         G > 0 ? G + 1 : 0, (const int32_t*)sid, reinterpret_cast<int32_t*>(si), G,
+                                         (const int32_t*)pmd, reinterpret_cast<int32_t*>(pm), perm_host ? T : 0,
+                                         stream) != cudaSuccess) {
+                cudaGetLastError();
+                return LML_ERR_CUDA;
+            }
+            lml_status st = lora_mixed_linear(t, xs, W0, T, reinterpret_cast<int32_t*>(so), reinterpret_cast<int32_t*>(si), G,
+                                              perm_host ? reinterpret_cast<int32_t*>(pm) : nullptr, yd, p, inner, stream);
+            if (st == LML_OK) t->last_launches += 1;
+            return st;
+        }
+    }
     bool ok = cudaMemcpyAsync(xs, x_host, (size_t)T * t->d_in * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     if (G > 0) {
         ok = ok && cudaMemcpyAsync(so, seg_offsets_host, (size_t)(G + 1) * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;

@@ -73,6 +73,35 @@ cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream)
     return cudaGetLastError();
 }
 
+// Host-buffer form of a decode call whose host buffers are pinned: one kernel pulls the inputs out of
+// host memory (16-byte loads for x, all in flight at once: one trip over the host link instead of a DMA
+// copy per array) into the device staging that the decode kernel reads.
+__global__ void __launch_bounds__(256) stage_host_inputs_kernel(
+    const uint4* __restrict__ x_host, uint4* __restrict__ x_dev, int x_chunks, const int32_t* __restrict__ so_host,
+    int32_t* __restrict__ so_dev, int n_so, const int32_t* __restrict__ ids_host, int32_t* __restrict__ ids_dev, int n_ids,
+    const int32_t* __restrict__ perm_host, int32_t* __restrict__ perm_dev, int n_perm)
+{
+    ptx::grid_dependency_wait();   // the call before may still read the staging
+    ptx::grid_launch_dependents();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x, n = gridDim.x * blockDim.x;
+    for (int c = i; c < x_chunks; c += n) x_dev[c] = x_host[c];
+    for (int c = i; c < n_so; c += n) so_dev[c] = so_host[c];
+    for (int c = i; c < n_ids; c += n) ids_dev[c] = ids_host[c];
+    for (int c = i; c < n_perm; c += n) perm_dev[c] = perm_host[c];
+}
+
+cudaError_t launch_stage_host_inputs(const void* x_host, void* x_dev, size_t x_bytes, const int32_t* so_host, int32_t* so_dev,
+                                     int n_so, const int32_t* ids_host, int32_t* ids_dev, int n_ids,
+                                     const int32_t* perm_host, int32_t* perm_dev, int n_perm, cudaStream_t stream)
+{
+    const int chunks = (int)(x_bytes / 16);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3((unsigned)((chunks + 255) / 256 < 1 ? 1 : (chunks + 255) / 256)), dim3(256), 0, stream);
+    return cudaLaunchKernelEx(&cfg, stage_host_inputs_kernel, (const uint4*)x_host, (uint4*)x_dev, chunks, so_host, so_dev,
+                              n_so, ids_host, ids_dev, n_ids, perm_host, perm_dev, n_perm);
+}
+
 __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
     const __grid_constant__ SlotSnapshot snap, const int32_t* __restrict__ token_slots, int T,
     int32_t* __restrict__ perm, int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_slot_ids,

@@ -45,6 +45,10 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
                                 int d_in, int d_out, cudaStream_t stream);
 
 cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream);
+// inputs of a decode call out of pinned host memory (device-accessible pointers) into device staging; x_bytes a multiple of 16
+cudaError_t launch_stage_host_inputs(const void* x_host, void* x_dev, size_t x_bytes, const int32_t* so_host, int32_t* so_dev,
+                                     int n_so, const int32_t* ids_host, int32_t* ids_dev, int n_ids,
+                                     const int32_t* perm_host, int32_t* perm_dev, int n_perm, cudaStream_t stream);
 // (A', B') = (B^T, A^T) of a forward adapter A [rank][K], B [N][rank] into slot `slot` of the transposed table's arena
 cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const void* A, const void* B, int rank,
                                            int K, int N, cudaStream_t stream);

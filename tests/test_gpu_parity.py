@@ -361,6 +361,21 @@ def test_host_buffer_entry_point():
             site.table.lora_mixed_linear_host(xh, site.W0, so, ids, yh, perm_host=pm)
             torch.cuda.synchronize()
             assert np.array_equal(to_bits(yh), ref_y)
+            # pageable buffers (for up to 16 tokens the pinned form above takes no copies at all: a kernel
+            # reads the inputs from host memory and y is written straight into the caller's buffer)
+            xp = torch.from_numpy(w.x.view(np.int16).copy()).view(torch.bfloat16)
+            yp = torch.zeros((w.T, w.d_out), dtype=torch.bfloat16)
+            pmp = None if w.perm is None else torch.from_numpy(w.perm.copy())
+            site.table.lora_mixed_linear_host(xp, site.W0, torch.from_numpy(w.seg_offsets.copy()),
+                                              torch.from_numpy(site.slot_ids().copy()), yp, perm_host=pmp)
+            torch.cuda.synchronize()
+            assert np.array_equal(to_bits(yp), ref_y)
+            # twice in a row on the same pinned buffers, then a base-only call
+            yh.zero_()
+            site.table.lora_mixed_linear_host(xh, site.W0, so, ids, yh, perm_host=pm)
+            site.table.lora_mixed_linear_host(xh, site.W0, so, ids, yh, perm_host=pm)
+            torch.cuda.synchronize()
+            assert np.array_equal(to_bits(yh), ref_y)
         finally:
             site.close()
 
