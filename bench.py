@@ -509,7 +509,7 @@ def cpu_baseline(w, kind, unit, budget_s):
                       f"{secs * repeats:.1f} s wall on {cores} threads, scaled by rows"}
 
 
-def run_layer_sweep(device, peaks, steps):
+def run_layer_sweep(device, peaks, steps, only=None):
     """The decoder-layer sweep (three distinct projection shapes x five token counts), one cell after
     the other: microseconds per call of lora_mixed_linear_tokens and the fraction of the bound that
     holds for the cell (the slower of bytes / HBM peak and flops / tensor peak)."""
@@ -518,6 +518,8 @@ def run_layer_sweep(device, peaks, steps):
     cells = []
     for proj, same_as in (("q", "q k v o"), ("gate", "gate up"), ("down", "down")):
         for T in wl.SWEEP_TOKENS:
+            if only and (proj, T) not in only:
+                continue
             w = wl.layer_sweep(proj, T)
             rot = Rotation(w, device, 3 * L2_BYTES)
             n = max(rot.R, min(steps, 400 if T <= 16 else (100 if T <= 1024 else 30)))
@@ -587,6 +589,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=2000)
     ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS) + ["layer_sweep"],
                     help="layer_sweep: per-cell timings of the decoder-layer sweep (1 GPU, its own JSON line)")
+    ap.add_argument("--sweep-cells", default="", help="layer_sweep: only these cells, e.g. q:128,down:16 (projections q, gate, down)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-secondary", action="store_true", help="skip the prefill line object")
     args = ap.parse_args()
@@ -613,10 +616,11 @@ def main():
     peaks = measured_peaks()
     warmup = max(3, args.warmup)
     if args.workload == "layer_sweep":
+        only = {(c.split(":")[0], int(c.split(":")[1])) for c in args.sweep_cells.split(",") if c} or None
         if rank == 0:
             print(json.dumps({"metric": "decoder-layer sweep, per-cell time of lora_mixed_linear_tokens", "unit": "us",
                               "n_gpus": 1, "dtype": "bf16", "data": "synthetic", "peak_source": peaks["source"],
-                              "cells": run_layer_sweep(device, peaks, args.steps)}), flush=True)
+                              "cells": run_layer_sweep(device, peaks, args.steps, only)}), flush=True)
         barrier()
         return
     primary = run_workload(args.workload, args.steps, warmup, device, world, peaks, rank == 0,
