@@ -30,6 +30,7 @@ constexpr int kShrinkWarps = 8;
 constexpr int kShrinkRows = 32;       // rows of one CTA (two 16-row MMA tiles)
 constexpr int kShrinkUnroll = 4;
 constexpr int kShrinkMaxCluster = 8;
+constexpr int kShrinkSegCache = 256;
 
 template <int NB> struct ShrinkSmem {
     static constexpr int kCols = NB * 8;
@@ -58,6 +59,7 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     float* red = shrink_smem;                                           // [warp][row][pitch]
     float* partial = shrink_smem + kShrinkWarps * kShrinkRows * S::kPitch;   // [row][cols]
     __shared__ int sh_piece[4];   // slot, lo, hi, found
+    __shared__ int seg_s[kShrinkSegCache + 1];   // the segment offsets, when they fit: the search below is then one round trip to memory, not one per step
 
     cg::cluster_group cluster = cg::this_cluster();
     const int KS = (int)gridDim.z, ks = (int)blockIdx.z;
@@ -85,16 +87,22 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     }
 
     // Which piece, if any, has block index b?  Largest g with g + tile_first(g) <= b.
+    const bool seg_cached = G <= kShrinkSegCache;
+    if (seg_cached) {
+        for (int g = tid; g <= G; g += blockDim.x) seg_s[g] = __ldg(seg_offsets + g);
+        __syncthreads();
+    }
     if (tid == 0) {
         int lo = 0, hi = G;   // invariant: candidates in [lo, hi)
         while (hi - lo > 1) {
             int mid = (lo + hi) >> 1;
-            if (mid + (__ldg(seg_offsets + mid) / kTileM) <= b) lo = mid; else hi = mid;
+            const int off = seg_cached ? seg_s[mid] : __ldg(seg_offsets + mid);
+            if (mid + (off / kTileM) <= b) lo = mid; else hi = mid;
         }
         int g = lo, found = 0, slot = -1, plo = 0, phi = 0;
         if (G > 0) {
             int m = b - g;
-            int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
+            int s0 = seg_cached ? seg_s[g] : __ldg(seg_offsets + g), s1 = seg_cached ? seg_s[g + 1] : __ldg(seg_offsets + g + 1);
             if (m >= 0 && m < num_tiles) {
                 plo = max(max(s0, m * kTileM), 0);
                 phi = min(min(s1, (m + 1) * kTileM), T);
