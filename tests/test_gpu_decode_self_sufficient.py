@@ -26,7 +26,11 @@ out = {}
 cases = [wl.ragged(T=8, d_in=264, d_out=136, ranks=(4, 16, 1, 33, 64)),
          wl.ragged(T=16, d_in=520, d_out=264, ranks=(4, 16, 1, 33, 64)),
          wl.ragged(T=16, d_in=1024, d_out=4104, ranks=(64, 64, 64, 64, 64), shuffled=True),
-         wl.ragged(T=5, d_in=4096, d_out=512, ranks=(16, 16, 16, 16, 16))]
+         wl.ragged(T=5, d_in=4096, d_out=512, ranks=(16, 16, 16, 16, 16)),
+         # CTAs with several rounds of rows: the expand of early rounds is put off until u is there
+         wl.ragged(T=8, d_in=264, d_out=5200, ranks=(4, 16, 1, 33, 64)),
+         wl.ragged(T=16, d_in=264, d_out=10360, ranks=(8, 16, 16, 64, 2), shuffled=True),
+         wl.ragged(T=3, d_in=4104, d_out=16000, ranks=(16, 16, 16, 16, 16))]
 for i, w in enumerate(cases):
     site = Site(w)
     y, flags = site.run()
@@ -57,6 +61,6 @@ def _run(tmp_path, name, patience):
 def test_self_sufficient_path_matches_normal_path(tmp_path):
     normal = _run(tmp_path, "normal.npz", None)
     alone = _run(tmp_path, "alone.npz", 0)
-    assert sorted(normal.files) == sorted(alone.files) and len(normal.files) == 4
+    assert sorted(normal.files) == sorted(alone.files) and len(normal.files) == 7
     for k in normal.files:
         assert np.array_equal(normal[k], alone[k]), k
