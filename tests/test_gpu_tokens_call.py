@@ -26,7 +26,9 @@ def _table(K, N, ranks, seed):
     return tbl, entries
 
 
-@pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384)])
+@pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384),
+                                   (17, 264, 136), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
+                                   (200, 1536, 520)])
 def test_tokens_call_equals_segment_then_layer(T, K, N):
     import torch
     tbl, entries = _table(K, N, (4, 16, 33), seed=21)
@@ -56,13 +58,14 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
     tbl.close()
 
 
-def test_tokens_call_flags_ids_without_adapter():
+@pytest.mark.parametrize("reps", [1, 20])
+def test_tokens_call_flags_ids_without_adapter(reps):
     import torch
-    K, N, T = 264, 136, 8
+    K, N, T = 264, 136, 8 * reps
     tbl, entries = _table(K, N, (8,), seed=5)
     good = entries[0][0]
     free = [s for s in range(tbl.max_slots) if s != good][0]
-    token_slots = np.array([good, free, -1, 99, good, -7, good, -1], np.int32)
+    token_slots = np.tile(np.array([good, free, -1, 99, good, -7, good, -1], np.int32), reps)
     x, W = to_dev(wl.normal_bf16(5, 1, (T, K), 1.0)), to_dev(wl.normal_bf16(5, 2, (N, K), 0.05))
     y = to_bits(tbl.lora_mixed_linear_tokens(x, W, torch.from_numpy(token_slots).cuda()))
     torch.cuda.synchronize()
