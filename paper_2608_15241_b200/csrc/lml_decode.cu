@@ -31,6 +31,11 @@
 //                       for their shares it computes all of u itself (same arithmetic, same bits).  So
 //                       the launch is an ordinary one and needs no co-residency guarantee.
 // d_in wider than a span is walked span by span.  All waits are bounded.
+// CTAs with more than one round of 32 rows (wide layers) come in two further builds of the kernel: the
+// spans are walked forwards and backwards in turn, so that the x fragments a round ends with serve the
+// next one without a reload; and, with adapters, the expand of early rounds is put off until u has
+// arrived (the base sums wait in shared memory), so only a CTA's last round can wait for the grid.  The
+// expand's operand B is staged compactly (the chunks a row really has) for all of a CTA's rows at once.
 #include <cstdlib>
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
@@ -46,7 +51,7 @@ constexpr int kDecUnitRows = 8;                  // W0 rows per unit = the 8-wid
 constexpr int kDecSpan = 4096;                   // columns whose x fragments fit in registers (half of it for T > 8)
 constexpr int kDecChunk = 2048;                  // columns per stage (one 4 KB bulk copy per row)
 constexpr int kDecChunksPerSpan = kDecSpan / kDecChunk;             // 4
-constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 4 k-steps per warp and stage
+constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 8 k-steps per warp and stage
 constexpr int kDecRowPitch = kDecChunk * 2 + 64; // bytes; a multiple of 16 that is 4 mod 8 in 16-byte chunks: rows land on different banks
 constexpr int kDecStageBytes = kDecUnitRows * kDecRowPitch;
 constexpr int kDecStages = 4;

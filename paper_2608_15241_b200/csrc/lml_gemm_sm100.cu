@@ -18,6 +18,8 @@
 // operands come from two more sets of u blocks (second slots; first slots negated), and the epilogue
 // reads the second output.  The producer slips those stages into the middle of the next tile's
 // k-blocks, by when the first read is long done.
+// For few tokens (tiles far fewer than SMs) a split-K variant follows below: a cluster of CTAs shares a
+// tile and exchanges partial sums through distributed shared memory; it also has a shrink mode.
 // Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
 #include <cstdio>
 #include <cstdlib>
