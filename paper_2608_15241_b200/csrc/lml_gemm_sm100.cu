@@ -23,6 +23,7 @@
 // Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
@@ -1176,7 +1177,7 @@ struct SplitChoice { int bn, split; };
 static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
 {
     static int max_clusters[2][kSplitMaxS + 1];
-    static bool probed = false;
+    static std::once_flag probed;
     if (const char* e = getenv("LML_GEMM_SPLIT")) {   // test knob: "<bn>x<split>", or 0 for no split
         int bn = 0, sp = 0;
         if (sscanf(e, "%dx%d", &bn, &sp) == 2 && (bn == 128 || bn == 256) && sp >= 2 && sp <= kSplitMaxS &&
@@ -1184,7 +1185,7 @@ static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
             return {bn, sp};
         return {0, 0};
     }
-    if (!probed) {   // clusters of each size that can be resident together
+    std::call_once(probed, [&]() {   // clusters of each size that can be resident together
         for (int w = 0; w < 2; ++w)
             for (int S = 2; S <= kSplitMaxS; ++S) {
                 cudaLaunchConfig_t cfg = {};
@@ -1201,8 +1202,7 @@ static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
                 if (e != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
                 max_clusters[w][S] = n;
             }
-        probed = true;
-    }
+    });
     const int num_m = (T + kBM - 1) / kBM, num_kb = (d_in + kBK - 1) / kBK;
     if (num_m * ((d_out + 127) / 128) * 4 > num_sms * 3) return {0, 0};   // enough tiles without splitting
     SplitChoice best = {0, 0};
@@ -1328,13 +1328,16 @@ cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const
 {
     static int max_clusters[kSplitMaxS + 1];
     static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return cudaErrorNotSupported;
+    static std::once_flag probed;
+    std::call_once(probed, [&]() {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return;
+        }
         for (int S = 1; S <= kSplitMaxS; ++S) {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(S, 1, num_sms / S);
+            cfg.gridDim = dim3(S, 1, sms / S);
             cfg.blockDim = dim3(kGemmThreads);
             cfg.dynamicSmemBytes = GemmCfg<64>::kSmemBytes;
             cudaLaunchAttribute attr[1];
@@ -1345,7 +1348,9 @@ cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const
             if (cudaOccupancyMaxActiveClusters(&n, lora_gemm_sm100_splitk_kernel<64, true>, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
             max_clusters[S] = n;
         }
-    }
+        num_sms = sms;
+    });
+    if (num_sms == 0) return cudaErrorNotSupported;
     const int num_m = (T + kBM - 1) / kBM, num_kb = (d_in + kBK - 1) / kBK;
     const int blocks = num_m + (G > 0 ? G : 1);
     // as many CTAs per piece as still leaves every block index a cluster that is resident at once
