@@ -284,6 +284,12 @@ lml_status lora_mixed_linear_adapters(lml_table* t, const void* x, const void* W
  * cudaHostRegister; x_host and y_host 16-byte aligned), no copy is enqueued at all: one kernel
  * reads the inputs out of host memory into the staging and the decode kernel writes y straight
  * into y_host (two launches).  Pageable buffers, and larger calls, take the copies.
+ * From 2048 tokens on, with pinned x_host and y_host and no perm, the call runs in eight chunks of
+ * whole 128-row tiles: the copy of the next chunk's x, the layer on this chunk and the copy of the
+ * last chunk's y proceed side by side on the caller's stream and two streams that belong to the
+ * table (created with it; the call creates nothing), and the caller's stream is made to wait for
+ * the last copy, so stream order is what the caller sees.  Results are those of lora_mixed_linear
+ * on the same rows.
  */
 size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);
 lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* W0, int T,

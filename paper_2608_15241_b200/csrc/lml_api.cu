@@ -32,6 +32,20 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
 
 }  // namespace
 
+static void free_table_resources(lml_table* t)
+{
+    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
+    if (t->copy_in) cudaStreamDestroy(t->copy_in);
+    if (t->copy_out) cudaStreamDestroy(t->copy_out);
+    if (t->ev_begin) cudaEventDestroy(t->ev_begin);
+    if (t->ev_done) cudaEventDestroy(t->ev_done);
+    for (int c = 0; c < lml_table::kHostChunks; ++c) {
+        if (t->ev_in[c]) cudaEventDestroy(t->ev_in[c]);
+        if (t->ev_layer[c]) cudaEventDestroy(t->ev_layer[c]);
+    }
+    (void)cudaGetLastError();
+}
+
 extern "C" {
 
 const char* lml_status_string(lml_status s)
@@ -87,10 +101,18 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && decode_init() == cudaSuccess;
     ok = ok && encode_tmap_3d(&t->tmap_B256, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
+    ok = ok && cudaStreamCreateWithFlags(&t->copy_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&t->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&t->ev_begin, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&t->ev_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; c < lml_table::kHostChunks; ++c) {
+        ok = ok && cudaEventCreateWithFlags(&t->ev_in[c], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&t->ev_layer[c], cudaEventDisableTiming) == cudaSuccess;
+    }
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
+        free_table_resources(t);
         delete t;
         return LML_ERR_CUDA;
     }
@@ -103,7 +125,7 @@ lml_status lml_table_destroy(lml_table* t)
     if (!t) return LML_ERR_INVALID_ARG;
     {
         DeviceGuard guard(t->device);
-        cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
+        free_table_resources(t);
     }
     delete t;
     return LML_OK;
@@ -582,6 +604,7 @@ size_t lml_host_workspace_bytes(const lml_table* t, int max_tokens, int max_segm
     n += round_up((size_t)max_tokens * t->d_out * 2, 1024);   // y staging
     n += round_up((size_t)(max_segments + 1) * 4, 1024) + round_up((size_t)max_segments * 4 + 4, 1024);
     n += round_up((size_t)max_tokens * 4 + 4, 1024);          // perm staging
+    n += lml_table::kHostChunks * round_up((size_t)(2 * max_segments + 2) * 4, 256);   // per-chunk segment arrays
     return n;
 }
 
@@ -633,6 +656,62 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
                                               perm_host ? reinterpret_cast<int32_t*>(pm) : nullptr, yd, p, inner, stream);
             if (st == LML_OK) t->last_launches += 1;
             return st;
+        }
+    }
+    // Large calls on pinned buffers, rows in segment order: in chunks of whole row tiles, the copy of the next
+    // chunk's x, the layer on this chunk and the copy of the last chunk's y side by side on three streams
+    // (the caller's and two of the table's), joined again before the call's last operation.
+    constexpr int kChunks = lml_table::kHostChunks;
+    if (T >= 256 * kChunks && !perm_host) {
+        auto pinned = [](const void* h) {
+            cudaPointerAttributes a;
+            if (cudaPointerGetAttributes(&a, h) != cudaSuccess) { cudaGetLastError(); return false; }
+            return a.type == cudaMemoryTypeHost;
+        };
+        if (pinned(x_host) && pinned(y_host)) {
+            const int rows = (int)round_up((size_t)(T + kChunks - 1) / kChunks, kTileM);
+            const int stride = (int)(round_up((size_t)(2 * G + 2) * 4, 256) / 4);
+            int32_t* chunk_arrays = reinterpret_cast<int32_t*>(pm + round_up((size_t)T * 4 + 4, 1024));
+            bool ok = true;
+            int launches = 0;
+            if (G > 0) {
+                ok = ok && cudaMemcpyAsync(so, seg_offsets_host, (size_t)(G + 1) * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+                ok = ok && cudaMemcpyAsync(si, slot_ids_host, (size_t)G * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+                ok = ok && launch_clip_segments(reinterpret_cast<int32_t*>(so), reinterpret_cast<int32_t*>(si), G, T, rows,
+                                                (T + rows - 1) / rows, chunk_arrays, stride, stream) == cudaSuccess;
+                ++launches;
+            }
+            ok = ok && cudaEventRecord(t->ev_begin, stream) == cudaSuccess;        // everything before this call on the caller's stream
+            ok = ok && cudaStreamWaitEvent(t->copy_in, t->ev_begin, 0) == cudaSuccess;
+            const size_t xrow = (size_t)t->d_in * 2, yrow = (size_t)t->d_out * 2;
+            int c = 0;
+            for (int r0 = 0; r0 < T && ok; r0 += rows, ++c) {
+                const int Tc = T - r0 < rows ? T - r0 : rows;
+                ok = ok && cudaMemcpyAsync(xs + r0 * xrow, static_cast<const uint8_t*>(x_host) + r0 * xrow, Tc * xrow,
+                                           cudaMemcpyHostToDevice, t->copy_in) == cudaSuccess;
+                ok = ok && cudaEventRecord(t->ev_in[c], t->copy_in) == cudaSuccess;
+            }
+            if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
+            c = 0;
+            for (int r0 = 0; r0 < T; r0 += rows, ++c) {
+                const int Tc = T - r0 < rows ? T - r0 : rows;
+                if (cudaStreamWaitEvent(stream, t->ev_in[c], 0) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+                const int32_t* so_c = chunk_arrays + (size_t)c * stride;
+                lml_status st = lora_mixed_linear(t, xs + r0 * xrow, W0, Tc, G > 0 ? so_c : nullptr, G > 0 ? so_c + G + 1 : nullptr, G,
+                                                  nullptr, ys + r0 * yrow, p, inner, stream);
+                if (st != LML_OK) return st;
+                launches += t->last_launches;
+                ok = ok && cudaEventRecord(t->ev_layer[c], stream) == cudaSuccess;
+                ok = ok && cudaStreamWaitEvent(t->copy_out, t->ev_layer[c], 0) == cudaSuccess;
+                ok = ok && cudaMemcpyAsync(static_cast<uint8_t*>(y_host) + r0 * yrow, ys + r0 * yrow, Tc * yrow,
+                                           cudaMemcpyDeviceToHost, t->copy_out) == cudaSuccess;
+                if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
+            }
+            ok = ok && cudaEventRecord(t->ev_done, t->copy_out) == cudaSuccess;
+            ok = ok && cudaStreamWaitEvent(stream, t->ev_done, 0) == cudaSuccess;   // the caller's stream ends with y in place
+            if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
+            t->last_launches = launches;
+            return LML_OK;
         }
     }
     bool ok = cudaMemcpyAsync(xs, x_host, (size_t)T * t->d_in * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;

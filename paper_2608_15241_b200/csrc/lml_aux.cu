@@ -102,6 +102,42 @@ cudaError_t launch_stage_host_inputs(const void* x_host, void* x_dev, size_t x_b
                               n_so, ids_host, ids_dev, n_ids, perm_host, perm_dev, n_perm);
 }
 
+// Host-buffer form of large calls, done chunk by chunk: the segment arrays of chunk c (rows [c * rows,
+// (c + 1) * rows) of the call), offsets relative to the chunk and clipped to it.  Malformed offsets are
+// detected on the whole call and poison every chunk's array, so that every chunk falls back to the base
+// output, as the unchunked call does.
+__global__ void __launch_bounds__(256) clip_segments_kernel(const int32_t* __restrict__ seg_offsets,
+                                                            const int32_t* __restrict__ slot_ids, int G, int T, int rows,
+                                                            int32_t* __restrict__ out, int stride)
+{
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
+    const int c = blockIdx.x, r0 = c * rows, Tc = min(rows, T - r0);
+    int32_t* so = out + (size_t)c * stride;
+    int32_t* ids = so + G + 1;
+    int bad = 0;
+    for (int g = threadIdx.x; g < G; g += blockDim.x) {
+        const int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
+        if (s1 < s0 || s0 < 0 || s1 > T) bad = 1;
+    }
+    if (threadIdx.x == 0 && (__ldg(seg_offsets) != 0 || __ldg(seg_offsets + G) != T)) bad = 1;
+    bad = __syncthreads_or(bad);
+    for (int g = threadIdx.x; g <= G; g += blockDim.x) {
+        const int v = min(max(__ldg(seg_offsets + g) - r0, 0), Tc);
+        so[g] = bad ? (g == 0 ? 1 : 0) : v;   // (an array that starts at 1 is malformed for every chunk)
+        if (g < G) ids[g] = __ldg(slot_ids + g);
+    }
+}
+
+cudaError_t launch_clip_segments(const int32_t* seg_offsets, const int32_t* slot_ids, int G, int T, int rows, int chunks,
+                                 int32_t* out, int stride, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3((unsigned)chunks), dim3(256), 0, stream);
+    return cudaLaunchKernelEx(&cfg, clip_segments_kernel, seg_offsets, slot_ids, G, T, rows, out, stride);
+}
+
 __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
     const __grid_constant__ SlotSnapshot snap, const int32_t* __restrict__ token_slots, int T,
     int32_t* __restrict__ perm, int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_slot_ids,

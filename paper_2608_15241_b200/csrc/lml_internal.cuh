@@ -45,6 +45,9 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
                                 int d_in, int d_out, cudaStream_t stream);
 
 cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream);
+// per-chunk segment arrays ([offsets (G + 1) | slot ids (G)] every `stride` ints) of a call done in chunks of `rows` rows
+cudaError_t launch_clip_segments(const int32_t* seg_offsets, const int32_t* slot_ids, int G, int T, int rows, int chunks,
+                                 int32_t* out, int stride, cudaStream_t stream);
 // inputs of a decode call out of pinned host memory (device-accessible pointers) into device staging; x_bytes a multiple of 16
 cudaError_t launch_stage_host_inputs(const void* x_host, void* x_dev, size_t x_bytes, const int32_t* so_host, int32_t* so_dev,
                                      int n_so, const int32_t* ids_host, int32_t* ids_dev, int n_ids,

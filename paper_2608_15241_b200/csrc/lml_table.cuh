@@ -17,6 +17,11 @@ struct lml_table {
     lml::Arena arena{};
     CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
     int last_launches = 0;
+    // host-buffer form of large calls: the copies of x in and of y out run on two streams of the table's own,
+    // chunk by chunk beside the layer (created with the table: the call itself creates nothing)
+    static constexpr int kHostChunks = 8;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_begin = nullptr, ev_done = nullptr, ev_in[kHostChunks] = {}, ev_layer[kHostChunks] = {};
     mutable std::mutex mu;
 };
 

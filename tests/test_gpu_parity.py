@@ -380,6 +380,50 @@ def test_host_buffer_entry_point():
             site.close()
 
 
+@pytest.mark.parametrize("kw", [dict(T=2100, d_in=256, d_out=520), dict(T=2048, d_in=520, d_out=264),
+                                dict(T=4000, d_in=264, d_out=1000)])
+def test_host_buffer_call_in_chunks(kw):
+    """Large calls (2048 tokens and more) on pinned buffers run in eight chunks of whole row tiles with the copies on the table's own
+    streams.  Same results as the device-buffer call (up to the order of the split-K sums where a chunk is
+    small enough for that kernel), the oracle within tolerance, malformed offsets caught for the whole
+    call, and back-to-back calls on the same buffers stay ordered."""
+    import torch
+    from paper_2608_15241_b200 import binding
+    w = wl.ragged(ranks=(4, 16, 1, 33, 64), **kw)
+    site = Site(w)
+    try:
+        ref_y, _ = site.run()
+        xh = torch.from_numpy(w.x.view(np.int16)).view(torch.bfloat16).pin_memory()
+        yh = torch.zeros((w.T, w.d_out), dtype=torch.bfloat16).pin_memory()
+        so = torch.from_numpy(w.seg_offsets).pin_memory()
+        ids = torch.from_numpy(site.slot_ids()).pin_memory()
+        for _ in range(3):
+            site.table.lora_mixed_linear_host(xh, site.W0, so, ids, yh)
+        torch.cuda.synchronize()
+        assert site.table.device_status() == 0
+        got = to_bits(yh)
+        ref, _ = oracle.forward(w.x, w.W0, w.entries, w.seg_offsets, w.seg_entry, None)
+        assert oracle.compare(got, ref)["ok"]
+        diff = np.abs(wl.bf16_bits_to_f64(got) - wl.bf16_bits_to_f64(ref_y))
+        assert (diff <= 2.0 ** -7 * np.maximum(1.0, np.abs(wl.bf16_bits_to_f64(ref_y)))).all()
+        # no adapters at all
+        yh.zero_()
+        site.table.lora_mixed_linear_host(xh, site.W0, None, None, yh)
+        torch.cuda.synchronize()
+        base = oracle.forward(w.x, w.W0, [], [0, w.T], [-1])[0]
+        assert oracle.compare(to_bits(yh), base)["ok"]
+        # malformed offsets: base output everywhere, flag raised
+        bad = w.seg_offsets.copy()
+        bad[1], bad[2] = bad[2], bad[1]
+        if bad[1] != bad[2]:
+            site.table.lora_mixed_linear_host(xh, site.W0, torch.from_numpy(bad).pin_memory(), ids, yh)
+            torch.cuda.synchronize()
+            assert site.table.device_status() & binding.FLAG_BAD_OFFSETS
+            assert oracle.compare(to_bits(yh), base)["ok"]
+    finally:
+        site.close()
+
+
 @pytest.mark.parametrize("T,G", [(16, 200), (7, 129), (16, 128)])
 def test_decode_with_many_mostly_empty_segments(T, G):
     """More segments than the decode kernel caches in shared memory (128): the lookup then searches
