@@ -442,6 +442,37 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
         x_secs, _, _ = timed_graph_loop(rot.backward_dx, rot.R, bsteps, 3, stream)
         a_secs, _, _ = timed_graph_loop(rot.backward_adapters, rot.R, bsteps, 3, stream)
         backward = {"dx_us": x_secs / bsteps * 1e6, "adapter_gradients_us": a_secs / bsteps * 1e6}
+    # context: spread of the layer-only time over repeats, one call alone (launch to completion seen from the
+    # host), and the plain library GEMM of the same base shape (harness only: not a target, not part of the path)
+    reps = []
+    rsteps = max(rot.R, min(ksteps, 400 if kind == "decode" else 60))
+    for _ in range(5):
+        r_secs, _, _ = timed_graph_loop(rot.layer_only, rot.R, rsteps, 3, stream)
+        reps.append(r_secs / rsteps * 1e6)
+    lat = []
+    with torch.cuda.stream(stream):
+        for i in range(40):
+            stream.synchronize()
+            t_a = time.perf_counter()
+            rot.layer_only(i)
+            stream.synchronize()
+            lat.append((time.perf_counter() - t_a) * 1e6)
+    mm_us = None
+    try:
+        with torch.cuda.stream(stream):
+            outs = [torch.empty((w.T, w.d_out), dtype=torch.bfloat16, device=device) for _ in range(2)]
+            def mm(i):
+                s_ = rot.sets[i % rot.R]
+                torch.matmul(s_["x"], s_["W0"].t(), out=outs[i & 1])
+                return 1
+            mm_secs, _, _ = timed_graph_loop(mm, rot.R, rsteps, 3, stream)
+            mm_us = mm_secs / rsteps * 1e6
+    except Exception:
+        mm_us = None
+    context = {"layer_only_us_min": min(reps), "layer_only_us_median": float(np.median(reps)), "repeats": len(reps),
+               "single_call_latency_us_median": float(np.median(lat)), "single_call_latency_us_min": min(lat),
+               "torch_matmul_base_only_us": mm_us,
+               "l2_bytes": int(getattr(torch.cuda.get_device_properties(device), "L2_cache_size", 0))}
     roof["traffic"] = ncu_traffic(name)
     roof["algorithmic"] = w.bytes() if kind == "decode" else w.flops()
     esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
@@ -451,7 +482,7 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
 
     # quick sampled parity of the last timed step against the oracle (rank 0)
     out = {"metric": spec["metric"], "value": value, "unit": spec["unit"], "ms_per_step": secs / steps * 1e3,
-           "gpu_launches": launches, "roofline": roof, "e2e": e2e, "clocks": clocks,
+           "gpu_launches": launches, "roofline": roof, "e2e": e2e, "clocks": clocks, "context": context,
            "config": {"workload": name, "tokens": w.T, "d_in": w.d_in, "d_out": w.d_out,
                       "resident_entries": len(w.entries), "segments": w.G, "rotation_sets": rot.R,
                       "l2_policy": f"inputs larger than L2: {rot.R} distinct weight/activation sets "
@@ -505,6 +536,7 @@ def cpu_baseline(w, kind, unit, budget_s):
     frac = len(pos) / w.T
     v = units_of(w, kind) * frac / secs
     return {"value": v, "unit": unit, "cores": cores, "kind": "oracle",
+            "single_thread_value": units_of(w, kind) / (per_row * w.T),   # one row on one thread, scaled by rows
             "sample": f"{len(pos)} of {w.T} token rows (all output columns) x {repeats} passes, "
                       f"{secs * repeats:.1f} s wall on {cores} threads, scaled by rows"}
 
