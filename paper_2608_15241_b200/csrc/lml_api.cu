@@ -388,7 +388,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
         if (e == cudaSuccess && G > 0) {
             e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids, G, x, tile_identity, plan,
-                                     u_blocks, stream);
+                                     u_blocks, stream, perm ? 2 : 0);
             if (e == cudaSuccess) ++launches;
         }
         if (e == cudaSuccess) {

@@ -69,7 +69,7 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                  const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                 __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained = false,   // chained: a further pass of the same call, may run beside the one before
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream, int chained = 0,   // 1: a further pass of the same call, may run beside the one before; 2: behind the call's row-gather kernel
                                  __nv_bfloat16* u_blocks_neg = nullptr);                              // optional second copy of the blocks, negated
 
 // The same pass on the tcgen05 tensor cores (the split-K kernel's shrink form); same arguments.

@@ -48,11 +48,14 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
     PlanWord* __restrict__ plan, __nv_bfloat16* __restrict__ u_blocks, int num_tiles, int chained,
     __nv_bfloat16* __restrict__ u_blocks_neg)   // optional second copy of the blocks with the sign flipped
 {
-    // Launched with a full dependency on the work before it, so nothing to wait for; the GEMM that
-    // follows may start its main loop right away.  (chained: this is a further shrink pass of the same
-    // call, launched as a programmatic dependent of the first, which had that full dependency: the
-    // passes run side by side.  One CTA then stays until the pass before is complete, so that whoever
-    // waits for this grid has waited for all of them.)
+    // chained 0: launched with a full dependency on the work before it, so nothing to wait for; the GEMM that
+    // follows may start its main loop right away.  chained 1: this is a further shrink pass of the same call,
+    // launched as a programmatic dependent of the first, which had that full dependency: the passes run side by
+    // side; one CTA then stays until the pass before is complete, so that whoever waits for this grid has
+    // waited for all of them.  chained 2: the predecessor is the call's own short row-gather kernel; launched
+    // as its programmatic dependent (the launch latency hides behind it), every CTA waits for it here before
+    // it lets the GEMM go, so that the GEMM finds the gathered rows complete as well.
+    if (chained == 2) ptx::grid_dependency_wait();
     ptx::grid_launch_dependents();
     extern __shared__ float shrink_smem[];
     using S = ShrinkSmem<NB>;
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(kShrinkWarps * 32, NB <= 2 ? 2 : 1) shrink_pie
 
     // One CTA validates the segment arrays for the whole call.
     if (b == 0 && sub == 0 && ks == 0) {
-        if (chained && tid == 0) ptx::grid_dependency_wait();
+        if (chained == 1 && tid == 0) ptx::grid_dependency_wait();
         int bad_off = 0, bad_slot = 0;
         for (int g = tid; g < G; g += blockDim.x) {
             int s0 = __ldg(seg_offsets + g), s1 = __ldg(seg_offsets + g + 1);
@@ -228,7 +231,7 @@ template <int NB>
 static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
                                     const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                     const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                    __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
+                                    __nv_bfloat16* u_blocks, cudaStream_t stream, int chained, __nv_bfloat16* u_blocks_neg)
 {
     const int num_tiles = (T + kTileM - 1) / kTileM;
     int ks = (d_in + 1023) / 1024;
@@ -252,7 +255,7 @@ static cudaError_t launch_shrink_nb(const Arena& ar, const SlotSnapshot& snap, c
     const __nv_bfloat16* xb = (const __nv_bfloat16*)x;
     const __nv_bfloat16* xip = (const __nv_bfloat16*)x_in_place;
     return cudaLaunchKernelEx(&cfg, shrink_pieces_kernel<NB>, snap, arenaA, status, xb, T, d_in, seg_offsets,
-                              slot_ids, G, xip, tile_identity, plan, u_blocks, num_tiles, chained ? 1 : 0, u_blocks_neg);
+                              slot_ids, G, xip, tile_identity, plan, u_blocks, num_tiles, chained, u_blocks_neg);
 }
 
 cudaError_t shrink_init()
@@ -267,7 +270,7 @@ cudaError_t shrink_init()
 cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, const void* x, int T,
                                  int d_in, const int32_t* seg_offsets, const int32_t* slot_ids, int G,
                                  const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
-                                 __nv_bfloat16* u_blocks, cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
+                                 __nv_bfloat16* u_blocks, cudaStream_t stream, int chained, __nv_bfloat16* u_blocks_neg)
 {
     // LML_SHRINK=tensor selects the tcgen05 form (the split-K kernel's shrink mode).  Measured on B200 it is
     // no faster than the kernel of this file (prefill_q_proj 65.7 against 64.6 us per layer call, 128 tokens
@@ -276,7 +279,7 @@ cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, cons
         const char* env = getenv("LML_SHRINK");
         if (env && env[0] == 't') {
             cudaError_t e = launch_shrink_sm100(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan,
-                                                u_blocks, stream, chained, u_blocks_neg);
+                                                u_blocks, stream, chained == 1, u_blocks_neg);
             if (e != cudaErrorNotSupported) return e;
         }
     }
