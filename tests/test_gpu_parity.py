@@ -182,7 +182,7 @@ def test_mlp_up_gate_shuffled_through_segmentation_pass():
 
 
 @pytest.mark.parametrize("proj,T", [("q", 1), ("q", 16), ("down", 16), ("gate", 128), ("down", 128),
-                                    ("q", 1024), ("o", 8192)])
+                                    ("q", 1024), ("o", 8192), ("k", 128), ("gate", 16), ("up", 1), ("gate", 1024)])
 def test_layer_sweep_cells_sampled(proj, T):
     check_sampled(wl.layer_sweep(proj, T), count=40)
 
