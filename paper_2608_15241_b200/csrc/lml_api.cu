@@ -34,7 +34,7 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
 
 static void free_table_resources(lml_table* t)
 {
-    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
+    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.Bc); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
     if (t->copy_in) cudaStreamDestroy(t->copy_in);
     if (t->copy_out) cudaStreamDestroy(t->copy_out);
     if (t->ev_begin) cudaEventDestroy(t->ev_begin);
@@ -90,6 +90,9 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     const size_t b_bytes = (size_t)max_slots * d_out * kRankPad * sizeof(__nv_bfloat16);
     bool ok = cudaMalloc(&t->arena.A, a_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&t->arena.B, b_bytes) == cudaSuccess;
+    const size_t bc_bytes = (size_t)max_slots * d_out * kRankCompact * sizeof(__nv_bfloat16);
+    ok = ok && cudaMalloc(&t->arena.Bc, bc_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.Bc, 0, bc_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&t->arena.status, 256) == cudaSuccess;
     ok = ok && cudaMalloc(&t->arena.adapter_map, kMaxAdapterIds * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.A, 0, a_bytes) == cudaSuccess;

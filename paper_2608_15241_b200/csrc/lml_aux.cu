@@ -10,6 +10,7 @@ namespace lml {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pack_adapter_kernel(__nv_bfloat16* __restrict__ dstA,
                                                            __nv_bfloat16* __restrict__ dstB,
+                                                           __nv_bfloat16* __restrict__ dstBc,
                                                            const __nv_bfloat16* __restrict__ A,
                                                            const __nv_bfloat16* __restrict__ B,
                                                            int rank, int d_in, int d_out)
@@ -32,6 +33,14 @@ __global__ void __launch_bounds__(256) pack_adapter_kernel(__nv_bfloat16* __rest
         long long n = i / kRankPad;
         Bd[i] = (j < rank) ? Bs[n * rank + j] : (unsigned short)0;
     }
+    if (rank <= kRankCompact) {   // the compact copy: [d_out][kRankCompact]
+        unsigned short* Bcd = reinterpret_cast<unsigned short*>(dstBc);
+        for (long long i = tid; i < (long long)d_out * kRankCompact; i += stride) {
+            const int j = (int)(i % kRankCompact);
+            const long long n = i / kRankCompact;
+            Bcd[i] = (j < rank) ? Bs[n * rank + j] : (unsigned short)0;
+        }
+    }
 }
 
 cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const void* B, int rank,
@@ -42,7 +51,8 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
     long long work = (long long)d_out * kRankPad;
     int blocks = (int)((work + 255) / 256);
     if (blocks > 1184) blocks = 1184;
-    pack_adapter_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, (const __nv_bfloat16*)A,
+    __nv_bfloat16* dstBc = ar.Bc + (size_t)slot * d_out * kRankCompact;
+    pack_adapter_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, dstBc, (const __nv_bfloat16*)A,
                                                     (const __nv_bfloat16*)B, rank, d_in, d_out);
     return cudaGetLastError();
 }
@@ -276,6 +286,7 @@ cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) pack_adapter_transposed_kernel(__nv_bfloat16* __restrict__ dstA,
                                                                       __nv_bfloat16* __restrict__ dstB,
+                                                                      __nv_bfloat16* __restrict__ dstBc,
                                                                       const __nv_bfloat16* __restrict__ A,
                                                                       const __nv_bfloat16* __restrict__ B,
                                                                       int rank, int K, int N)
@@ -296,6 +307,14 @@ __global__ void __launch_bounds__(256) pack_adapter_transposed_kernel(__nv_bfloa
         const long long k = i / kRankPad;
         Bd[i] = j < rank ? As[(long long)j * K + k] : (unsigned short)0;
     }
+    if (rank <= kRankCompact) {   // the compact copy of B': [K][kRankCompact]
+        unsigned short* Bcd = reinterpret_cast<unsigned short*>(dstBc);
+        for (long long i = tid; i < (long long)K * kRankCompact; i += stride) {
+            const int j = (int)(i % kRankCompact);
+            const long long k = i / kRankCompact;
+            Bcd[i] = j < rank ? As[(long long)j * K + k] : (unsigned short)0;
+        }
+    }
 }
 
 cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const void* A, const void* B, int rank,
@@ -306,7 +325,8 @@ cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const voi
     long long work = (long long)(K > N ? K : N) * kRankPad;
     int blocks = (int)((work + 255) / 256);
     if (blocks > 1184) blocks = 1184;
-    pack_adapter_transposed_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, (const __nv_bfloat16*)A,
+    __nv_bfloat16* dstBc = arT.Bc + (size_t)slot * K * kRankCompact;
+    pack_adapter_transposed_kernel<<<blocks, 256, 0, stream>>>(dstA, dstB, dstBc, (const __nv_bfloat16*)A,
                                                                (const __nv_bfloat16*)B, rank, K, N);
     return cudaGetLastError();
 }

@@ -136,7 +136,7 @@ __device__ __forceinline__ void prefetch_l2(const void* p)
 template <bool kTwo, bool kMulti, bool kPutOff>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
     const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
-    const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ x,
+    const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ arenaBc, const __nv_bfloat16* __restrict__ x,
     const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
     const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
     const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, const int32_t* __restrict__ adapter_map, uint32_t* status, int T, int K, int N,
@@ -451,15 +451,19 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             for (int t = 0; t < T; ++t) {
                 if (!ctrl->b_lead[t]) continue;
                 const int r8 = (lk->rank_of_row[t] + 7) >> 3;
-                const char* b = reinterpret_cast<const char*>(arenaB + ((size_t)ctrl->slot_of_row[t] * N + row_begin) * kRankPad);
+                // (ranks up to 16 are read from the compact copy of B: 32-byte rows back to back, not a quarter of a padded row each)
+                const bool compact = lk->rank_of_row[t] <= kRankCompact;
+                const int pitch = compact ? kRankCompact * 2 : kRankPad * 2;
+                const char* b = compact ? reinterpret_cast<const char*>(arenaBc + ((size_t)ctrl->slot_of_row[t] * N + row_begin) * kRankCompact)
+                                        : reinterpret_cast<const char*>(arenaB + ((size_t)ctrl->slot_of_row[t] * N + row_begin) * kRankPad);
                 const int off = ctrl->b_of_row[t];
                 if (off >= 0) {
                     for (int i = me; i < rows_cta * r8; i += kDecShrinkWarps * 32) {
                         const int c = i / rows_cta, r = i - c * rows_cta;
-                        cp_async_16(smem_u32(dot_s) + off + i * 16, b + (size_t)r * kRankPad * 2 + c * 16);
+                        cp_async_16(smem_u32(dot_s) + off + i * 16, b + (size_t)r * pitch + c * 16);
                     }
                 } else {
-                    for (int r = me; r < rows_cta; r += kDecShrinkWarps * 32) prefetch_l2(b + (size_t)r * kRankPad * 2);
+                    for (int r = me; r < rows_cta; r += kDecShrinkWarps * 32) prefetch_l2(b + (size_t)r * pitch);
                 }
             }
         };
@@ -746,7 +750,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 const int slot = lora ? ctrl->slot_of_row[t] : -1;
                 if (slot >= 0) {
                     const int r8 = (lk->rank_of_row[t] + 7) >> 3;
-                    const uint4* bp = reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
+                    const uint4* bp = lk->rank_of_row[t] <= kRankCompact
+                                          ? reinterpret_cast<const uint4*>(arenaBc + ((size_t)slot * N + n) * kRankCompact)
+                                          : reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
                     const int bb = ctrl->b_of_row[t];
                     const uint4* bs = reinterpret_cast<const uint4*>(dot_s + bb) + (n - row_begin);
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
@@ -853,6 +859,7 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     float* up = a.u;
     const __nv_bfloat16* arenaA = ar.A;
     const __nv_bfloat16* arenaB = ar.B;
+    const __nv_bfloat16* arenaBc = ar.Bc;
     uint32_t* status = ar.status;
     const int32_t* so = a.seg_offsets;
     const int32_t* ids = a.slot_ids;
@@ -866,7 +873,7 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
     const bool put_off = multi && a.G > 0;
     auto launch = [&](auto kernel) {
-        return cudaLaunchKernelEx(&cfg, kernel, snap, arenaA, arenaB, xb, wb, yb, up, so, ids, pm, ts, amap, status, a.T,
+        return cudaLaunchKernelEx(&cfg, kernel, snap, arenaA, arenaB, arenaBc, xb, wb, yb, up, so, ids, pm, ts, amap, status, a.T,
                                   a.d_in, a.d_out, a.G, g_dec_patience);
     };
     cudaError_t e;

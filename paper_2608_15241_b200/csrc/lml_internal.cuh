@@ -13,6 +13,7 @@ namespace lml {
 
 constexpr int kMaxSlots = LML_MAX_SLOTS;
 constexpr int kRankPad = 64;          // adapters are stored zero-padded to this rank
+constexpr int kRankCompact = 16;      // ... and B a second time, padded to this rank only, where the rank allows
 constexpr int kTileM = 128;           // token rows per GEMM tile and per shrink piece block
 constexpr int kDecodeMaxT = LML_DECODE_MAX_TOKENS;
 constexpr int kMaxAdapterIds = LML_MAX_ADAPTER_IDS;   // adapter ids that can be resolved on the device
@@ -29,6 +30,8 @@ struct SlotSnapshot {
 struct Arena {
     __nv_bfloat16* A;   // [max_slots][kRankPad][d_in]   rows >= rank are zero
     __nv_bfloat16* B;   // [max_slots][d_out][kRankPad]  columns >= rank are zero
+    __nv_bfloat16* Bc;  // [max_slots][d_out][kRankCompact]: the same rows, 32 bytes each, for slots of rank <= kRankCompact
+                        // (what the decode kernel reads: it needs a row's real columns only, a quarter of the padded row)
     uint32_t* status;   // sticky LML_FLAG_* bits
     int32_t* adapter_map;   // [kMaxAdapterIds] serving slot of each adapter id, -1 = none; written by lml_publish
 };
