@@ -525,17 +525,15 @@ lml_status lora_mixed_linear_backward_adapters(lml_table* t, lml_table* t_T, con
     cudaError_t e = launch_shrink_pieces(t->arena, snap, x, T, t->d_in, seg_offsets, slot_ids, G, x, nullptr, plan, u_blocks, stream);
     if (e == cudaSuccess) {
         ++launches;
+        // (a further pass of the same call: it runs beside the first)
         e = launch_shrink_pieces(t_T->arena, snap_T, dy, T, t_T->d_in, seg_offsets, slot_ids_T, G, dy, nullptr, plan,
-                                 u_blocks + set_elems, stream);
+                                 u_blocks + set_elems, stream, 1);
     }
     if (e == cudaSuccess) {
         ++launches;
-        // dA_s[j][k] += sum_t scale.(dy.B)[t][j] x[t][k];   dB_s[n][j] += sum_t dy[t][n] scale.(x.A^T)[t][j]
-        e = launch_weight_grad(snap, u_blocks + set_elems, x, T, t->d_in, seg_offsets, slot_ids, G, dA, 0, stream);
-    }
-    if (e == cudaSuccess) {
-        ++launches;
-        e = launch_weight_grad(snap, u_blocks, dy, T, t->d_out, seg_offsets, slot_ids, G, dB, 1, stream);
+        // dA_s[j][k] += sum_t scale.(dy.B)[t][j] x[t][k];   dB_s[n][j] += sum_t dy[t][n] scale.(x.A^T)[t][j]: one launch
+        e = launch_weight_grad(snap, u_blocks + set_elems, x, T, t->d_in, seg_offsets, slot_ids, G, dA, 0, stream,
+                               u_blocks, dy, t->d_out, dB, 1);
     }
     if (e == cudaSuccess) ++launches;
     t->last_launches = launches;

@@ -360,16 +360,27 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
 // runs over positions, 16 at a time.  P is staged as [position][j] and Q as [position][column], so both
 // operands are read with ldmatrix .trans.  Warp w owns columns 32w .. 32w+31 (four 8-wide tiles) and all
 // 16-row groups of j that the slot's rank needs.
-__global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant__ SlotSnapshot snap,
-                                                          const __nv_bfloat16* __restrict__ pieces,
-                                                          const __nv_bfloat16* __restrict__ Q, int T, int C,
+// One launch does both gradients side by side: blockIdx.z = 0 takes the first set of arguments, 1 the second.
+struct GradJob {
+    const __nv_bfloat16* pieces;
+    const __nv_bfloat16* Q;
+    float* out;
+    int C, mode;
+};
+__global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant__ SlotSnapshot snap, const GradJob job0,
+                                                          const GradJob job1, int T,
                                                           const int32_t* __restrict__ seg_offsets,
-                                                          const int32_t* __restrict__ slot_ids, int G,
-                                                          float* __restrict__ out, int mode)
+                                                          const int32_t* __restrict__ slot_ids, int G)
 {
     extern __shared__ __align__(16) unsigned char grad_smem[];
     ptx::grid_dependency_wait();     // the shrink passes before this kernel are complete now
     ptx::grid_launch_dependents();
+    const GradJob& job = blockIdx.z == 0 ? job0 : job1;
+    const __nv_bfloat16* __restrict__ pieces = job.pieces;
+    const __nv_bfloat16* __restrict__ Q = job.Q;
+    float* __restrict__ out = job.out;
+    const int C = job.C, mode = job.mode;
+    if ((int)blockIdx.x * kGradCols >= C) return;
     const int slot = blockIdx.y;
     const int rank = slot < snap.max_slots ? (int)snap.rank[slot] : 0;
     if (rank == 0) return;
@@ -480,7 +491,7 @@ __global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant_
 
 cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pieces, const void* Q, int T, int C,
                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, float* out, int mode,
-                               cudaStream_t stream)
+                               cudaStream_t stream, const __nv_bfloat16* pieces2, const void* Q2, int C2, float* out2, int mode2)
 {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -490,9 +501,11 @@ cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pi
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    pdl_config(cfg, attr, dim3((C + kGradCols - 1) / kGradCols, snap.max_slots), dim3(256), kGradSmemBytes, stream);
-    return cudaLaunchKernelEx(&cfg, weight_grad_kernel, snap, pieces, (const __nv_bfloat16*)Q, T, C, seg_offsets, slot_ids, G,
-                              out, mode);
+    const int cmax = (out2 && C2 > C) ? C2 : C;
+    pdl_config(cfg, attr, dim3((cmax + kGradCols - 1) / kGradCols, snap.max_slots, out2 ? 2 : 1), dim3(256), kGradSmemBytes, stream);
+    const GradJob j0 = {pieces, (const __nv_bfloat16*)Q, out, C, mode};
+    const GradJob j1 = {pieces2, (const __nv_bfloat16*)Q2, out2, C2, mode2};
+    return cudaLaunchKernelEx(&cfg, weight_grad_kernel, snap, j0, j1, T, seg_offsets, slot_ids, G);
 }
 
 }  // namespace lml

@@ -61,7 +61,9 @@ cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const voi
 // out_s += P_s^T . Q_s per slot (adapter gradients); mode 0: out[slot][j][c], mode 1: out[slot][c][j]
 cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pieces, const void* Q, int T, int C,
                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, float* out, int mode,
-                               cudaStream_t stream);
+                               cudaStream_t stream,   // optionally a second gradient in the same launch:
+                               const __nv_bfloat16* pieces2 = nullptr, const void* Q2 = nullptr, int C2 = 0,
+                               float* out2 = nullptr, int mode2 = 0);
 cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots,
                                   int T, int32_t* perm, int32_t* seg_offsets, int32_t* seg_slot_ids,
                                   cudaStream_t stream, bool by_adapter = false);   // by_adapter: the ids are adapter ids, resolved through ar.adapter_map
