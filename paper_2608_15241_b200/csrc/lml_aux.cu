@@ -339,7 +339,7 @@ cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const voi
 // keeps the sums in registers, so the result does not depend on scheduling.  fp32 accumulation, added
 // onto what out holds.  mode 0: out[slot][j][c] (dA);  mode 1: out[slot][c][j] (dB).
 // ---------------------------------------------------------------------------------------------
-constexpr int kGradCols = 256;                                  // columns of Q (and of the output) per CTA
+constexpr int kGradCols = 128;                                  // columns of Q (and of the output) per CTA: two CTAs fit on an SM
 constexpr int kGradQPitch = kGradCols * 2 + 16;                 // bytes per row of the staged Q tile (16 more: no bank conflicts in ldmatrix)
 constexpr int kGradPPitch = kRankPad * 2 + 16;                  // bytes per row of the staged piece block
 constexpr int kGradQBytes = kTileM * kGradQPitch;
@@ -358,7 +358,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
 
 // out_s (64 x C) += P_s^T (64 x positions) . Q_s (positions x C) on mma.sync m16n8k16: the contraction
 // runs over positions, 16 at a time.  P is staged as [position][j] and Q as [position][column], so both
-// operands are read with ldmatrix .trans.  Warp w owns columns 32w .. 32w+31 (four 8-wide tiles) and all
+// operands are read with ldmatrix .trans.  Warp w owns columns 16w .. 16w+15 (two 8-wide tiles) and all
 // 16-row groups of j that the slot's rank needs.
 // One launch does both gradients side by side: blockIdx.z = 0 takes the first set of arguments, 1 the second.
 struct GradJob {
@@ -367,7 +367,7 @@ struct GradJob {
     float* out;
     int C, mode;
 };
-__global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant__ SlotSnapshot snap, const GradJob job0,
+__global__ void __launch_bounds__(256, 2) weight_grad_kernel(const __grid_constant__ SlotSnapshot snap, const GradJob job0,
                                                           const GradJob job1, int T,
                                                           const int32_t* __restrict__ seg_offsets,
                                                           const int32_t* __restrict__ slot_ids, int G)
@@ -388,11 +388,11 @@ __global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int c0 = blockIdx.x * kGradCols;
     const int ncols = min(kGradCols, C - c0);
-    float acc[4][4][4];   // [16-row group of j][8-column tile][fragment]
+    float acc[4][2][4];   // [16-row group of j][8-column tile][fragment]
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int n = 0; n < 4; ++n) acc[a][n][0] = acc[a][n][1] = acc[a][n][2] = acc[a][n][3] = 0.f;
+        for (int n = 0; n < 2; ++n) acc[a][n][0] = acc[a][n][1] = acc[a][n][2] = acc[a][n][3] = 0.f;
     const uint32_t smem = (uint32_t)__cvta_generic_to_shared(grad_smem);
     auto q_off = [](int buf) { return (uint32_t)(buf * (kGradQBytes + kGradPBytes)); };
     auto p_off = [](int buf) { return (uint32_t)(buf * (kGradQBytes + kGradPBytes) + kGradQBytes); };
@@ -445,12 +445,11 @@ __global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant_
 #pragma unroll 2
         for (int ks = 0; ks < kTileM / 16; ++ks) {
             const int p0 = ks * 16;
-            // B operand for the warp's four column tiles: matrices (p 0-7 | 8-15) x (tile 2h | tile 2h+1)
-            uint32_t bq[4][2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t addr = qb + (uint32_t)((p0 + (mi & 1) * 8 + rr) * kGradQPitch + (warp * 32 + h * 16 + (mi >> 1) * 8) * 2);
-                ldmatrix_x4_trans(addr, bq[2 * h][0], bq[2 * h][1], bq[2 * h + 1][0], bq[2 * h + 1][1]);
+            // B operand for the warp's two column tiles: matrices (p 0-7 | 8-15) x (tile 0 | tile 1)
+            uint32_t bq[2][2];
+            {
+                const uint32_t addr = qb + (uint32_t)((p0 + (mi & 1) * 8 + rr) * kGradQPitch + (warp * 16 + (mi >> 1) * 8) * 2);
+                ldmatrix_x4_trans(addr, bq[0][0], bq[0][1], bq[1][0], bq[1][1]);
             }
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
@@ -461,7 +460,7 @@ __global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant_
                     const uint32_t addr = pb + (uint32_t)((p0 + (mi >> 1) * 8 + rr) * kGradPPitch + (a * 16 + (mi & 1) * 8) * 2);
                     ldmatrix_x4_trans(addr, a0, a1, a2, a3);
 #pragma unroll
-                    for (int n = 0; n < 4; ++n) mma_bf16_16816(acc[a][n], a0, a1, a2, a3, bq[n][0], bq[n][1]);
+                    for (int n = 0; n < 2; ++n) mma_bf16_16816(acc[a][n], a0, a1, a2, a3, bq[n][0], bq[n][1]);
                 }
             }
         }
@@ -475,11 +474,11 @@ __global__ void __launch_bounds__(256) weight_grad_kernel(const __grid_constant_
     for (int a = 0; a < 4; ++a) {
         if (a >= mtiles) continue;
 #pragma unroll
-        for (int n = 0; n < 4; ++n) {
+        for (int n = 0; n < 2; ++n) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int j = a * 16 + gq + (e >> 1) * 8;
-                const int c = c0 + warp * 32 + n * 8 + tq * 2 + (e & 1);
+                const int c = c0 + warp * 16 + n * 8 + tq * 2 + (e & 1);
                 if (j < rank && c < C) {
                     float* o = mode == 0 ? out + ((size_t)slot * kRankPad + j) * C + c : out + ((size_t)slot * C + c) * kRankPad + j;
                     *o += acc[a][n][e];
