@@ -326,7 +326,7 @@ def timed_e2e_loop(rot, steps, warmup, stream):
     from paper_2608_15241_b200 import binding as b
     w = rot.w
     hosts = []
-    for s in rot.sets[: min(rot.R, 4)]:
+    for s in rot.sets:          # all R sets: successive steps never find their weights in L2
         xh = s["x"].cpu().pin_memory()
         yh = torch.empty((w.T, w.d_out), dtype=torch.bfloat16).pin_memory()
         so = s["so_pre"].cpu().pin_memory()
@@ -388,7 +388,8 @@ def units_of(w, kind):
     return w.bytes() / 1e9 if kind == "decode" else w.flops() / 1e12   # GB or TFLOP per step
 
 
-def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e2e_steps):
+def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e2e_steps,
+                 extras=("dual", "backward", "context", "e2e", "shuffled")):
     import torch
     spec = WORKLOADS[name]
     w = spec["make"]()
@@ -410,8 +411,9 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
     secs = max_over_ranks(secs)
 
     # the layer's own launches (pre-segmented input): what the roofline fraction is computed from
-    ksteps = max(rot.R, min(steps, 2000 if kind == "decode" else 200))
-    ksecs, klaunches, _ = timed_graph_loop(rot.layer_only, rot.R, ksteps, max(3, warmup // 4), stream)
+    # (its length does not follow --steps: a kernel time from a handful of calls is not a measurement)
+    ksteps = max(rot.R, 2000 if kind == "decode" else (200 if w.flops() < 2e11 else 60))
+    ksecs, klaunches, _ = timed_graph_loop(rot.layer_only, rot.R, ksteps, max(3 * rot.R, 20), stream)
     per_launch = ksecs / ksteps
     achieved = unit_per_step / per_launch
     if kind == "decode":
@@ -427,7 +429,7 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                 "traffic": None, "us_per_launch": per_launch * 1e6}
 
     dual = None
-    if kind != "decode" and w.G >= 1:
+    if kind != "decode" and w.G >= 1 and "dual" in extras:
         # the same tokens under two bindings: one call with a shared base product against two ordinary calls
         rot.prepare_dual()
         dsteps = max(rot.R, min(steps, 100))
@@ -435,7 +437,7 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
         t_secs, _, _ = timed_graph_loop(rot.two_singles, rot.R, dsteps, 3, stream)
         dual = {"us_per_call": d_secs / dsteps * 1e6, "two_single_calls_us": t_secs / dsteps * 1e6}
     backward = None
-    if kind != "decode" and w.G >= 1 and w.perm is None:
+    if kind != "decode" and w.G >= 1 and w.perm is None and "backward" in extras:
         # the training task's pass through the layer: dx (the layer on the transposed table) and the adapter gradients
         rot.prepare_backward()
         bsteps = max(rot.R, min(steps, 100))
@@ -446,12 +448,12 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
     # host), and the plain library GEMM of the same base shape (harness only: not a target, not part of the path)
     reps = []
     rsteps = max(rot.R, min(ksteps, 400 if kind == "decode" else 60))
-    for _ in range(5):
+    for _ in range(5 if "context" in extras else 1):
         r_secs, _, _ = timed_graph_loop(rot.layer_only, rot.R, rsteps, 3, stream)
         reps.append(r_secs / rsteps * 1e6)
     lat = []
     with torch.cuda.stream(stream):
-        for i in range(40):
+        for i in range(40 if "context" in extras else 3):
             stream.synchronize()
             t_a = time.perf_counter()
             rot.layer_only(i)
@@ -459,6 +461,8 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
             lat.append((time.perf_counter() - t_a) * 1e6)
     mm_us = None
     try:
+        if "context" not in extras:
+            raise RuntimeError("skipped")
         with torch.cuda.stream(stream):
             outs = [torch.empty((w.T, w.d_out), dtype=torch.bfloat16, device=device) for _ in range(2)]
             def mm(i):
@@ -475,27 +479,50 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                "l2_bytes": int(getattr(torch.cuda.get_device_properties(device), "L2_cache_size", 0))}
     roof["traffic"] = ncu_traffic(name)
     roof["algorithmic"] = w.bytes() if kind == "decode" else w.flops()
-    esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
-    esecs = max_over_ranks(esecs)
-    e2e = {"value": world * e2e_steps * unit_per_step / esecs, "unit": spec["unit"], "steps": e2e_steps,
-           "ms_per_step": esecs / e2e_steps * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    e2e = None
+    if "e2e" in extras:
+        esecs, h2d, d2h = timed_e2e_loop(rot, e2e_steps, 3, stream)
+        esecs = max_over_ranks(esecs)
+        e2e = {"value": world * e2e_steps * unit_per_step / esecs, "unit": spec["unit"], "steps": e2e_steps,
+               "ms_per_step": esecs / e2e_steps * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "host_buffer_sets": rot.R}
 
     # quick sampled parity of the last timed step against the oracle (rank 0)
     out = {"metric": spec["metric"], "value": value, "unit": spec["unit"], "ms_per_step": secs / steps * 1e3,
-           "gpu_launches": launches, "roofline": roof, "e2e": e2e, "clocks": clocks, "context": context,
+           "gpu_launches": launches, "roofline": roof, "clocks": clocks, "context": context,
            "config": {"workload": name, "tokens": w.T, "d_in": w.d_in, "d_out": w.d_out,
                       "resident_entries": len(w.entries), "segments": w.G, "rotation_sets": rot.R,
                       "l2_policy": f"inputs larger than L2: {rot.R} distinct weight/activation sets "
                                    f"({rot.R * w.bytes() / 1e6:.0f} MB) visited round-robin",
                       "timing": "CUDA-graph replay of R-step chunks, CUDA events on the launch stream"}}
+    if e2e:
+        out["e2e"] = e2e
     if dual:
         out["dual_version_call"] = dual
     if backward:
         out["backward"] = backward
     if want_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(w, kind, spec["unit"], budget_s=6.0)
+        out["cpu_baseline"] = cpu_baseline(w, kind, spec["unit"], budget_s=6.0 if "context" in extras else 2.0)
         out["parity_sample"] = sampled_parity(rot)
     rot.close()
+    del rot
+    torch.cuda.empty_cache()
+    if kind != "decode" and "shuffled" in extras:
+        # the same batch with its rows in arrival order: per-token ids through the segmentation pass, the
+        # row gather and the scatter epilogue, all inside the timed step
+        ws = wl.mlp_up_gate(shuffled=True) if name == "mlp_up_gate" else wl.shuffle_rows(w)
+        rot_s = Rotation(ws, device, 4 * L2_BYTES)
+        ssteps = max(rot_s.R, min(steps, 200 if ws.flops() < 2e11 else 60))
+        s_secs, s_launches, _ = timed_graph_loop(rot_s.step, rot_s.R, ssteps, max(3 * rot_s.R, 10), stream)
+        s_secs = max_over_ranks(s_secs)
+        out["shuffled_rows"] = {"ms_per_step": s_secs / ssteps * 1e3, "value": world * ssteps * units_of(ws, kind) / s_secs,
+                                "unit": spec["unit"], "steps": ssteps, "launches_per_step": s_launches // ssteps,
+                                "frac_of_measured_burst": units_of(ws, kind) / (s_secs / ssteps) / peaks["tensor_burst"]}
+        if want_cpu_baseline:
+            out["shuffled_rows"]["parity_sample"] = sampled_parity(rot_s)
+        rot_s.close()
+        del rot_s
+        torch.cuda.empty_cache()
     return out
 
 
@@ -541,7 +568,7 @@ def cpu_baseline(w, kind, unit, budget_s):
                       f"{secs * repeats:.1f} s wall on {cores} threads, scaled by rows"}
 
 
-def run_layer_sweep(device, peaks, steps, only=None):
+def run_layer_sweep(device, peaks, steps, only=None, parity=False):
     """The decoder-layer sweep (three distinct projection shapes x five token counts), one cell after
     the other: microseconds per call of lora_mixed_linear_tokens and the fraction of the bound that
     holds for the cell (the slower of bytes / HBM peak and flops / tensor peak)."""
@@ -563,6 +590,10 @@ def run_layer_sweep(device, peaks, steps, only=None):
                           "us_per_call": us, "launches_per_call": launches // n, "GB/s": w.bytes() / secs * n / 1e9,
                           "TFLOP/s": w.flops() / secs * n / 1e12, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
                           "frac_of_bound": max(t_hbm, t_tensor) / (secs / n)})
+            if parity:
+                r = sampled_parity(rot)
+                cells[-1]["parity_sample"] = {"ok": r["ok"], "rows": r["rows"], "rel_fro": r["rel_fro"],
+                                              "worst_tol_ratio": r["worst_tol_ratio"]}
             rot.close()
             del rot
             torch.cuda.empty_cache()
@@ -664,11 +695,23 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
     line.update(primary)
     if not args.no_secondary and args.workload == "decode_q_proj":
+        # the other configurations of the workload, each an object of its own in the same line
         psteps = max(3, min(args.steps, 400))
         sec = run_workload("prefill_q_proj", psteps, max(3, min(warmup, 40)), device, world, peaks, rank == 0,
                            e2e_steps=max(3, min(psteps, 50)))
         sec["steps"] = psteps
         line["prefill"] = sec
+        msteps = max(3, min(args.steps, 100))
+        sec = run_workload("mlp_up_gate", msteps, max(3, min(warmup, 10)), device, world, peaks, rank == 0,
+                           e2e_steps=3, extras=("dual", "shuffled"))
+        sec["steps"] = msteps
+        line["mlp_up_gate"] = sec
+        if rank == 0:
+            line["layer_sweep"] = {"what": "us per lora_mixed_linear_tokens call (segmentation included) and fraction of the "
+                                           "cell's bound = max(bytes / measured HBM peak, flops / measured burst tensor peak) / time; "
+                                           "16 adapters of rank 16, two of them in two versions (18 resident entries), Zipf(1.1) binding",
+                                   "cells": run_layer_sweep(device, peaks, 200, parity=True)}
+        barrier()
     if rank == 0:
         print(json.dumps(line), flush=True)
     if _DIST["on"]:

@@ -99,21 +99,33 @@ lml_status lml_table_destroy(lml_table* t);
  * The new entry is visible to calls issued after this returns; work on OTHER streams must be
  * ordered after `stream` by the caller.  *slot_out receives the physical slot index to use in
  * slot_ids / token_slots (lowest free index).  A rejected call changes nothing: no
- * half-registered entry is ever visible.
+ * half-registered entry is ever visible.  (`stream` is this library's addition to the call: the copy
+ * into the arena is a kernel, and the caller says where it runs.)
  * Errors: INVALID_ARG, DUPLICATE, TABLE_FULL, CUDA.
  */
 lml_status register_adapter(lml_table* t, int adapter_id, int version, const void* A, const void* B,
                             int rank, float scale, void* stream, int* slot_out);
 
 /*
- * retire_version — drop a resident (adapter_id, version) entry (Section 5.3: the old version
- * goes away once in-flight work bound to it is done).  Host-side and immediate for later
- * calls; work already enqueued keeps the slot description it was launched with, but the
- * slot's arena space may be reused by the next register_adapter, so retire only after work
- * bound to that slot has been ordered before the registering stream.  Other slots keep their
- * indices.  Errors: INVALID_ARG, NOT_FOUND.
+ * retire_version / retire_version_on — drop a resident (adapter_id, version) entry (Section 5.3: the
+ * old version goes away once in-flight work bound to it is done).  On the host the entry is gone for
+ * every later call; work already enqueued keeps the slot description it was launched with, but the
+ * slot's arena space may be reused by the next register_adapter, so retire only after work bound to
+ * that slot has been ordered before the registering stream.  Other slots keep their indices.  A pinned
+ * entry only becomes RETIRING (see lml_pin).
+ * Retiring the SERVING version of an adapter also takes it out of the device map that the *_adapters
+ * calls resolve through: a one-thread kernel, enqueued on `stream`, clears the adapter's word if it still
+ * names this entry.  Pass the stream the entry was published on (or one ordered behind it), so that the
+ * clear cannot overtake the publish.  retire_version is retire_version_on with the legacy default stream,
+ * which orders against blocking streams only.  Every later register_adapter makes its stream wait for the
+ * clear before it overwrites a slot.  Independently of all ordering, a word of the map names the
+ * registration it was published for: once that entry is retired, or its slot holds another registration,
+ * the word resolves to "no serving version" (base output, LML_FLAG_BAD_SLOT), never to the slot's new
+ * tenant.  Neither call may be made while `stream` is being captured.
+ * Errors: INVALID_ARG, NOT_FOUND, CUDA (the clear could not be enqueued; the entry stays).
  */
 lml_status retire_version(lml_table* t, int adapter_id, int version);
+lml_status retire_version_on(lml_table* t, int adapter_id, int version, void* stream);
 
 /* Slot index of a resident (adapter_id, version).  Errors: INVALID_ARG, NOT_FOUND. */
 lml_status lml_lookup(const lml_table* t, int adapter_id, int version, int* slot_out);
@@ -142,7 +154,11 @@ size_t lml_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
  * that served before.  The switch is a single 4-byte store on the device, so no call sees a
  * mixture.  The version that served before becomes RETIRING: it stays resident while work is
  * pinned to it and is retired (slot free again) by the unpin that brings its count to zero, or at
- * once if nothing is pinned.  previous_version_out (may be NULL) receives that version, or -1.
+ * once if nothing is pinned.  So work that spans two calls and must see one version (ids resolved by
+ * lml_segment_tokens_adapters, the layer run later by lora_mixed_linear) pins the slot it resolved to,
+ * or does not straddle a publish: without the pin the old slot is free by the time the second call
+ * takes its snapshot, and its tokens get base output and LML_FLAG_BAD_SLOT.
+ * previous_version_out (may be NULL) receives that version, or -1.
  * 0 <= adapter_id < LML_MAX_ADAPTER_IDS.  Errors: INVALID_ARG, NOT_FOUND, CUDA.
  *
  * lml_pin / lml_unpin count work in flight that is bound to a slot (a request that started under
@@ -183,7 +199,8 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * segment whose slot holds no live adapter gets base output and sets LML_FLAG_BAD_SLOT).  Segment g
  * covers positions [seg_offsets[g], seg_offsets[g+1]); position p is row perm[p] of x and y
  * if perm (device int32[T], a permutation) is given, else row p.  G == 0 means "no adapter
- * anywhere".  T == 0 returns LML_OK without launching.
+ * anywhere": the base product is still computed and y written (one launch).  T == 0 returns LML_OK
+ * without launching.
  * T <= 16 runs the bandwidth-bound decode kernel (W0 read once through a bulk-copy ring; with
  * segments its CTAs hand one another their share of the shrink result and count themselves in
  * the table's status block, so two decode calls on the SAME table must not overlap on the GPU:
@@ -315,8 +332,9 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
  * Limits and rules
  *   - T <= LML_DECODE_MAX_TOKENS (16).  A larger T is refused with LML_ERR_TOO_LARGE before
  *     anything is launched; use lora_mixed_linear with a workspace for it.
- *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
- *     that device current).  Make that first call outside any stream capture.
+ *   - Every call looks up the array's device address (cudaGetSymbolAddress, with the table's device
+ *     current; no allocation).  The first call on a device may load the library's device code:
+ *     make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.
  *     Nothing in it has to start at zero: the kernel writes every element it later reads.
  *     Two calls that overlap on the GPU (different streams without ordering, or concurrent

@@ -33,7 +33,7 @@ EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "regist
            "lml_publish", "lml_pin", "lml_unpin", "lml_resolve", "lml_slot_state",
            "lml_segment_tokens_adapters", "lora_mixed_linear_adapters",
            "lml_dual_workspace_bytes", "lora_mixed_linear_dual", "register_adapter_transposed",
-           "lml_backward_workspace_bytes", "lora_mixed_linear_backward_adapters")
+           "lml_backward_workspace_bytes", "lora_mixed_linear_backward_adapters", "retire_version_on")
 
 
 class LmlError(RuntimeError):
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.lml_table_destroy.argtypes = [vp]
         L.register_adapter.argtypes = [vp, i32, i32, vp, vp, i32, ctypes.c_float, vp, ctypes.POINTER(i32)]
         L.retire_version.argtypes = [vp, i32, i32]
+        L.retire_version_on.argtypes = [vp, i32, i32, vp]
         L.lml_lookup.argtypes = [vp, i32, i32, ctypes.POINTER(i32)]
         L.lml_slot_info.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
                                     ctypes.POINTER(ctypes.c_float)]
@@ -129,6 +130,11 @@ def register_adapter(table: int, adapter_id: int, version: int, A_ptr: int, B_pt
 
 def retire_version(table: int, adapter_id: int, version: int) -> None:
     _check(lib().retire_version(table, adapter_id, version), "retire_version")
+
+
+def retire_version_on(table: int, adapter_id: int, version: int, stream: int = 0) -> None:
+    """retire_version whose device-side part (the serving entry leaves the adapter map) runs on `stream`."""
+    _check(lib().retire_version_on(table, adapter_id, version, stream), "retire_version_on")
 
 
 def lml_lookup(table: int, adapter_id: int, version: int) -> int:
@@ -346,8 +352,13 @@ class Table:
         return register_adapter(self.handle, adapter_id, version, _ptr(A), _ptr(B), rank, float(scale),
                                 _stream(stream))
 
-    def retire_version(self, adapter_id: int, version: int) -> None:
-        retire_version(self.handle, adapter_id, version)
+    def retire_version(self, adapter_id: int, version: int, stream="legacy") -> None:
+        """stream="legacy": the C call retire_version (legacy default stream); a torch stream or None (the
+        current stream): retire_version_on."""
+        if isinstance(stream, str):
+            retire_version(self.handle, adapter_id, version)
+        else:
+            retire_version_on(self.handle, adapter_id, version, _stream(stream))
 
     def lookup(self, adapter_id: int, version: int) -> int:
         return lml_lookup(self.handle, adapter_id, version)

@@ -39,6 +39,7 @@ static void free_table_resources(lml_table* t)
     if (t->copy_out) cudaStreamDestroy(t->copy_out);
     if (t->ev_begin) cudaEventDestroy(t->ev_begin);
     if (t->ev_done) cudaEventDestroy(t->ev_done);
+    if (t->ev_map) cudaEventDestroy(t->ev_map);
     for (int c = 0; c < lml_table::kHostChunks; ++c) {
         if (t->ev_in[c]) cudaEventDestroy(t->ev_in[c]);
         if (t->ev_layer[c]) cudaEventDestroy(t->ev_layer[c]);
@@ -102,8 +103,13 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && gemm_sm100_init(device) == cudaSuccess;
     ok = ok && shrink_init() == cudaSuccess;
     ok = ok && decode_init() == cudaSuccess;
+    ok = ok && aux_init() == cudaSuccess;
     ok = ok && encode_tmap_3d(&t->tmap_B256, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
+    ok = ok && encode_tmap_3d(&t->tmap_B128, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
+                              kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 128, 1);
+    gemm_split_override(&t->split_bn, &t->split_s);   // the test knob is read here, never on the hot path
+    ok = ok && cudaEventCreateWithFlags(&t->ev_map, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_in, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_out, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&t->ev_begin, cudaEventDisableTiming) == cudaSuccess;
@@ -150,6 +156,11 @@ lml_status register_adapter(lml_table* t, int adapter_id, int version, const voi
     if (free_slot < 0) return LML_ERR_TABLE_FULL;
     DeviceGuard guard(t->device);
     if (!guard.ok) return LML_ERR_CUDA;
+    // a slot that a retire freed is overwritten only behind the kernel that took it out of the device map
+    if (t->map_clear_recorded && cudaStreamWaitEvent((cudaStream_t)stream, t->ev_map, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
     if (launch_pack_adapter(t->arena, free_slot, A, B, rank, t->d_in, t->d_out, (cudaStream_t)stream) != cudaSuccess) {
         cudaGetLastError();
         return LML_ERR_CUDA;
@@ -157,6 +168,7 @@ lml_status register_adapter(lml_table* t, int adapter_id, int version, const voi
     auto& e = t->entries[free_slot];
     e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
     e.state = LML_STATE_RESIDENT; e.pins = 0;
+    e.gen = ++t->next_gen;
     e.live = true;   // published last: the entry is complete before it becomes visible
     *slot_out = free_slot;
     return LML_OK;
@@ -178,6 +190,10 @@ lml_status register_adapter_transposed(lml_table* t_T, int adapter_id, int versi
     if (free_slot < 0) return LML_ERR_TABLE_FULL;
     DeviceGuard guard(t_T->device);
     if (!guard.ok) return LML_ERR_CUDA;
+    if (t_T->map_clear_recorded && cudaStreamWaitEvent((cudaStream_t)stream, t_T->ev_map, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return LML_ERR_CUDA;
+    }
     if (launch_pack_adapter_transposed(t_T->arena, free_slot, A, B, rank, /*K=*/t_T->d_out, /*N=*/t_T->d_in,
                                        (cudaStream_t)stream) != cudaSuccess) {
         cudaGetLastError();
@@ -186,12 +202,13 @@ lml_status register_adapter_transposed(lml_table* t_T, int adapter_id, int versi
     auto& e = t_T->entries[free_slot];
     e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
     e.state = LML_STATE_RESIDENT; e.pins = 0;
+    e.gen = ++t_T->next_gen;
     e.live = true;
     *slot_out = free_slot;
     return LML_OK;
 }
 
-lml_status retire_version(lml_table* t, int adapter_id, int version)
+lml_status retire_version_on(lml_table* t, int adapter_id, int version, void* stream)
 {
     if (!t) return LML_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(t->mu);
@@ -199,13 +216,19 @@ lml_status retire_version(lml_table* t, int adapter_id, int version)
         auto& e = t->entries[i];
         if (e.live && e.adapter_id == adapter_id && e.version == version) {
             if (e.state == LML_STATE_SERVING) {
-                // no longer the adapter's serving version: calls that name the adapter must stop resolving to it
+                // No longer the adapter's serving version: calls that name the adapter must stop resolving to it.
+                // The word is cleared in stream order, like the publish that set it, and only if it still names
+                // this entry (a newer publish of the adapter stays).  The event lets later registrations order
+                // themselves behind the clear before they reuse the slot.
                 DeviceGuard guard(t->device);
-                const int32_t none = -1;
-                if (!guard.ok || cudaMemcpy(t->arena.adapter_map + adapter_id, &none, sizeof none, cudaMemcpyHostToDevice) != cudaSuccess) {
+                bool ok = guard.ok;
+                ok = ok && launch_clear_word_if(t->arena.adapter_map + adapter_id, adapter_map_word(i, e.gen), (cudaStream_t)stream) == cudaSuccess;
+                ok = ok && cudaEventRecord(t->ev_map, (cudaStream_t)stream) == cudaSuccess;
+                if (!ok) {
                     cudaGetLastError();
                     return LML_ERR_CUDA;
                 }
+                t->map_clear_recorded = true;
             }
             if (e.pins > 0) e.state = LML_STATE_RETIRING;   // freed by the last unpin
             else e.live = false;
@@ -213,6 +236,11 @@ lml_status retire_version(lml_table* t, int adapter_id, int version)
         }
     }
     return LML_ERR_NOT_FOUND;
+}
+
+lml_status retire_version(lml_table* t, int adapter_id, int version)
+{
+    return retire_version_on(t, adapter_id, version, nullptr);   // the legacy default stream
 }
 
 lml_status lml_publish(lml_table* t, int adapter_id, int version, void* stream, int* previous_version_out)
@@ -232,7 +260,7 @@ lml_status lml_publish(lml_table* t, int adapter_id, int version, void* stream, 
     DeviceGuard guard(t->device);
     if (!guard.ok) return LML_ERR_CUDA;
     // the controlled publication point: one 4-byte store, in stream order
-    if (launch_set_word(t->arena.adapter_map + adapter_id, slot, (cudaStream_t)stream) != cudaSuccess) {
+    if (launch_set_word(t->arena.adapter_map + adapter_id, adapter_map_word(slot, t->entries[slot].gen), (cudaStream_t)stream) != cudaSuccess) {
         cudaGetLastError();
         return LML_ERR_CUDA;
     }
@@ -383,8 +411,7 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         int32_t* tile_identity = nullptr;
         if (perm) {
             tile_identity = reinterpret_cast<int32_t*>(wsb + ws.ident_off);
-            e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, tile_identity, !gemm_pairs_forced(),
-                                   t->arena.status, stream);
+            e = launch_gather_rows(x, perm, T, t->d_in, wsb + ws.xg_off, tile_identity, true, t->arena.status, stream);
             if (e == cudaSuccess) { ++launches; xg = wsb + ws.xg_off; }
         }
         PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
@@ -400,8 +427,9 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
             a.plan = plan; a.u_blocks = u_blocks ? u_blocks : reinterpret_cast<const __nv_bfloat16*>(x);
             a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
             a.overlap_with_previous = G > 0;
+            a.split_bn = t->split_bn; a.split_s = t->split_s;
             if (G == 0) a.u_blocks = reinterpret_cast<const __nv_bfloat16*>(W0);   // never read; map needs a valid base
-            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
+            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, &t->tmaps, a, stream);
             if (e == cudaSuccess) ++launches;
         }
     }
@@ -482,7 +510,8 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
         a.plan = plan; a.u_blocks = u_blocks;
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         a.overlap_with_previous = true;
-        e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, a, stream);
+        a.split_bn = 0; a.split_s = 0;   // the dual form runs on whole-K tiles
+        e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, &t->tmaps, a, stream);
         if (e == cudaSuccess) ++launches;
     }
     t->last_launches = launches;

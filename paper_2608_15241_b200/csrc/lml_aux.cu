@@ -66,16 +66,14 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
 // ---------------------------------------------------------------------------------------------
 constexpr int kSegWarps = 32;
 
-// adapter id -> serving slot through the table's device map; -1 stays -1, anything else unknown is -2 (flagged)
-__device__ __forceinline__ int resolve_adapter(const int32_t* __restrict__ adapter_map, int id)
-{
-    if (id == -1) return -1;
-    if (id < 0 || id >= kMaxAdapterIds) return -2;
-    const int s = __ldg(adapter_map + id);
-    return s < 0 ? -2 : s;
-}
-
 __global__ void set_word_kernel(int32_t* dst, int32_t value) { *dst = value; }
+__global__ void clear_word_if_kernel(int32_t* dst, int32_t expected) { if (*dst == expected) *dst = -1; }
+
+cudaError_t launch_clear_word_if(int32_t* dst, int32_t expected, cudaStream_t stream)
+{
+    clear_word_if_kernel<<<1, 1, 0, stream>>>(dst, expected);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream)
 {
@@ -172,7 +170,7 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
         int i = c + lane;
         if (i < end) {
             int s = __ldg(token_slots + i);
-            if (adapter_map) s = resolve_adapter(adapter_map, s);
+            if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
             if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) { bad = true; s = -1; }
             int key = s < 0 ? snap.max_slots : s;
             atomicAdd(&hist[warp][key], 1);
@@ -204,7 +202,7 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
         int key = nk;                          // sentinel for lanes past the end
         if (i < end) {
             int s = __ldg(token_slots + i);
-            if (adapter_map) s = resolve_adapter(adapter_map, s);
+            if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
             if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) s = -1;
             key = s < 0 ? snap.max_slots : s;
         }
@@ -334,10 +332,11 @@ cudaError_t launch_pack_adapter_transposed(const Arena& arT, int slot, const voi
 // ---------------------------------------------------------------------------------------------
 // Adapter gradients: out_s += P_s^T . Q_s over the tokens bound to slot s, where P holds one
 // 64-wide row per position (the piece blocks a shrink pass wrote: scale.(dy.B) for dA, scale.(x.A^T)
-// for dB) and Q is x (for dA, C = d_in) or dy (for dB, C = d_out).  One CTA per (256 columns, slot);
-// a thread owns one column and all 64 rows j of the output, walks the slot's positions in order and
-// keeps the sums in registers, so the result does not depend on scheduling.  fp32 accumulation, added
-// onto what out holds.  mode 0: out[slot][j][c] (dA);  mode 1: out[slot][c][j] (dB).
+// for dB) and Q is x (for dA, C = d_in) or dy (for dB, C = d_out).  One CTA of eight warps per
+// (128 columns, slot), two CTAs to an SM; the contraction over positions runs on mma.sync (see the
+// kernel), the slot's positions are walked in order and the sums stay in registers, so the result does
+// not depend on scheduling.  fp32 accumulation, added onto what out holds.
+// mode 0: out[slot][j][c] (dA);  mode 1: out[slot][c][j] (dB).
 // ---------------------------------------------------------------------------------------------
 constexpr int kGradCols = 128;                                  // columns of Q (and of the output) per CTA: two CTAs fit on an SM
 constexpr int kGradQPitch = kGradCols * 2 + 16;                 // bytes per row of the staged Q tile (16 more: no bank conflicts in ldmatrix)
@@ -494,17 +493,16 @@ cudaError_t launch_weight_grad(const SlotSnapshot& snap, const __nv_bfloat16* pi
 {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(weight_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGradSmemBytes);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     const int cmax = (out2 && C2 > C) ? C2 : C;
     pdl_config(cfg, attr, dim3((cmax + kGradCols - 1) / kGradCols, snap.max_slots, out2 ? 2 : 1), dim3(256), kGradSmemBytes, stream);
     const GradJob j0 = {pieces, (const __nv_bfloat16*)Q, out, C, mode};
     const GradJob j1 = {pieces2, (const __nv_bfloat16*)Q2, out2, C2, mode2};
     return cudaLaunchKernelEx(&cfg, weight_grad_kernel, snap, j0, j1, T, seg_offsets, slot_ids, G);
+}
+
+cudaError_t aux_init()   // called with the table's device current, once per table
+{
+    return cudaFuncSetAttribute(weight_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGradSmemBytes);
 }
 
 }  // namespace lml

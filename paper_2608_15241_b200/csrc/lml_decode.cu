@@ -322,11 +322,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             int my_token_slot = -1;
             if (by_token && lane < T) {
                 my_token_slot = __ldg(token_slots + lane);
-                if (adapter_map) {   // the ids are adapter ids: the table's device map names the serving slot (-2: none, flagged below)
-                    const int id = my_token_slot;
-                    my_token_slot = id == -1 ? -1 : ((id < 0 || id >= kMaxAdapterIds) ? -2 : __ldg(adapter_map + id));
-                    if (id != -1 && my_token_slot < 0) my_token_slot = -2;
-                }
+                // the ids are adapter ids: the table's device map names the serving slot (-2: none, flagged below)
+                if (adapter_map) my_token_slot = resolve_adapter(snap, adapter_map, my_token_slot);
             }
             asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp

@@ -477,11 +477,7 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// kShrink: the same machinery computes the LoRA shrink.  A work item is a piece (block index b = tile m +
-// segment g, see the shrink kernel): u = scale * x_tile . A_slot^T, a 128 x 64 product over all of K with
-// the slot's 64 (zero-padded) rows of A in the place of W0; rows outside the segment are zeroed and the
-// result is written as a bf16 u block.  Launched with a full dependency on the work before it.
-template <int BN, bool kShrink = false>
+template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel(
     const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x0,
     const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_u,
@@ -501,7 +497,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = (int)gridDim.x, rank = (int)blockIdx.x;   // the cluster spans the grid's x dimension
     const int n = (int)blockIdx.y;
-    int m = (int)blockIdx.z;   // (shrink: the block index b; the tile follows from the lookup below)
+    const int m = (int)blockIdx.z;
     const int num_kb = (p.K + kBK - 1) / kBK;
     const bool seg_cached = p.G <= kSegCache;
     // chunks of the tile's 256 columns that CTA r reduces: [first(r), first(r + 1))
@@ -527,60 +523,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
             slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
         }
     }
-    int piece_slot_id = -1, piece_lo = 0, piece_hi = 0;
-    if (kShrink) {
-        grid_launch_dependents();   // the GEMM behind this kernel may start on its base k-blocks
-        const int b = (int)blockIdx.z;
-        if (b == 0 && rank == 0) {   // one CTA validates the segment arrays for the whole call
-            if (p.u_set_rows && threadIdx.x == 0) grid_dependency_wait();   // (a chained pass: see the launcher)
-            int bad_off = 0, bad_slot = 0;
-            for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
-                const int s0 = __ldg(p.seg_offsets + g), s1 = __ldg(p.seg_offsets + g + 1);
-                if (s1 < s0 || s0 < 0 || s1 > p.T) bad_off = 1;
-                const int sl = __ldg(p.slot_ids + g);
-                if (sl != -1 && s1 > s0 && slot_rank(snap, sl) == 0) bad_slot = 1;   // an empty segment may name anything
-            }
-            if (threadIdx.x == 0 && (__ldg(p.seg_offsets) != 0 || __ldg(p.seg_offsets + p.G) != p.T)) bad_off = 1;
-            bad_off = __syncthreads_or(bad_off);
-            bad_slot = __syncthreads_or(bad_slot);
-            if (threadIdx.x == 0) {
-                const_cast<PlanWord*>(p.plan)->lora_ok = bad_off ? 0 : 1;
-                const unsigned f = (bad_off ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u);
-                if (f) atomicOr(p.status, f);
-            }
-        }
-        __syncthreads();   // the segment cache is loaded
-        if (threadIdx.x == 0) {   // which piece has block index b: the largest g with g + first tile of g <= b
-            int lo = 0, hi = p.G;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                const int off = seg_cached ? seg_cache[mid] : __ldg(p.seg_offsets + mid);
-                if (mid + off / kBM <= b) lo = mid; else hi = mid;
-            }
-            const int g = lo, mm = b - g;
-            int found = 0, sl = -1, plo = 0, phi = 0;
-            if (p.G > 0 && mm >= 0 && mm < p.num_m) {
-                const int s0 = seg_cached ? seg_cache[g] : __ldg(p.seg_offsets + g);
-                const int s1 = seg_cached ? seg_cache[g + 1] : __ldg(p.seg_offsets + g + 1);
-                plo = max(max(s0, mm * kBM), 0);
-                phi = min(min(s1, (mm + 1) * kBM), p.T);
-                sl = __ldg(p.slot_ids + g);
-                found = plo < phi && slot_rank(snap, sl) > 0;
-            }
-            ctrl->piece[0] = found; ctrl->piece[1] = sl; ctrl->piece[2] = plo; ctrl->piece[3] = phi;
-        }
-        __syncthreads();
-        if (!ctrl->piece[0]) return;   // every CTA of the cluster shares b and leaves together; nothing reads this block
-        piece_slot_id = ctrl->piece[1]; piece_lo = ctrl->piece[2]; piece_hi = ctrl->piece[3];
-        m = piece_lo / kBM;
-    }
     if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), BN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile int* abort = &ctrl->abort;
-    if (!kShrink && p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
         grid_dependency_wait();
         grid_launch_dependents();
     }
@@ -615,13 +564,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                 if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
                 else tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
-                if (kShrink) tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, kb * kBK, 0, piece_slot_id);   // (tmap_b: the arena of A here)
-                else tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
+                tma_load_2d(a_dst + Cfg::kABytes, &tmap_w, bar, kb * kBK, n * BN);
                 advance();
             }
             // this CTA's share of the tile's LoRA pieces
             bool lora = false;
-            if (!kShrink && p.G > 0) {
+            if (p.G > 0) {
                 grid_dependency_wait();
                 grid_launch_dependents();
                 lora = p.plan->lora_ok != 0;
@@ -752,25 +700,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 }
             }
             const int col0 = n * BN + c * kEpiChunkCols;
-            if (kShrink) {
-                // the piece's u block: scale, zero outside the segment's rows, round; all 128 rows are written
-                const bool mine = pos >= piece_lo && pos < piece_hi;
-                const float sc = mine ? snap.scale[piece_slot_id] : 0.f;
-                __nv_bfloat16* out = p.y + ((size_t)blockIdx.z * kBM + row) * kRankPad + col0;
-                __nv_bfloat16* out_neg = p.y2 ? p.y2 + ((size_t)blockIdx.z * kBM + row) * kRankPad + col0 : nullptr;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint4 v;
-                    v.x = pack_bf16(acc[8 * j + 0] * sc, acc[8 * j + 1] * sc);
-                    v.y = pack_bf16(acc[8 * j + 2] * sc, acc[8 * j + 3] * sc);
-                    v.z = pack_bf16(acc[8 * j + 4] * sc, acc[8 * j + 5] * sc);
-                    v.w = pack_bf16(acc[8 * j + 6] * sc, acc[8 * j + 7] * sc);
-                    if (!mine) v = make_uint4(0, 0, 0, 0);   // (0 * garbage may be a NaN)
-                    *reinterpret_cast<uint4*>(out + j * 8) = v;
-                    if (out_neg) *reinterpret_cast<uint4*>(out_neg + j * 8) = make_uint4(v.x ^ 0x80008000u, v.y ^ 0x80008000u, v.z ^ 0x80008000u, v.w ^ 0x80008000u);
-                }
-                continue;
-            }
             if (!row_ok) continue;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -789,298 +718,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, BN);
-    }
-}
-
-// ---- CTA-pair variant ---------------------------------------------------------------------------------
-// Two CTAs of a cluster share a 256 x 256 tile (cta_group::2).  CTA r of the pair owns rows
-// [256 m2 + 128 r, +128): it stages its own 128 x 64 block of x and HALF of the W0 block (rows
-// n0 + 128 r .. of W0), so a stage is 32 KB instead of 48 KB and the ring is six stages deep — the
-// single-CTA kernel's four stages barely cover one TMA round trip.  The even CTA's MMA thread issues
-// every MMA for both CTAs; the tensor cores fetch the other half of the W0 block from the peer's
-// shared memory.  Barriers: full[] lives in the even CTA and counts both CTAs' TMA bytes; empty[] and
-// tmem_full[] exist in both CTAs and are signalled by one commit addressed to both; tmem_empty[] lives
-// in the even CTA and collects the epilogue warps of both.
-// LoRA pieces: the pair walks the union of the segments that touch either half.  A CTA whose half
-// does not meet a segment loads that stage's u operand from beyond the end of the u blocks, which
-// TMA fills with zeros, so it adds nothing.
-constexpr int kPairStages = 6;
-constexpr int kPairBN = 256;
-constexpr int kPairABytes = kBM * kBK * 2;                 // 16 KB: this CTA's rows of x (or of u)
-constexpr int kPairBBytes = (kPairBN / 2) * kBK * 2;       // 16 KB: this CTA's half of the W0 (or B) block
-constexpr int kPairStageBytes = kPairABytes + kPairBBytes;
-constexpr int kPairEpiBytes = 4 * 2 * kEpiBufBytes;
-constexpr int kPairCtrlBytes = 256 + (kSegCache + 1) * 4 + kSegCache;
-constexpr int kPairSmemBytes = 1024 + kPairStages * kPairStageBytes + kPairEpiBytes + ((kPairCtrlBytes + 15) & ~15);
-
-__global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_pair_kernel(
-    const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-    const __grid_constant__ CUtensorMap tmap_u, const __grid_constant__ CUtensorMap tmap_b,
-    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ SlotSnapshot snap,
-    const GemmParams p)
-{
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw_addr = smem_u32(smem_raw);
-    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
-    uint8_t* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-    const uint32_t epi_addr = tiles_addr + kPairStages * kPairStageBytes;
-    uint8_t* epi_ptr = tiles_ptr + kPairStages * kPairStageBytes;
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(epi_ptr + kPairEpiBytes);
-    int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
-    int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();          // 0 = even CTA: issues the MMAs, owns full[] / tmem_empty[]
-    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int num_m2 = (p.num_m + 1) >> 1;             // 256-row tiles
-    const int num_tiles = num_m2 * p.num_n;
-    const int num_kb = (p.K + kBK - 1) / kBK;
-    const bool seg_cached = p.G <= kSegCache;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->empty[s]), 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&ctrl->tmem_full[a]), 1);
-            mbar_init(smem_u32(&ctrl->tmem_empty[a]), 8);   // four epilogue warps in each CTA
-        }
-        ctrl->abort = 0;
-        fence_mbar_init();
-    }
-    if (warp == 0 && lane == 0) {
-        prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_u);
-        prefetch_tmap(&tmap_b); prefetch_tmap(&tmap_y);
-    }
-    if (seg_cached && p.G > 0) {
-        for (int g = threadIdx.x; g <= p.G; g += kGemmThreads) seg_cache[g] = __ldg(p.seg_offsets + g);
-        for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
-            int s = __ldg(p.slot_ids + g);
-            slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
-        }
-    }
-    if (warp == 1) tmem_alloc_pair(smem_u32(&ctrl->tmem_base), 2 * kPairBN);
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();   // both CTAs' barriers exist before either signals the other
-    tc_fence_after();
-    const uint32_t tmem_base = ctrl->tmem_base;
-    volatile int* abort = &ctrl->abort;
-    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
-        grid_dependency_wait();
-        grid_launch_dependents();
-    }
-
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) {
-            bool lora = false, lora_known = (p.G == 0);
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            auto acquire = [&]() -> bool { return mbar_wait(smem_u32(&ctrl->empty[stage]), phase ^ 1u, abort); };
-            auto advance = [&]() { if (++stage == kPairStages) { stage = 0; phase ^= 1u; } };
-            const int u_rows_total = (p.num_m + (p.G > 0 ? p.G : 1)) * kBM;   // first row coordinate that TMA zero-fills
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                const int m2 = tile % num_m2, n = tile / num_m2;
-                const int m = m2 * 2 + (int)rank;                      // this CTA's 128-row tile
-                const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
-                const int prow0 = m2 * 2 * kBM, prow1 = min(prow0 + 2 * kBM, p.T);   // the pair's rows
-                int g_first = 0, g_end = 0, last_piece = -1;
-                auto seg_at = [&](int g, int& s0, int& s1, int& s) {
-                    if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
-                    else {
-                        s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1); s = __ldg(p.slot_ids + g);
-                        if (slot_rank(snap, s) == 0) s = -1;
-                    }
-                };
-                // slot of the pair's piece for segment g (-1: none) and whether this CTA's half meets it
-                auto pair_piece = [&](int g, bool& mine) -> int {
-                    int s0, s1, s;
-                    seg_at(g, s0, s1, s);
-                    mine = min(s1, row1) > max(s0, row0);
-                    if (min(s1, prow1) <= max(s0, prow0)) return -1;
-                    return s;
-                };
-                for (int kb = 0; kb < num_kb && ok; ++kb) {
-                    if (kb == num_kb - 1) {
-                        if (!lora_known) {
-                            grid_dependency_wait();   // plan word and u blocks come from the shrink kernel
-                            grid_launch_dependents();
-                            lora = p.plan->lora_ok != 0;
-                            lora_known = true;
-                        }
-                        if (lora) {
-                            if (seg_cached) {
-                                int lo = 0, hi = p.G;
-                                while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > prow0) hi = mid; else lo = mid + 1; }
-                                g_first = lo;
-                                g_end = g_first;
-                                while (g_end < p.G && seg_cache[g_end] < prow1) ++g_end;
-                            } else {
-                                g_first = seg_upper(p.seg_offsets, p.G, prow0);
-                                g_end = g_first;
-                                while (g_end < p.G && __ldg(p.seg_offsets + g_end) < prow1) ++g_end;
-                            }
-                            bool mine;
-                            for (int g = g_first; g < g_end; ++g) if (pair_piece(g, mine) >= 0) last_piece = g;
-                        }
-                    }
-                    ok = acquire();
-                    if (!ok) break;
-                    const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
-                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                    if (rank == 0) {
-                        ctrl->stage_info[stage] = 4u | ((kb == num_kb - 1 && last_piece < 0) ? 0x100u : 0u);
-                        mbar_arrive_expect_tx(bar, 2 * kPairStageBytes);   // both CTAs' bytes land on this barrier
-                    }
-                    tma_load_2d_pair(a_dst, &tmap_x, bar, kb * kBK, row0);
-                    tma_load_2d_pair(a_dst + kPairABytes, &tmap_w, bar, kb * kBK, n * kPairBN + (int)rank * (kPairBN / 2));
-                    advance();
-                }
-                for (int g = g_first; g < g_end && ok; ++g) {
-                    bool mine;
-                    const int s = pair_piece(g, mine);
-                    if (s < 0) continue;
-                    ok = acquire();
-                    if (!ok) break;
-                    const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
-                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                    if (rank == 0) {
-                        const uint32_t ksteps = (uint32_t)((snap.rank[s] + 15) >> 4);
-                        ctrl->stage_info[stage] = ksteps | (g == last_piece ? 0x100u : 0u);
-                        mbar_arrive_expect_tx(bar, 2 * kPairStageBytes);
-                    }
-                    tma_load_2d_pair(a_dst, &tmap_u, bar, 0, mine ? (m + g) * kBM : u_rows_total);
-                    tma_load_3d_pair(a_dst + kPairABytes, &tmap_b, bar, 0, n * kPairBN + (int)rank * (kPairBN / 2), s);
-                    advance();
-                }
-            }
-            for (int i = 0; i < kPairStages && ok; ++i) { ok = acquire(); advance(); }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (even CTA only)
-        if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(2 * kBM, kPairBN);
-            int stage = 0;
-            uint32_t phase = 0;
-            int acc = 0;
-            uint32_t acc_phase = 0;
-            bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                ok = mbar_wait(smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1u, abort);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
-                uint32_t accumulate = 0;
-                bool more = true;
-                for (int kb = 0; more; ++kb) {
-                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
-                    if (!ok) break;
-                    const uint32_t a_addr = tiles_addr + stage * kPairStageBytes;
-                    const uint64_t adesc = umma_desc_k128(a_addr);
-                    const uint64_t bdesc = umma_desc_k128(a_addr + kPairABytes);
-                    int ksteps = 4;
-                    if (kb >= num_kb - 1) {
-                        const uint32_t info = ctrl->stage_info[stage];
-                        ksteps = (int)(info & 0xffu);
-                        more = (info & 0x100u) == 0;
-                    }
-#pragma unroll 4
-                    for (int k = 0; k < ksteps; ++k) {
-                        umma_bf16_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
-                        accumulate = 1;
-                    }
-                    umma_commit_pair(smem_u32(&ctrl->empty[stage]));   // frees the stage in both CTAs
-                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
-                }
-                if (!ok) break;
-                umma_commit_pair(smem_u32(&ctrl->tmem_full[acc]));     // both CTAs' epilogues may read
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ epilogue warps (both CTAs)
-        const int q = warp & 3;
-        const int ew = warp - 2;
-        const uint32_t buf_addr0 = epi_addr + (uint32_t)(ew * 2 * kEpiBufBytes);
-        uint8_t* buf_ptr0 = epi_ptr + ew * 2 * kEpiBufBytes;
-        int acc = 0;
-        uint32_t acc_phase = 0;
-        int buf = 0;
-        bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-            const int m2 = tile % num_m2, n = tile / num_m2;
-            const int row_base = (m2 * 2 + (int)rank) * kBM + q * 32;
-            ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), acc_phase, abort);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kPairBN);
-#pragma unroll 1
-            for (int c = 0; c < kPairBN / kEpiChunkCols; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(t_addr + (uint32_t)(c * kEpiChunkCols), r);
-                tmem_ld_wait();
-                if (c == kPairBN / kEpiChunkCols - 1) {
-                    // accumulator fully read: tell the even CTA's MMA thread
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctrl->tmem_empty[acc]), 0));
-                }
-                const int col0 = n * kPairBN + c * kEpiChunkCols;
-                if (col0 >= p.N || row_base >= p.T) continue;
-                if (lane == 0) tma_store_wait_read<1>();
-                __syncwarp();
-                uint8_t* bp = buf_ptr0 + buf * kEpiBufBytes;
-                const uint32_t ba = buf_addr0 + (uint32_t)(buf * kEpiBufBytes);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(r[8 * j + 0]), __uint_as_float(r[8 * j + 1]));
-                    v.y = pack_bf16(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                    v.z = pack_bf16(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                    v.w = pack_bf16(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                    const int phys = j ^ ((lane >> 1) & 3);
-                    *reinterpret_cast<uint4*>(bp + lane * 64 + phys * 16) = v;
-                }
-                if (p.perm == nullptr) {
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmap_y, ba, col0, row_base);
-                        tma_store_commit();
-                    }
-                } else {
-                    __syncwarp();
-#pragma unroll
-                    for (int pass = 0; pass < 4; ++pass) {
-                        const int rr = pass * 8 + (lane >> 2), j = lane & 3;
-                        const int pos = row_base + rr;
-                        if (pos < p.T && col0 + j * 8 < p.N) {
-                            const int row = __ldg(p.perm + pos);
-                            if (row >= 0 && row < p.T) {
-                                const int phys = j ^ ((rr >> 1) & 3);
-                                uint4 v = *reinterpret_cast<const uint4*>(bp + rr * 64 + phys * 16);
-                                *reinterpret_cast<uint4*>(p.y + (size_t)row * p.N + col0 + j * 8) = v;
-                            }
-                        }
-                    }
-                    __syncwarp();
-                }
-                buf ^= 1;
-            }
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        }
-        if (lane == 0) tma_store_wait_all();
-    }
-
-    __syncthreads();
-    cluster_sync_all();   // neither CTA leaves while the other may still read its tiles or signal its barriers
-    if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.status, LML_FLAG_TIMEOUT);
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc_pair(tmem_base, 2 * kPairBN);
     }
 }
 
@@ -1143,16 +780,11 @@ cudaError_t gemm_sm100_init(int /*device*/)
     cudaError_t e = cudaFuncSetAttribute(lora_gemm_sm100_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          GemmCfg<256>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(lora_gemm_sm100_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
-    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              GemmCfg<256>::kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              GemmCfg<128>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(lora_gemm_sm100_splitk_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             GemmCfg<64>::kSmemBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(lora_gemm_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 GemmCfg<128>::kSmemBytes);
@@ -1174,17 +806,28 @@ int gemm_pick_bn(int T, int d_out, int num_sms)
 // fit the machine at once, take the one with the most CTAs, and among equals the smaller cluster (less
 // to exchange); every CTA keeps at least two k-blocks, and the exchange area must fit the stage memory.
 struct SplitChoice { int bn, split; };
-static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
+// The table's override (LML_GEMM_SPLIT, read once when the table is created; a test knob): "<bn>x<split>"
+// forces that shape, 0 switches the split-K kernel off.  Returns false when the variable is not set.
+bool gemm_split_override(int* bn_out, int* split_out)
+{
+    *bn_out = -1; *split_out = -1;
+    const char* e = getenv("LML_GEMM_SPLIT");
+    if (!e) return false;
+    int bn = 0, sp = 0;
+    if (sscanf(e, "%dx%d", &bn, &sp) == 2 && (bn == 128 || bn == 256) && sp >= 2 && sp <= kSplitMaxS &&
+        sp * ((bn / 32 + sp - 1) / sp) * 16384 <= GemmCfg<128>::kStages * GemmCfg<128>::kStageBytes) {
+        *bn_out = bn; *split_out = sp;
+    } else {
+        *bn_out = 0; *split_out = 0;
+    }
+    return true;
+}
+
+static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms, int forced_bn, int forced_split)
 {
     static int max_clusters[2][kSplitMaxS + 1];
     static std::once_flag probed;
-    if (const char* e = getenv("LML_GEMM_SPLIT")) {   // test knob: "<bn>x<split>", or 0 for no split
-        int bn = 0, sp = 0;
-        if (sscanf(e, "%dx%d", &bn, &sp) == 2 && (bn == 128 || bn == 256) && sp >= 2 && sp <= kSplitMaxS &&
-            sp * ((bn / 32 + sp - 1) / sp) * 16384 <= GemmCfg<128>::kStages * GemmCfg<128>::kStageBytes)
-            return {bn, sp};
-        return {0, 0};
-    }
+    if (forced_bn >= 0) return {forced_bn, forced_split};
     std::call_once(probed, [&]() {   // clusters of each size that can be resident together
         for (int w = 0; w < 2; ++w)
             for (int S = 2; S <= kSplitMaxS; ++S) {
@@ -1219,57 +862,57 @@ static SplitChoice gemm_pick_split(int T, int d_in, int d_out, int num_sms)
     return best;
 }
 
-// LML_FORCE_GEMM=pair|single overrides the choice below (a test knob: small problems would
-// otherwise never reach the pair kernel).
-static int gemm_forced_mode()
+// Tensor maps of the caller's buffers are kept per table: a serving loop calls with the same few
+// (pointer, shape) combinations over and over, and encoding a map costs a driver call each time.
+bool TmapCache::get_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t stride_bytes,
+                       uint32_t box_inner, uint32_t box_outer)
 {
-    static int mode = -1;
-    if (mode < 0) {
-        const char* e = getenv("LML_FORCE_GEMM");
-        mode = !e ? 0 : (e[0] == 'p' ? 1 : (e[0] == 's' ? 2 : 0));
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i) {
+        const Key& k = keys[i];
+        if (k.base == base && k.inner == inner && k.outer == outer && k.stride == stride_bytes && k.box_inner == box_inner &&
+            k.box_outer == box_outer) {
+            *out = maps[i];
+            return true;
+        }
     }
-    return mode;
+    CUtensorMap m;
+    if (!encode_tmap_2d(&m, base, inner, outer, stride_bytes, box_inner, box_outer)) return false;
+    const int slot = used < kEntries ? used++ : (next = (next + 1) % kEntries);
+    keys[slot] = Key{base, inner, outer, stride_bytes, box_inner, box_outer};
+    maps[slot] = m;
+    *out = m;
+    return true;
 }
 
-bool gemm_pairs_forced() { return gemm_forced_mode() == 1; }
-
-static bool gemm_use_pairs(int /*T*/, int /*d_out*/, int /*num_sms*/)
+cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B256,
+                              const CUtensorMap& tmap_B128, TmapCache* cache, const GemmArgs& a, cudaStream_t stream)
 {
-    // Measured on B200 (prefill_q_proj / mlp_up_gate, us per call): single-CTA tiles 66 / 314, CTA
-    // pairs 74 / 349.  Pairs halve the W0 bytes each SM stages and give a six-stage ring, but the
-    // cross-CTA barrier round trip costs more than that buys, so the single-CTA kernel is the
-    // default and the pair kernel is selected only on request.
-    return gemm_forced_mode() == 1;
-}
-
-cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B,
-                              const GemmArgs& a, cudaStream_t stream)
-{
-    const bool pairs = gemm_use_pairs(a.T, a.d_out, a.num_sms);
-    const SplitChoice sc = (pairs || a.slot_ids2 != nullptr) ? SplitChoice{0, 0} : gemm_pick_split(a.T, a.d_in, a.d_out, a.num_sms);
+    const bool dual = a.slot_ids2 != nullptr;
+    if (dual && (a.G <= 0 || !a.y2)) return cudaErrorInvalidValue;
+    const SplitChoice sc = gemm_pick_split(a.T, a.d_in, a.d_out, a.num_sms, a.split_bn, a.split_s);
     const int split = sc.split;
-    const int bn = pairs ? kPairBN : (split ? sc.bn : gemm_pick_bn(a.T, a.d_out, a.num_sms));
+    const int bn = split ? sc.bn : gemm_pick_bn(a.T, a.d_out, a.num_sms);
     const int num_m = (a.T + kBM - 1) / kBM;
     const int num_n = (a.d_out + bn - 1) / bn;
-    const uint32_t w_box_rows = pairs ? (uint32_t)(kPairBN / 2) : (uint32_t)bn;
-    const bool dual = a.slot_ids2 != nullptr;
-    if (dual && (pairs || a.G <= 0 || !a.y2)) return cudaErrorInvalidValue;
-    CUtensorMap tx, tx0, tw, tu, ty, ty2, tb = tmap_B;
-    if (!encode_tmap_2d(&tx, a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
-    if (!encode_tmap_2d(&tx0, a.x_in_place ? a.x_in_place : a.x, (uint64_t)a.d_in, (uint64_t)a.T, (uint64_t)a.d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
-    if (!encode_tmap_2d(&tw, a.W0, (uint64_t)a.d_in, (uint64_t)a.d_out, (uint64_t)a.d_in * 2, kBK, w_box_rows)) return cudaErrorInvalidValue;
+    TmapCache local;   // (a call without a table-owned cache encodes its maps afresh)
+    TmapCache* tc = cache ? cache : &local;
+    CUtensorMap tx, tx0, tw, tu, ty, ty2;
+    const CUtensorMap& tb = bn == 256 ? tmap_B256 : tmap_B128;
     const uint64_t u_set_rows = (uint64_t)(num_m + (a.G > 0 ? a.G : 1)) * kBM;
     const uint64_t u_rows = u_set_rows * (dual ? 3 : 1);
-    if (!encode_tmap_2d(&tu, a.u_blocks, kRankPad, u_rows, kRankPad * 2, kBK, kBM)) return cudaErrorInvalidValue;
-    if (!encode_tmap_2d(&ty, a.y, (uint64_t)a.d_out, (uint64_t)a.T, (uint64_t)a.d_out * 2, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
-    if (!encode_tmap_2d(&ty2, dual ? a.y2 : a.y, (uint64_t)a.d_out, (uint64_t)a.T, (uint64_t)a.d_out * 2, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
-    if (pairs || bn != 256) {
-        if (!encode_tmap_3d(&tb, ar.B, kRankPad, (uint64_t)a.d_out, (uint64_t)snap.max_slots, kRankPad * 2,
-                            (uint64_t)a.d_out * kRankPad * 2, kBK, w_box_rows, 1)) return cudaErrorInvalidValue;
+    const uint64_t xs = (uint64_t)a.d_in * 2, ys = (uint64_t)a.d_out * 2;
+    if (!tc->get_2d(&tx, a.x, (uint64_t)a.d_in, (uint64_t)a.T, xs, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!tc->get_2d(&tx0, a.x_in_place ? a.x_in_place : a.x, (uint64_t)a.d_in, (uint64_t)a.T, xs, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!tc->get_2d(&tw, a.W0, (uint64_t)a.d_in, (uint64_t)a.d_out, xs, kBK, (uint32_t)bn)) return cudaErrorInvalidValue;
+    if (!tc->get_2d(&tu, a.u_blocks, kRankPad, u_rows, kRankPad * 2, kBK, kBM)) return cudaErrorInvalidValue;
+    if (!split) {   // (the split-K kernel stores its outputs with plain stores)
+        if (!tc->get_2d(&ty, a.y, (uint64_t)a.d_out, (uint64_t)a.T, ys, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
+        if (!tc->get_2d(&ty2, dual ? a.y2 : a.y, (uint64_t)a.d_out, (uint64_t)a.T, ys, kEpiChunkCols, 32)) return cudaErrorInvalidValue;
     }
     GemmParams p;
     p.seg_offsets = a.seg_offsets; p.slot_ids = a.slot_ids; p.perm = a.perm; p.plan = a.plan;
-    p.tile_identity = pairs ? nullptr : a.tile_identity;
+    p.tile_identity = a.tile_identity;
     p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
     p.slot_ids2 = a.slot_ids2; p.y2 = (__nv_bfloat16*)a.y2; p.u_set_rows = (int)u_set_rows;
     p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
@@ -1282,20 +925,6 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
         attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[nattr].val.programmaticStreamSerializationAllowed = 1;
         ++nattr;
-    }
-    if (pairs) {
-        const int pair_tiles = ((num_m + 1) / 2) * num_n;
-        const int npairs = min(pair_tiles, a.num_sms / 2);
-        cfg.gridDim = dim3(2 * npairs);
-        cfg.dynamicSmemBytes = kPairSmemBytes;
-        attr[nattr].id = cudaLaunchAttributeClusterDimension;
-        attr[nattr].val.clusterDim.x = 2;
-        attr[nattr].val.clusterDim.y = 1;
-        attr[nattr].val.clusterDim.z = 1;
-        ++nattr;
-        cfg.attrs = attr;
-        cfg.numAttrs = nattr;
-        return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_pair_kernel, tx, tw, tu, tb, ty, snap, p);
     }
     if (split) {
         cfg.gridDim = dim3(split, num_n, num_m);
@@ -1316,71 +945,6 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.numAttrs = nattr;
     if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
     return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
-}
-
-
-// The LoRA shrink on the tensor cores: the shrink form of the split-K kernel, one cluster per block index.
-// Returns cudaErrorNotSupported when the caller should use the mma.sync kernel instead.
-cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
-                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, const void* x_in_place,
-                                const int32_t* tile_identity, PlanWord* plan, __nv_bfloat16* u_blocks,
-                                cudaStream_t stream, bool chained, __nv_bfloat16* u_blocks_neg)
-{
-    static int max_clusters[kSplitMaxS + 1];
-    static int num_sms = 0;
-    static std::once_flag probed;
-    std::call_once(probed, [&]() {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return;
-        }
-        for (int S = 1; S <= kSplitMaxS; ++S) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(S, 1, sms / S);
-            cfg.blockDim = dim3(kGemmThreads);
-            cfg.dynamicSmemBytes = GemmCfg<64>::kSmemBytes;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr; cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, lora_gemm_sm100_splitk_kernel<64, true>, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
-            max_clusters[S] = n;
-        }
-        num_sms = sms;
-    });
-    if (num_sms == 0) return cudaErrorNotSupported;
-    const int num_m = (T + kBM - 1) / kBM, num_kb = (d_in + kBK - 1) / kBK;
-    const int blocks = num_m + (G > 0 ? G : 1);
-    // as many CTAs per piece as still leaves every block index a cluster that is resident at once
-    int split = 1;
-    for (int S = 2; S <= kSplitMaxS; ++S)
-        if (blocks <= max_clusters[S] && num_kb >= 2 * S) split = S;
-    CUtensorMap tx, tx0, ta;
-    if (!encode_tmap_2d(&tx, x, (uint64_t)d_in, (uint64_t)T, (uint64_t)d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
-    if (!encode_tmap_2d(&tx0, x_in_place ? x_in_place : x, (uint64_t)d_in, (uint64_t)T, (uint64_t)d_in * 2, kBK, kBM)) return cudaErrorInvalidValue;
-    if (!encode_tmap_3d(&ta, ar.A, (uint64_t)d_in, kRankPad, (uint64_t)snap.max_slots, (uint64_t)d_in * 2,
-                        (uint64_t)d_in * kRankPad * 2, kBK, kRankPad, 1)) return cudaErrorInvalidValue;
-    GemmParams p = {};
-    p.seg_offsets = seg_offsets; p.slot_ids = slot_ids; p.perm = nullptr; p.plan = plan;
-    p.tile_identity = tile_identity;
-    p.y = u_blocks; p.y2 = u_blocks_neg; p.status = ar.status; p.slot_ids2 = nullptr;
-    p.u_set_rows = chained ? 1 : 0;
-    p.T = T; p.K = d_in; p.N = kRankPad; p.G = G; p.num_m = num_m; p.num_n = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(split, 1, blocks);
-    cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = GemmCfg<64>::kSmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // only a chained pass starts before its predecessor ends
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = chained ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_splitk_kernel<64, true>, tx, tx0, tx, tx, ta, snap, p);
 }
 
 }  // namespace lml

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "lora_mixed_linear.h"
 
 namespace lml {
@@ -24,6 +26,7 @@ struct SlotSnapshot {
     uint8_t rank[kMaxSlots];   // 0 = slot not live.  First, with max_slots right behind: what a kernel needs
     int32_t max_slots;         // first sits in one or two lines of the parameter cache (a miss there costs
     float scale[kMaxSlots];    // as much as a trip to L2)
+    uint16_t gen[kMaxSlots];   // registration counter of the entry in the slot: what a word of the adapter map must name
 };
 
 // Device-resident pieces of a table.
@@ -33,8 +36,10 @@ struct Arena {
     __nv_bfloat16* Bc;  // [max_slots][d_out][kRankCompact]: the same rows, 32 bytes each, for slots of rank <= kRankCompact
                         // (what the decode kernel reads: it needs a row's real columns only, a quarter of the padded row)
     uint32_t* status;   // sticky LML_FLAG_* bits
-    int32_t* adapter_map;   // [kMaxAdapterIds] serving slot of each adapter id, -1 = none; written by lml_publish
+    int32_t* adapter_map;   // [kMaxAdapterIds] serving entry of each adapter id: slot | generation << 8, -1 = none; written by lml_publish
 };
+
+inline int32_t adapter_map_word(int slot, uint16_t gen) { return (int32_t)((uint32_t)slot | ((uint32_t)gen << 8)); }
 
 // Workspace header written by the shrink kernels and read by the kernels that follow.
 struct PlanWord {
@@ -48,6 +53,8 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
                                 int d_in, int d_out, cudaStream_t stream);
 
 cudaError_t launch_set_word(int32_t* dst, int32_t value, cudaStream_t stream);
+cudaError_t launch_clear_word_if(int32_t* dst, int32_t expected, cudaStream_t stream);   // *dst = -1 if it still holds `expected`
+cudaError_t aux_init();   // sets the dynamic shared memory attribute of the gradient kernel
 // per-chunk segment arrays ([offsets (G + 1) | slot ids (G)] every `stride` ints) of a call done in chunks of `rows` rows
 cudaError_t launch_clip_segments(const int32_t* seg_offsets, const int32_t* slot_ids, int G, int T, int rows, int chunks,
                                  int32_t* out, int stride, cudaStream_t stream);
@@ -77,16 +84,9 @@ cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, cons
                                  __nv_bfloat16* u_blocks, cudaStream_t stream, int chained = 0,   // 1: a further pass of the same call, may run beside the one before; 2: behind the call's row-gather kernel
                                  __nv_bfloat16* u_blocks_neg = nullptr);                              // optional second copy of the blocks, negated
 
-// The same pass on the tcgen05 tensor cores (the split-K kernel's shrink form); same arguments.
-cudaError_t launch_shrink_sm100(const Arena& ar, const SlotSnapshot& snap, const void* x, int T, int d_in,
-                                const int32_t* seg_offsets, const int32_t* slot_ids, int G, const void* x_in_place,
-                                const int32_t* tile_identity, PlanWord* plan, __nv_bfloat16* u_blocks,
-                                cudaStream_t stream, bool chained = false, __nv_bfloat16* u_blocks_neg = nullptr);
-
 // tile_identity[m] = 1: tile m's perm is the identity, its rows were not copied and stay in place.
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
                                int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream);
-bool gemm_pairs_forced();   // the CTA-pair kernel does not read tile_identity
 
 struct GemmArgs {
     const void* x;            // rows in position order (already gathered when perm is used)
@@ -103,11 +103,25 @@ struct GemmArgs {
     void* y2 = nullptr;                   // (num_m + G) blocks: first slots, second slots, first slots negated
     int T, d_in, d_out, G;
     int num_sms;
+    int split_bn = -1, split_s = -1;   // the table's split-K override: -1 = the library chooses, 0 = off, else the forced shape
     bool overlap_with_previous;   // launch as a programmatic dependent of the shrink kernel before it
 };
+// Tensor maps of caller buffers, kept per table and found again by (pointer, shape, box).
+struct TmapCache {
+    static constexpr int kEntries = 32;
+    struct Key { const void* base; uint64_t inner, outer, stride; uint32_t box_inner, box_outer; };
+    Key keys[kEntries];
+    CUtensorMap maps[kEntries];
+    int used = 0, next = 0;
+    std::mutex mu;
+    bool get_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t stride_bytes,
+                uint32_t box_inner, uint32_t box_outer);
+};
+bool gemm_split_override(int* bn_out, int* split_out);
+// tmap_B256 / tmap_B128: the table's maps of its packed B arena for 256- and 128-column tiles.
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
-cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B,
-                              const GemmArgs& a, cudaStream_t stream);
+cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B256,
+                              const CUtensorMap& tmap_B128, TmapCache* cache, const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_sm100_init(int device);
 cudaError_t shrink_init();   // both set the dynamic shared memory attributes of their kernels
 bool encode_tmap_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,
@@ -199,6 +213,20 @@ __device__ __forceinline__ int seg_upper(const int32_t* __restrict__ seg_offsets
 __device__ __forceinline__ int slot_rank(const SlotSnapshot& snap, int slot)
 {
     return (slot >= 0 && slot < snap.max_slots) ? (int)snap.rank[slot] : 0;
+}
+
+// adapter id -> serving slot through the table's device map.  -1 stays -1 (no adapter); an id out of range,
+// without a serving version, or whose map word names an entry that is no longer the one in that slot
+// (retired, slot taken by another registration since) gives -2: no adapter, and the caller raises the flag.
+__device__ __forceinline__ int resolve_adapter(const SlotSnapshot& snap, const int32_t* __restrict__ adapter_map, int id)
+{
+    if (id == -1) return -1;
+    if (id < 0 || id >= kMaxAdapterIds) return -2;
+    const int v = __ldg(adapter_map + id);
+    if (v < 0) return -2;
+    const int slot = v & 0xff;
+    if (slot >= snap.max_slots || snap.rank[slot] == 0 || snap.gen[slot] != (uint16_t)((uint32_t)v >> 8)) return -2;
+    return slot;
 }
 
 }  // namespace lml

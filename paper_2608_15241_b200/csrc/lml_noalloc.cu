@@ -17,27 +17,19 @@ constexpr size_t kStaticScratchBytes = 4096;
 static_assert(kStaticU <= kStaticScratchBytes, "static scratch too small");
 
 // In host code this name is only a handle for the runtime, not a device address: the address the
-// kernels get is looked up once per device with cudaGetSymbolAddress below.
+// kernels get is looked up with cudaGetSymbolAddress below, with the table's device current.
 static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-std::mutex g_setup_mu;
-void* g_scratch_ptr[kMaxDevices] = {};
-
-// Device address of the scratch array on `device` (which must be the current device).  The first
-// call on a device asks the runtime for it; later calls reuse the answer.
-cudaError_t scratch_address(int device, void** out)
+// Device address of the scratch array on the current device.  Asked of the runtime on every call: the
+// lookup allocates nothing and costs little, and an address remembered across a tear-down of the device's
+// context (cudaDeviceReset and a new table on the same ordinal) would be stale.
+cudaError_t scratch_address(void** out)
 {
-    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(g_setup_mu);
-    if (!g_scratch_ptr[device]) {
-        void* p = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&p, g_decode_scratch);
-        if (e != cudaSuccess) return e;
-        if (!p) return cudaErrorInvalidSymbol;
-        g_scratch_ptr[device] = p;
-    }
-    *out = g_scratch_ptr[device];
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_decode_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    *out = p;
     return cudaSuccess;
 }
 
@@ -59,7 +51,7 @@ extern "C" lml_status lora_mixed_linear_decode_static(lml_table* t, const void* 
     if (!guard.ok) return LML_ERR_CUDA;
 
     void* scratch = nullptr;
-    if (scratch_address(t->device, &scratch) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+    if (scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
     float* u = static_cast<float*>(scratch);
 
     // The array keeps whatever the previous call left.  Nothing has to start at zero: the kernel

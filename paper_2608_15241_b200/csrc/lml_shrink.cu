@@ -272,17 +272,6 @@ cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, cons
                                  const void* x_in_place, const int32_t* tile_identity, PlanWord* plan,
                                  __nv_bfloat16* u_blocks, cudaStream_t stream, int chained, __nv_bfloat16* u_blocks_neg)
 {
-    // LML_SHRINK=tensor selects the tcgen05 form (the split-K kernel's shrink mode).  Measured on B200 it is
-    // no faster than the kernel of this file (prefill_q_proj 65.7 against 64.6 us per layer call, 128 tokens
-    // 31 against 27 us; 8192 tokens 259 against 267 us), so it stays a switch with its own test.
-    if (G > 0) {
-        const char* env = getenv("LML_SHRINK");
-        if (env && env[0] == 't') {
-            cudaError_t e = launch_shrink_sm100(ar, snap, x, T, d_in, seg_offsets, slot_ids, G, x_in_place, tile_identity, plan,
-                                                u_blocks, stream, chained == 1, u_blocks_neg);
-            if (e != cudaErrorNotSupported) return e;
-        }
-    }
     int max_rank = 0;
     for (int i = 0; i < snap.max_slots; ++i) max_rank = snap.rank[i] > max_rank ? snap.rank[i] : max_rank;
     if (max_rank <= 16)

@@ -13,9 +13,17 @@ struct lml_table {
         float scale = 0.f;
         int state = 0;   // LML_STATE_*: resident (staged or plain), serving, retiring
         int pins = 0;    // work in flight that is bound to this entry
+        uint16_t gen = 0;   // the table's registration counter when the entry was made (see the adapter map)
     } entries[lml::kMaxSlots];
+    uint16_t next_gen = 0;
     lml::Arena arena{};
-    CUtensorMap tmap_B256;   // packed B arena as [max_slots][d_out][64], box 64 x 256 x 1
+    CUtensorMap tmap_B256, tmap_B128;   // packed B arena as [max_slots][d_out][64], boxes 64 x 256 x 1 and 64 x 128 x 1
+    lml::TmapCache tmaps;               // tensor maps of the caller's buffers seen so far
+    int split_bn = -1, split_s = -1;    // LML_GEMM_SPLIT as it stood when the table was created (-1: not set)
+    // Retiring a serving entry clears its word of the device map with a kernel on a stream; the event marks
+    // that point, and every later registration makes its own stream wait for it before it overwrites a slot.
+    cudaEvent_t ev_map = nullptr;
+    bool map_clear_recorded = false;
     int last_launches = 0;
     // host-buffer form of large calls: the copies of x in and of y out run on two streams of the table's own,
     // chunk by chunk beside the layer (created with the table: the call itself creates nothing)
@@ -50,6 +58,7 @@ inline SlotSnapshot snapshot_locked(const lml_table* t)
         const bool live = i < t->max_slots && t->entries[i].live;
         s.rank[i] = live ? (uint8_t)t->entries[i].rank : 0;
         s.scale[i] = live ? t->entries[i].scale : 0.f;
+        s.gen[i] = live ? t->entries[i].gen : (uint16_t)0;
     }
     s.max_slots = t->max_slots;
     return s;

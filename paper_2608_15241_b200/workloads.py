@@ -210,6 +210,18 @@ def prefill_q_proj(seed: int = 0) -> Workload:
     return Workload("prefill_q_proj", K, N, T, x, W0, entries, off, seg_entry, tok)
 
 
+def shuffle_rows(w: Workload, seed: int = 3) -> Workload:
+    """The same batch with its rows in arrival order instead of grouped: row r of the result is a
+    random row of `w`; perm / seg_offsets / seg_entry are the stable grouping of the shuffled
+    per-token binding (what the token-segmentation pass has to produce)."""
+    assert w.perm is None
+    order = _rng(seed, _STREAM_ASSIGN + 2).permutation(w.T).astype(np.int32)
+    tok = w.token_entry[order].astype(np.int32)
+    perm, off, seg_entry = group_tokens(tok, len(w.entries))
+    return Workload(w.name + "_shuffled", w.d_in, w.d_out, w.T, np.ascontiguousarray(w.x[order]), w.W0,
+                    w.entries, off, seg_entry, tok, perm)
+
+
 def zipf_assign(seed: int, stream: int, count: int, num: int, s: float) -> np.ndarray:
     """count i.i.d. draws from p_i proportional to (i+1)^-s over i = 0..num-1."""
     p = np.arange(1, num + 1, dtype=np.float64) ** (-s)

@@ -12,6 +12,33 @@ def to_bits(t) -> np.ndarray:
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
+class Guarded:
+    """A device buffer between two canary bands.  The library is handed the middle; after the call the
+    bands must still hold the canary byte: a write before or behind a buffer is caught even without a
+    memory checker.  The payload starts out as 0xFF bytes (a bf16 / fp32 NaN), so an element the
+    library should have written and did not shows up in any comparison."""
+
+    BAND = 4096
+    CANARY = 0xA5
+
+    def __init__(self, nbytes, device="cuda:0", fill=0xFF):
+        import torch
+        self.nbytes = int(nbytes)
+        pad = (-self.nbytes) % 256
+        self.raw = torch.full((2 * self.BAND + self.nbytes + pad,), self.CANARY, dtype=torch.uint8, device=device)
+        self.payload = self.raw[self.BAND:self.BAND + self.nbytes]
+        if self.nbytes:
+            self.payload.fill_(fill)
+
+    def view(self, dtype, shape):
+        return self.payload.view(dtype).view(*shape)
+
+    def intact(self) -> bool:
+        head = self.raw[:self.BAND]
+        tail = self.raw[self.BAND + self.nbytes:]
+        return bool((head == self.CANARY).all().item()) and bool((tail == self.CANARY).all().item())
+
+
 class Site:
     """A table with a workload's entries registered and its tensors resident on the GPU."""
 
@@ -42,12 +69,35 @@ class Site:
         dids = torch.from_numpy(ids).to(self.device) if len(ids) else None
         dpm = None if pm is None else torch.from_numpy(np.ascontiguousarray(pm, dtype=np.int32)).to(self.device)
         xx = self.x if x is None else x
-        y = self.table.lora_mixed_linear(xx, self.W0, dso, dids, dpm)
+        # output and workspace sit between canary bands; the workspace is exactly as large as the library asks
+        T, G = int(xx.shape[0]), len(ids)
+        gy = Guarded(T * w.d_out * 2, self.device)
+        gws = Guarded(max(self.table.workspace_bytes(T, G), 256), self.device)
+        y = gy.view(torch.bfloat16, (T, w.d_out))
+        self.table.lora_mixed_linear(xx, self.W0, dso, dids, dpm, y=y, workspace=gws.payload)
         torch.cuda.synchronize()
+        assert gy.intact(), "the call wrote outside y"
+        assert gws.intact(), "the call wrote outside its workspace"
         return to_bits(y), self.table.device_status()
 
     def close(self):
         self.table.close()
+
+
+def sample_positions_every_tile(w, count, tile=128, seed=0):
+    """At least `count` positions: one in every `tile`-row band (so that no row tile of the GEMM goes
+    unchecked), every segment's first and last row, and random ones."""
+    rng = np.random.default_rng(seed)
+    pos = set()
+    for t0 in range(0, w.T, tile):
+        pos.add(int(rng.integers(t0, min(t0 + tile, w.T))))
+    for g in range(w.G):
+        a, b = int(w.seg_offsets[g]), int(w.seg_offsets[g + 1])
+        if b > a:
+            pos.update((a, b - 1))
+    while len(pos) < min(count, w.T):
+        pos.add(int(rng.integers(0, w.T)))
+    return np.array(sorted(pos), dtype=np.int32)
 
 
 def sample_positions(w, count, seed=0):

@@ -54,5 +54,14 @@ def test_fused_qkv_equals_separate_calls(T):
     tbl.close()
 
     assert np.array_equal(y_fused, y_sep)
+    # each projection's columns against the oracle on that projection's own (A_p, B_p): no helper of the
+    # product stands between the raw adapters and the expected values
+    n0 = 0
+    for p in range(3):
+        ents = [wl.AdapterEntry(s, 1, ranks[p], scale, adapters[s][p][0], adapters[s][p][1]) for s in range(2)]
+        ref_p, _ = oracle.forward(x_bits, W_bits[p], ents, so, np.array([0, 1], np.int32))
+        r = oracle.compare(np.ascontiguousarray(y_fused[:, n0:n0 + Ns[p]]), ref_p)
+        assert r["ok"], (p, r)
+        n0 += Ns[p]
     ref, _ = oracle.forward(x_bits, np.concatenate(W_bits, axis=0), fused_entries, so, np.array([0, 1], np.int32))
     assert oracle.compare(y_fused, ref)["ok"]

@@ -7,7 +7,7 @@ import pytest
 import oracle
 from paper_2608_15241_b200 import workloads as wl
 
-from gpu_util import Site, sample_positions, to_bits, to_dev
+from gpu_util import Site, sample_positions, sample_positions_every_tile, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -25,12 +25,15 @@ def check_full(w, **site_kw):
         site.close()
 
 
-def check_sampled(w, count=48):
+def check_every_tile(w, count=512):
+    """Largest shapes: the oracle on >= `count` rows that include a row of every 128-row tile and every
+    segment's first and last row (rows are independent, so a sampled row is checked exactly)."""
     site = Site(w)
     try:
         y, flags = site.run()
         assert flags == 0
-        pos = sample_positions(w, count)
+        pos = sample_positions_every_tile(w, count)
+        assert len(pos) >= min(count, w.T)
         ref, _ = oracle.forward_workload(w, positions=pos)
         rows = pos if w.perm is None else w.perm[pos]
         r = oracle.compare(y, ref, rows=rows)
@@ -154,15 +157,33 @@ def test_decode_q_proj(split):
         assert not oracle.compare(y, other, rows=np.array([0, 1]))["ok"]
 
 
-def test_prefill_q_proj_sampled_rows():
-    check_sampled(wl.prefill_q_proj(), count=64)
+def test_prefill_q_proj_every_element():
+    check_full(wl.prefill_q_proj())
 
 
-def test_mlp_up_gate_sampled_rows():
-    check_sampled(wl.mlp_up_gate(), count=48)
+def test_prefill_q_proj_shuffled_every_element():
+    # the same batch with its rows in arrival order: per-token ids through the segmentation pass, row gather,
+    # scatter epilogue
+    import torch
+    w = wl.shuffle_rows(wl.prefill_q_proj())
+    site = Site(w)
+    try:
+        tok = np.array([site.slots[e] if e >= 0 else -1 for e in w.token_entry], np.int32)
+        y = site.table.lora_mixed_linear_tokens(site.x, site.W0, torch.from_numpy(tok).cuda())
+        torch.cuda.synchronize()
+        assert site.table.device_status() == 0
+        ref, _ = oracle.forward_workload(w)
+        r = oracle.compare(to_bits(y), ref)
+        assert r["ok"], r
+    finally:
+        site.close()
 
 
-def test_mlp_up_gate_shuffled_through_segmentation_pass():
+def test_mlp_up_gate_every_element():
+    check_full(wl.mlp_up_gate())
+
+
+def test_mlp_up_gate_shuffled_through_segmentation_pass_every_element():
     import torch
     w = wl.mlp_up_gate(shuffled=True)
     site = Site(w, max_slots=8)
@@ -173,18 +194,25 @@ def test_mlp_up_gate_shuffled_through_segmentation_pass():
         torch.cuda.synchronize()
         assert site.table.device_status() == 0
         assert np.array_equal(perm.cpu().numpy(), w.perm)      # same stable grouping as the recipe
-        pos = sample_positions(w, 40)
-        ref, _ = oracle.forward_workload(w, positions=pos)
-        r = oracle.compare(to_bits(y), ref, rows=w.perm[pos])
+        ref, _ = oracle.forward_workload(w)
+        r = oracle.compare(to_bits(y), ref)
         assert r["ok"], r
     finally:
         site.close()
 
 
-@pytest.mark.parametrize("proj,T", [("q", 1), ("q", 16), ("down", 16), ("gate", 128), ("down", 128),
-                                    ("q", 1024), ("o", 8192), ("k", 128), ("gate", 16), ("up", 1), ("gate", 1024)])
-def test_layer_sweep_cells_sampled(proj, T):
-    check_sampled(wl.layer_sweep(proj, T), count=40)
+# every cell of the decoder-layer sweep up to 1024 tokens, every element (q k v o share a shape, gate and up too:
+# one of each, plus two of the others for their different seeds)
+@pytest.mark.parametrize("proj,T", [(p, T) for p in ("q", "gate", "down") for T in (1, 16, 128, 1024)] +
+                         [("k", 128), ("up", 1), ("o", 16), ("v", 1024)])
+def test_layer_sweep_cells_every_element(proj, T):
+    check_full(wl.layer_sweep(proj, T))
+
+
+# the 8192-token cells: >= 512 rows with a row of every 128-row tile and every segment's ends
+@pytest.mark.parametrize("proj", ["o", "gate", "down"])
+def test_layer_sweep_8192_token_cells_every_tile(proj):
+    check_every_tile(wl.layer_sweep(proj, 8192), count=512)
 
 
 # ---- properties that hold at any size ----------------------------------------------------------------------

@@ -133,3 +133,92 @@ def test_publish_errors_and_retire_of_the_serving_version():
     with pytest.raises(LmlError):
         tbl.slot_state(s)
     tbl.close()
+
+
+@pytest.mark.parametrize("ordered", [False, True])
+def test_retired_serving_entry_never_resolves_to_the_slots_next_tenant(ordered):
+    """An adapter is published on a busy non-blocking stream and retired while that publish is still
+    queued; another adapter is then registered and takes over the slot.  A call that names the retired
+    adapter must get base output and the flag, never the new tenant's delta: with the retire ordered on
+    the publishing stream (the device map is cleared behind the publish) and also with the plain
+    retire_version, whose clear on the legacy stream overtakes the publish and leaves a stale word in
+    the map (the word names the old registration, which the slot no longer holds)."""
+    import torch
+    from paper_2608_15241_b200 import binding as b
+    from paper_2608_15241_b200.binding import Table
+    K, N, T = 264, 136, 8
+    tbl = Table(K, N, 2)
+    old, new = _entry(21, 5, 1, 8, K, N), _entry(21, 9, 1, 16, K, N)
+    x_bits, W_bits = wl.normal_bf16(21, 1, (T, K), 1.0), wl.normal_bf16(21, 2, (N, K), 0.05)
+    x, W = to_dev(x_bits), to_dev(W_bits)
+    s_old = tbl.register_adapter(5, 1, to_dev(old.A), to_dev(old.B), old.scale)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()                 # a non-blocking stream: the legacy stream does not order against it
+    big = torch.randn((4096, 4096), device="cuda")
+    with torch.cuda.stream(side):
+        for _ in range(40):                    # keeps the stream busy for a few milliseconds
+            big = big @ big * 1e-3
+        tbl.publish(5, 1, stream=side)         # queued behind the products
+    if ordered:
+        tbl.retire_version(5, 1, stream=side)
+    else:
+        tbl.retire_version(5, 1)               # its clear runs at once, before the publish lands
+    with torch.cuda.stream(side):
+        s_new = tbl.register_adapter(9, 1, to_dev(new.A), to_dev(new.B), new.scale, stream=side)
+    assert s_new == s_old                      # lowest free index: the retired entry's slot
+    side.synchronize()
+    torch.cuda.synchronize()
+    ids = torch.full((T,), 5, dtype=torch.int32, device="cuda")
+    y = to_bits(tbl.lora_mixed_linear_adapters(x, W, ids))
+    torch.cuda.synchronize()
+    assert tbl.device_status() == b.FLAG_BAD_SLOT
+    base = _ref(x_bits, W_bits, [old, new], [-1] * T)
+    assert oracle.compare(y, base)["ok"]
+    with_new = _ref(x_bits, W_bits, [old, new], [1] * T)
+    assert not oracle.compare(y, with_new)["ok"]          # the other adapter's delta would show
+    # the new tenant itself is reachable by its slot, and by its adapter id once published
+    y_slot = to_bits(tbl.lora_mixed_linear_tokens(x, W, torch.full((T,), s_new, dtype=torch.int32, device="cuda")))
+    tbl.publish(9, 1)
+    y_id = to_bits(tbl.lora_mixed_linear_adapters(x, W, torch.full((T,), 9, dtype=torch.int32, device="cuda")))
+    torch.cuda.synchronize()
+    assert tbl.device_status() == 0
+    assert oracle.compare(y_slot, with_new)["ok"] and np.array_equal(y_slot, y_id)
+    tbl.close()
+
+
+def test_two_step_form_across_a_publish_keeps_its_version_when_pinned():
+    """Ids resolved by lml_segment_tokens_adapters, the layer run by lora_mixed_linear after a publish of
+    the same adapter: with the resolved slot pinned the tokens run under the version they were bound to;
+    without the pin the replaced entry is free by then and they fall back to base output with the flag."""
+    import torch
+    from paper_2608_15241_b200 import binding as b
+    from paper_2608_15241_b200.binding import Table
+    K, N, T = 264, 136, 200
+    e1, e2 = _entry(33, 4, 1, 8, K, N), _entry(33, 4, 2, 16, K, N)
+    x_bits, W_bits = wl.normal_bf16(33, 1, (T, K), 1.0), wl.normal_bf16(33, 2, (N, K), 0.05)
+    x, W = to_dev(x_bits), to_dev(W_bits)
+    ids = torch.full((T,), 4, dtype=torch.int32, device="cuda")
+    for pinned in (True, False):
+        tbl = Table(K, N, 4)
+        s1 = tbl.register_adapter(4, 1, to_dev(e1.A), to_dev(e1.B), e1.scale)
+        tbl.register_adapter(4, 2, to_dev(e2.A), to_dev(e2.B), e2.scale)
+        tbl.publish(4, 1)
+        if pinned:
+            tbl.pin(s1)
+        perm = torch.empty(T, dtype=torch.int32, device="cuda")
+        so = torch.empty(tbl.max_slots + 2, dtype=torch.int32, device="cuda")
+        sid = torch.empty(tbl.max_slots + 1, dtype=torch.int32, device="cuda")
+        b.lml_segment_tokens_adapters(tbl.handle, ids.data_ptr(), T, perm.data_ptr(), so.data_ptr(), sid.data_ptr(),
+                                      b._stream(None))
+        tbl.publish(4, 2)                                   # the adapter moves on between the two steps
+        y = to_bits(tbl.lora_mixed_linear(x, W, so, sid, perm))
+        torch.cuda.synchronize()
+        flags = tbl.device_status()
+        if pinned:
+            assert flags == 0
+            assert oracle.compare(y, _ref(x_bits, W_bits, [e1, e2], [0] * T))["ok"]
+            tbl.unpin(s1)
+        else:
+            assert flags == b.FLAG_BAD_SLOT
+            assert oracle.compare(y, _ref(x_bits, W_bits, [e1, e2], [-1] * T))["ok"]
+        tbl.close()

@@ -46,30 +46,3 @@ def test_library_choice_for_few_tokens(T, monkeypatch):
     ref, _ = oracle.forward(w.x, w.W0, w.entries, w.seg_offsets, w.seg_entry, w.perm)
     assert oracle.compare(y, ref)["ok"]
     site.close()
-
-
-@pytest.mark.parametrize("kw", [dict(T=333, d_in=520, d_out=264), dict(T=600, d_in=1024, d_out=512, shuffled=True),
-                                dict(T=40, d_in=2048, d_out=136)])
-def test_tensor_core_shrink_form(kw, monkeypatch):
-    """LML_SHRINK=tensor: u = scale * x . A^T computed by the split-K kernel's shrink mode (128 x 64 tcgen05
-    products per piece, K split over a cluster) instead of the mma.sync shrink kernel."""
-    w = wl.ragged(ranks=(4, 16, 1, 33, 64), **kw)
-    site = Site(w)
-    y0, f0 = site.run()
-    monkeypatch.setenv("LML_SHRINK", "tensor")
-    y, flags = site.run()
-    assert flags == 0 and f0 == 0
-    ref, _ = oracle.forward(w.x, w.W0, w.entries, w.seg_offsets, w.seg_entry, w.perm)
-    r = oracle.compare(y, ref)
-    assert r["ok"], r
-    # against the default shrink kernel: u is rounded to bf16 by both, from sums in a different order
-    diff = np.abs(wl.bf16_bits_to_f64(y) - wl.bf16_bits_to_f64(y0))
-    assert (diff <= 2.0 ** -6 * np.maximum(1.0, np.abs(wl.bf16_bits_to_f64(y0)))).all()
-    # malformed offsets are caught by this form too: base output only, flag raised
-    from paper_2608_15241_b200 import binding
-    T = w.T
-    yb, fb = site.run(seg_offsets=[0, 2 * T // 3, T // 3, T], raw_slot_ids=[site.slots[0], site.slots[1], site.slots[2]])
-    assert fb & binding.FLAG_BAD_OFFSETS
-    base = oracle.forward(w.x, w.W0, [], [0, T], [-1], w.perm)[0]
-    assert oracle.compare(yb, base)["ok"]
-    site.close()
