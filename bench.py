@@ -600,6 +600,87 @@ def run_layer_sweep(device, peaks, steps, only=None, parity=False):
     return cells
 
 
+def run_multi_decode(device, peaks, want_parity):
+    """Several projections of one decode step in one lora_mixed_linear_multi call: q/k/v (3 x 4096 x 4096) and
+    gate/up (2 x 11008 x 4096) of a 7B-class layer, 8 tokens of 4 agents, 5 resident entries of rank 16 per
+    projection.  Per cell: microseconds per call, algorithmic GB/s and fraction of the measured HBM peak, against
+    the same projections as one call each."""
+    import torch
+    from paper_2608_15241_b200 import binding as b
+    from paper_2608_15241_b200.binding import Table
+    stream = torch.cuda.Stream(device=device)
+    dev = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(device)
+    cells = []
+    for name, Ns in (("decode_qkv", (4096, 4096, 4096)), ("decode_gate_up", (11008, 11008))):
+        K, T, n_ad, rank = 4096, 8, 5, 16
+        P = len(Ns)
+        x_bits = wl.normal_bf16(5, 1, (T, K), 1.0)
+        W_bits = [wl.normal_bf16(5, 10 + p, (n, K), 0.02) for p, n in enumerate(Ns)]
+        ents = [[wl.AdapterEntry(a, 1, rank, 2.0, wl.normal_bf16(5, 100 + 10 * p + a, (rank, K), 0.02),
+                                 wl.normal_bf16(5, 300 + 10 * p + a, (n, rank), 0.02)) for a in range(n_ad)]
+                for p, n in enumerate(Ns)]
+        tok_np = np.array([0, 0, 1, 1, 2, 2, 3, 3], np.int32)     # 4 agents x 2 tokens; the fifth entry is resident, unused
+        used = 4
+        nbytes = sum(2.0 * K * n + 2.0 * T * n + used * 2.0 * rank * (K + n) for n in Ns) + 2.0 * T * K + 4.0 * T * P
+        R = max(2, int(math.ceil(3 * L2_BYTES / nbytes)))
+        x0, W0s = dev(x_bits), [dev(w) for w in W_bits]
+        A0 = [[dev(e.A) for e in pe] for pe in ents]
+        B0 = [[dev(e.B) for e in pe] for pe in ents]
+        tok = torch.from_numpy(tok_np).to(device)
+        sets = []
+        for i in range(R):
+            roll = lambda t_: t_ if i == 0 else torch.roll(t_, shifts=i, dims=0).contiguous()
+            tabs = [Table(K, n, n_ad, device=torch.device(device).index or 0) for n in Ns]
+            for p, t in enumerate(tabs):
+                for a in range(n_ad):
+                    t.register_adapter(a, 1, roll(A0[p][a]), roll(B0[p][a]), 2.0)
+            s_ = dict(tabs=tabs, h=[t.handle for t in tabs], x=roll(x0), W=[roll(w) for w in W0s],
+                      ys=[torch.empty((T, n), dtype=torch.bfloat16, device=device) for n in Ns])
+            s_["ws"] = torch.empty(b.lml_multi_workspace_bytes(s_["h"], T), dtype=torch.uint8, device=device)
+            sets.append(s_)
+        torch.cuda.synchronize()
+
+        def multi(i):
+            s_ = sets[i % R]
+            b.lora_mixed_linear_multi(s_["h"], s_["x"].data_ptr(), [w.data_ptr() for w in s_["W"]], T, [tok.data_ptr()] * P,
+                                      [y.data_ptr() for y in s_["ys"]], s_["ws"].data_ptr(), s_["ws"].numel(), b._stream(None))
+            return sum(t.last_launch_count() for t in s_["tabs"])
+
+        def separate(i):
+            s_ = sets[i % R]
+            for p in range(P):
+                b.lora_mixed_linear_tokens(s_["h"][p], s_["x"].data_ptr(), s_["W"][p].data_ptr(), T, tok.data_ptr(),
+                                           s_["ys"][p].data_ptr(), s_["ws"].data_ptr(), s_["ws"].numel(), b._stream(None))
+            return P
+
+        n = max(R, 600)
+        m_secs, m_launches, _ = timed_graph_loop(multi, R, n, 3 * R, stream)
+        s_secs, _, _ = timed_graph_loop(separate, R, n, 3 * R, stream)
+        cell = {"workload": name, "projections": P, "d_in": K, "d_out": list(Ns), "tokens": T,
+                "us_per_call": m_secs / n * 1e6, "launches_per_call": m_launches // n,
+                "GB/s": nbytes / (m_secs / n) / 1e9, "frac_of_measured_hbm": nbytes / (m_secs / n) / 1e9 / peaks["hbm"],
+                "one_call_per_projection_us": s_secs / n * 1e6, "algorithmic_bytes": nbytes, "rotation_sets": R}
+        if want_parity:
+            import oracle
+            multi(0)
+            torch.cuda.synchronize()
+            worst = {"ok": True, "rel_fro": 0.0, "worst_tol_ratio": 0.0}
+            for p in range(P):
+                ref, _ = oracle.forward(x_bits, W_bits[p], ents[p], np.arange(T + 1, dtype=np.int32), tok_np)
+                r = oracle.compare(sets[0]["ys"][p].view(torch.int16).cpu().numpy().view(np.uint16), ref)
+                worst = {"ok": worst["ok"] and r["ok"], "rel_fro": max(worst["rel_fro"], r["rel_fro"]),
+                         "worst_tol_ratio": max(worst["worst_tol_ratio"], r["worst_tol_ratio"])}
+            worst["rows"] = T * P
+            cell["parity"] = worst
+        cells.append(cell)
+        for s_ in sets:
+            for t in s_["tabs"]:
+                t.close()
+        del sets
+        torch.cuda.empty_cache()
+    return cells
+
+
 def run_reference(args):
     """The reference arm of this tier: the fp64 oracle on host cores, a bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -707,6 +788,7 @@ def main():
         sec["steps"] = msteps
         line["mlp_up_gate"] = sec
         if rank == 0:
+            line["multi_projection_decode"] = run_multi_decode(device, peaks, True)
             line["layer_sweep"] = {"what": "us per lora_mixed_linear_tokens call (segmentation included) and fraction of the "
                                            "cell's bound = max(bytes / measured HBM peak, flops / measured burst tensor peak) / time; "
                                            "16 adapters of rank 16, two of them in two versions (18 resident entries), Zipf(1.1) binding",

@@ -75,6 +75,7 @@ typedef enum {
 #define LML_MAX_RANK 64   /* upper bound for an adapter's rank */
 #define LML_MAX_ADAPTER_IDS 4096 /* adapter ids 0 .. this-1 can be published and resolved on the device */
 #define LML_DECODE_MAX_TOKENS 16 /* T <= this takes the bandwidth-bound decode kernel */
+#define LML_MAX_PROJECTIONS 4 /* projections one lora_mixed_linear_multi call can take */
 
 const char* lml_status_string(lml_status s);
 
@@ -277,6 +278,35 @@ size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens);
 lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0, int T,
                                     const int32_t* token_slots, void* y, void* workspace,
                                     size_t workspace_bytes, void* stream);
+
+/*
+ * lora_mixed_linear_multi — several projections that read the same x in one call: q / k / v of an
+ * attention block, gate / up of an MLP (a decoder layer runs all of its projections at every step;
+ * the paper's runtime replays decode steps from CUDA graphs, Section 7.7).  Projection p has its own
+ * table tables[p] (its own adapters, ranks, scales), base weight W0[p] (device bf16
+ * [d_out_p][d_in]), per-token binding token_slots[p] (device int32[T]: slot of tables[p] per row of
+ * x, or -1; the pointers may be equal when the tables were filled in the same order) and output
+ * y[p] (device bf16 [T][d_out_p], distinct buffers).  tables, W0, token_slots and y are HOST arrays of
+ * P pointers, 1 <= P <= LML_MAX_PROJECTIONS; all tables share d_in and the device.
+ * T <= 16: ONE launch of the decode kernel.  The rows of all base weights form one stream that the
+ * grid shares out evenly, x is read once, the fixed cost of a launch is paid once; results per
+ * projection are those of lora_mixed_linear_tokens on that projection, to fp32 summation order.  The
+ * library falls back to one decode call per projection where that is the faster way or the only one:
+ * weights so large that a launch's fixed cost no longer counts (gate / up of a 7B-class MLP), and
+ * tables whose resident adapters have more rows than the one-launch kernel streams (more than
+ * an eighth of the weights' rows, or more than 1024).
+ * T > 16: the projections run one after the other on `stream`, each exactly as
+ * lora_mixed_linear_tokens(tables[p], ...).
+ * The call counts its CTAs in tables[0]'s status block: two multi calls that share tables[0], or a multi
+ * call and a decode call on tables[0], must not overlap on the GPU.  Device-detected errors set the
+ * flags of the table they concern (malformed input that concerns all: tables[0]).
+ * workspace: device, 256-byte aligned, at least lml_multi_workspace_bytes(tables, P, T).
+ * Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+size_t lml_multi_workspace_bytes(lml_table* const* tables, int P, int max_tokens);
+lml_status lora_mixed_linear_multi(lml_table* const* tables, int P, const void* x, const void* const* W0, int T,
+                                   const int32_t* const* token_slots, void* const* y, void* workspace,
+                                   size_t workspace_bytes, void* stream);
 
 /*
  * The same two calls for callers that hold ADAPTER ids per token instead of slots: every id is

@@ -33,7 +33,8 @@ EXPORTS = ("lml_status_string", "lml_table_create", "lml_table_destroy", "regist
            "lml_publish", "lml_pin", "lml_unpin", "lml_resolve", "lml_slot_state",
            "lml_segment_tokens_adapters", "lora_mixed_linear_adapters",
            "lml_dual_workspace_bytes", "lora_mixed_linear_dual", "register_adapter_transposed",
-           "lml_backward_workspace_bytes", "lora_mixed_linear_backward_adapters", "retire_version_on")
+           "lml_backward_workspace_bytes", "lora_mixed_linear_backward_adapters", "retire_version_on",
+           "lml_multi_workspace_bytes", "lora_mixed_linear_multi")
 
 
 class LmlError(RuntimeError):
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
         L.lml_dual_workspace_bytes.restype = sz
         L.lml_dual_workspace_bytes.argtypes = [vp, i32, i32]
         L.lora_mixed_linear_dual.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.lml_multi_workspace_bytes.restype = sz
+        L.lml_multi_workspace_bytes.argtypes = [ctypes.POINTER(vp), i32, i32]
+        L.lora_mixed_linear_multi.argtypes = [ctypes.POINTER(vp), i32, vp, ctypes.POINTER(vp), i32, ctypes.POINTER(vp),
+                                              ctypes.POINTER(vp), vp, sz, vp]
         L.lml_publish.argtypes = [vp, i32, i32, vp, ctypes.POINTER(i32)]
         L.lml_pin.argtypes = [vp, i32]
         L.lml_unpin.argtypes = [vp, i32]
@@ -93,7 +98,8 @@ def lib() -> ctypes.CDLL:
         L.lml_last_launch_count.argtypes = [vp]
         for name in EXPORTS:
             if name not in ("lml_status_string", "lml_workspace_bytes", "lml_host_workspace_bytes",
-                            "lml_tokens_workspace_bytes", "lml_dual_workspace_bytes", "lml_backward_workspace_bytes"):
+                            "lml_tokens_workspace_bytes", "lml_dual_workspace_bytes", "lml_backward_workspace_bytes",
+                            "lml_multi_workspace_bytes"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -188,6 +194,27 @@ def lora_mixed_linear_tokens(table: int, x_ptr: int, W0_ptr: int, T: int, token_
     """Segmentation and layer in one call: one slot id per token instead of segments."""
     _check(lib().lora_mixed_linear_tokens(table, x_ptr, W0_ptr, T, token_slots_ptr, y_ptr, workspace_ptr,
                                           workspace_bytes, stream), "lora_mixed_linear_tokens")
+
+
+def _ptr_array(values):
+    arr = (ctypes.c_void_p * len(values))()
+    for i, v in enumerate(values):
+        arr[i] = v
+    return arr
+
+
+def lml_multi_workspace_bytes(tables, max_tokens: int) -> int:
+    return int(lib().lml_multi_workspace_bytes(_ptr_array(tables), len(tables), max_tokens))
+
+
+def lora_mixed_linear_multi(tables, x_ptr: int, W0_ptrs, T: int, token_slots_ptrs, y_ptrs, workspace_ptr: int,
+                            workspace_bytes: int, stream: int = 0) -> None:
+    """Several projections of the same x in one call (table handles and per-projection pointers as lists)."""
+    P = len(tables)
+    assert len(W0_ptrs) == P and len(token_slots_ptrs) == P and len(y_ptrs) == P
+    _check(lib().lora_mixed_linear_multi(_ptr_array(tables), P, x_ptr, _ptr_array(W0_ptrs), T,
+                                         _ptr_array(token_slots_ptrs), _ptr_array(y_ptrs), workspace_ptr,
+                                         workspace_bytes, stream), "lora_mixed_linear_multi")
 
 
 def register_adapter_transposed(table_T: int, adapter_id: int, version: int, A_ptr: int, B_ptr: int, rank: int,
@@ -322,6 +349,23 @@ def fuse_projection_adapters(parts):
         n0 += n
         r0 += r
     return A, B
+
+
+def multi_projection(tables, x, W0s, token_slots, ys=None, workspace=None, stream=None):
+    """lora_mixed_linear_multi for torch tensors: tables = [Table, ...], W0s / token_slots per projection
+    (token_slots may also be one tensor for all).  Returns the list of outputs."""
+    import torch
+    P, T = len(tables), int(x.shape[0])
+    if not isinstance(token_slots, (list, tuple)):
+        token_slots = [token_slots] * P
+    if ys is None:
+        ys = [torch.empty((T, t.d_out), dtype=torch.bfloat16, device=x.device) for t in tables]
+    handles = [t.handle for t in tables]
+    if workspace is None:
+        workspace = torch.empty(max(lml_multi_workspace_bytes(handles, T), 256), dtype=torch.uint8, device=x.device)
+    lora_mixed_linear_multi(handles, _ptr(x), [_ptr(w) for w in W0s], T, [_ptr(s) for s in token_slots],
+                            [_ptr(y) for y in ys], _ptr(workspace), int(workspace.numel()), _stream(stream))
+    return ys
 
 
 class Table:

@@ -39,6 +39,8 @@
 #include <cstdlib>
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
+#include "lml_decode_common.cuh"
+#include "lml_decode_stream.cuh"
 
 namespace lml {
 
@@ -91,44 +93,6 @@ struct DecCtrl {
     uint8_t b_lead[16];  // 1: this row of x is the first with its slot (it stands for the slot's block of B)
 };
 static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control block");
-
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v)
-{
-    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
-{
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)   // 16-byte aligned, multiple of 16
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)   // global -> shared, past L1, no registers
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all()
-{
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-__device__ __forceinline__ void prefetch_l2(const void* p)
-{
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
 
 // kTwo false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers.
 // kMulti: the CTAs have more than one round of rows; compiled with the code that saves reloads of x between rounds.
@@ -828,8 +792,11 @@ cudaError_t decode_init()
     };
     set(decode_main_kernel<false, false, false>); set(decode_main_kernel<false, true, false>); set(decode_main_kernel<false, true, true>);
     set(decode_main_kernel<true, false, false>);  set(decode_main_kernel<true, true, false>);  set(decode_main_kernel<true, true, true>);
+    if (e == cudaSuccess) e = decode_stream_init();
     return e;
 }
+
+int decode_patience() { return g_dec_patience; }
 
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a, cudaStream_t stream,
                           int* launches)

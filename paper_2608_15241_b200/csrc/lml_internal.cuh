@@ -143,7 +143,8 @@ struct DecodeArgs {
     int T, d_in, d_out, G;
     int num_sms;
 };
-cudaError_t decode_init();   // sets the dynamic shared memory attribute
+cudaError_t decode_init();   // sets the dynamic shared memory attributes
+int decode_patience();       // LML_DECODE_PATIENCE or the default, in clock cycles
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
                           cudaStream_t stream, int* launches);
 
