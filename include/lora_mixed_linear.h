@@ -225,8 +225,9 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
  * adapter, either side).  y_a = x.W0 + delta_a, y_b = x.W0 + delta_b, both device bf16 [T][d_out],
  * distinct buffers.  For T > 16 the base product x.W0 is computed once: y_a is read out of the
  * accumulator, then (delta_b - delta_a) is added to it with a few more tensor-core steps and y_b is
- * read out, so y_a is bit-identical to lora_mixed_linear with slot_ids_a and y_b agrees with
- * lora_mixed_linear with slot_ids_b to fp32 rounding of the accumulator.  For T <= 16 the call is two
+ * read out, so y_a agrees with lora_mixed_linear with slot_ids_a to the bf16 rounding of u (bit for
+ * bit when that call takes u from the same shrink kernel) and y_b with lora_mixed_linear with
+ * slot_ids_b to fp32 rounding of the accumulator as well.  For T <= 16 the call is two
  * decode calls.  G >= 1.  workspace: at least lml_dual_workspace_bytes(t, T, G).  Other arguments,
  * flags and errors as lora_mixed_linear.
  */

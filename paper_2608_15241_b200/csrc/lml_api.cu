@@ -1,5 +1,6 @@
 // Host side of the C ABI: the adapter slot table, argument validation, workspace layout and
 // dispatch to the decode / prefill kernels.  See include/lora_mixed_linear.h for the contract.
+#include <cstdlib>
 #include <new>
 
 #include "lml_table.cuh"
@@ -35,7 +36,7 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
 
 static void free_table_resources(lml_table* t)
 {
-    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.Bc); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map);
+    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.Bc); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map); cudaFree(t->arena.tile_flags);
     if (t->copy_in) cudaStreamDestroy(t->copy_in);
     if (t->copy_out) cudaStreamDestroy(t->copy_out);
     if (t->ev_begin) cudaEventDestroy(t->ev_begin);
@@ -101,6 +102,8 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && cudaMemset(t->arena.B, 0, b_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.adapter_map, 0xff, kMaxAdapterIds * sizeof(int32_t)) == cudaSuccess;   // -1: no serving version
+    ok = ok && cudaMalloc(&t->arena.tile_flags, kFuseMaxTiles * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.tile_flags, 0, kFuseMaxTiles * sizeof(int32_t)) == cudaSuccess;
     ok = ok && gemm_sm100_init(device) == cudaSuccess;
     ok = ok && shrink_init() == cudaSuccess;
     ok = ok && decode_init() == cudaSuccess;
@@ -109,7 +112,10 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 256, 1);
     ok = ok && encode_tmap_3d(&t->tmap_B128, t->arena.B, kRankPad, (uint64_t)d_out, (uint64_t)max_slots,
                               kRankPad * 2, (uint64_t)d_out * kRankPad * 2, 64, 128, 1);
-    gemm_split_override(&t->split_bn, &t->split_s);   // the test knob is read here, never on the hot path
+    ok = ok && encode_tmap_3d(&t->tmap_A, t->arena.A, (uint64_t)d_in, kRankPad, (uint64_t)max_slots, (uint64_t)d_in * 2,
+                              (uint64_t)d_in * kRankPad * 2, 64, 64, 1);
+    gemm_split_override(&t->split_bn, &t->split_s);   // the test knobs are read here, never on the hot path
+    if (const char* e = getenv("LML_FUSE_SHRINK")) t->fuse_shrink = e[0] != '0';
     ok = ok && cudaEventCreateWithFlags(&t->ev_map, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_in, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -419,20 +425,25 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
         }
         PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
         __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
-        if (e == cudaSuccess && G > 0) {
+        // With whole-K tiles the shrink runs inside the GEMM kernel (on the CTAs that own the fewest tiles, ahead of
+        // their tiles); otherwise a shrink kernel goes first and the GEMM is its programmatic dependent.
+        const bool fused = G > 0 && t->fuse_shrink &&
+                           gemm_can_fuse_shrink(T, t->d_in, t->d_out, G, t->num_sms, t->split_bn, t->split_s);
+        if (e == cudaSuccess && G > 0 && !fused) {
             e = launch_shrink_pieces(t->arena, snap, xg, T, t->d_in, seg_offsets, slot_ids, G, x, tile_identity, plan,
                                      u_blocks, stream, perm ? 2 : 0);
             if (e == cudaSuccess) ++launches;
         }
         if (e == cudaSuccess) {
             GemmArgs a;
+            a.fused_shrink = fused;
             a.x = xg; a.x_in_place = x; a.tile_identity = tile_identity; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
             a.plan = plan; a.u_blocks = u_blocks ? u_blocks : reinterpret_cast<const __nv_bfloat16*>(x);
             a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
             a.overlap_with_previous = G > 0;
             a.split_bn = t->split_bn; a.split_s = t->split_s;
             if (G == 0) a.u_blocks = reinterpret_cast<const __nv_bfloat16*>(W0);   // never read; map needs a valid base
-            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, &t->tmaps, a, stream);
+            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, t->tmap_A, &t->tmaps, a, stream);
             if (e == cudaSuccess) ++launches;
         }
     }
@@ -514,7 +525,7 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         a.overlap_with_previous = true;
         a.split_bn = 0; a.split_s = 0;   // the dual form runs on whole-K tiles
-        e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, &t->tmaps, a, stream);
+        e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, t->tmap_A, &t->tmaps, a, stream);
         if (e == cudaSuccess) ++launches;
     }
     t->last_launches = launches;

@@ -18,6 +18,12 @@
 // operands come from two more sets of u blocks (second slots; first slots negated), and the epilogue
 // reads the second output.  The producer slips those stages into the middle of the next tile's
 // k-blocks, by when the first read is long done.
+// Fused shrink (the plain call): no shrink kernel runs before this one.  The CTAs at the end of the grid, which
+// own the fewest output tiles, first compute u = scale * x.A^T for a row tile each, as 128 x 64 tcgen05 products
+// (x k-blocks against the A k-blocks of the segments that touch the tile, side by side in an accumulator), write
+// the u blocks and raise the row tile's flag in the table's device memory; a producer waits for that flag (a
+// bounded wait) before it loads the tile's u blocks.  The table's epoch, advanced by the last CTA of every such
+// call, tells this call's flags from the last call's.
 // For few tokens (tiles far fewer than SMs) a split-K variant follows below: a cluster of CTAs shares a
 // tile and exchanges partial sums through distributed shared memory; it also has a shrink mode.
 // Every wait is bounded; on give-up the CTA sets LML_FLAG_TIMEOUT, drains and frees its TMEM.
@@ -46,7 +52,7 @@ template <int BN> struct GemmCfg {
     static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
     static constexpr int kTmemCols = 2 * BN;
-    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache;   // barriers + segment cache (two slot arrays)
+    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache + 512;   // barriers + segment cache (two slot arrays) + shrink plan
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiBytes + ((kCtrlBytes + 15) & ~15);
 };
 
@@ -69,6 +75,28 @@ constexpr uint32_t kStageFresh = 0x400u;    // first stage of a tile: wait for t
 constexpr uint32_t kStageDelta = 0x800u;    // dual form: first stage of a tile's second output: wait until the first was read
 
 static_assert(sizeof(GemmCtrl) <= 256, "control block");
+constexpr uint32_t kStageShrink = 0x1000u;  // a stage of a shrink pass: x tile and bits 16..18 blocks of A; as many 128 x 64 products
+
+// Fused shrink (the plain call on whole-K tiles): the CTAs at the end of the grid, which own one tile fewer than
+// the others or none more, first compute u = scale * x.A^T for a row tile each: one pass multiplies the tile's x
+// k-blocks with the A blocks of up to BN / 64 segments that touch the tile (128 x 64 tcgen05 products side by side
+// in an accumulator), its epilogue writes the u blocks and raises the tile's flag in the table's device memory.
+constexpr int kShrMaxPasses = 8;
+struct ShrPass {
+    int32_t m;          // row tile
+    int32_t n;          // pieces in this pass
+    int32_t last;       // the tile's last pass: raise its flag afterwards
+    int32_t g[4];       // segment of each piece
+    int32_t slot[4];
+};
+struct ShrPlan {
+    int32_t npass;
+    int32_t lora_ok;
+    int32_t epoch;
+    int32_t pad;
+    ShrPass pass[kShrMaxPasses];
+};
+static_assert(sizeof(ShrPlan) <= 512, "shrink plan");
 
 struct GemmParams {
     const int32_t* seg_offsets;
@@ -83,6 +111,10 @@ struct GemmParams {
     uint32_t* status;
     int T, K, N, G;
     int num_m, num_n;
+    int fused;                  // the shrink runs inside this kernel (else a shrink kernel ran before it)
+    int32_t* tile_flags;        // fused: [row tile] = epoch + 1 once the tile's u blocks are written
+    uint32_t* fuse_sync;        // fused: [0] the table's epoch, [1] CTAs that have finished (the last one advances the epoch)
+    __nv_bfloat16* u_out;       // fused: the u blocks, for writing
 };
 
 template <int BN>
@@ -91,9 +123,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     const __grid_constant__ CUtensorMap tmap_w,
     const __grid_constant__ CUtensorMap tmap_u, const __grid_constant__ CUtensorMap tmap_b,
     const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_y2,
-    const __grid_constant__ SlotSnapshot snap, const GemmParams p)
+    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ SlotSnapshot snap, const GemmParams p)
 {
     using Cfg = GemmCfg<BN>;
+    constexpr int kShrPerPass = BN / 64;   // 128 x 64 products that fit side by side in one accumulator
     const bool dual = p.slot_ids2 != nullptr;
     extern __shared__ uint8_t smem_raw[];
     // 128-byte swizzled tiles need 1024-byte alignment
@@ -106,6 +139,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
     int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
     int8_t* slot_cache2 = slot_cache + kSegCache;   // dual form: the second slot per segment
+    ShrPlan* shr = reinterpret_cast<ShrPlan*>(slot_cache2 + kSegCache);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = p.num_m * p.num_n;
@@ -148,9 +182,51 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile int* abort = &ctrl->abort;
-    if (p.G == 0) {   // no shrink kernel ran before this one in the call: wait for foreign work here
+    if (p.G == 0 || p.fused) {   // no shrink kernel ran before this one in the call: wait for foreign work here
         grid_dependency_wait();
         grid_launch_dependents();
+    }
+    if (p.fused) {
+        // The segment arrays are checked here (every CTA reaches the same verdict from its own copy), and the CTA's
+        // shrink passes are laid out: row tiles grid-1-blockIdx, +grid, ... (the CTAs at the end of the grid own
+        // the fewest output tiles), and for each the live segments that touch it, kShrPerPass to a pass.
+        int bad_off = 0, bad_slot = 0;
+        for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
+            const int s0 = seg_cache[g], s1 = seg_cache[g + 1];
+            if (s1 < s0 || s0 < 0 || s1 > p.T) bad_off = 1;
+            const int sl = __ldg(p.slot_ids + g);
+            if (sl != -1 && s1 > s0 && slot_rank(snap, sl) == 0) bad_slot = 1;   // an empty segment may name anything
+        }
+        if (threadIdx.x == 0 && (seg_cache[0] != 0 || seg_cache[p.G] != p.T)) bad_off = 1;
+        bad_off = __syncthreads_or(bad_off);
+        bad_slot = __syncthreads_or(bad_slot);
+        if (threadIdx.x == 0) {
+            if (blockIdx.x == 0) {
+                const unsigned f = (bad_off ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u);
+                if (f) atomicOr(p.status, f);
+            }
+            shr->lora_ok = bad_off ? 0 : 1;
+            shr->epoch = (int32_t)(*reinterpret_cast<volatile uint32_t*>(p.fuse_sync));
+            int np = 0;
+            for (int m = (int)gridDim.x - 1 - (int)blockIdx.x; m < p.num_m && !bad_off; m += (int)gridDim.x) {
+                const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+                int lo = 0, hi = p.G;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+                const int first_pass = np;
+                int n = 0;
+                for (int g = lo; g < p.G && seg_cache[g] < row1 && np < kShrMaxPasses; ++g) {
+                    const int s = slot_cache[g];
+                    if (s < 0 || min(seg_cache[g + 1], row1) <= max(seg_cache[g], row0)) continue;
+                    ShrPass& ps = shr->pass[np];
+                    ps.m = m; ps.g[n] = g; ps.slot[n] = s; ps.last = 0;
+                    if (++n == kShrPerPass) { ps.n = n; n = 0; ++np; }
+                }
+                if (n > 0 && np < kShrMaxPasses) { shr->pass[np].n = n; ++np; }
+                if (np > first_pass) shr->pass[np - 1].last = 1;   // (a tile that no live segment touches has no pass and no flag: nobody waits for it)
+            }
+            shr->npass = np;
+        }
+        __syncthreads();
     }
 
     if (warp == 0) {
@@ -175,11 +251,28 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 // Everything the shrink kernel wrote (plan word, u blocks) is first touched after the
                 // base k-blocks of the first tile are already in flight.
                 if (!lora_known) {
-                    grid_dependency_wait();
-                    grid_launch_dependents();
-                    lora = p.plan->lora_ok != 0;
+                    if (p.fused) lora = shr->lora_ok != 0;
+                    else {
+                        grid_dependency_wait();
+                        grid_launch_dependents();
+                        lora = p.plan->lora_ok != 0;
+                    }
                     lora_known = true;
                 }
+            };
+            // fused shrink: the u blocks of row tile m are written by another CTA of this grid, which raises the
+            // tile's flag when they are complete (bounded wait; the flag's writer runs its shrink passes first thing)
+            int flag_seen_m = -1;
+            auto wait_u = [&](int m) {
+                if (!p.fused || m == flag_seen_m) return;
+                const int want = shr->epoch + 1;
+                const long long t0 = clock64();
+                while (ld_acquire_gpu_s32(p.tile_flags + m) != want) {
+                    if (*abort) { ok = false; return; }
+                    if (clock64() - t0 > (1ll << 31)) { *abort = 1; ok = false; return; }
+                }
+                fence_proxy_async_all();   // what those CTAs wrote with ordinary stores is read by TMA from here on
+                flag_seen_m = m;
             };
             // slot of segment g as far as tile rows [row0, row1) are concerned; -1 = no piece
             auto piece_slot = [&](int g, int row0, int row1, bool second) -> int {
@@ -217,6 +310,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                     for (int g = g_first; g < g_end; ++g) if (piece_slot(g, row0, row1, second) >= 0) { last_piece = g; ++count; }
                 }
                 if (count_only) return count;
+                if (count > 0) wait_u(m);
+                if (!ok) return count;
                 bool first = true;
                 for (int g = g_first; g < g_end && ok; ++g) {
                     const int s = piece_slot(g, row0, row1, second);
@@ -252,6 +347,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 if (ok && n_old > 0) emit_pieces(m, n, 2, false, acc_flag, n_new == 0 ? kStageDelta : 0u, kStageCommit, false);
             };
             int ordinal = 0, prev_m = -1, prev_n = -1;
+            // this CTA's shrink passes: a pass is num_kb stages of [x k-block | A k-blocks of its pieces]
+            for (int ps = 0; p.fused && ps < shr->npass && ok; ++ps, ++ordinal) {
+                const ShrPass& sp = shr->pass[ps];
+                const uint32_t acc_flag = (ordinal & 1) ? kStageAcc1 : 0u;
+                const bool in_place = p.tile_identity && __ldg(p.tile_identity + sp.m);
+                // (a pass with one piece moves 24 KB per k-block: two k-blocks share a stage, so that as many bytes
+                // are on their way as in the tiles' stages)
+                const int sub_bytes = Cfg::kABytes + sp.n * (64 * kBK * 2);
+                const int per_stage = 2 * sub_bytes <= Cfg::kStageBytes ? 2 : 1;
+                for (int kb = 0; kb < num_kb && ok; kb += per_stage) {
+                    ok = acquire();
+                    if (!ok) break;
+                    const int nsub = min(per_stage, num_kb - kb);
+                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                    ctrl->stage_info[stage] = 4u | acc_flag | kStageShrink | ((uint32_t)sp.n << 16) | ((uint32_t)nsub << 20) |
+                                              (kb == 0 ? kStageFresh : 0u) | (kb + nsub >= num_kb ? kStageCommit : 0u);
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nsub * sub_bytes));
+                    for (int j = 0; j < nsub; ++j) {
+                        const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes + j * sub_bytes;
+                        if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, (kb + j) * kBK, sp.m * kBM);
+                        else tma_load_2d(a_dst, &tmap_x, bar, (kb + j) * kBK, sp.m * kBM);
+                        for (int i = 0; i < sp.n; ++i)
+                            tma_load_3d(a_dst + Cfg::kABytes + i * (64 * kBK * 2), &tmap_a, bar, (kb + j) * kBK, 0, sp.slot[i]);
+                    }
+                    advance();
+                }
+            }
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ordinal) {
                 const int m = tile % p.num_m, n = tile / p.num_m;
                 const int row0 = m * kBM;
@@ -341,6 +463,42 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 flagged_stages(acc, accumulate);
             };
             int ordinal = 0;
+            // this CTA's shrink passes: per stage, one 128 x 64 product per piece, side by side in the accumulator
+            for (int ps = 0; p.fused && ps < shr->npass && ok; ++ps, ++ordinal) {
+                constexpr uint32_t idesc64 = umma_idesc_bf16(kBM, 64);
+                const int acc = ordinal & 1;
+                uint32_t& eph = acc ? empty_ph1 : empty_ph0;
+                ok = mbar_wait(smem_u32(&ctrl->tmem_empty[acc]), eph ^ 1u, abort);
+                if (!ok) break;
+                eph ^= 1u;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                bool fresh = true;
+                for (bool more = true; more && ok;) {
+                    ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
+                    if (!ok) break;
+                    const uint32_t info = ctrl->stage_info[stage];
+                    more = (info & kStageCommit) == 0;
+                    const int npc = (int)((info >> 16) & 7u), nsub = (int)((info >> 20) & 3u);
+                    const int sub_bytes = Cfg::kABytes + npc * (64 * kBK * 2);
+                    tc_fence_after();
+                    for (int j = 0; j < nsub; ++j) {
+                        const uint32_t a_addr = tiles_addr + stage * Cfg::kStageBytes + j * sub_bytes;
+                        const uint64_t adesc = umma_desc_k128(a_addr);
+                        for (int i = 0; i < npc; ++i) {
+                            const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes + i * (64 * kBK * 2));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_bf16(d_tmem + (uint32_t)(64 * i), adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc64,
+                                          (!fresh || k > 0) ? 1u : 0u);
+                        }
+                        fresh = false;
+                    }
+                    umma_commit(smem_u32(&ctrl->empty[stage]));
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(smem_u32(&ctrl->tmem_full[acc]));
+            }
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ordinal) {
                 const int acc = ordinal & 1;
                 uint32_t& eph = acc ? empty_ph1 : empty_ph0;
@@ -373,6 +531,48 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         uint32_t full_ph0 = 0, full_ph1 = 0;
         int buf = 0;
         bool ok = true;
+        // this CTA's shrink passes: scale, zero the rows outside the segment, round, write the u blocks; after a
+        // tile's last pass its flag goes up (release: the four warps' stores are complete)
+        for (int ps = 0; p.fused && ps < shr->npass && ok; ++ps) {
+            const ShrPass& sp = shr->pass[ps];
+            uint32_t& fph = acc ? full_ph1 : full_ph0;
+            ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[acc]), fph, abort);
+            if (!ok) break;
+            fph ^= 1u;
+            tc_fence_after();
+            const int pos = sp.m * kBM + q * 32 + lane;
+            const int row0 = sp.m * kBM, row1 = min(row0 + kBM, p.T);
+            for (int i = 0; i < sp.n; ++i) {
+                const int g = sp.g[i];
+                const bool mine = pos >= max(seg_cache[g], row0) && pos < min(seg_cache[g + 1], row1);
+                const float sc = mine ? snap.scale[sp.slot[i]] : 0.f;
+                __nv_bfloat16* out = p.u_out + ((size_t)(sp.m + g) * kBM + q * 32 + lane) * kRankPad;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + 64 * i + 32 * c), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(r[8 * j + 0]) * sc, __uint_as_float(r[8 * j + 1]) * sc);
+                        v.y = pack_bf16(__uint_as_float(r[8 * j + 2]) * sc, __uint_as_float(r[8 * j + 3]) * sc);
+                        v.z = pack_bf16(__uint_as_float(r[8 * j + 4]) * sc, __uint_as_float(r[8 * j + 5]) * sc);
+                        v.w = pack_bf16(__uint_as_float(r[8 * j + 6]) * sc, __uint_as_float(r[8 * j + 7]) * sc);
+                        if (!mine) v = make_uint4(0, 0, 0, 0);   // (0 * garbage may be a NaN)
+                        *reinterpret_cast<uint4*>(out + c * 32 + j * 8) = v;
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[acc]));
+            fence_proxy_async_all();   // the blocks will be read by TMA
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+            if (sp.last && warp == 2 && lane == 0) st_release_gpu_s32(p.tile_flags + sp.m, shr->epoch + 1);
+            acc ^= 1;
+        }
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int m = tile % p.num_m, n = tile / p.num_m;
             const int row_base = m * kBM + q * 32;
@@ -453,6 +653,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
 
     __syncthreads();
     if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.status, LML_FLAG_TIMEOUT);
+    if (threadIdx.x == 0 && p.fused) {
+        // the last CTA to finish moves the table's epoch on: the flags of this call mean nothing to the next one
+        __threadfence();
+        if (atomicAdd(p.fuse_sync + 1, 1u) == gridDim.x - 1) {
+            p.fuse_sync[1] = 0u;
+            p.fuse_sync[0] = (uint32_t)(shr->epoch + 1);
+        }
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
@@ -885,8 +1093,26 @@ bool TmapCache::get_2d(CUtensorMap* out, const void* base, uint64_t inner, uint6
     return true;
 }
 
+// Whether the shrink can run inside the GEMM kernel for this call: whole-K tiles, the segment arrays in the
+// kernel's shared-memory cache, a flag per row tile in the table's array, and no CTA with more shrink passes
+// than its plan holds (worst case: every segment touches every one of its row tiles).
+bool gemm_can_fuse_shrink(int T, int d_in, int d_out, int G, int num_sms, int split_bn, int split_s)
+{
+    if (G <= 0 || G > kSegCache) return false;
+    if (gemm_pick_split(T, d_in, d_out, num_sms, split_bn, split_s).split) return false;
+    const int bn = gemm_pick_bn(T, d_out, num_sms);
+    const int num_m = (T + kBM - 1) / kBM, num_n = (d_out + bn - 1) / bn;
+    if (num_m > kFuseMaxTiles) return false;
+    const int grid = min(num_m * num_n, num_sms);
+    const int tiles_per_cta = (num_m + grid - 1) / grid;
+    const int per_pass = bn / 64;
+    const int passes_per_tile = (min(G, kBM) + per_pass - 1) / per_pass;
+    return tiles_per_cta * passes_per_tile <= kShrMaxPasses;
+}
+
 cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B256,
-                              const CUtensorMap& tmap_B128, TmapCache* cache, const GemmArgs& a, cudaStream_t stream)
+                              const CUtensorMap& tmap_B128, const CUtensorMap& tmap_A, TmapCache* cache, const GemmArgs& a,
+                              cudaStream_t stream)
 {
     const bool dual = a.slot_ids2 != nullptr;
     if (dual && (a.G <= 0 || !a.y2)) return cudaErrorInvalidValue;
@@ -916,6 +1142,9 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     p.y = (__nv_bfloat16*)a.y; p.status = ar.status;
     p.slot_ids2 = a.slot_ids2; p.y2 = (__nv_bfloat16*)a.y2; p.u_set_rows = (int)u_set_rows;
     p.T = a.T; p.K = a.d_in; p.N = a.d_out; p.G = a.G; p.num_m = num_m; p.num_n = num_n;
+    p.fused = (a.fused_shrink && !split && !dual) ? 1 : 0;
+    p.tile_flags = ar.tile_flags; p.fuse_sync = ar.status + 4; p.u_out = const_cast<__nv_bfloat16*>(a.u_blocks);
+    if (a.fused_shrink && !p.fused) return cudaErrorInvalidValue;   // (the caller asked gemm_can_fuse_shrink first)
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kGemmThreads);
     cfg.stream = stream;
@@ -943,8 +1172,8 @@ cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const C
     cfg.dynamicSmemBytes = bn == 256 ? GemmCfg<256>::kSmemBytes : GemmCfg<128>::kSmemBytes;
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
-    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
-    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, ty2, snap, p);
+    if (bn == 256) return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<256>, tx, tx0, tw, tu, tb, ty, ty2, tmap_A, snap, p);
+    return cudaLaunchKernelEx(&cfg, lora_gemm_sm100_kernel<128>, tx, tx0, tw, tu, tb, ty, ty2, tmap_A, snap, p);
 }
 
 }  // namespace lml

@@ -18,7 +18,8 @@ constexpr int kRankPad = 64;          // adapters are stored zero-padded to this
 constexpr int kRankCompact = 16;      // ... and B a second time, padded to this rank only, where the rank allows
 constexpr int kTileM = 128;           // token rows per GEMM tile and per shrink piece block
 constexpr int kDecodeMaxT = LML_DECODE_MAX_TOKENS;
-constexpr int kMaxAdapterIds = LML_MAX_ADAPTER_IDS;   // adapter ids that can be resolved on the device
+constexpr int kMaxAdapterIds = LML_MAX_ADAPTER_IDS;
+constexpr int kFuseMaxTiles = 4096;   // row tiles of a call whose shrink can run inside the GEMM kernel (524288 tokens)   // adapter ids that can be resolved on the device
 
 // Per-call snapshot of the slot table, passed by value as a kernel parameter so that a later
 // register / retire cannot change a call that is already enqueued.
@@ -36,6 +37,7 @@ struct Arena {
     __nv_bfloat16* Bc;  // [max_slots][d_out][kRankCompact]: the same rows, 32 bytes each, for slots of rank <= kRankCompact
                         // (what the decode kernel reads: it needs a row's real columns only, a quarter of the padded row)
     uint32_t* status;   // sticky LML_FLAG_* bits
+    int32_t* tile_flags;    // [kFuseMaxTiles] fused shrink of the prefill GEMM: row tile m's u blocks are written (= epoch + 1; the epoch is word 4 of status)
     int32_t* adapter_map;   // [kMaxAdapterIds] serving entry of each adapter id: slot | generation << 8, -1 = none; written by lml_publish
 };
 
@@ -103,6 +105,7 @@ struct GemmArgs {
     void* y2 = nullptr;                   // (num_m + G) blocks: first slots, second slots, first slots negated
     int T, d_in, d_out, G;
     int num_sms;
+    bool fused_shrink = false;         // no shrink kernel ran: the GEMM kernel computes the u blocks itself (see gemm_can_fuse_shrink)
     int split_bn = -1, split_s = -1;   // the table's split-K override: -1 = the library chooses, 0 = off, else the forced shape
     bool overlap_with_previous;   // launch as a programmatic dependent of the shrink kernel before it
 };
@@ -120,8 +123,11 @@ struct TmapCache {
 bool gemm_split_override(int* bn_out, int* split_out);
 // tmap_B256 / tmap_B128: the table's maps of its packed B arena for 256- and 128-column tiles.
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
+bool gemm_can_fuse_shrink(int T, int d_in, int d_out, int G, int num_sms, int split_bn, int split_s);
+// tmap_A: the table's map of its packed A arena ([max_slots][64][d_in], box 64 x 64 x 1), for the fused shrink.
 cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B256,
-                              const CUtensorMap& tmap_B128, TmapCache* cache, const GemmArgs& a, cudaStream_t stream);
+                              const CUtensorMap& tmap_B128, const CUtensorMap& tmap_A, TmapCache* cache, const GemmArgs& a,
+                              cudaStream_t stream);
 cudaError_t gemm_sm100_init(int device);
 cudaError_t shrink_init();   // both set the dynamic shared memory attributes of their kernels
 bool encode_tmap_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer,

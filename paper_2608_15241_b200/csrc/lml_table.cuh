@@ -19,6 +19,8 @@ struct lml_table {
     uint16_t next_gen = 0;
     lml::Arena arena{};
     CUtensorMap tmap_B256, tmap_B128;   // packed B arena as [max_slots][d_out][64], boxes 64 x 256 x 1 and 64 x 128 x 1
+    CUtensorMap tmap_A;                 // packed A arena as [max_slots][64][d_in], box 64 x 64 x 1
+    bool fuse_shrink = true;            // LML_FUSE_SHRINK=0 when the table was created: always the separate shrink kernel (a test knob)
     lml::TmapCache tmaps;               // tensor maps of the caller's buffers seen so far
     int split_bn = -1, split_s = -1;    // LML_GEMM_SPLIT as it stood when the table was created (-1: not set)
     // Retiring a serving entry clears its word of the device map with a kernel on a stream; the event marks
