@@ -524,7 +524,7 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
         a.plan = plan; a.u_blocks = u_blocks;
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         a.overlap_with_previous = true;
-        a.split_bn = 0; a.split_s = 0;   // the dual form runs on whole-K tiles
+        a.split_bn = t->split_bn; a.split_s = t->split_s;   // (few tokens: the split-K kernel, both bindings' accumulators side by side)
         e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, t->tmap_A, &t->tmaps, a, stream);
         if (e == cudaSuccess) ++launches;
     }

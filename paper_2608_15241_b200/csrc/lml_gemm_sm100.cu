@@ -75,6 +75,7 @@ constexpr uint32_t kStageFresh = 0x400u;    // first stage of a tile: wait for t
 constexpr uint32_t kStageDelta = 0x800u;    // dual form: first stage of a tile's second output: wait until the first was read
 
 static_assert(sizeof(GemmCtrl) <= 256, "control block");
+constexpr uint32_t kStageBoth = 0x2000u;    // split-K dual form: the stage's product goes into both bindings' accumulators
 constexpr uint32_t kStageShrink = 0x1000u;  // a stage of a shrink pass: x tile and bits 16..18 blocks of A; as many 128 x 64 products
 
 // Fused shrink (the plain call on whole-K tiles): the CTAs at the end of the grid, which own one tile fewer than
@@ -701,6 +702,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
     GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(epi_ptr + Cfg::kEpiBytes);
     int32_t* seg_cache = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctrl) + 256);
     int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
+    int8_t* slot_cache2 = slot_cache + kSegCache;   // dual form: the second slot per segment
+    // Dual form (two bindings of the same segments, two outputs): the k-blocks pass through shared memory once and
+    // are multiplied into two accumulators (with few tokens the tensor cores have time to spare: the kernel is
+    // bound by the read of W0); each binding's pieces go to its own accumulator, and the exchange runs twice.
+    const bool dual = p.slot_ids2 != nullptr;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = (int)gridDim.x, rank = (int)blockIdx.x;   // the cluster spans the grid's x dimension
@@ -729,9 +735,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
         for (int g = threadIdx.x; g < p.G; g += kGemmThreads) {
             int s = __ldg(p.slot_ids + g);
             slot_cache[g] = (int8_t)((s >= 0 && s < snap.max_slots && snap.rank[s] > 0) ? s : -1);
+            if (dual) {
+                const int s2 = __ldg(p.slot_ids2 + g);
+                slot_cache2[g] = (int8_t)((s2 >= 0 && s2 < snap.max_slots && snap.rank[s2] > 0) ? s2 : -1);
+            }
         }
     }
-    if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), BN);
+    if (warp == 1) tmem_alloc(smem_u32(&ctrl->tmem_base), dual ? 2 * BN : BN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -753,11 +763,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
             const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
             const bool in_place = p.tile_identity && __ldg(p.tile_identity + m);
             const int kb0 = rank * num_kb / S, kb1 = (rank + 1) * num_kb / S;
-            auto piece_slot = [&](int g) -> int {
+            auto piece_slot = [&](int g, bool second) -> int {
                 int s0, s1, s;
-                if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = slot_cache[g]; }
+                if (seg_cached) { s0 = seg_cache[g]; s1 = seg_cache[g + 1]; s = second ? slot_cache2[g] : slot_cache[g]; }
                 else {
-                    s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1); s = __ldg(p.slot_ids + g);
+                    s0 = __ldg(p.seg_offsets + g); s1 = __ldg(p.seg_offsets + g + 1);
+                    s = __ldg((second ? p.slot_ids2 : p.slot_ids) + g);
                     if (slot_rank(snap, s) == 0) s = -1;
                 }
                 return min(s1, row1) <= max(s0, row0) ? -1 : s;
@@ -768,7 +779,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 if (!ok) break;
                 const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
                 const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                ctrl->stage_info[stage] = 4u;
+                ctrl->stage_info[stage] = 4u | (dual ? kStageBoth : 0u);
                 mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
                 if (in_place) tma_load_2d(a_dst, &tmap_x0, bar, kb * kBK, row0);
                 else tma_load_2d(a_dst, &tmap_x, bar, kb * kBK, row0);
@@ -797,20 +808,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 }
                 // segment g's piece goes to CTA g mod S: which CTA adds a row's LoRA term depends only on the
                 // row's own segment, so a row's bits do not change with what other segments are bound to
-                for (int g = g_first; g < g_end && ok; ++g) {
-                    if (g % S != rank) continue;
-                    const int s = piece_slot(g);
-                    if (s < 0) continue;
-                    ok = acquire();
-                    if (!ok) break;
-                    const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
-                    const uint32_t bar = smem_u32(&ctrl->full[stage]);
-                    ctrl->stage_info[stage] = (uint32_t)((snap.rank[s] + 15) >> 4);
-                    mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
-                    tma_load_2d(a_dst, &tmap_u, bar, 0, (m + g) * kBM);
-                    tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
-                    advance();
-                }
+                for (int side = 0; side < (dual ? 2 : 1) && ok; ++side)
+                    for (int g = g_first; g < g_end && ok; ++g) {
+                        if (g % S != rank) continue;
+                        const int s = piece_slot(g, side == 1);
+                        if (s < 0) continue;
+                        ok = acquire();
+                        if (!ok) break;
+                        const uint32_t a_dst = tiles_addr + stage * Cfg::kStageBytes;
+                        const uint32_t bar = smem_u32(&ctrl->full[stage]);
+                        ctrl->stage_info[stage] = (uint32_t)((snap.rank[s] + 15) >> 4) | (side ? kStageAcc1 : 0u);
+                        mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+                        tma_load_2d(a_dst, &tmap_u, bar, 0, side * p.u_set_rows + (m + g) * kBM);   // (the second binding's u blocks: the second set)
+                        tma_load_3d(a_dst + Cfg::kABytes, &tmap_b, bar, 0, n * BN, s);
+                        advance();
+                    }
             }
             if (ok) {   // end of this CTA's K: a stage without operands
                 ok = acquire();
@@ -828,7 +840,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN);
             int stage = 0;
-            uint32_t phase = 0, accumulate = 0;
+            uint32_t phase = 0, accumulate = 0, accumulate2 = 0;
             bool ok = true;
             for (bool more = true; more && ok;) {
                 ok = mbar_wait(smem_u32(&ctrl->full[stage]), phase, abort);
@@ -840,16 +852,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 const uint64_t adesc = umma_desc_k128(a_addr);
                 const uint64_t bdesc = umma_desc_k128(a_addr + Cfg::kABytes);
                 tc_fence_after();
+                if ((info & kStageAcc1) == 0) {
 #pragma unroll 4
-                for (int k = 0; k < ksteps; ++k) {
-                    umma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
-                    accumulate = 1;
+                    for (int k = 0; k < ksteps; ++k) {
+                        umma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                }
+                if (info & (kStageAcc1 | kStageBoth)) {   // the second binding's accumulator
+#pragma unroll 4
+                    for (int k = 0; k < ksteps; ++k) {
+                        umma_bf16(tmem_base + (uint32_t)BN, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, accumulate2);
+                        accumulate2 = 1;
+                    }
                 }
                 umma_commit(smem_u32(&ctrl->empty[stage]));
                 if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
             }
             if (ok) umma_commit(smem_u32(&ctrl->tmem_full[0]));
-            ctrl->pad[0] = (int32_t)accumulate;   // 0: this CTA had no K at all, its accumulator holds nothing
+            ctrl->pad[0] = (int32_t)accumulate;    // 0: this CTA had no K at all, its accumulator holds nothing
+            ctrl->pad[1] = (int32_t)accumulate2;   // the same for the second binding's
         }
     }
     // ---------------------------------------------------------------------- exchange and reduction
@@ -859,12 +881,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
         ok = mbar_wait_warp(smem_u32(&ctrl->tmem_full[0]), 0u, abort);   // this CTA's MMAs are complete: so are its loads
         tc_fence_after();
     }
-    cluster_sync_all();   // every CTA of the cluster is done with its stage memory
     const int q = warp & 3;   // TMEM lane quarter an epilogue warp may read
     const int row = q * 32 + lane;
+    for (int o = 0; o < (dual ? 2 : 1); ++o) {   // one exchange per output
+    __nv_bfloat16* const yout = o ? p.y2 : p.y;
+    cluster_sync_all();   // every CTA of the cluster is done with its stage memory (and with the exchange before this one)
     if (warp >= 2 && ok) {
-        const bool have = ctrl->pad[0] != 0;
-        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const bool have = ctrl->pad[o] != 0;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(o * BN);
         int owner = 0;
 #pragma unroll 1
         for (int c = 0; c < kSplitChunks; ++c) {
@@ -917,15 +941,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_splitk_kernel
                 v.y = pack_bf16(acc[8 * j + 2], acc[8 * j + 3]);
                 v.z = pack_bf16(acc[8 * j + 4], acc[8 * j + 5]);
                 v.w = pack_bf16(acc[8 * j + 6], acc[8 * j + 7]);
-                *reinterpret_cast<uint4*>(p.y + (size_t)out_row * p.N + col0 + j * 8) = v;
+                *reinterpret_cast<uint4*>(yout + (size_t)out_row * p.N + col0 + j * 8) = v;
             }
         }
     }
+    }   // outputs
     __syncthreads();
     if (threadIdx.x == 0 && ctrl->abort) atomicOr(p.status, LML_FLAG_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, BN);
+        tmem_dealloc(tmem_base, dual ? 2 * BN : BN);
     }
 }
 

@@ -65,6 +65,32 @@ def test_dual_matches_two_single_calls(kw, monkeypatch):
     site.close()
 
 
+@pytest.mark.parametrize("kw", [dict(T=128, d_in=2048, d_out=1544), dict(T=77, d_in=1024, d_out=2056, shuffled=True),
+                                dict(T=300, d_in=2048, d_out=1032), dict(T=64, d_in=4096, d_out=4096)])
+def test_dual_with_few_tokens_takes_the_split_k_kernel(kw, monkeypatch):
+    """The chunk sizes of the paper's stale-coverage prefill (64 to 128 tokens, Section 5.3 / 7.5): the library picks
+    the split-K kernel, which multiplies the k-blocks into both bindings' accumulators.  First output bit for bit
+    the single call's (same kernel, same order), second within tolerance of the oracle."""
+    monkeypatch.delenv("LML_GEMM_SPLIT", raising=False)
+    w = wl.ragged(ranks=(4, 16, 1, 33, 64), **kw)
+    E = len(w.entries)
+    rng = np.random.default_rng(w.T + 1)
+    se_a = w.seg_entry.copy()
+    se_b = np.array([[int(rng.integers(0, E)), int(se_a[g]), -1][int(rng.integers(0, 3))] for g in range(w.G)], np.int32)
+    site = Site(w)
+    y_a, y_b, flags = _dual(site, w, se_a, se_b)
+    assert flags == 0
+    y_a1, f1 = site.run(seg_entry=se_a)
+    assert f1 == 0 and np.array_equal(y_a, y_a1)
+    for se, y in ((se_a, y_a), (se_b, y_b)):
+        ref, _ = oracle.forward(w.x, w.W0, w.entries, w.seg_offsets, se, w.perm)
+        r = oracle.compare(y, ref)
+        assert r["ok"], r
+    y_a2, y_b2, _ = _dual(site, w, se_a, se_b)
+    assert np.array_equal(y_a, y_a2) and np.array_equal(y_b, y_b2)
+    site.close()
+
+
 def test_dual_on_prefill_q_proj_sampled_rows():
     w = wl.prefill_q_proj()
     se_b = np.roll(w.seg_entry, 1)
