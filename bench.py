@@ -600,7 +600,7 @@ def run_layer_sweep(device, peaks, steps, only=None, parity=False):
     return cells
 
 
-def run_multi_decode(device, peaks, want_parity):
+def run_multi_decode(device, peaks, want_parity, calls=600):
     """Several projections of one decode step in one lora_mixed_linear_multi call: q/k/v (3 x 4096 x 4096) and
     gate/up (2 x 11008 x 4096) of a 7B-class layer, 8 tokens of 4 agents, 5 resident entries of rank 16 per
     projection.  Per cell: microseconds per call, algorithmic GB/s and fraction of the measured HBM peak, against
@@ -653,7 +653,7 @@ def run_multi_decode(device, peaks, want_parity):
                                            s_["ys"][p].data_ptr(), s_["ws"].data_ptr(), s_["ws"].numel(), b._stream(None))
             return P
 
-        n = max(R, 600)
+        n = max(R, calls)
         m_secs, m_launches, _ = timed_graph_loop(multi, R, n, 3 * R, stream)
         s_secs, _, _ = timed_graph_loop(separate, R, n, 3 * R, stream)
         cell = {"workload": name, "projections": P, "d_in": K, "d_out": list(Ns), "tokens": T,
@@ -733,7 +733,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=2000)
-    ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS) + ["layer_sweep"],
+    ap.add_argument("--workload", default="decode_q_proj", choices=sorted(WORKLOADS) + ["layer_sweep", "multi_decode"],
                     help="layer_sweep: per-cell timings of the decoder-layer sweep (1 GPU, its own JSON line)")
     ap.add_argument("--sweep-cells", default="", help="layer_sweep: only these cells, e.g. q:128,down:16 (projections q, gate, down)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -761,6 +761,13 @@ def main():
     barrier()
     peaks = measured_peaks()
     warmup = max(3, args.warmup)
+    if args.workload == "multi_decode":
+        if rank == 0:
+            print(json.dumps({"metric": "several projections of one decode step in one lora_mixed_linear_multi call", "unit": "us",
+                              "n_gpus": 1, "dtype": "bf16", "data": "synthetic", "peak_source": peaks["source"],
+                              "cells": run_multi_decode(device, peaks, True, calls=max(8, min(args.steps, 600)))}), flush=True)
+        barrier()
+        return
     if args.workload == "layer_sweep":
         only = {(c.split(":")[0], int(c.split(":")[1])) for c in args.sweep_cells.split(",") if c} or None
         if rank == 0:
