@@ -422,7 +422,7 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                 "peak_source": peaks["source"], "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None,
                 "us_per_launch": per_launch * 1e6}
     else:
-        roof = {"bound": "tensor", "kernel": "lora_gemm_sm100_kernel (time includes the shrink kernel before it)",
+        roof = {"bound": "tensor", "kernel": "lora_gemm_sm100_kernel (the LoRA shrink runs inside it)",
                 "achieved": achieved, "peak": peaks["tensor_burst"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["tensor_burst"], "peak_source": peaks["source"] + " burst",
                 "frac_of_sustained": achieved / peaks["tensor_sustained"], "frac_of_nominal_2250": achieved / 2250.0,

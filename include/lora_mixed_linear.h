@@ -238,8 +238,9 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
                                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Backward pass of the layer, for the training task that shares the GPU with inference (Section 3.1,
- * Section 4.1).  With y = x.W0^T + s (x.A^T).B^T per segment and an upstream gradient dy [T][d_out]:
+ * Backward pass of the layer, for the training task that shares the GPU with inference (Section 2.2:
+ * adapters are updated online in the background; Section 4.1: the task model's training task).
+ * With y = x.W0^T + s (x.A^T).B^T per segment and an upstream gradient dy [T][d_out]:
  *
  *   dx = dy.W0 + s (dy.B).A  is the layer itself on the transposed problem: a second table t_T with
  *   d_in = d_out(t), d_out = d_in(t), the caller's W0^T [d_in][d_out] as base weight and every adapter

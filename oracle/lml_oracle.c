@@ -220,8 +220,9 @@ int lml_oracle_segment(const int32_t *token_entry, int T, int num_entries, int32
 }
 
 /*
- * Backward pass of the layer for the training task (Section 3.1: adapters are trained in the
- * background; Section 4.1: the training step is one of the tasks that share the GPU).  With
+ * Backward pass of the layer for the training task (Section 2.2, online RL: adapters are updated
+ * in the background; Section 4.1, task model: the training step is one of the tasks that share
+ * the GPU).  With
  *     y[t] = x[t].W0^T + s_e (x[t].A_e^T).B_e^T          (e = entry of the position of row t)
  * and an upstream gradient dy [T][N] (bf16 like every activation), the definitions are
  *     dx[t]     = dy[t].W0 + s_e (dy[t].B_e).A_e

@@ -52,7 +52,7 @@ template <int BN> struct GemmCfg {
     static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;
     static constexpr int kTmemCols = 2 * BN;
-    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache + 512;   // barriers + segment cache (two slot arrays) + shrink plan
+    static constexpr int kCtrlBytes = 256 + (kSegCache + 1) * 4 + 2 * kSegCache + 512 + 1040;   // barriers + segment cache (two slot arrays) + shrink plan + its per-tile table
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiBytes + ((kCtrlBytes + 15) & ~15);
 };
 
@@ -83,10 +83,11 @@ constexpr uint32_t kStageShrink = 0x1000u;  // a stage of a shrink pass: x tile 
 // k-blocks with the A blocks of up to BN / 64 segments that touch the tile (128 x 64 tcgen05 products side by side
 // in an accumulator), its epilogue writes the u blocks and raises the tile's flag in the table's device memory.
 constexpr int kShrMaxPasses = 8;
+constexpr int kFuseTilesInKernel = 512;   // row tiles of a call whose shrink runs inside the kernel (the per-tile table in shared memory)
 struct ShrPass {
     int32_t m;          // row tile
     int32_t n;          // pieces in this pass
-    int32_t last;       // the tile's last pass: raise its flag afterwards
+    int32_t flag;       // the pass's number among all passes of the call: the flag it raises
     int32_t g[4];       // segment of each piece
     int32_t slot[4];
 };
@@ -127,7 +128,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ SlotSnapshot snap, const GemmParams p)
 {
     using Cfg = GemmCfg<BN>;
-    constexpr int kShrPerPass = BN / 64;   // 128 x 64 products that fit side by side in one accumulator
+    // One piece to a pass: a pass with one piece moves two k-blocks per stage and takes about as long as an output
+    // tile; more pieces side by side (up to BN / 64 fit an accumulator) halve that rate, and every CTA's first
+    // tile would wait for the longest pass.  A row tile's pieces run on different CTAs instead.
+    constexpr int kShrPerPass = 1;
     const bool dual = p.slot_ids2 != nullptr;
     extern __shared__ uint8_t smem_raw[];
     // 128-byte swizzled tiles need 1024-byte alignment
@@ -141,6 +145,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
     int8_t* slot_cache = reinterpret_cast<int8_t*>(seg_cache + kSegCache + 1);
     int8_t* slot_cache2 = slot_cache + kSegCache;   // dual form: the second slot per segment
     ShrPlan* shr = reinterpret_cast<ShrPlan*>(slot_cache2 + kSegCache);
+    uint16_t* shr_base = reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(shr) + 512);   // [row tile] first pass; kFuseTilesInKernel + 1 entries
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = p.num_m * p.num_n;
@@ -201,6 +206,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
         if (threadIdx.x == 0 && (seg_cache[0] != 0 || seg_cache[p.G] != p.T)) bad_off = 1;
         bad_off = __syncthreads_or(bad_off);
         bad_slot = __syncthreads_or(bad_slot);
+        // Passes of every row tile: its live pieces, kShrPerPass to a pass (threads share the tiles out) ...
+        auto live_pieces = [&](int m, int skip, int take, ShrPass* out) -> int {   // counts the tile's pieces; fills `out` with pieces skip .. skip+take-1
+            const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
+            int lo = 0, hi = p.G;
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
+            int c = 0;
+            for (int g = lo; g < p.G && seg_cache[g] < row1; ++g) {
+                const int sl = slot_cache[g];
+                if (sl < 0 || min(seg_cache[g + 1], row1) <= max(seg_cache[g], row0)) continue;
+                if (out && c >= skip && c < skip + take) { out->g[c - skip] = g; out->slot[c - skip] = sl; }
+                ++c;
+            }
+            return c;
+        };
+        for (int m = threadIdx.x; m < p.num_m; m += kGemmThreads)
+            shr_base[m + 1] = (uint16_t)(bad_off ? 0 : (live_pieces(m, 0, 0, nullptr) + kShrPerPass - 1) / kShrPerPass);
+        __syncthreads();
         if (threadIdx.x == 0) {
             if (blockIdx.x == 0) {
                 const unsigned f = (bad_off ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u);
@@ -208,22 +230,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
             }
             shr->lora_ok = bad_off ? 0 : 1;
             shr->epoch = (int32_t)(*reinterpret_cast<volatile uint32_t*>(p.fuse_sync));
-            int np = 0;
-            for (int m = (int)gridDim.x - 1 - (int)blockIdx.x; m < p.num_m && !bad_off; m += (int)gridDim.x) {
-                const int row0 = m * kBM, row1 = min(row0 + kBM, p.T);
-                int lo = 0, hi = p.G;
-                while (lo < hi) { const int mid = (lo + hi) >> 1; if (seg_cache[mid + 1] > row0) hi = mid; else lo = mid + 1; }
-                const int first_pass = np;
-                int n = 0;
-                for (int g = lo; g < p.G && seg_cache[g] < row1 && np < kShrMaxPasses; ++g) {
-                    const int s = slot_cache[g];
-                    if (s < 0 || min(seg_cache[g + 1], row1) <= max(seg_cache[g], row0)) continue;
-                    ShrPass& ps = shr->pass[np];
-                    ps.m = m; ps.g[n] = g; ps.slot[n] = s; ps.last = 0;
-                    if (++n == kShrPerPass) { ps.n = n; n = 0; ++np; }
-                }
-                if (n > 0 && np < kShrMaxPasses) { shr->pass[np].n = n; ++np; }
-                if (np > first_pass) shr->pass[np - 1].last = 1;   // (a tile that no live segment touches has no pass and no flag: nobody waits for it)
+            // ... numbered through all row tiles (shr_base[m] = first pass of tile m); pass i is the work of CTA
+            // grid-1 - (i mod grid): the CTAs at the end of the grid own the fewest output tiles, and the passes
+            // of a row tile with many pieces run side by side on different CTAs
+            shr_base[0] = 0;
+            for (int m = 0; m < p.num_m; ++m) shr_base[m + 1] = (uint16_t)(shr_base[m] + shr_base[m + 1]);
+            const int total = shr_base[p.num_m];
+            int np = 0, m = 0;
+            for (int i = (int)gridDim.x - 1 - (int)blockIdx.x; i < total && np < kShrMaxPasses; i += (int)gridDim.x) {
+                while (shr_base[m + 1] <= i) ++m;
+                ShrPass& ps = shr->pass[np++];
+                ps.m = m; ps.flag = i;
+                const int c = live_pieces(m, (i - shr_base[m]) * kShrPerPass, kShrPerPass, &ps);
+                ps.n = min(kShrPerPass, c - (i - shr_base[m]) * kShrPerPass);
             }
             shr->npass = np;
         }
@@ -268,10 +287,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
                 if (!p.fused || m == flag_seen_m) return;
                 const int want = shr->epoch + 1;
                 const long long t0 = clock64();
-                while (ld_acquire_gpu_s32(p.tile_flags + m) != want) {
-                    if (*abort) { ok = false; return; }
-                    if (clock64() - t0 > (1ll << 31)) { *abort = 1; ok = false; return; }
-                }
+                for (int i = shr_base[m]; i < shr_base[m + 1]; ++i)
+                    while (ld_acquire_gpu_s32(p.tile_flags + i) != want) {
+                        if (*abort) { ok = false; return; }
+                        if (clock64() - t0 > (1ll << 31)) { *abort = 1; ok = false; return; }
+                    }
                 fence_proxy_async_all();   // what those CTAs wrote with ordinary stores is read by TMA from here on
                 flag_seen_m = m;
             };
@@ -571,7 +591,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lora_gemm_sm100_kernel(
             fence_proxy_async_all();   // the blocks will be read by TMA
             __threadfence();
             asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
-            if (sp.last && warp == 2 && lane == 0) st_release_gpu_s32(p.tile_flags + sp.m, shr->epoch + 1);
+            if (warp == 2 && lane == 0) st_release_gpu_s32(p.tile_flags + sp.flag, shr->epoch + 1);
             acc ^= 1;
         }
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -1125,14 +1145,14 @@ bool gemm_can_fuse_shrink(int T, int d_in, int d_out, int G, int num_sms, int sp
 {
     if (G <= 0 || G > kSegCache) return false;
     if (gemm_pick_split(T, d_in, d_out, num_sms, split_bn, split_s).split) return false;
-    const int bn = gemm_pick_bn(T, d_out, num_sms);
-    const int num_m = (T + kBM - 1) / kBM, num_n = (d_out + bn - 1) / bn;
-    if (num_m > kFuseMaxTiles) return false;
-    const int grid = min(num_m * num_n, num_sms);
-    const int tiles_per_cta = (num_m + grid - 1) / grid;
-    const int per_pass = bn / 64;
-    const int passes_per_tile = (min(G, kBM) + per_pass - 1) / per_pass;
-    return tiles_per_cta * passes_per_tile <= kShrMaxPasses;
+    // A shrink pass takes about as long as an output tile, whatever its width.  It pays where some CTAs have a
+    // tile's time to spare and the others do not reach their first pieces before it is over: 256-column tiles in
+    // more than one wave, and few enough passes that no CTA gets two.
+    if (gemm_pick_bn(T, d_out, num_sms) != 256) return false;
+    const int num_m = (T + kBM - 1) / kBM, num_n = (d_out + 255) / 256;
+    if (num_m > kFuseTilesInKernel || num_m * num_n <= num_sms) return false;
+    const int worst_passes = num_m + G;   // (every segment boundary inside a row tile adds a piece)
+    return worst_passes <= num_sms / 2;
 }
 
 cudaError_t launch_gemm_sm100(const Arena& ar, const SlotSnapshot& snap, const CUtensorMap& tmap_B256,

@@ -1,7 +1,7 @@
 """The LoRA shrink inside the GEMM kernel (whole-K tiles: the CTAs with the fewest output tiles first compute
 u = scale * x.A^T for a row tile each on the tensor cores and raise a flag per row tile) against the oracle and
 against the separate shrink kernel (LML_FUSE_SHRINK=0, read when a table is created): the two differ only in
-the rounding of u to bf16.  Shapes are wide enough that the library does not pick the split-K kernel."""
+the rounding of u to bf16.  Shapes are such that the library chooses the fused form (256-column tiles in more than one wave)."""
 import numpy as np
 import pytest
 
@@ -33,7 +33,7 @@ def _both(w, monkeypatch, **run_kw):
     return y_fused
 
 
-@pytest.mark.parametrize("kw", [dict(T=700, d_in=520, d_out=3000), dict(T=1300, d_in=1032, d_out=2056, shuffled=True),
+@pytest.mark.parametrize("kw", [dict(T=700, d_in=520, d_out=8192), dict(T=1300, d_in=1032, d_out=4104, shuffled=True),
                                 dict(T=2100, d_in=264, d_out=5000)])
 def test_fused_shrink_matches_oracle_and_separate_kernel(kw, monkeypatch):
     w = wl.ragged(ranks=(4, 16, 1, 33, 64), **kw)
@@ -44,8 +44,8 @@ def test_fused_shrink_matches_oracle_and_separate_kernel(kw, monkeypatch):
 
 
 def test_many_segments_in_one_row_tile_take_several_passes(monkeypatch):
-    # 14 segments over 700 rows: several pieces in a 128-row tile, two to a pass with 128-column tiles
-    w = wl.ragged(T=700, d_in=520, d_out=3000, ranks=(8, 16, 4, 32, 64))
+    # 14 segments over 700 rows: several pieces in a 128-row tile, each a pass of its own on another CTA
+    w = wl.ragged(T=700, d_in=520, d_out=8192, ranks=(8, 16, 4, 32, 64))
     rng = np.random.default_rng(5)
     cuts = np.sort(rng.integers(0, w.T + 1, size=13))
     so = np.concatenate([[0], cuts, [w.T]]).astype(np.int32)
@@ -59,7 +59,7 @@ def test_many_segments_in_one_row_tile_take_several_passes(monkeypatch):
 def test_malformed_offsets_are_caught_by_the_fused_form(monkeypatch):
     from paper_2608_15241_b200 import binding
     monkeypatch.delenv("LML_FUSE_SHRINK", raising=False)
-    w = wl.ragged(T=700, d_in=520, d_out=3000, ranks=(8, 16, 4))
+    w = wl.ragged(T=700, d_in=520, d_out=8192, ranks=(8, 16, 4))
     T = w.T
     site = Site(w)
     y, flags = site.run(seg_offsets=[0, 2 * T // 3, T // 3, T], raw_slot_ids=[site.slots[0], site.slots[1], site.slots[2]])

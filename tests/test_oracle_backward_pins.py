@@ -1,4 +1,4 @@
-"""Pins for the oracle's backward pass (the gradients of Section 3.1's training task through the
+"""Pins for the oracle's backward pass (the gradients that the training task of Sections 2.2 and 4.1 takes through the
 mixed-adapter linear layer).  Nothing here calls the CUDA path.
 
 * The forward oracle is linear in x, in A and in B, so a central difference of the scalar
