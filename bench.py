@@ -279,28 +279,31 @@ def timed_graph_loop(fn, R, steps, warmup, stream, min_warm_seconds=0.0):
     Returns (seconds, kernel launches inside the timed region, (t0, t1) wall clock)."""
     import torch
     launches_per = [0] * R
+    # One graph holds several rounds over the R input sets (at least 64 calls when the run is long enough): consecutive
+    # calls inside a graph overlap as programmatic dependents, consecutive graph launches do not.
+    Rg = R * max(1, min(-(-64 // R), steps // R)) if steps >= R else R
     with torch.cuda.stream(stream):
         for i in range(R):          # eager pass: allocations, lazy init
             launches_per[i] = fn(i)
         stream.synchronize()
         g_full = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g_full, stream=stream):
-            for i in range(R):
+            for i in range(Rg):
                 fn(i)
-        tail = steps % R
+        tail = steps % Rg
         g_tail = None
         if tail:
             g_tail = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g_tail, stream=stream):
                 for i in range(tail):
                     fn(i)
-        warm_replays = max(1, -(-warmup // R))
+        warm_replays = max(1, -(-warmup // Rg))
         t_w = time.time()
         n = 0
         while n < warm_replays or time.time() - t_w < min_warm_seconds:
             g_full.replay()
             n += 1
-            if n % 64 == 0:
+            if n % 16 == 0:
                 stream.synchronize()
         stream.synchronize()
         barrier()
@@ -308,7 +311,7 @@ def timed_graph_loop(fn, R, steps, warmup, stream, min_warm_seconds=0.0):
         torch.cuda.synchronize()
         t0 = time.time()
         ev0.record(stream)
-        for _ in range(steps // R):
+        for _ in range(steps // Rg):
             g_full.replay()
         if g_tail is not None:
             g_tail.replay()
@@ -316,7 +319,7 @@ def timed_graph_loop(fn, R, steps, warmup, stream, min_warm_seconds=0.0):
         torch.cuda.synchronize()
         t1 = time.time()
         barrier()
-    launches = (steps // R) * sum(launches_per) + sum(launches_per[:tail])
+    launches = (steps // R) * sum(launches_per) + sum(launches_per[:steps % R])
     return ev0.elapsed_time(ev1) / 1e3, launches, (t0, t1)
 
 

@@ -54,7 +54,7 @@ constexpr int kDecSpan = 4096;                   // columns whose x fragments fi
 constexpr int kDecChunk = 2048;                  // columns per stage (one 4 KB bulk copy per row)
 constexpr int kDecChunksPerSpan = kDecSpan / kDecChunk;             // 4
 constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 8 k-steps per warp and stage
-constexpr int kDecRowPitch = kDecChunk * 2 + 64; // bytes; a multiple of 16 that is 4 mod 8 in 16-byte chunks: rows land on different banks
+constexpr int kDecRowPitch = kDecChunk * 2 + 16; // bytes; one 16-byte chunk more than a multiple of 128: a quarter-warp's reads (2 rows x 4 lanes, 32 bytes apart) cover all banks
 constexpr int kDecStageBytes = kDecUnitRows * kDecRowPitch;
 constexpr int kDecStages = 4;
 constexpr int kDecRoundUnits = 4;                // units (= 32 rows) reduced together
@@ -197,14 +197,30 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
 
     // This warp's x fragments (chunk kc, k-steps warp*S .. warp*S+S-1 of a span) stay in registers.
     uint4 xa[kChunksPerSpan * kDecStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDecStepsPerChunk : 1];
+    // Fragment i of a chunk (i = 0..7 per warp) holds the 8 columns warp*256 + (i/2)*64 + tq*16 + (i&1)*8 ..: a lane's
+    // fragments 2j and 2j+1 are 32 consecutive bytes of its row of x, so one 32-byte load fetches both and a warp's load
+    // covers whole 128-byte lines (half as many requests to L2 as 16-byte loads).  The ring is read with the same
+    // permutation, which a dot product does not see.
+    const bool x_wide = ((reinterpret_cast<uintptr_t>(x) | (uintptr_t)((size_t)K * 2)) & 31u) == 0;
     auto load_x = [&](int k_begin, int span) {
         const bool ta = gq < T, tb = gq + 8 < T;
 #pragma unroll
-        for (int i = 0; i < kChunksPerSpan * kDecStepsPerChunk; ++i) {
-            const int c = (i / kDecStepsPerChunk) * kDecChunk + (warp * kDecStepsPerChunk + i % kDecStepsPerChunk) * 32 + tq * 8;
-            const bool lv = c < span;
-            xa[i] = (lv && ta) ? ldg_nc_v4(x + (size_t)gq * K + k_begin + c) : make_uint4(0, 0, 0, 0);
-            if (kTwo) xc[i] = (lv && tb) ? ldg_nc_v4(x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < kChunksPerSpan * kDecStepsPerChunk; i += 2) {
+            const int c = (i / kDecStepsPerChunk) * kDecChunk + (warp * kDecStepsPerChunk + i % kDecStepsPerChunk) * 32 + tq * 16;
+            const __nv_bfloat16* pa = x + (size_t)gq * K + k_begin + c;
+            const __nv_bfloat16* pb = x + (size_t)(gq + 8) * K + k_begin + c;
+            if (x_wide && c + 16 <= span) {
+                if (ta) ldg_nc_v8(pa, xa[i], xa[i + 1]); else xa[i] = xa[i + 1] = make_uint4(0, 0, 0, 0);
+                if (kTwo) { if (tb) ldg_nc_v8(pb, xc[i], xc[i + 1]); else xc[i] = xc[i + 1] = make_uint4(0, 0, 0, 0); }
+            } else {
+                const bool l0 = c < span, l1 = c + 8 < span;
+                xa[i] = (l0 && ta) ? ldg_nc_v4(pa) : make_uint4(0, 0, 0, 0);
+                xa[i + 1] = (l1 && ta) ? ldg_nc_v4(pa + 8) : make_uint4(0, 0, 0, 0);
+                if (kTwo) {
+                    xc[i] = (l0 && tb) ? ldg_nc_v4(pb) : make_uint4(0, 0, 0, 0);
+                    xc[i + 1] = (l1 && tb) ? ldg_nc_v4(pb + 8) : make_uint4(0, 0, 0, 0);
+                }
+            }
         }
     };
 
@@ -622,7 +638,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                         if (kc < nchunks && ok) {
                             ok = mbar_wait_warp(smem_u32(&ctrl->full[stage]), phase, abort);
                             if (ok) {
-                                const uint32_t wbase = ring + stage * kDecStageBytes + gq * kDecRowPitch + tq * 16;
+                                const uint32_t wbase = ring + stage * kDecStageBytes + gq * kDecRowPitch + tq * 32 + warp * (kDecStepsPerChunk * 64);
                                 // all of the stage's operand reads first, then the stage can go back to the producer
                                 // before the MMAs run
                                 uint4 w[kDecStepsPerChunk];
@@ -630,7 +646,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                                     // a full stage (all but the ragged edges): no predicates
 #pragma unroll
                                     for (int i = 0; i < kDecStepsPerChunk; ++i)
-                                        w[i] = lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64));
+                                        w[i] = lds128(wbase + (uint32_t)((i >> 1) * 128 + (i & 1) * 16));
 #pragma unroll
                                     for (int i = 0; i < kDecStepsPerChunk; ++i) {
                                         const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
@@ -641,13 +657,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                                 } else {
 #pragma unroll
                                     for (int i = 0; i < kDecStepsPerChunk; ++i) {
-                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
-                                        w[i] = (rv && c0 + tq * 8 < span) ? lds128(wbase + (uint32_t)((warp * kDecStepsPerChunk + i) * 64))
-                                                                          : make_uint4(0, 0, 0, 0);
+                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + (i & ~1)) * 32;   // the pair's 64 columns start here
+                                        w[i] = (rv && c0 + tq * 16 + (i & 1) * 8 < span) ? lds128(wbase + (uint32_t)((i >> 1) * 128 + (i & 1) * 16))
+                                                                                         : make_uint4(0, 0, 0, 0);
                                     }
 #pragma unroll
                                     for (int i = 0; i < kDecStepsPerChunk; ++i) {
-                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + i) * 32;
+                                        const int c0 = kc * kDecChunk + (warp * kDecStepsPerChunk + (i & ~1)) * 32;
                                         if (c0 < span) {   // uniform across the warp: all lanes issue the MMAs or none
                                             const uint4 a0 = xa[kc * kDecStepsPerChunk + i];
                                             const uint4 a1 = kTwo ? xc[kc * kDecStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
