@@ -46,7 +46,7 @@ constexpr int kDsUnitRows = 8;                   // rows per unit = the 8-wide M
 constexpr int kDsSpan = 4096;                    // columns whose x fragments fit in registers (half of it for T > 8)
 constexpr int kDsChunk = 2048;                   // columns per stage (one 4 KB bulk copy per row)
 constexpr int kDsStepsPerChunk = kDsChunk / 32 / kDsConsumers;   // 8 k-steps per warp and stage
-constexpr int kDsRowPitch = kDsChunk * 2 + 64;   // bytes; rows land on different banks
+constexpr int kDsRowPitch = kDsChunk * 2 + 16;   // bytes; a quarter-warp's reads (2 rows x 4 lanes, 32 bytes apart) cover all banks
 constexpr int kDsStageBytes = kDsUnitRows * kDsRowPitch;
 constexpr int kDsStages = 4;
 constexpr int kDsRoundUnits = 4;                 // units (<= 32 rows) reduced together
@@ -570,18 +570,32 @@ __global__ void __launch_bounds__(kDsThreads, 1) decode_stream_kernel(const __gr
     const int gq = lane >> 2, tq = lane & 3;
     uint4 xa[kChunksPerSpan * kDsStepsPerChunk], xc[kTwo ? kChunksPerSpan * kDsStepsPerChunk : 1];
     int span_loaded = -1;
-    // The x fragments of span sp into registers (plain 16-byte loads: x is small and sits in L2).
+    // The x fragments of span sp into registers.  Fragment i of a chunk holds the 8 columns warp*256 + (i/2)*64 + tq*16 +
+    // (i&1)*8 ..: fragments 2j and 2j+1 of a lane are 32 consecutive bytes of its row, fetched by one 32-byte load, so a
+    // warp's load covers whole 128-byte lines.  The weights are read with the same permutation on either route.
+    const bool x_wide = ((reinterpret_cast<uintptr_t>(prm.x) | (uintptr_t)((size_t)K * 2)) & 31u) == 0;
     auto ensure_x = [&](int sp) {
         if (sp == span_loaded) return;
         span_loaded = sp;
         const int k_begin = sp * kSpan, span = min(kSpan, K - k_begin);
         const bool ta = gq < T, tb = gq + 8 < T;
 #pragma unroll
-        for (int i = 0; i < kChunksPerSpan * kDsStepsPerChunk; ++i) {
-            const int c = (i / kDsStepsPerChunk) * kDsChunk + (warp * kDsStepsPerChunk + i % kDsStepsPerChunk) * 32 + tq * 8;
-            const bool lv = c < span;
-            xa[i] = (lv && ta) ? ldg_nc_v4(prm.x + (size_t)gq * K + k_begin + c) : make_uint4(0, 0, 0, 0);
-            if (kTwo) xc[i] = (lv && tb) ? ldg_nc_v4(prm.x + (size_t)(gq + 8) * K + k_begin + c) : make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < kChunksPerSpan * kDsStepsPerChunk; i += 2) {
+            const int c = (i / kDsStepsPerChunk) * kDsChunk + (warp * kDsStepsPerChunk + i % kDsStepsPerChunk) * 32 + tq * 16;
+            const __nv_bfloat16* pa = prm.x + (size_t)gq * K + k_begin + c;
+            const __nv_bfloat16* pb = prm.x + (size_t)(gq + 8) * K + k_begin + c;
+            if (x_wide && c + 16 <= span) {
+                if (ta) ldg_nc_v8(pa, xa[i], xa[i + 1]); else xa[i] = xa[i + 1] = make_uint4(0, 0, 0, 0);
+                if (kTwo) { if (tb) ldg_nc_v8(pb, xc[i], xc[i + 1]); else xc[i] = xc[i + 1] = make_uint4(0, 0, 0, 0); }
+            } else {
+                const bool l0 = c < span, l1 = c + 8 < span;
+                xa[i] = (l0 && ta) ? ldg_nc_v4(pa) : make_uint4(0, 0, 0, 0);
+                xa[i + 1] = (l1 && ta) ? ldg_nc_v4(pa + 8) : make_uint4(0, 0, 0, 0);
+                if (kTwo) {
+                    xc[i] = (l0 && tb) ? ldg_nc_v4(pb) : make_uint4(0, 0, 0, 0);
+                    xc[i + 1] = (l1 && tb) ? ldg_nc_v4(pb + 8) : make_uint4(0, 0, 0, 0);
+                }
+            }
         }
     };
     // One unit (up to eight rows) times one span of x: this warp's partial sums [token][row] into `out` (set on the
@@ -601,14 +615,14 @@ __global__ void __launch_bounds__(kDsThreads, 1) decode_stream_kernel(const __gr
             if (kc < nchunks && ok) {
                 if (!kGlobal) ok = mbar_wait_warp(smem_u32(&ctrl->full[stage]), phase, abort);
                 if (ok) {
-                    const uint32_t wbase = ring + stage * kDsStageBytes + gq * kDsRowPitch + tq * 16;
+                    const uint32_t wbase = ring + stage * kDsStageBytes + gq * kDsRowPitch + tq * 32 + warp * (kDsStepsPerChunk * 64);
                     uint4 w[kDsStepsPerChunk];
                     if (!kGlobal && rows == kDsUnitRows && span - kc * kDsChunk >= kDsChunk) {
                         // a full stage (all but the ragged edges): straight-line code, no predicates: all of the
                         // stage's operand reads first, then its MMAs
 #pragma unroll
                         for (int i = 0; i < kDsStepsPerChunk; ++i)
-                            w[i] = lds128(wbase + (uint32_t)((warp * kDsStepsPerChunk + i) * 64));
+                            w[i] = lds128(wbase + (uint32_t)((i >> 1) * 128 + (i & 1) * 16));
 #pragma unroll
                         for (int i = 0; i < kDsStepsPerChunk; ++i) {
                             const uint4 a0 = xa[kc * kDsStepsPerChunk + i];
@@ -619,14 +633,15 @@ __global__ void __launch_bounds__(kDsThreads, 1) decode_stream_kernel(const __gr
                     } else {
 #pragma unroll
                         for (int i = 0; i < kDsStepsPerChunk; ++i) {
-                            const int c0 = kc * kDsChunk + (warp * kDsStepsPerChunk + i) * 32;
-                            const bool lv = rv && c0 + tq * 8 < span;
-                            if (kGlobal) w[i] = lv ? ldg_nc_v4(grow + k_begin + c0 + tq * 8) : make_uint4(0, 0, 0, 0);
-                            else w[i] = lv ? lds128(wbase + (uint32_t)((warp * kDsStepsPerChunk + i) * 64)) : make_uint4(0, 0, 0, 0);
+                            const int c0 = kc * kDsChunk + (warp * kDsStepsPerChunk + (i & ~1)) * 32;   // the pair's 64 columns start here
+                            const int cl = c0 + tq * 16 + (i & 1) * 8;                                   // this lane's 8 columns
+                            const bool lv = rv && cl < span;
+                            if (kGlobal) w[i] = lv ? ldg_nc_v4(grow + k_begin + cl) : make_uint4(0, 0, 0, 0);
+                            else w[i] = lv ? lds128(wbase + (uint32_t)((i >> 1) * 128 + (i & 1) * 16)) : make_uint4(0, 0, 0, 0);
                         }
 #pragma unroll
                         for (int i = 0; i < kDsStepsPerChunk; ++i) {
-                            const int c0 = kc * kDsChunk + (warp * kDsStepsPerChunk + i) * 32;
+                            const int c0 = kc * kDsChunk + (warp * kDsStepsPerChunk + (i & ~1)) * 32;
                             if (c0 < span) {   // uniform across the warp: all lanes issue the MMAs or none
                                 const uint4 a0 = xa[kc * kDsStepsPerChunk + i];
                                 const uint4 a1 = kTwo ? xc[kc * kDsStepsPerChunk + i] : make_uint4(0, 0, 0, 0);
