@@ -290,18 +290,16 @@ lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0,
  * x, or -1; the pointers may be equal when the tables were filled in the same order) and output
  * y[p] (device bf16 [T][d_out_p], distinct buffers).  tables, W0, token_slots and y are HOST arrays of
  * P pointers, 1 <= P <= LML_MAX_PROJECTIONS; all tables share d_in and the device.
- * T <= 16: ONE launch of the decode kernel.  The rows of all base weights form one stream that the
- * grid shares out evenly, x is read once, the fixed cost of a launch is paid once; results per
- * projection are those of lora_mixed_linear_tokens on that projection, to fp32 summation order.  The
- * library falls back to one decode call per projection where that is the faster way or the only one:
- * weights so large that a launch's fixed cost no longer counts (gate / up of a 7B-class MLP), and
- * tables whose resident adapters have more rows than the one-launch kernel streams (more than
- * an eighth of the weights' rows, or more than 1024).
+ * T <= 16: ONE launch of the decode kernel for all projections.  Its CTAs are dealt out over the projections in
+ * proportion to their rows; each works on its projection exactly as in a call of its own, so results per
+ * projection are bit for bit those of lora_mixed_linear_tokens on that projection, and the fixed cost of a
+ * call (the wait for the preceding work, the fetch of x, the tail) is paid once.  A single projection, or a
+ * table named twice, runs as one decode call per projection.
  * T > 16: the projections run one after the other on `stream`, each exactly as
  * lora_mixed_linear_tokens(tables[p], ...).
- * The call counts its CTAs in tables[0]'s status block: two multi calls that share tables[0], or a multi
- * call and a decode call on tables[0], must not overlap on the GPU.  Device-detected errors set the
- * flags of the table they concern (malformed input that concerns all: tables[0]).
+ * Every projection's CTAs count themselves in that table's status block, as in a decode call: two calls
+ * that share a table must not overlap on the GPU.  Device-detected errors set the flags of the table they
+ * concern.
  * workspace: device, 256-byte aligned, at least lml_multi_workspace_bytes(tables, P, T).
  * Errors: INVALID_ARG, WORKSPACE, CUDA.
  */

@@ -17,7 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "liblora_mixed_linear.so")
-SOURCES = ["lml_api.cu", "lml_aux.cu", "lml_shrink.cu", "lml_decode.cu", "lml_decode_stream.cu", "lml_gemm_sm100.cu",
+SOURCES = ["lml_api.cu", "lml_aux.cu", "lml_shrink.cu", "lml_decode.cu", "lml_gemm_sm100.cu",
            "lml_noalloc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

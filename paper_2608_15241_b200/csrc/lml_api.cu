@@ -24,8 +24,8 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
     w.ident_off = round_up(sizeof(PlanWord), 256);
     w.u_off = round_up(w.ident_off + (num_m + 1) * sizeof(int32_t), 1024);
     size_t u_bytes = (size_t)u_sets * (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
-    // the decode kernels' scratch: u[16][64] fp32 for one projection, the exchange buffer of the one-launch form for several
-    const size_t dec_bytes = kDsExchangeBytes;
+    // the decode kernel's scratch: u[16][64] fp32 per projection of a launch
+    const size_t dec_bytes = (size_t)LML_MAX_PROJECTIONS * 16 * kRankPad * sizeof(float);
     if (u_bytes < dec_bytes) u_bytes = dec_bytes;
     w.xg_off = w.u_off + round_up(u_bytes, 1024);
     w.total = w.xg_off + round_up((size_t)T * t->d_in * sizeof(__nv_bfloat16), 1024);
@@ -176,7 +176,6 @@ lml_status register_adapter(lml_table* t, int adapter_id, int version, const voi
     e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
     e.state = LML_STATE_RESIDENT; e.pins = 0;
     e.gen = ++t->next_gen;
-    t->arena_dirty = true;
     e.live = true;   // published last: the entry is complete before it becomes visible
     *slot_out = free_slot;
     return LML_OK;
@@ -211,7 +210,6 @@ lml_status register_adapter_transposed(lml_table* t_T, int adapter_id, int versi
     e.adapter_id = adapter_id; e.version = version; e.rank = rank; e.scale = scale;
     e.state = LML_STATE_RESIDENT; e.pins = 0;
     e.gen = ++t_T->next_gen;
-    t_T->arena_dirty = true;
     e.live = true;
     *slot_out = free_slot;
     return LML_OK;
@@ -642,7 +640,7 @@ lml_status lora_mixed_linear_adapters(lml_table* t, const void* x, const void* W
 
 size_t lml_multi_workspace_bytes(lml_table* const* tables, int P, int max_tokens)
 {
-    if (!tables || P < 1 || P > kDsMaxProj || max_tokens < 0 || max_tokens > kMaxTokens) return 0;
+    if (!tables || P < 1 || P > LML_MAX_PROJECTIONS || max_tokens < 0 || max_tokens > kMaxTokens) return 0;
     size_t n = 0;
     for (int p = 0; p < P; ++p) {
         if (!tables[p]) return 0;
@@ -656,7 +654,7 @@ lml_status lora_mixed_linear_multi(lml_table* const* tables, int P, const void* 
                                    const int32_t* const* token_slots, void* const* y, void* workspace,
                                    size_t workspace_bytes, void* stream_v)
 {
-    if (!tables || !W0 || !token_slots || !y || P < 1 || P > kDsMaxProj || T < 0 || T > kMaxTokens) return LML_ERR_INVALID_ARG;
+    if (!tables || !W0 || !token_slots || !y || P < 1 || P > LML_MAX_PROJECTIONS || T < 0 || T > kMaxTokens) return LML_ERR_INVALID_ARG;
     for (int p = 0; p < P; ++p) {
         if (!tables[p] || tables[p]->d_in != tables[0]->d_in || tables[p]->device != tables[0]->device) return LML_ERR_INVALID_ARG;
         for (int q = 0; q < p; ++q) if (y[q] == y[p] && T > 0) return LML_ERR_INVALID_ARG;
@@ -668,48 +666,34 @@ lml_status lora_mixed_linear_multi(lml_table* const* tables, int P, const void* 
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < lml_multi_workspace_bytes(tables, P, T))
         return LML_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)stream_v;
-    if (T <= kDecodeMaxT) {
-        SlotSnapshot snaps[kDsMaxProj];
-        int d_out[kDsMaxProj];
-        bool early = true;
+    bool distinct = true;   // (a table's counters serve one projection of a launch)
+    for (int p = 0; p < P; ++p)
+        for (int q = 0; q < p; ++q) distinct = distinct && tables[p] != tables[q];
+    if (T <= kDecodeMaxT && P > 1 && distinct) {
+        // One launch of the decode kernel for all projections: its CTAs are dealt out over them, each works on its
+        // projection as in a call of its own, and the fixed costs of a call are paid once.
+        DeviceGuard guard(tables[0]->device);
+        if (!guard.ok) return LML_ERR_CUDA;
+        SlotSnapshot snaps[LML_MAX_PROJECTIONS];
+        DecodeArgs args[LML_MAX_PROJECTIONS];
+        const Arena* ars[LML_MAX_PROJECTIONS];
+        const WsLayout ws = ws_layout(tables[0], T, 1);
         for (int p = 0; p < P; ++p) {
             snaps[p] = snapshot_locked(tables[p]);
-            d_out[p] = tables[p]->d_out;
-            early = early && !tables[p]->arena_dirty;
+            ars[p] = &tables[p]->arena;
+            DecodeArgs& a = args[p];
+            a.x = x; a.W0 = W0[p]; a.y = y[p]; a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
+            a.token_slots = token_slots[p];
+            a.by_adapter = false;
+            a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.u_off) + (size_t)p * 16 * kRankPad;
+            a.T = T; a.d_in = tables[0]->d_in; a.d_out = tables[p]->d_out; a.G = 1; a.num_sms = tables[0]->num_sms;
         }
-        // One launch for all projections pays when what it saves (the fixed cost of the other P - 1 launches, about
-        // 5 us each) outweighs what its kernel loses against the single-projection one on the stream itself
-        // (measured on B200: a little under a fifth of the time the weights take at the HBM rate).
-        long long n_total = 0;
-        for (int p = 0; p < P; ++p) n_total += d_out[p];
-        const double stream_us = (double)n_total * tables[0]->d_in * 2.0 / 6.3e6;
-        if (P > 1 && (P - 1) * 5.0 > 0.18 * stream_us &&
-            decode_stream_eligible(snaps, d_out, P, tables[0]->d_in, true, tables[0]->num_sms)) {
-            DeviceGuard guard(tables[0]->device);
-            if (!guard.ok) return LML_ERR_CUDA;
-            const WsLayout ws = ws_layout(tables[0], T, 1);
-            DsParams prm = {};
-            for (int p = 0; p < P; ++p) {
-                DsProj& pj = prm.proj[p];
-                const Arena& ar = tables[p]->arena;
-                pj.W0 = (const __nv_bfloat16*)W0[p]; pj.y = (__nv_bfloat16*)y[p];
-                pj.arenaA = ar.A; pj.arenaB = ar.B; pj.arenaBc = ar.Bc;
-                pj.token_slots = token_slots[p]; pj.adapter_map = nullptr;
-                pj.status = ar.status; pj.N = tables[p]->d_out;
-            }
-            prm.x = (const __nv_bfloat16*)x;
-            prm.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.u_off);
-            prm.sync_words = tables[0]->arena.status + 1;
-            prm.P = P; prm.T = T; prm.K = tables[0]->d_in; prm.G = 1;
-            prm.patience = decode_patience();
-            prm.early_adapters = early ? 1 : 0;
-            const cudaError_t e = launch_decode_stream(snaps, prm, tables[0]->num_sms, stream);
-            if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
-            for (int p = 0; p < P; ++p) { tables[p]->arena_dirty = false; tables[p]->last_launches = p == 0 ? 1 : 0; }
-            return LML_OK;
-        }
+        const cudaError_t e = launch_decode_multi(ars, snaps, args, P, stream);
+        if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+        for (int p = 0; p < P; ++p) tables[p]->last_launches = p == 0 ? 1 : 0;
+        return LML_OK;
     }
-    // one projection after the other: larger batches (the GEMM path), or tables too large for the one-launch decode form
+    // one projection after the other: larger batches (the GEMM path), a single projection, or a table named twice
     for (int p = 0; p < P; ++p) {
         const lml_status st = tokens_impl(tables[p], x, W0[p], T, token_slots[p], y[p], workspace, workspace_bytes, stream_v, false);
         if (st != LML_OK) return st;

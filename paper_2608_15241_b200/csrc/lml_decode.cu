@@ -40,12 +40,12 @@
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
 #include "lml_decode_common.cuh"
-#include "lml_decode_stream.cuh"
 
 namespace lml {
 
 using namespace ptx;
 
+constexpr int kDecMaxProj = LML_MAX_PROJECTIONS;  // projections that one launch can serve
 constexpr int kDecConsumers = 8;                 // consumer warps
 constexpr int kDecShrinkWarps = 3;               // warps after the producer warp: the LoRA shrink
 constexpr int kDecThreads = (kDecConsumers + 1 + kDecShrinkWarps) * 32;
@@ -97,15 +97,57 @@ static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control b
 // kTwo false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers.
 // kMulti: the CTAs have more than one round of rows; compiled with the code that saves reloads of x between rounds.
 // kPutOff: compiled with the code that puts the expand of early rounds off (kMulti calls with adapters).
-template <bool kTwo, bool kMulti, bool kPutOff>
-__global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
-    const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
-    const __nv_bfloat16* __restrict__ arenaB, const __nv_bfloat16* __restrict__ arenaBc, const __nv_bfloat16* __restrict__ x,
-    const __nv_bfloat16* __restrict__ W0, __nv_bfloat16* __restrict__ y, float* u,
-    const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ slot_ids,
-    const int32_t* __restrict__ perm, const int32_t* __restrict__ token_slots, const int32_t* __restrict__ adapter_map, uint32_t* status, int T, int K, int N,
-    int G, int patience)
+// One projection of a launch: its table, base weight, binding and output, and the CTAs that work on it.
+struct DecProj {
+    const __nv_bfloat16* arenaA;
+    const __nv_bfloat16* arenaB;
+    const __nv_bfloat16* arenaBc;
+    const __nv_bfloat16* W0;
+    __nv_bfloat16* y;
+    float* u;
+    const int32_t* seg_offsets;
+    const int32_t* slot_ids;
+    const int32_t* perm;
+    const int32_t* token_slots;
+    const int32_t* adapter_map;
+    uint32_t* status;
+    int N, G;
+    int cta_begin, cta_count;   // CTAs [cta_begin, cta_begin + cta_count) of the grid
+};
+// kP projections that read the same x (kP = 1: the plain call).  With several, the grid is dealt out over the
+// projections in proportion to their rows; a CTA works on one projection as if that were the whole call (its own
+// rows, its own share of that table's dot products, that table's counters), so one launch pays the fixed costs of a
+// call (the wait for the preceding work, the fetch of x, the tail) once for all of them.
+template <int kP> struct DecLaunch {
+    SlotSnapshot snap[kP];
+    DecProj proj[kP];
+    const __nv_bfloat16* x;
+    int T, K, P, patience;
+};
+
+template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1>
+__global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __grid_constant__ DecLaunch<kP> prm)
 {
+    int pi = 0;
+    if (kP > 1)
+        while (pi + 1 < prm.P && (int)blockIdx.x >= prm.proj[pi + 1].cta_begin) ++pi;
+    const SlotSnapshot& snap = prm.snap[pi];
+    const DecProj& pj = prm.proj[pi];
+    const int cta = (int)blockIdx.x - pj.cta_begin, ncta = pj.cta_count;   // this CTA among those of its projection
+    const __nv_bfloat16* __restrict__ arenaA = pj.arenaA;
+    const __nv_bfloat16* __restrict__ arenaB = pj.arenaB;
+    const __nv_bfloat16* __restrict__ arenaBc = pj.arenaBc;
+    const __nv_bfloat16* __restrict__ x = prm.x;
+    const __nv_bfloat16* __restrict__ W0 = pj.W0;
+    __nv_bfloat16* __restrict__ y = pj.y;
+    float* u = pj.u;
+    const int32_t* __restrict__ seg_offsets = pj.seg_offsets;
+    const int32_t* __restrict__ slot_ids = pj.slot_ids;
+    const int32_t* __restrict__ perm = pj.perm;
+    const int32_t* __restrict__ token_slots = pj.token_slots;
+    const int32_t* __restrict__ adapter_map = pj.adapter_map;
+    uint32_t* status = pj.status;
+    const int T = prm.T, K = prm.K, N = pj.N, G = pj.G, patience = prm.patience;
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
     const uint32_t ring = (raw + 127u) & ~127u;
@@ -119,8 +161,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
-    const int row_begin = (int)((long long)blockIdx.x * N / gridDim.x);
-    const int row_end = (int)((long long)(blockIdx.x + 1) * N / gridDim.x);
+    const int row_begin = (int)((long long)cta * N / ncta);
+    const int row_end = (int)((long long)(cta + 1) * N / ncta);
     // x fragments of a span live in registers; with two 8-token blocks a span is half as wide, so
     // both variants hold 64 fragment registers and stay clear of spills
     constexpr int kSpan = kTwo ? kDecSpan / 2 : kDecSpan;
@@ -261,7 +303,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
             const int live_rows = total0 + __shfl_sync(0xffffffffu, incl1, 31);
             if ((long long)live_rows * K * 16 <= (long long)N * K) {
                 // lane L of this CTA takes live row blockIdx + L * grid
-                const int i = (int)blockIdx.x + lane * (int)gridDim.x;
+                const int i = cta + lane * ncta;
                 // find the slot holding live row i: the first whose inclusive count exceeds i
                 const unsigned m0 = __ballot_sync(0xffffffffu, incl0 > 0);   // (dummy use keeps the shuffles converged)
                 (void)m0;
@@ -365,7 +407,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
                 ctrl->bad_offsets = bad;
                 const unsigned f = (bad ? LML_FLAG_BAD_OFFSETS : 0u) | (bad_slot ? LML_FLAG_BAD_SLOT : 0u) |
                                    (bad_perm ? LML_FLAG_BAD_PERM : 0u);
-                if (f && blockIdx.x == 0) atomicOr(status, f);
+                if (f && cta == 0) atomicOr(status, f);
             }
             __syncwarp();
             // Per row of x: rank, scale, and where its dot products end in the grid-wide numbering (rows
@@ -418,7 +460,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         const int total = lk->dot_end[15];
         // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
         // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
-        const int gsize = total <= (int)gridDim.x ? 1 : (total <= 2 * (int)gridDim.x ? 2 : kDecDotGroup);
+        const int gsize = total <= ncta ? 1 : (total <= 2 * ncta ? 2 : kDecDotGroup);
         const int ngroups = total / gsize;
         const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
         // Brings the blocks of B into the staging buffer (16-byte asynchronous copies, all in flight at
@@ -539,16 +581,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         };
         const long long t_shrink = clock64();
         if (gsize == 1) {
-            if ((int)blockIdx.x < total) {
+            if (cta < total) {
                 int t, j;
-                const float val = single((int)blockIdx.x, t, j);
+                const float val = single(cta, t, j);
                 if (me == 0) {
                     u[t * kRankPad + j] = val;
                     red_release_gpu_add(sync_words, 1u);
                 }
             }
         } else
-        for (int g = (int)blockIdx.x; g < ngroups; g += (int)gridDim.x) {
+        for (int g = cta; g < ngroups; g += ncta) {
             float val[kDecDotGroup];
             int t, j0;
             group(g, val, t, j0);
@@ -601,7 +643,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(
         // both counters back to zero for the next call on this table.
         if (sw == 0 && lane == 0) {
             __threadfence();
-            if (atomicAdd(sync_words + 1, 1u) == gridDim.x - 1) {
+            if (atomicAdd(sync_words + 1, 1u) == (unsigned)ncta - 1u) {
                 sync_words[0] = 0u;
                 sync_words[1] = 0u;
             }
@@ -806,65 +848,128 @@ cudaError_t decode_init()
     auto set = [&](auto kernel) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes);
     };
-    set(decode_main_kernel<false, false, false>); set(decode_main_kernel<false, true, false>); set(decode_main_kernel<false, true, true>);
-    set(decode_main_kernel<true, false, false>);  set(decode_main_kernel<true, true, false>);  set(decode_main_kernel<true, true, true>);
-    if (e == cudaSuccess) e = decode_stream_init();
+    set(decode_main_kernel<false, false, false, 1>); set(decode_main_kernel<false, true, false, 1>); set(decode_main_kernel<false, true, true, 1>);
+    set(decode_main_kernel<true, false, false, 1>);  set(decode_main_kernel<true, true, false, 1>);  set(decode_main_kernel<true, true, true, 1>);
+    set(decode_main_kernel<false, false, false, kDecMaxProj>); set(decode_main_kernel<false, true, false, kDecMaxProj>); set(decode_main_kernel<false, true, true, kDecMaxProj>);
+    set(decode_main_kernel<true, false, false, kDecMaxProj>);  set(decode_main_kernel<true, true, false, kDecMaxProj>);  set(decode_main_kernel<true, true, true, kDecMaxProj>);
     return e;
 }
 
 int decode_patience() { return g_dec_patience; }
+
+namespace {
+
+void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
+{
+    pj.arenaA = ar.A; pj.arenaB = ar.B; pj.arenaBc = ar.Bc;
+    pj.W0 = (const __nv_bfloat16*)a.W0;
+    pj.y = (__nv_bfloat16*)a.y;
+    pj.u = a.u;
+    pj.seg_offsets = a.seg_offsets; pj.slot_ids = a.slot_ids; pj.perm = a.perm; pj.token_slots = a.token_slots;
+    pj.adapter_map = a.by_adapter ? ar.adapter_map : nullptr;
+    pj.status = ar.status;
+    pj.N = a.d_out; pj.G = a.G;
+}
+
+// An ordinary launch, as a programmatic dependent of whatever precedes it on the stream (the kernel waits for that
+// work itself, after it has started on W0).  The CTAs hand one another their share of u, but none of them depends on
+// the others being resident (see the kernel), so no cooperative launch is needed, and the kernel can start while its
+// predecessor drains.  Three builds of the kernel per token count: CTAs with one round of rows (the plain loop), with
+// several rounds (x is kept between rounds), and with several rounds and adapters (the expand of early rounds is put
+// off until u has arrived).
+template <int kP>
+cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_cta, bool adapters, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kDecThreads);
+    cfg.dynamicSmemBytes = kDecSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
+    const bool put_off = multi && adapters;
+    auto launch = [&](auto kernel) { return cudaLaunchKernelEx(&cfg, kernel, prm); };
+    if (prm.T > 8)
+        return put_off ? launch(decode_main_kernel<true, true, true, kP>)
+                       : (multi ? launch(decode_main_kernel<true, true, false, kP>) : launch(decode_main_kernel<true, false, false, kP>));
+    return put_off ? launch(decode_main_kernel<false, true, true, kP>)
+                   : (multi ? launch(decode_main_kernel<false, true, false, kP>) : launch(decode_main_kernel<false, false, false, kP>));
+}
+
+}  // namespace
 
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a, cudaStream_t stream,
                           int* launches)
 {
     *launches = 0;
     const int row_pairs = (a.d_out + 1) / 2;   // at least two rows per CTA
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(row_pairs < a.num_sms ? row_pairs : a.num_sms);
-    cfg.blockDim = dim3(kDecThreads);
-    cfg.dynamicSmemBytes = kDecSmemBytes;
-    cfg.stream = stream;
-    // An ordinary launch, as a programmatic dependent of whatever precedes it on the stream (the kernel
-    // waits for that work itself, after it has started on W0).  The CTAs hand one another their share of
-    // u, but none of them depends on the others being resident (see the kernel), so no cooperative
-    // launch is needed, and the kernel can start while its predecessor drains.
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const __nv_bfloat16* xb = (const __nv_bfloat16*)a.x;
-    const __nv_bfloat16* wb = (const __nv_bfloat16*)a.W0;
-    __nv_bfloat16* yb = (__nv_bfloat16*)a.y;
-    float* up = a.u;
-    const __nv_bfloat16* arenaA = ar.A;
-    const __nv_bfloat16* arenaB = ar.B;
-    const __nv_bfloat16* arenaBc = ar.Bc;
-    uint32_t* status = ar.status;
-    const int32_t* so = a.seg_offsets;
-    const int32_t* ids = a.slot_ids;
-    const int32_t* pm = a.perm;
-    const int32_t* ts = a.token_slots;
-    const int32_t* amap = a.by_adapter ? ar.adapter_map : nullptr;
-    // Three builds of the kernel per token count: CTAs with one round of rows (the plain loop), with
-    // several rounds (x is kept between rounds), and with several rounds and adapters (the expand of
-    // early rounds is put off until u has arrived).
-    const int rows_per_cta = (a.d_out + (int)cfg.gridDim.x - 1) / (int)cfg.gridDim.x;
-    const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
-    const bool put_off = multi && a.G > 0;
-    auto launch = [&](auto kernel) {
-        return cudaLaunchKernelEx(&cfg, kernel, snap, arenaA, arenaB, arenaBc, xb, wb, yb, up, so, ids, pm, ts, amap, status, a.T,
-                                  a.d_in, a.d_out, a.G, g_dec_patience);
-    };
-    cudaError_t e;
-    if (a.T > 8)
-        e = put_off ? launch(decode_main_kernel<true, true, true>)
-                    : (multi ? launch(decode_main_kernel<true, true, false>) : launch(decode_main_kernel<true, false, false>));
-    else
-        e = put_off ? launch(decode_main_kernel<false, true, true>)
-                    : (multi ? launch(decode_main_kernel<false, true, false>) : launch(decode_main_kernel<false, false, false>));
+    const int grid = row_pairs < a.num_sms ? row_pairs : a.num_sms;
+    DecLaunch<1> prm;
+    prm.snap[0] = snap;
+    fill_proj(prm.proj[0], ar, a);
+    prm.proj[0].cta_begin = 0; prm.proj[0].cta_count = grid;
+    prm.x = (const __nv_bfloat16*)a.x;
+    prm.T = a.T; prm.K = a.d_in; prm.P = 1; prm.patience = g_dec_patience;
+    const cudaError_t e = launch_decode_grid<1>(prm, grid, (a.d_out + grid - 1) / grid, a.G > 0, stream);
     if (e == cudaSuccess) ++*launches;
     return e;
+}
+
+// Several projections of one decode step (the same x, T and d_in) in one launch: the SMs are dealt out in proportion to
+// the projections' rows (every projection gets at least one CTA, none more than it has pairs of rows).
+cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* snaps, const DecodeArgs* args, int P, cudaStream_t stream)
+{
+    if (P < 1 || P > kDecMaxProj) return cudaErrorInvalidValue;
+    const int num_sms = args[0].num_sms;
+    long long rows_total = 0;
+    for (int p = 0; p < P; ++p) rows_total += args[p].d_out;
+    int count[kDecMaxProj], given = 0;
+    for (int p = 0; p < P; ++p) {
+        int c = (int)((long long)num_sms * args[p].d_out / rows_total);
+        const int cap = (args[p].d_out + 1) / 2;
+        c = c < 1 ? 1 : (c > cap ? cap : c);
+        count[p] = c;
+        given += c;
+    }
+    // what the rounding left over goes, one CTA at a time, to the projection with the most rows per CTA
+    while (given < num_sms) {
+        int best = -1;
+        double worst = 0.0;
+        for (int p = 0; p < P; ++p) {
+            const double load = (double)args[p].d_out / count[p];
+            if (count[p] < (args[p].d_out + 1) / 2 && load > worst) { worst = load; best = p; }
+        }
+        if (best < 0) break;
+        ++count[best];
+        ++given;
+    }
+    while (given > num_sms) {   // (more projections than SMs cannot happen with P <= 4; kept for safety)
+        int best = 0;
+        for (int p = 1; p < P; ++p) if (count[p] > count[best]) best = p;
+        if (count[best] <= 1) break;
+        --count[best];
+        --given;
+    }
+    DecLaunch<kDecMaxProj> prm;
+    int begin = 0, rows_per_cta = 0;
+    bool adapters = false;
+    for (int p = 0; p < P; ++p) {
+        prm.snap[p] = snaps[p];
+        fill_proj(prm.proj[p], *ars[p], args[p]);
+        prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = count[p];
+        begin += count[p];
+        const int r = (args[p].d_out + count[p] - 1) / count[p];
+        rows_per_cta = r > rows_per_cta ? r : rows_per_cta;
+        adapters = adapters || args[p].G > 0;
+    }
+    for (int p = P; p < kDecMaxProj; ++p) { prm.snap[p] = snaps[0]; prm.proj[p] = prm.proj[0]; prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = 0; }
+    prm.x = (const __nv_bfloat16*)args[0].x;
+    prm.T = args[0].T; prm.K = args[0].d_in; prm.P = P; prm.patience = g_dec_patience;
+    return launch_decode_grid<kDecMaxProj>(prm, begin, rows_per_cta, adapters, stream);
 }
 
 }  // namespace lml

@@ -153,6 +153,9 @@ cudaError_t decode_init();   // sets the dynamic shared memory attributes
 int decode_patience();       // LML_DECODE_PATIENCE or the default, in clock cycles
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
                           cudaStream_t stream, int* launches);
+// P <= LML_MAX_PROJECTIONS projections that read the same x (args[p].x, T, d_in, num_sms equal for all p) in one launch.
+cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* snaps, const DecodeArgs* args, int P,
+                                cudaStream_t stream);
 
 // Every kernel of the library is launched as a programmatic dependent of whatever precedes it on
 // the stream and executes griddepcontrol.wait before it touches global memory (unless its

@@ -4,7 +4,6 @@
 #include <mutex>
 
 #include "lml_internal.cuh"
-#include "lml_decode_stream.cuh"
 
 struct lml_table {
     int device = 0, d_in = 0, d_out = 0, max_slots = 0, num_sms = 0;
@@ -27,9 +26,6 @@ struct lml_table {
     // that point, and every later registration makes its own stream wait for it before it overwrites a slot.
     cudaEvent_t ev_map = nullptr;
     bool map_clear_recorded = false;
-    // A registration has been enqueued since the table's last streaming decode call: that kernel fetches rows of
-    // the adapter arena before it waits for the work in front of it, which the copy into the arena may be.
-    bool arena_dirty = true;
     int last_launches = 0;
     // host-buffer form of large calls: the copies of x in and of y out run on two streams of the table's own,
     // chunk by chunk beside the layer (created with the table: the call itself creates nothing)

@@ -1,7 +1,8 @@
 """lora_mixed_linear_multi: several projections of the same x (q/k/v, gate/up) in one call, every projection
 with its own table (ranks up to 64, its own scales, its own slot numbering).  Each output is compared with
-the oracle run on that projection alone; for up to 16 tokens (one launch for all projections) also with the
-separate lora_mixed_linear_tokens calls, which may differ in the last place only (fp32 summation order)."""
+the oracle run on that projection alone and, bit for bit, with the separate lora_mixed_linear_tokens calls: up to
+16 tokens are one launch of the decode kernel for all projections, whose CTAs each work on one projection exactly as
+in a call of its own (a row's arithmetic does not depend on how the rows are dealt out)."""
 import numpy as np
 import pytest
 
@@ -78,8 +79,7 @@ def _check(out, sep, flags, x, W, ents, tok_adapter, last_place=True):
         r = oracle.compare(out[p], ref)
         assert r["ok"], (p, r)
         if last_place:
-            a, s = wl.bf16_bits_to_f64(out[p]), wl.bf16_bits_to_f64(sep[p])
-            assert (np.abs(a - s) <= 2.0 ** -7 * np.maximum(1.0, np.abs(s))).all(), p
+            assert np.array_equal(out[p], sep[p]), p
 
 
 @pytest.mark.parametrize("T", [1, 8, 16, 128, 2048])
@@ -94,8 +94,8 @@ def test_three_projections_with_their_own_ranks_and_scales(T):
 
 @pytest.mark.parametrize("T", [3, 16])
 def test_wide_projections_take_one_launch(T):
-    """q/k/v-like widths where the tables' live rows are few: one launch of the streaming decode kernel, rows of
-    the three weights shared out over the grid (CTA ranges cross projection boundaries)."""
+    """q/k/v-like widths of unequal size: one launch, the CTAs dealt out over the projections in proportion to their
+    rows."""
     import torch
     from paper_2608_15241_b200 import binding as b
     K, Ns = 1032, (4104, 2056, 3080)
@@ -143,14 +143,13 @@ def test_multi_launch_count_and_bad_ids():
         t.close()
 
 
-def test_tables_too_large_for_one_launch_fall_back_to_one_call_per_projection():
+def test_tables_with_many_wide_adapters():
     K, Ns, T = 264, (520, 264), 8
-    ranks = [(64,) * 12, (64,) * 12]          # 768 live rows per table: far more than an eighth of the weight rows
+    ranks = [(64,) * 12, (64,) * 12]          # 768 rows of A per table: more than the weights have rows
     scales = [(1.0,) * 12, (2.0,) * 12]
     x, W, ents, tok = _case(11, K, Ns, ranks, scales, T)
     out, sep, flags = _run_multi(K, Ns, x, W, ents, tok)
     _check(out, sep, flags, x, W, ents, tok)
-    assert all(np.array_equal(o, s) for o, s in zip(out, sep))     # the very same kernels
 
 
 def test_seven_b_class_qkv_decode():
