@@ -432,10 +432,11 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                 "traffic": None, "us_per_launch": per_launch * 1e6}
 
     dual = None
-    if kind != "decode" and w.G >= 1 and "dual" in extras:
-        # the same tokens under two bindings: one call with a shared base product against two ordinary calls
+    if w.G >= 1 and "dual" in extras:
+        # the same tokens under two bindings: one call with a shared base product (decode: one launch, W0 out of HBM
+        # once) against two ordinary calls
         rot.prepare_dual()
-        dsteps = max(rot.R, min(steps, 100))
+        dsteps = max(rot.R, min(steps, 100)) if kind != "decode" else max(rot.R, min(10 * steps, 1200))
         d_secs, _, _ = timed_graph_loop(rot.dual_only, rot.R, dsteps, 3, stream)
         t_secs, _, _ = timed_graph_loop(rot.two_singles, rot.R, dsteps, 3, stream)
         dual = {"us_per_call": d_secs / dsteps * 1e6, "two_single_calls_us": t_secs / dsteps * 1e6}

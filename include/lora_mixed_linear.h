@@ -227,8 +227,9 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
  * accumulator, then (delta_b - delta_a) is added to it with a few more tensor-core steps and y_b is
  * read out, so y_a agrees with lora_mixed_linear with slot_ids_a to the bf16 rounding of u (bit for
  * bit when that call takes u from the same shrink kernel) and y_b with lora_mixed_linear with
- * slot_ids_b to fp32 rounding of the accumulator as well.  For T <= 16 the call is two
- * decode calls.  G >= 1.  workspace: at least lml_dual_workspace_bytes(t, T, G).  Other arguments,
+ * slot_ids_b to fp32 rounding of the accumulator as well.  For T <= 16 the call is one launch of
+ * the decode kernel with half of its CTAs per binding (the two halves walk W0 together, so it
+ * leaves HBM once); y_a and y_b are bit for bit those of two lora_mixed_linear calls.  G >= 1.  workspace: at least lml_dual_workspace_bytes(t, T, G).  Other arguments,
  * flags and errors as lora_mixed_linear.
  */
 size_t lml_dual_workspace_bytes(const lml_table* t, int max_tokens, int max_segments);

@@ -475,13 +475,28 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
         !aligned16(W0) || !aligned16(y_a) || !aligned16(y_b))
         return LML_ERR_INVALID_ARG;
     if (T <= kDecodeMaxT) {
-        // The decode kernel has no two-output form: two calls, W0 streamed twice.
-        lml_status st = lora_mixed_linear(t, x, W0, T, seg_offsets, slot_ids_a, G, perm, y_a, workspace, workspace_bytes, stream_v);
-        if (st != LML_OK) return st;
-        const int first = t->last_launches;
-        st = lora_mixed_linear(t, x, W0, T, seg_offsets, slot_ids_b, G, perm, y_b, workspace, workspace_bytes, stream_v);
-        if (st == LML_OK) t->last_launches += first;
-        return st;
+        // One launch of the decode kernel with the two bindings as two projections over the same W0: half of the CTAs
+        // per binding, each half exactly a single call (so y_a and y_b are bit for bit those of two calls).  The two
+        // halves walk the same rows of W0 at the same time, so the second reader of a line finds it in L2.
+        const WsLayout ws1 = ws_layout(t, T, G);
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < ws1.xg_off) return LML_ERR_WORKSPACE;
+        const SlotSnapshot snap = snapshot_locked(t);
+        DeviceGuard guard(t->device);
+        if (!guard.ok) return LML_ERR_CUDA;
+        SlotSnapshot snaps[2] = {snap, snap};
+        const Arena* ars[2] = {&t->arena, &t->arena};
+        DecodeArgs args[2];
+        for (int p = 0; p < 2; ++p) {
+            DecodeArgs& a = args[p];
+            a.x = x; a.W0 = W0; a.y = p == 0 ? y_a : y_b; a.perm = perm; a.seg_offsets = seg_offsets;
+            a.slot_ids = p == 0 ? slot_ids_a : slot_ids_b;
+            a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws1.u_off) + (size_t)p * 16 * kRankPad;
+            a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
+        }
+        const cudaError_t e = launch_decode_multi(ars, snaps, args, 2, (cudaStream_t)stream_v);
+        t->last_launches = e == cudaSuccess ? 1 : 0;
+        if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+        return LML_OK;
     }
     const WsLayout ws = ws_layout(t, T, G, 3);
     const size_t need = perm ? ws.total : ws.xg_off;
@@ -847,6 +862,7 @@ lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
     bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     // also puts the decode kernel's two grid counters (words 1 and 2) back to zero, in case a call gave up
     ok = ok && cudaMemsetAsync(t->arena.status, 0, 3 * sizeof v, stream) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(t->arena.status + 8, 0, 2 * sizeof v, stream) == cudaSuccess;   // (the counters of a dual decode call's second binding)
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
     *flags_out = v;

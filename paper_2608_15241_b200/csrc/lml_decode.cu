@@ -111,6 +111,7 @@ struct DecProj {
     const int32_t* token_slots;
     const int32_t* adapter_map;
     uint32_t* status;
+    unsigned int* sync_words;   // [0] elements of u that are written, [1] CTAs that have left: two words of the table's status block
     int N, G;
     int cta_begin, cta_count;   // CTAs [cta_begin, cta_begin + cta_count) of the grid
 };
@@ -274,7 +275,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     // dot product, sixteen 16-byte loads in flight per lane.  The results go to u in global memory; a
     // counter in the table's status block tells every CTA when all of u is there.  The consumers look at
     // it only in their first epilogue.
-    unsigned int* sync_words = status + 1;   // [0] elements of u that are written, [1] CTAs that have left
+    unsigned int* sync_words = pj.sync_words;
     const bool shrinker = warp > kDecConsumers;
     if (consumer && G > 0)   // let the lookup's loads go first through the load/store path (see below)
         asm volatile("bar.sync 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
@@ -868,6 +869,7 @@ void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
     pj.seg_offsets = a.seg_offsets; pj.slot_ids = a.slot_ids; pj.perm = a.perm; pj.token_slots = a.token_slots;
     pj.adapter_map = a.by_adapter ? ar.adapter_map : nullptr;
     pj.status = ar.status;
+    pj.sync_words = ar.status + 1;
     pj.N = a.d_out; pj.G = a.G;
 }
 
@@ -960,6 +962,8 @@ cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* sna
     for (int p = 0; p < P; ++p) {
         prm.snap[p] = snaps[p];
         fill_proj(prm.proj[p], *ars[p], args[p]);
+        for (int q = 0; q < p; ++q)   // a table that serves two projections of the launch (the two bindings of a dual call): its second pair of counters
+            if (ars[q] == ars[p]) prm.proj[p].sync_words = ars[p]->status + 8;
         prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = count[p];
         begin += count[p];
         const int r = (args[p].d_out + count[p] - 1) / count[p];

@@ -65,6 +65,29 @@ def test_dual_matches_two_single_calls(kw, monkeypatch):
     site.close()
 
 
+@pytest.mark.parametrize("kw", [dict(T=1, d_in=1032, d_out=2056), dict(T=8, d_in=4096, d_out=4096),
+                                dict(T=16, d_in=2056, d_out=1000, shuffled=True), dict(T=11, d_in=264, d_out=40)])
+def test_dual_decode_is_one_launch_and_bit_identical_to_two_calls(kw):
+    """Up to 16 tokens: one launch of the decode kernel, half of its CTAs per binding, each half a single call."""
+    w = wl.ragged(ranks=(4, 16, 1, 33, 64), **kw)
+    E = len(w.entries)
+    rng = np.random.default_rng(7 + w.T)
+    se_a = w.seg_entry.copy()
+    se_b = np.array([[int(rng.integers(0, E)), int(se_a[g]), -1][int(rng.integers(0, 3))] for g in range(w.G)], se_a.dtype)
+    site = Site(w)
+    y_a, y_b, flags = _dual(site, w, se_a, se_b)
+    assert flags == 0 and site.table.last_launch_count() == 1
+    y_a1, f1 = site.run(seg_entry=se_a)
+    y_b1, f2 = site.run(seg_entry=se_b)
+    assert f1 == 0 and f2 == 0
+    assert np.array_equal(y_a, y_a1) and np.array_equal(y_b, y_b1)
+    for y, se in ((y_a, se_a), (y_b, se_b)):
+        ref, _ = oracle.forward(w.x, w.W0, w.entries, w.seg_offsets, se, w.perm)
+        r = oracle.compare(y, ref)
+        assert r["ok"], r
+    site.close()
+
+
 @pytest.mark.parametrize("kw", [dict(T=128, d_in=2048, d_out=1544), dict(T=77, d_in=1024, d_out=2056, shuffled=True),
                                 dict(T=300, d_in=2048, d_out=1032), dict(T=64, d_in=4096, d_out=4096)])
 def test_dual_with_few_tokens_takes_the_split_k_kernel(kw, monkeypatch):
