@@ -31,6 +31,10 @@
 //                       for their shares it computes all of u itself (same arithmetic, same bits).  So
 //                       the launch is an ordinary one and needs no co-residency guarantee.
 // d_in wider than a span is walked span by span.  All waits are bounded.
+// Several projections that read the same x (q / k / v, gate / up, or the two bindings of a dual-version call over
+// one W0) run as one launch: the grid is dealt out over the projections in proportion to their rows, and a CTA
+// works on its projection as if that were the whole call, so the results are those of separate calls bit for bit
+// and the fixed costs of a call (the wait for the preceding work, the fetch of x, the tail) are paid once.
 // CTAs with more than one round of 32 rows (wide layers) come in two further builds of the kernel: the
 // spans are walked forwards and backwards in turn, so that the x fragments a round ends with serve the
 // next one without a reload; and, with adapters, the expand of early rounds is put off until u has
