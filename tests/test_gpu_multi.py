@@ -106,6 +106,17 @@ def test_wide_projections_take_one_launch(T):
     _check(out, sep, flags, x, W, ents, tok)
 
 
+@pytest.mark.parametrize("T", [2, 16])
+def test_four_projections_some_with_very_few_rows(T):
+    """LML_MAX_PROJECTIONS projections, two of them with fewer pairs of rows than their share of the SMs."""
+    K, Ns = 264, (3080, 16, 1032, 40)
+    ranks = [(16, 8, 64), (4, 16, 1), (64, 2, 16), (8, 8, 8)]
+    scales = [(2.0, 0.5, 1.0), (1.0, 2.0, 0.25), (0.5, 1.5, 2.0), (1.0, 1.0, 3.0)]
+    x, W, ents, tok = _case(90 + T, K, Ns, ranks, scales, T)
+    out, sep, flags = _run_multi(K, Ns, x, W, ents, tok)
+    _check(out, sep, flags, x, W, ents, tok)
+
+
 def test_multi_launch_count_and_bad_ids():
     import torch
     from paper_2608_15241_b200 import binding as b
