@@ -65,6 +65,7 @@ cudaError_t launch_pack_adapter(const Arena& ar, int slot, const void* A, const 
 // chunk.  Everything is order-deterministic.
 // ---------------------------------------------------------------------------------------------
 constexpr int kSegWarps = 32;
+constexpr int kSegKeyCache = 16384;   // tokens whose keys are kept in shared memory between the two passes
 
 __global__ void set_word_kernel(int32_t* dst, int32_t value) { *dst = value; }
 __global__ void clear_word_if_kernel(int32_t* dst, int32_t expected) { if (*dst == expected) *dst = -1; }
@@ -153,11 +154,24 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
 {
     __shared__ int hist[kSegWarps][kMaxSlots + 1];
     __shared__ int base[kMaxSlots + 2];
+    __shared__ uint8_t keys_s[kSegKeyCache];
     const int nk = snap.max_slots + 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < kSegWarps * (kMaxSlots + 1); i += blockDim.x) (&hist[0][0])[i] = 0;
     ptx::grid_dependency_wait();      // launched as a programmatic dependent: whatever ran before is complete now
     ptx::grid_launch_dependents();    // the next kernel may get resident; it waits for this one the same way
+    // Up to kSegKeyCache tokens: every key is fetched once, all loads in flight together (one trip to memory instead of
+    // one per 32 tokens of a warp's range and pass), and both passes read shared memory.  0xff marks an id that names
+    // no live slot (it counts as "none" and raises the flag).
+    const bool cached = T <= kSegKeyCache;
+    if (cached) {
+        for (int i = threadIdx.x; i < T; i += blockDim.x) {
+            int s = __ldg(token_slots + i);
+            if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
+            const bool bad_id = s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0);
+            keys_s[i] = bad_id ? (uint8_t)0xff : (uint8_t)(s < 0 ? snap.max_slots : s);
+        }
+    }
     __syncthreads();
 
     int per = (T + kSegWarps - 1) / kSegWarps;
@@ -169,10 +183,16 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
     for (int c = begin; c < end; c += 32) {
         int i = c + lane;
         if (i < end) {
-            int s = __ldg(token_slots + i);
-            if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
-            if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) { bad = true; s = -1; }
-            int key = s < 0 ? snap.max_slots : s;
+            int key;
+            if (cached) {
+                key = keys_s[i];
+                if (key == 0xff) { bad = true; key = snap.max_slots; }
+            } else {
+                int s = __ldg(token_slots + i);
+                if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
+                if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) { bad = true; s = -1; }
+                key = s < 0 ? snap.max_slots : s;
+            }
             atomicAdd(&hist[warp][key], 1);
         }
     }
@@ -201,10 +221,14 @@ __global__ void __launch_bounds__(kSegWarps * 32) segment_tokens_kernel(
         int i = c + lane;
         int key = nk;                          // sentinel for lanes past the end
         if (i < end) {
-            int s = __ldg(token_slots + i);
-            if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
-            if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) s = -1;
-            key = s < 0 ? snap.max_slots : s;
+            if (cached) {
+                key = keys_s[i] == 0xff ? snap.max_slots : (int)keys_s[i];
+            } else {
+                int s = __ldg(token_slots + i);
+                if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
+                if (s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0)) s = -1;
+                key = s < 0 ? snap.max_slots : s;
+            }
         }
         unsigned m = __match_any_sync(0xffffffffu, key);
         int before = __popc(m & ((1u << lane) - 1u));
