@@ -288,7 +288,7 @@ def test_segmentation_matches_reference_grouping():
         for a in range(18):
             tbl.register_adapter(a, 1, A, B, 1.0)
         rng = np.random.default_rng(1)
-        for T in (0, 1, 31, 32, 33, 1000, 8192, 50000):
+        for T in (0, 1, 31, 32, 33, 1000, 8192, 16384, 16385, 50000):   # (up to 16384 tokens the kernel keeps the keys in shared memory)
             tok = rng.integers(-1, 18, size=T).astype(np.int32)
             perm, so, ids = tbl.segment_tokens(torch.from_numpy(tok).cuda())
             torch.cuda.synchronize()
