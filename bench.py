@@ -581,7 +581,7 @@ def cpu_baseline(w, kind, unit, budget_s):
                       f"{secs * repeats:.1f} s wall on {cores} threads, scaled by rows"}
 
 
-def run_layer_sweep(device, peaks, steps, only=None, parity=False):
+def run_layer_sweep(device, peaks, steps, only=None, parity=False, tokens=None):
     """The decoder-layer sweep (three distinct projection shapes x five token counts), one cell after
     the other: microseconds per call of lora_mixed_linear_tokens and the fraction of the bound that
     holds for the cell (the slower of bytes / HBM peak and flops / tensor peak)."""
@@ -589,7 +589,7 @@ def run_layer_sweep(device, peaks, steps, only=None, parity=False):
     stream = torch.cuda.Stream(device=device)
     cells = []
     for proj, same_as in (("q", "q k v o"), ("gate", "gate up"), ("down", "down")):
-        for T in wl.SWEEP_TOKENS:
+        for T in (tokens or wl.SWEEP_TOKENS):
             if only and (proj, T) not in only:
                 continue
             w = wl.layer_sweep(proj, T)
@@ -813,6 +813,8 @@ def main():
                                            "cell's bound = max(bytes / measured HBM peak, flops / measured burst tensor peak) / time; "
                                            "16 adapters of rank 16, two of them in two versions (18 resident entries), Zipf(1.1) binding",
                                    "cells": run_layer_sweep(device, peaks, 200, parity=True)}
+            line["few_blocks_of_16_tokens"] = {"what": "the same sweep at 32 tokens: two blocks of 16 on the decode kernel in one launch",
+                                               "cells": run_layer_sweep(device, peaks, 200, parity=True, tokens=(32,))}
         barrier()
     if rank == 0:
         print(json.dumps(line), flush=True)

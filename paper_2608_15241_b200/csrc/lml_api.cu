@@ -25,7 +25,7 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
     w.u_off = round_up(w.ident_off + (num_m + 1) * sizeof(int32_t), 1024);
     size_t u_bytes = (size_t)u_sets * (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
     // the decode kernel's scratch: u[16][64] fp32 per projection of a launch
-    const size_t dec_bytes = (size_t)LML_MAX_PROJECTIONS * 16 * kRankPad * sizeof(float);
+    const size_t dec_bytes = (size_t)kDecMaxBlocks * 16 * kRankPad * sizeof(float);
     if (u_bytes < dec_bytes) u_bytes = dec_bytes;
     w.xg_off = w.u_off + round_up(u_bytes, 1024);
     w.total = w.xg_off + round_up((size_t)T * t->d_in * sizeof(__nv_bfloat16), 1024);
@@ -116,6 +116,7 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
                               (uint64_t)d_in * kRankPad * 2, 64, 64, 1);
     gemm_split_override(&t->split_bn, &t->split_s);   // the test knobs are read here, never on the hot path
     if (const char* e = getenv("LML_FUSE_SHRINK")) t->fuse_shrink = e[0] != '0';
+    if (const char* e = getenv("LML_DECODE_BLOCK_TOKENS")) t->dec_block_tokens = atoi(e) < 0 ? 0 : (atoi(e) > kDecMaxBlocks * kDecodeMaxT ? kDecMaxBlocks * kDecodeMaxT : atoi(e));
     ok = ok && cudaEventCreateWithFlags(&t->ev_map, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_in, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -626,6 +627,43 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
         if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
         return LML_OK;
     }
+    // (measured on B200 against the GEMM path: two blocks win on every layer of a 7B-class model, 15 us against 29 us
+    // on 4096 x 4096 and 33 against 39 - 45 us on the MLP's; three win on the 4096 x 4096 layers only, 24 against 29 us;
+    // four or more lose: every block's CTAs take all of W0 in from L2)
+    const int block_limit = t->dec_block_tokens >= 0 ? t->dec_block_tokens
+                                                     : ((long long)t->d_in * t->d_out <= (1ll << 24) ? 3 : 2) * kDecodeMaxT;
+    if (T <= block_limit) {
+        // A few blocks of 16 tokens: one launch of the decode kernel with the blocks as its parts, an equal share of the
+        // CTAs each.  The shares walk W0 together, so a line leaves HBM once and the other readers find it in L2; no
+        // grouping, no row copy, no shrink kernel.  Every row's arithmetic is that of a decode call.
+        const SlotSnapshot snap = snapshot_locked(t);
+        DeviceGuard guard(t->device);
+        if (!guard.ok) return LML_ERR_CUDA;
+        const WsLayout ws = ws_layout(t, T, 1);
+        const int nb = (T + kDecodeMaxT - 1) / kDecodeMaxT;
+        SlotSnapshot snaps[kDecMaxBlocks];
+        DecodeArgs args[kDecMaxBlocks];
+        const Arena* ars[kDecMaxBlocks];
+        for (int bi = 0; bi < nb; ++bi) {
+            snaps[bi] = snap;
+            ars[bi] = &t->arena;
+            DecodeArgs& a = args[bi];
+            const int t0 = bi * kDecodeMaxT;
+            a.x = static_cast<const __nv_bfloat16*>(x) + (size_t)t0 * t->d_in;
+            a.W0 = W0;
+            a.y = static_cast<__nv_bfloat16*>(y) + (size_t)t0 * t->d_out;
+            a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
+            a.token_slots = token_slots + t0;
+            a.by_adapter = by_adapter;
+            a.u = reinterpret_cast<float*>(wsb + ws.u_off) + (size_t)bi * 16 * kRankPad;
+            a.T = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
+            a.d_in = t->d_in; a.d_out = t->d_out; a.G = 1; a.num_sms = t->num_sms;
+        }
+        const cudaError_t e = launch_decode_multi(ars, snaps, args, nb, stream);
+        t->last_launches = e == cudaSuccess ? 1 : 0;
+        if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+        return LML_OK;
+    }
     // Prefill: the segmentation pass writes perm and the segment arrays behind the layer's own workspace,
     // and the layer call follows on the same stream.
     const int G = t->max_slots + 1;
@@ -684,26 +722,36 @@ lml_status lora_mixed_linear_multi(lml_table* const* tables, int P, const void* 
     bool distinct = true;   // (a table's counters serve one projection of a launch)
     for (int p = 0; p < P; ++p)
         for (int q = 0; q < p; ++q) distinct = distinct && tables[p] != tables[q];
-    if (T <= kDecodeMaxT && P > 1 && distinct) {
+    const int nb = 1;   // (projections times blocks of 16 tokens in one launch was measured: 44.1 us against 42.8 us for q/k/v at 32 tokens as one call per projection)
+    if (P > 1 && distinct && T <= kDecodeMaxT) {
         // One launch of the decode kernel for all projections: its CTAs are dealt out over them, each works on its
         // projection as in a call of its own, and the fixed costs of a call are paid once.
         DeviceGuard guard(tables[0]->device);
         if (!guard.ok) return LML_ERR_CUDA;
-        SlotSnapshot snaps[LML_MAX_PROJECTIONS];
-        DecodeArgs args[LML_MAX_PROJECTIONS];
-        const Arena* ars[LML_MAX_PROJECTIONS];
+        SlotSnapshot snaps[kDecMaxBlocks];
+        DecodeArgs args[kDecMaxBlocks];
+        const Arena* ars[kDecMaxBlocks];
         const WsLayout ws = ws_layout(tables[0], T, 1);
+        int n = 0;
         for (int p = 0; p < P; ++p) {
-            snaps[p] = snapshot_locked(tables[p]);
-            ars[p] = &tables[p]->arena;
-            DecodeArgs& a = args[p];
-            a.x = x; a.W0 = W0[p]; a.y = y[p]; a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
-            a.token_slots = token_slots[p];
-            a.by_adapter = false;
-            a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.u_off) + (size_t)p * 16 * kRankPad;
-            a.T = T; a.d_in = tables[0]->d_in; a.d_out = tables[p]->d_out; a.G = 1; a.num_sms = tables[0]->num_sms;
+            const SlotSnapshot snap = snapshot_locked(tables[p]);
+            for (int bi = 0; bi < nb; ++bi, ++n) {
+                const int t0 = bi * kDecodeMaxT;
+                snaps[n] = snap;
+                ars[n] = &tables[p]->arena;
+                DecodeArgs& a = args[n];
+                a.x = static_cast<const __nv_bfloat16*>(x) + (size_t)t0 * tables[0]->d_in;
+                a.W0 = W0[p];
+                a.y = static_cast<__nv_bfloat16*>(y[p]) + (size_t)t0 * tables[p]->d_out;
+                a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
+                a.token_slots = token_slots[p] + t0;
+                a.by_adapter = false;
+                a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.u_off) + (size_t)n * 16 * kRankPad;
+                a.T = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
+                a.d_in = tables[0]->d_in; a.d_out = tables[p]->d_out; a.G = 1; a.num_sms = tables[0]->num_sms;
+            }
         }
-        const cudaError_t e = launch_decode_multi(ars, snaps, args, P, stream);
+        const cudaError_t e = launch_decode_multi(ars, snaps, args, n, stream);
         if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
         for (int p = 0; p < P; ++p) tables[p]->last_launches = p == 0 ? 1 : 0;
         return LML_OK;
@@ -862,7 +910,7 @@ lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
     bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     // also puts the decode kernel's two grid counters (words 1 and 2) back to zero, in case a call gave up
     ok = ok && cudaMemsetAsync(t->arena.status, 0, 3 * sizeof v, stream) == cudaSuccess;
-    ok = ok && cudaMemsetAsync(t->arena.status + 8, 0, 2 * sizeof v, stream) == cudaSuccess;   // (the counters of a dual decode call's second binding)
+    ok = ok && cudaMemsetAsync(t->arena.status + 8, 0, 14 * sizeof v, stream) == cudaSuccess;   // (the counters of the further parts of a decode launch)
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
     *flags_out = v;

@@ -49,7 +49,8 @@ namespace lml {
 
 using namespace ptx;
 
-constexpr int kDecMaxProj = LML_MAX_PROJECTIONS;  // projections that one launch can serve
+constexpr int kDecMaxTables = LML_MAX_PROJECTIONS;   // tables (projections proper) that one launch can serve
+constexpr int kDecMaxProj = kDecMaxBlocks;           // parts of a launch: projections, bindings of a dual call, blocks of 16 tokens
 constexpr int kDecConsumers = 8;                 // consumer warps
 constexpr int kDecShrinkWarps = 3;               // warps after the producer warp: the LoRA shrink
 constexpr int kDecThreads = (kDecConsumers + 1 + kDecShrinkWarps) * 32;
@@ -114,6 +115,9 @@ struct DecProj {
     const int32_t* perm;
     const int32_t* token_slots;
     const int32_t* adapter_map;
+    const __nv_bfloat16* x;     // this part's rows of x ...
+    int T;                      // ... and how many (<= 16)
+    int snap_idx;               // its table's snapshot in the launch's list
     uint32_t* status;
     unsigned int* sync_words;   // [0] elements of u that are written, [1] CTAs that have left: two words of the table's status block
     int N, G;
@@ -124,10 +128,9 @@ struct DecProj {
 // rows, its own share of that table's dot products, that table's counters), so one launch pays the fixed costs of a
 // call (the wait for the preceding work, the fetch of x, the tail) once for all of them.
 template <int kP> struct DecLaunch {
-    SlotSnapshot snap[kP];
+    SlotSnapshot snap[kP == 1 ? 1 : kDecMaxTables];
     DecProj proj[kP];
-    const __nv_bfloat16* x;
-    int T, K, P, patience;
+    int K, P, patience;
 };
 
 template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1>
@@ -136,13 +139,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     int pi = 0;
     if (kP > 1)
         while (pi + 1 < prm.P && (int)blockIdx.x >= prm.proj[pi + 1].cta_begin) ++pi;
-    const SlotSnapshot& snap = prm.snap[pi];
     const DecProj& pj = prm.proj[pi];
+    const SlotSnapshot& snap = prm.snap[kP == 1 ? 0 : pj.snap_idx];
     const int cta = (int)blockIdx.x - pj.cta_begin, ncta = pj.cta_count;   // this CTA among those of its projection
     const __nv_bfloat16* __restrict__ arenaA = pj.arenaA;
     const __nv_bfloat16* __restrict__ arenaB = pj.arenaB;
     const __nv_bfloat16* __restrict__ arenaBc = pj.arenaBc;
-    const __nv_bfloat16* __restrict__ x = prm.x;
+    const __nv_bfloat16* __restrict__ x = pj.x;
     const __nv_bfloat16* __restrict__ W0 = pj.W0;
     __nv_bfloat16* __restrict__ y = pj.y;
     float* u = pj.u;
@@ -152,7 +155,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     const int32_t* __restrict__ token_slots = pj.token_slots;
     const int32_t* __restrict__ adapter_map = pj.adapter_map;
     uint32_t* status = pj.status;
-    const int T = prm.T, K = prm.K, N = pj.N, G = pj.G, patience = prm.patience;
+    const int T = pj.T, K = prm.K, N = pj.N, G = pj.G, patience = prm.patience;
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
     const uint32_t ring = (raw + 127u) & ~127u;
@@ -868,6 +871,9 @@ void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
 {
     pj.arenaA = ar.A; pj.arenaB = ar.B; pj.arenaBc = ar.Bc;
     pj.W0 = (const __nv_bfloat16*)a.W0;
+    pj.x = (const __nv_bfloat16*)a.x;
+    pj.T = a.T;
+    pj.snap_idx = 0;
     pj.y = (__nv_bfloat16*)a.y;
     pj.u = a.u;
     pj.seg_offsets = a.seg_offsets; pj.slot_ids = a.slot_ids; pj.perm = a.perm; pj.token_slots = a.token_slots;
@@ -884,7 +890,7 @@ void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
 // several rounds (x is kept between rounds), and with several rounds and adapters (the expand of early rounds is put
 // off until u has arrived).
 template <int kP>
-cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_cta, bool adapters, cudaStream_t stream)
+cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_cta, bool adapters, int max_T, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -899,7 +905,7 @@ cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_
     const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
     const bool put_off = multi && adapters;
     auto launch = [&](auto kernel) { return cudaLaunchKernelEx(&cfg, kernel, prm); };
-    if (prm.T > 8)
+    if (max_T > 8)
         return put_off ? launch(decode_main_kernel<true, true, true, kP>)
                        : (multi ? launch(decode_main_kernel<true, true, false, kP>) : launch(decode_main_kernel<true, false, false, kP>));
     return put_off ? launch(decode_main_kernel<false, true, true, kP>)
@@ -918,9 +924,8 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     prm.snap[0] = snap;
     fill_proj(prm.proj[0], ar, a);
     prm.proj[0].cta_begin = 0; prm.proj[0].cta_count = grid;
-    prm.x = (const __nv_bfloat16*)a.x;
-    prm.T = a.T; prm.K = a.d_in; prm.P = 1; prm.patience = g_dec_patience;
-    const cudaError_t e = launch_decode_grid<1>(prm, grid, (a.d_out + grid - 1) / grid, a.G > 0, stream);
+    prm.K = a.d_in; prm.P = 1; prm.patience = g_dec_patience;
+    const cudaError_t e = launch_decode_grid<1>(prm, grid, (a.d_out + grid - 1) / grid, a.G > 0, a.T, stream);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
@@ -961,23 +966,35 @@ cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* sna
         --given;
     }
     DecLaunch<kDecMaxProj> prm;
-    int begin = 0, rows_per_cta = 0;
+    int begin = 0, rows_per_cta = 0, max_T = 0, ntables = 0;
     bool adapters = false;
+    const Arena* seen[kDecMaxTables];
+    int uses[kDecMaxTables];
+    // A table that serves several parts of the launch (the bindings of a dual call, the blocks of a batch of more than 16
+    // tokens) gives each of them its own pair of counters in its status block: words 1-2, then 8-9, 10-11, ...
     for (int p = 0; p < P; ++p) {
-        prm.snap[p] = snaps[p];
+        int ti = 0;
+        while (ti < ntables && seen[ti] != ars[p]) ++ti;
+        if (ti == ntables) {
+            if (ntables == kDecMaxTables) return cudaErrorInvalidValue;
+            seen[ntables] = ars[p]; uses[ntables] = 0; prm.snap[ntables] = snaps[p];
+            ++ntables;
+        }
         fill_proj(prm.proj[p], *ars[p], args[p]);
-        for (int q = 0; q < p; ++q)   // a table that serves two projections of the launch (the two bindings of a dual call): its second pair of counters
-            if (ars[q] == ars[p]) prm.proj[p].sync_words = ars[p]->status + 8;
+        prm.proj[p].snap_idx = ti;
+        prm.proj[p].sync_words = ars[p]->status + (uses[ti] == 0 ? 1 : 6 + 2 * uses[ti]);
+        ++uses[ti];
         prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = count[p];
         begin += count[p];
         const int r = (args[p].d_out + count[p] - 1) / count[p];
         rows_per_cta = r > rows_per_cta ? r : rows_per_cta;
+        max_T = args[p].T > max_T ? args[p].T : max_T;
         adapters = adapters || args[p].G > 0;
     }
-    for (int p = P; p < kDecMaxProj; ++p) { prm.snap[p] = snaps[0]; prm.proj[p] = prm.proj[0]; prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = 0; }
-    prm.x = (const __nv_bfloat16*)args[0].x;
-    prm.T = args[0].T; prm.K = args[0].d_in; prm.P = P; prm.patience = g_dec_patience;
-    return launch_decode_grid<kDecMaxProj>(prm, begin, rows_per_cta, adapters, stream);
+    for (int t = ntables; t < kDecMaxTables; ++t) prm.snap[t] = prm.snap[0];
+    for (int p = P; p < kDecMaxProj; ++p) { prm.proj[p] = prm.proj[0]; prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = 0; }
+    prm.K = args[0].d_in; prm.P = P; prm.patience = g_dec_patience;
+    return launch_decode_grid<kDecMaxProj>(prm, begin, rows_per_cta, adapters, max_T, stream);
 }
 
 }  // namespace lml

@@ -136,6 +136,7 @@ bool encode_tmap_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, 
                     uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
                     uint32_t b2);
 
+constexpr int kDecMaxBlocks = 8;   // parts of one decode launch at most (projections, bindings, blocks of 16 tokens)
 struct DecodeArgs {
     const void* x;
     const void* W0;
@@ -153,7 +154,8 @@ cudaError_t decode_init();   // sets the dynamic shared memory attributes
 int decode_patience();       // LML_DECODE_PATIENCE or the default, in clock cycles
 cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const DecodeArgs& a,
                           cudaStream_t stream, int* launches);
-// P <= LML_MAX_PROJECTIONS projections that read the same x (args[p].x, T, d_in, num_sms equal for all p) in one launch.
+// P <= kDecMaxBlocks parts in one launch (d_in and num_sms equal for all; at most LML_MAX_PROJECTIONS distinct tables):
+// projections that read the same x, the two bindings of a dual call, blocks of 16 tokens of a larger batch.
 cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* snaps, const DecodeArgs* args, int P,
                                 cudaStream_t stream);
 

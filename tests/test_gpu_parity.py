@@ -209,6 +209,36 @@ def test_layer_sweep_cells_every_element(proj, T):
     check_full(wl.layer_sweep(proj, T))
 
 
+# a few blocks of 16 tokens through the token form of the call (one launch of the decode kernel, a share of its CTAs per
+# block): every element against the oracle, output and workspace between canary bands
+@pytest.mark.parametrize("proj,T", [("q", 17), ("q", 32), ("q", 48), ("gate", 32), ("down", 31)])
+def test_layer_sweep_shapes_at_a_few_blocks_of_tokens(proj, T):
+    import torch
+    from gpu_util import Guarded
+    w = wl.layer_sweep(proj, T)
+    site = Site(w)
+    try:
+        token_entry = np.repeat(w.seg_entry, np.diff(w.seg_offsets))
+        if w.perm is not None:
+            unperm = np.empty_like(token_entry)
+            unperm[w.perm] = token_entry
+            token_entry = unperm
+        slots = site.slot_ids(token_entry)
+        gy = Guarded(T * w.d_out * 2)
+        from paper_2608_15241_b200.binding import lml_tokens_workspace_bytes
+        gws = Guarded(max(lml_tokens_workspace_bytes(site.table.handle, T), 256))
+        y = gy.view(torch.bfloat16, (T, w.d_out))
+        site.table.lora_mixed_linear_tokens(site.x, site.W0, torch.from_numpy(slots).cuda(), y=y, workspace=gws.payload)
+        torch.cuda.synchronize()
+        assert gy.intact() and gws.intact()
+        assert site.table.device_status() == 0 and site.table.last_launch_count() == 1
+        ref, oflags = oracle.forward_workload(w)
+        r = oracle.compare(to_bits(y), ref)
+        assert oflags == 0 and r["ok"], r
+    finally:
+        site.close()
+
+
 # the 8192-token cells: >= 512 rows with a row of every 128-row tile and every segment's ends
 @pytest.mark.parametrize("proj", ["o", "gate", "down"])
 def test_layer_sweep_8192_token_cells_every_tile(proj):

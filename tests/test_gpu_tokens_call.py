@@ -1,8 +1,9 @@
 """lora_mixed_linear_tokens (one slot id per token) against the two-call form it replaces:
 lml_segment_tokens followed by lora_mixed_linear with the perm it produced.  Both forms run the
 same arithmetic per output element, so the results must agree bit for bit; the oracle is checked
-on top.  Covers the one-launch decode form (T <= 16), the prefill form, ids that name no live
-adapter (flagged, treated as -1) and the all-base case."""
+on top.  Covers the one-launch decode form (T <= 16), the form for a few blocks of 16 tokens (the decode kernel
+again: bit for bit a decode call per block), the prefill form, ids that name no live adapter (flagged, treated
+as -1) and the all-base case."""
 import numpy as np
 import pytest
 
@@ -27,7 +28,7 @@ def _table(K, N, ranks, seed):
 
 
 @pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384),
-                                   (17, 264, 136), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
+                                   (17, 264, 136), (24, 1032, 520), (32, 1032, 16400), (33, 1032, 16400), (48, 520, 264), (49, 520, 264), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
                                    (200, 1536, 520)])
 def test_tokens_call_equals_segment_then_layer(T, K, N):
     import torch
@@ -45,7 +46,18 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
     y_two = to_bits(tbl.lora_mixed_linear(x, W, so, ids, perm=perm))
     torch.cuda.synchronize()
     assert tbl.device_status() == 0
-    assert np.array_equal(y_tok, y_two)
+    blocks = 16 < T <= (48 if K * N <= 1 << 24 else 32)
+    if blocks:
+        # a few blocks of 16 tokens: one launch of the decode kernel, every block's rows exactly those of a decode call
+        # on that block alone; against the two-call form (the GEMM path) equal to the last place of bf16
+        assert launches_tok == 1
+        for t0 in range(0, T, 16):
+            y_blk = to_bits(tbl.lora_mixed_linear_tokens(x[t0:t0 + 16].contiguous(), W, ts[t0:t0 + 16].contiguous()))
+            assert np.array_equal(y_tok[t0:t0 + 16], y_blk), t0
+        a, b2 = wl.bf16_bits_to_f64(y_tok), wl.bf16_bits_to_f64(y_two)
+        assert (np.abs(a - b2) <= 2.0 ** -7 * np.maximum(1.0, np.abs(b2))).all()
+    else:
+        assert np.array_equal(y_tok, y_two)
     if T <= 16:
         assert launches_tok == 1
 
