@@ -589,7 +589,7 @@ def run_layer_sweep(device, peaks, steps, only=None, parity=False, tokens=None):
     stream = torch.cuda.Stream(device=device)
     cells = []
     for proj, same_as in (("q", "q k v o"), ("gate", "gate up"), ("down", "down")):
-        for T in (tokens or wl.SWEEP_TOKENS):
+        for T in (tokens or (sorted({t_ for _, t_ in only}) if only else wl.SWEEP_TOKENS)):
             if only and (proj, T) not in only:
                 continue
             w = wl.layer_sweep(proj, T)
