@@ -508,6 +508,9 @@ def run_workload(name, steps, warmup, device, world, peaks, want_cpu_baseline, e
                       "l2_policy": f"inputs larger than L2: {rot.R} distinct weight/activation sets "
                                    f"({rot.R * w.bytes() / 1e6:.0f} MB) visited round-robin",
                       "timing": "CUDA-graph replay of R-step chunks, CUDA events on the launch stream"}}
+    if clocks and clocks.get("sm_mhz"):
+        # time x clock: comparable across power states (the long prefill loops run under the 1 kW cap at a lower SM clock)
+        out["us_per_step_times_sm_ghz"] = secs / steps * 1e6 * clocks["sm_mhz"] / 1e3
     if e2e:
         out["e2e"] = e2e
     if dual:
