@@ -287,7 +287,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     // it only in their first epilogue.
     unsigned int* sync_words = pj.sync_words;
     const bool shrinker = warp > kDecConsumers;
-    if (consumer && G > 0)   // let the lookup's loads go first through the load/store path (see below)
+    // Segments form: the lookup's loads (several small arrays) go first through the load/store path (see below).  With
+    // one slot id per row the lookup is a single load per row, and the order is not worth its price: 0.9 us on a
+    // batch in which no token is bound to an adapter.
+    if (consumer && G > 0 && token_slots == nullptr)
         asm volatile("bar.sync 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
     if (shrinker && G > 0) {
         const int sw = warp - kDecConsumers - 1;
@@ -358,7 +361,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 // the ids are adapter ids: the table's device map names the serving slot (-2: none, flagged below)
                 if (adapter_map) my_token_slot = resolve_adapter(snap, adapter_map, my_token_slot);
             }
-            asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
+            if (!by_token) asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
             if (cached) {
