@@ -204,7 +204,7 @@ lml_status lml_segment_tokens(lml_table* t, const int32_t* token_slots, int T, i
  * without launching.
  * T <= 16 runs the bandwidth-bound decode kernel (W0 read once through a bulk-copy ring; with
  * segments its CTAs hand one another their share of the shrink result and count themselves in
- * the table's status block, so two decode calls on the SAME table must not overlap on the GPU:
+ * a small exchange block that belongs to the table, so two decode calls on the SAME table must not overlap on the GPU:
  * put them on one stream or order them; a CTA whose peers are late computes their share itself,
  * so the call completes even when the grid cannot be resident all at once); larger T runs the
  * TMA / tcgen05 GEMM with the LoRA expand as extra tensor-core K-steps.
@@ -302,7 +302,7 @@ lml_status lora_mixed_linear_tokens(lml_table* t, const void* x, const void* W0,
  * table named twice, runs as one decode call per projection.
  * T > 16: the projections run one after the other on `stream`, each exactly as
  * lora_mixed_linear_tokens(tables[p], ...).
- * Every projection's CTAs count themselves in that table's status block, as in a decode call: two calls
+ * Every projection's CTAs count themselves in that table's exchange block, as in a decode call: two calls
  * that share a table must not overlap on the GPU.  Device-detected errors set the flags of the table they
  * concern.
  * workspace: device, 256-byte aligned, at least lml_multi_workspace_bytes(tables, P, T).
@@ -360,8 +360,8 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
  * was handed out completely at start-up.  Such a caller still passes its inputs and the output
  * (x, W0, seg_offsets, slot_ids, perm, y: same meaning, layout and alignment as in
  * lora_mixed_linear), but no workspace: the scratch the decode kernel needs between its two
- * phases (the scaled shrink result, 16 x 64 fp32) lives in a 4096-byte array inside the library
- * image.  Every GPU that loads the library holds that array until the
+ * phases (the scaled shrink result, 16 x 64 fp32, each value beside the mark of the launch that
+ * wrote it, and three counters) lives in an 8448-byte array inside the library image.  Every GPU that loads the library holds that array until the
  * process exits.  The call allocates and frees nothing, and calls no allocating routine.
  *
  * Limits and rules
@@ -370,9 +370,9 @@ lml_status lora_mixed_linear_host(lml_table* t, const void* x_host, const void* 
  *   - Every call looks up the array's device address (cudaGetSymbolAddress, with the table's device
  *     current; no allocation).  The first call on a device may load the library's device code:
  *     make that first call outside any stream capture.
- *   - All calls on a device share the one array, and it keeps the previous call's contents.
- *     Nothing in it has to start at zero: the kernel writes every element it later reads.
- *     Two calls that overlap on the GPU (different streams without ordering, or concurrent
+ *   - All calls on a device share the one array, and it keeps the previous call's contents:
+ *     it starts as zeros (a file-scope object), and its own launch counter tells a call's values
+ *     from those of earlier calls, whichever table they were for.  Two calls that overlap on the GPU (different streams without ordering, or concurrent
  *     graph branches) race on the array: order them.
  *   - Results are identical to lora_mixed_linear on the same inputs.
  * Errors: INVALID_ARG, TOO_LARGE, CUDA.
@@ -383,8 +383,8 @@ lml_status lora_mixed_linear_decode_static(lml_table* t, const void* x, const vo
 
 /*
  * Read and clear the sticky device status word (LML_FLAG_* bits).  Synchronises `stream`.
- * Also puts the decode kernel's grid counters back to zero, which matters only after a call
- * that reported LML_FLAG_TIMEOUT.
+ * Also puts the table's decode exchange blocks (values, marks, counters) back to zero, which matters only
+ * after a launch that ended abnormally.
  * Errors: INVALID_ARG, CUDA.
  */
 lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream);

@@ -24,9 +24,6 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
     w.ident_off = round_up(sizeof(PlanWord), 256);
     w.u_off = round_up(w.ident_off + (num_m + 1) * sizeof(int32_t), 1024);
     size_t u_bytes = (size_t)u_sets * (num_m + (size_t)(G > 0 ? G : 1)) * kTileM * kRankPad * sizeof(__nv_bfloat16);
-    // the decode kernel's scratch: u[16][64] fp32 per projection of a launch
-    const size_t dec_bytes = (size_t)kDecMaxBlocks * 16 * kRankPad * sizeof(float);
-    if (u_bytes < dec_bytes) u_bytes = dec_bytes;
     w.xg_off = w.u_off + round_up(u_bytes, 1024);
     w.total = w.xg_off + round_up((size_t)T * t->d_in * sizeof(__nv_bfloat16), 1024);
     return w;
@@ -36,7 +33,7 @@ WsLayout ws_layout(const lml_table* t, int T, int G, int u_sets = 1)
 
 static void free_table_resources(lml_table* t)
 {
-    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.Bc); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map); cudaFree(t->arena.tile_flags);
+    cudaFree(t->arena.A); cudaFree(t->arena.B); cudaFree(t->arena.Bc); cudaFree(t->arena.status); cudaFree(t->arena.adapter_map); cudaFree(t->arena.tile_flags); cudaFree(t->arena.dec_u);
     if (t->copy_in) cudaStreamDestroy(t->copy_in);
     if (t->copy_out) cudaStreamDestroy(t->copy_out);
     if (t->ev_begin) cudaEventDestroy(t->ev_begin);
@@ -101,6 +98,9 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
     ok = ok && cudaMemset(t->arena.A, 0, a_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.B, 0, b_bytes) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.status, 0, 256) == cudaSuccess;
+    const size_t dec_u_bytes = (size_t)kDecMaxBlocks * kDecExchStride * sizeof(unsigned long long);
+    ok = ok && cudaMalloc(&t->arena.dec_u, dec_u_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(t->arena.dec_u, 0, dec_u_bytes) == cudaSuccess;   // mark 0: written by no launch
     ok = ok && cudaMemset(t->arena.adapter_map, 0xff, kMaxAdapterIds * sizeof(int32_t)) == cudaSuccess;   // -1: no serving version
     ok = ok && cudaMalloc(&t->arena.tile_flags, kFuseMaxTiles * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMemset(t->arena.tile_flags, 0, kFuseMaxTiles * sizeof(int32_t)) == cudaSuccess;
@@ -411,7 +411,6 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
     if (decode) {
         DecodeArgs a;
         a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
-        a.u = G > 0 ? reinterpret_cast<float*>(wsb + ws.u_off) : nullptr;
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         e = launch_decode(t->arena, snap, a, stream, &launches);
     } else {
@@ -491,7 +490,6 @@ lml_status lora_mixed_linear_dual(lml_table* t, const void* x, const void* W0, i
             DecodeArgs& a = args[p];
             a.x = x; a.W0 = W0; a.y = p == 0 ? y_a : y_b; a.perm = perm; a.seg_offsets = seg_offsets;
             a.slot_ids = p == 0 ? slot_ids_a : slot_ids_b;
-            a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws1.u_off) + (size_t)p * 16 * kRankPad;
             a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
         }
         const cudaError_t e = launch_decode_multi(ars, snaps, args, 2, (cudaStream_t)stream_v);
@@ -619,7 +617,6 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
         a.x = x; a.W0 = W0; a.y = y; a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
         a.token_slots = token_slots;
         a.by_adapter = by_adapter;
-        a.u = reinterpret_cast<float*>(wsb + ws.u_off);
         a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = 1; a.num_sms = t->num_sms;
         int launches = 0;
         const cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
@@ -655,7 +652,6 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
             a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
             a.token_slots = token_slots + t0;
             a.by_adapter = by_adapter;
-            a.u = reinterpret_cast<float*>(wsb + ws.u_off) + (size_t)bi * 16 * kRankPad;
             a.T = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
             a.d_in = t->d_in; a.d_out = t->d_out; a.G = 1; a.num_sms = t->num_sms;
         }
@@ -746,7 +742,6 @@ lml_status lora_mixed_linear_multi(lml_table* const* tables, int P, const void* 
                 a.perm = nullptr; a.seg_offsets = nullptr; a.slot_ids = nullptr;
                 a.token_slots = token_slots[p] + t0;
                 a.by_adapter = false;
-                a.u = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.u_off) + (size_t)n * 16 * kRankPad;
                 a.T = T - t0 < kDecodeMaxT ? T - t0 : kDecodeMaxT;
                 a.d_in = tables[0]->d_in; a.d_out = tables[p]->d_out; a.G = 1; a.num_sms = tables[0]->num_sms;
             }
@@ -908,9 +903,9 @@ lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
     if (!guard.ok) return LML_ERR_CUDA;
     uint32_t v = 0;
     bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    // also puts the decode kernel's two grid counters (words 1 and 2) back to zero, in case a call gave up
-    ok = ok && cudaMemsetAsync(t->arena.status, 0, 3 * sizeof v, stream) == cudaSuccess;
-    ok = ok && cudaMemsetAsync(t->arena.status + 8, 0, 14 * sizeof v, stream) == cudaSuccess;   // (the counters of the further parts of a decode launch)
+    ok = ok && cudaMemsetAsync(t->arena.status, 0, sizeof v, stream) == cudaSuccess;
+    // (and the decode kernel's exchange blocks start over: a launch that ended abnormally may have left its counters behind)
+    ok = ok && cudaMemsetAsync(t->arena.dec_u, 0, (size_t)kDecMaxBlocks * kDecExchStride * sizeof(unsigned long long), stream) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
     *flags_out = v;

@@ -22,9 +22,11 @@
 //                       u[row][j] = scale_s * sum_k x[row][k] A_s[j][k] (fp32).  The dot products are dealt
 //                       out over the whole grid in groups of 1, 2 or 4 columns of one row; a group's
 //                       operands are staged in shared memory by asynchronous copies (one memory round
-//                       trip per group; single dot products stay in registers).  Each result is
-//                       published in global memory with a release-add on a grid-wide counter; the warps
-//                       wait for the counter and stage all of u in shared memory.  When the table's live
+//                       trip per group; single dot products stay in registers).  Each result goes to
+//                       the table's exchange block as one 64-bit word, the value beside this launch's
+//                       mark, followed by a plain add on a grid-wide counter (no fence anywhere); the
+//                       warps wait for the counter, then read the entries, taking only those that carry
+//                       the mark, and stage all of u in shared memory.  When the table's live
 //                       adapters are few, their rows of A are asked into L2 at kernel entry, ahead of
 //                       the weight stream.  The consumers meet the shrink warps once, at their first
 //                       epilogue.  No CTA depends on the others being resident: after a bounded wait
@@ -79,6 +81,8 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     int rank_of_row[16];
     float dot_part[kDecDotGroup][4];
     int u_complete;
+    unsigned epoch;         // this launch's mark on the entries of u
+    int pad[3];
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
 constexpr int kDecDeferBytes = 2048;   // base sums of rounds whose expand is put off: 16 x 32 or 2 x (8 x 32) fp32
@@ -109,14 +113,14 @@ struct DecProj {
     const __nv_bfloat16* arenaBc;
     const __nv_bfloat16* W0;
     __nv_bfloat16* y;
-    float* u;
+    unsigned long long* u;      // this part's exchange block: [16][kRankPad] entries (value | mark << 32), then its three words
     const int32_t* seg_offsets;
     const int32_t* slot_ids;
     const int32_t* perm;
     const int32_t* token_slots;
     const int32_t* adapter_map;
     uint32_t* status;
-    unsigned int* sync_words;   // [0] elements of u that are written, [1] CTAs that have left: two words of the table's status block
+    unsigned int* sync_words;   // the block's words: [0] the mark of the last launch that finished, [1] CTAs that have left, [2] entries written
     int N, G;
     int cta_begin, cta_count;   // CTAs [cta_begin, cta_begin + cta_count) of the grid
     // (what launches of several parts need comes last: the single-part build is sensitive to the layout of the fields above,
@@ -151,7 +155,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     const __nv_bfloat16* __restrict__ x = kP == 1 ? prm.x : pj.x;
     const __nv_bfloat16* __restrict__ W0 = pj.W0;
     __nv_bfloat16* __restrict__ y = pj.y;
-    float* u = pj.u;
+    unsigned long long* u = pj.u;
     const int32_t* __restrict__ seg_offsets = pj.seg_offsets;
     const int32_t* __restrict__ slot_ids = pj.slot_ids;
     const int32_t* __restrict__ perm = pj.perm;
@@ -282,9 +286,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     // The first of them works out the slot of every row of x, raises the status flags and pulls the B
     // rows this CTA will need into L2.  Then the (token, j) dot products u = scale * x.A_j are dealt
     // out round-robin to the CTAs of the grid and, inside a CTA, to its three shrink warps: one warp per
-    // dot product, sixteen 16-byte loads in flight per lane.  The results go to u in global memory; a
-    // counter in the table's status block tells every CTA when all of u is there.  The consumers look at
-    // it only in their first epilogue.
+    // dot product, sixteen 16-byte loads in flight per lane.  The results go to the exchange block in global
+    // memory; a counter there tells every CTA when to look for them.  The consumers look at u only in their
+    // first epilogue.
     unsigned int* sync_words = pj.sync_words;
     const bool shrinker = warp > kDecConsumers;
     // Segments form: the lookup's loads (several small arrays) go first through the load/store path (see below).  With
@@ -333,8 +337,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 (void)rows_before;
             }
         }
-        if (sw == kDecShrinkWarps - 1)
+        if (sw == kDecShrinkWarps - 1) {
+            // this launch's mark: one more than that of the last launch that finished on these words
+            unsigned last_epoch = 0;
+            if (lane == 0) last_epoch = ld_relaxed_gpu(sync_words);
             for (int sl = lane; sl < kMaxSlots; sl += 32) lk->scale_s[sl] = snap.scale[sl];
+            if (lane == 0) lk->epoch = last_epoch + 1u;
+        }
         if (sw == 0) {
             // One memory round trip for everything the lookup needs: the segment arrays go to shared
             // memory (all loads issued before the first is used), the search then runs there.  Calls
@@ -364,6 +373,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             if (!by_token) asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
+            if (lane == 0) lk->u_complete = 1;
             if (cached) {
 #pragma unroll
                 for (int i = 0; i <= kDecSegCache / 32; ++i) {
@@ -469,8 +479,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // m + 192, ... of the row in order, each warp adds its threads' sums up with the butterfly, and the
         // result is (w0 + w1) + w2 times the scale.  The operands of a whole group are brought into shared
         // memory with asynchronous 16-byte copies, all in flight at once (registers would hold a fraction of
-        // them), so a group costs one memory round trip.  A group's results are published with one
-        // release-add on the grid-wide counter: nobody waits for a fence.
+        // them), so a group costs one memory round trip.  A result is published as one 64-bit store (value and this
+        // launch's mark) and a relaxed add on the grid-wide counter: nobody waits for a fence.
         const int total = lk->dot_end[15];
         // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
         // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
@@ -594,13 +604,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             return val;
         };
         const long long t_shrink = clock64();
+        const unsigned epoch = lk->epoch;
         if (gsize == 1) {
             if (cta < total) {
                 int t, j;
                 const float val = single(cta, t, j);
                 if (me == 0) {
-                    u[t * kRankPad + j] = val;
-                    red_release_gpu_add(sync_words, 1u);
+                    st_relaxed_gpu_b64(u + t * kRankPad + j, pack_u(val, epoch));
+                    red_relaxed_gpu_add(sync_words + 2, 1u);
                 }
             }
         } else
@@ -609,8 +620,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             int t, j0;
             group(g, val, t, j0);
             if (me == 0) {
-                for (int i = 0; i < gsize; ++i) u[t * kRankPad + j0 + i] = val[i];
-                red_release_gpu_add(sync_words, (unsigned)gsize);
+                for (int i = 0; i < gsize; ++i) st_relaxed_gpu_b64(u + t * kRankPad + j0 + i, pack_u(val[i], epoch));
+                red_relaxed_gpu_add(sync_words + 2, (unsigned)gsize);
             }
         }
         if (gsize > 1) stage_b();   // the staging buffer is free now (the groups end with a barrier of these warps)
@@ -621,16 +632,45 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // bounded wait it simply computes every dot product itself, with the same arithmetic and hence the
         // same bits, finishes and makes room for whichever CTAs have not started yet.
         if (sw == 0 && lane == 0) {
-            int complete = 1;
-            while (ld_acquire_gpu(sync_words) < (unsigned)total) {
-                if (clock64() - t_shrink > (long long)patience) { complete = 0; break; }
+            while (ld_relaxed_gpu(sync_words + 2) < (unsigned)total) {
+                if (clock64() - t_shrink > (long long)patience) { lk->u_complete = 0; break; }
             }
-            lk->u_complete = complete;
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
         if (lk->u_complete) {
-            for (int i = me; i < T * kRankPad / 4; i += kDecShrinkWarps * 32)
-                reinterpret_cast<float4*>(u_s)[i] = __ldcg(reinterpret_cast<const float4*>(u) + i);
+            // Every entry of u is a 64-bit word, the value beside the mark of the launch that wrote it, and is written and
+            // read as one: an entry that carries this launch's mark is this launch's value, whatever order the stores and
+            // the counter's adds became visible in (the counter only says when looking is worth it: 148 CTAs that poll the
+            // entries themselves were measured 0.5 us and more slower than the counter they replaced).  A thread takes pairs
+            // of entries (16 bytes) of the columns that the expand reads, has all its loads in flight at once and asks
+            // again for what was not there yet.
+            constexpr int kPairs = (16 * kRankPad / 2 + kDecShrinkWarps * 32 - 1) / (kDecShrinkWarps * 32);   // 6
+            unsigned pending = 0;
+#pragma unroll
+            for (int k = 0; k < kPairs; ++k) {
+                const int i = me + k * kDecShrinkWarps * 32;
+                const int t = i / (kRankPad / 2), j = (i % (kRankPad / 2)) * 2;
+                if (t < T && j < ((lk->rank_of_row[t & 15] + 7) & ~7)) pending |= 1u << k;
+            }
+            while (pending) {
+                unsigned long long e0[kPairs], e1[kPairs];
+#pragma unroll
+                for (int k = 0; k < kPairs; ++k)
+                    if (pending >> k & 1u) ld_relaxed_gpu_v2_b64(u + 2 * (me + k * kDecShrinkWarps * 32), e0[k], e1[k]);
+#pragma unroll
+                for (int k = 0; k < kPairs; ++k) {
+                    if ((pending >> k & 1u) && (unsigned)(e0[k] >> 32) == epoch && (unsigned)(e1[k] >> 32) == epoch) {
+                        reinterpret_cast<float2*>(u_s)[me + k * kDecShrinkWarps * 32] =
+                            make_float2(__uint_as_float((unsigned)e0[k]), __uint_as_float((unsigned)e1[k]));
+                        pending &= ~(1u << k);
+                    }
+                }
+                if (pending && clock64() - t_shrink > (long long)patience) { lk->u_complete = 0; break; }
+            }
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+        if (lk->u_complete) {
+            // (u_s holds every column that the expand reads)
         } else if (gsize == 1) {   // (the staging buffer may hold B rows: stay in registers)
             for (int d = 0; d < total; ++d) {
                 int t, j;
@@ -653,13 +693,21 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // releases what it wrote)
         if (kPutOff) mbar_arrive(smem_u32(&ctrl->ufull));   // (the consumers can test this one without waiting)
         else asm volatile("bar.arrive 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
-        // Every CTA signs off once it has its copy of u and has published its own share; the last one puts
-        // both counters back to zero for the next call on this table.
+        // Every CTA signs off once it has its copy of u and has published its own share; the last one makes this
+        // launch's mark the table's last one, so that the next call on this table takes the next mark, and puts the
+        // counter back to zero.
         if (sw == 0 && lane == 0) {
             __threadfence();
             if (atomicAdd(sync_words + 1, 1u) == (unsigned)ncta - 1u) {
-                sync_words[0] = 0u;
+                if (epoch == 0xffffffffu) {   // the marks start over: no entry may keep one of the last round
+                    for (int i = 0; i < kDecExchEntries; ++i) u[i] = 0ull;
+                    __threadfence();
+                    sync_words[0] = 0u;
+                } else {
+                    sync_words[0] = epoch;
+                }
                 sync_words[1] = 0u;
+                sync_words[2] = 0u;
             }
         }
     }
@@ -881,11 +929,11 @@ void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
     pj.T = a.T;
     pj.snap_idx = 0;
     pj.y = (__nv_bfloat16*)a.y;
-    pj.u = a.u;
+    pj.u = a.exch ? a.exch : ar.dec_u;
     pj.seg_offsets = a.seg_offsets; pj.slot_ids = a.slot_ids; pj.perm = a.perm; pj.token_slots = a.token_slots;
     pj.adapter_map = a.by_adapter ? ar.adapter_map : nullptr;
     pj.status = ar.status;
-    pj.sync_words = ar.status + 1;
+    pj.sync_words = reinterpret_cast<unsigned int*>(pj.u + kDecExchEntries);
     pj.N = a.d_out; pj.G = a.G;
 }
 
@@ -978,7 +1026,7 @@ cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* sna
     const Arena* seen[kDecMaxTables];
     int uses[kDecMaxTables];
     // A table that serves several parts of the launch (the bindings of a dual call, the blocks of a batch of more than 16
-    // tokens) gives each of them its own pair of counters in its status block: words 1-2, then 8-9, 10-11, ...
+    // tokens) gives each of them an exchange block of its own
     for (int p = 0; p < P; ++p) {
         int ti = 0;
         while (ti < ntables && seen[ti] != ars[p]) ++ti;
@@ -989,7 +1037,10 @@ cudaError_t launch_decode_multi(const Arena* const* ars, const SlotSnapshot* sna
         }
         fill_proj(prm.proj[p], *ars[p], args[p]);
         prm.proj[p].snap_idx = ti;
-        prm.proj[p].sync_words = ars[p]->status + (uses[ti] == 0 ? 1 : 6 + 2 * uses[ti]);
+        if (!args[p].exch) {
+            prm.proj[p].u = ars[p]->dec_u + (size_t)uses[ti] * kDecExchStride;
+            prm.proj[p].sync_words = reinterpret_cast<unsigned int*>(prm.proj[p].u + kDecExchEntries);
+        }
         ++uses[ti];
         prm.proj[p].cta_begin = begin; prm.proj[p].cta_count = count[p];
         begin += count[p];

@@ -26,6 +26,30 @@ __device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v)
 {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_relaxed_gpu_add(unsigned* p, unsigned v)
+{
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_relaxed_gpu(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// An entry of the decode kernel's exchange buffer: a value and the mark of the launch that wrote it, one 64-bit
+// word that is stored and loaded whole.
+__device__ __forceinline__ unsigned long long pack_u(float v, unsigned mark)
+{
+    return (unsigned long long)__float_as_uint(v) | ((unsigned long long)mark << 32);
+}
+__device__ __forceinline__ void st_relaxed_gpu_b64(unsigned long long* p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void ld_relaxed_gpu_v2_b64(const unsigned long long* p, unsigned long long& a, unsigned long long& b)   // 16-byte aligned
+{
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
 {
     unsigned v;

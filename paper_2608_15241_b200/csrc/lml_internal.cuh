@@ -39,6 +39,7 @@ struct Arena {
     uint32_t* status;   // sticky LML_FLAG_* bits
     int32_t* tile_flags;    // [kFuseMaxTiles] fused shrink of the prefill GEMM: row tile m's u blocks are written (= epoch + 1; the epoch is word 4 of status)
     int32_t* adapter_map;   // [kMaxAdapterIds] serving entry of each adapter id: slot | generation << 8, -1 = none; written by lml_publish
+    unsigned long long* dec_u;   // [kDecMaxBlocks][kDecExchStride] the decode kernel's exchange blocks, one per part of a launch that works on this table
 };
 
 inline int32_t adapter_map_word(int slot, uint16_t gen) { return (int32_t)((uint32_t)slot | ((uint32_t)gen << 8)); }
@@ -136,6 +137,11 @@ bool encode_tmap_3d(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, 
                     uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1,
                     uint32_t b2);
 
+// The decode kernel's exchange block, through which the CTAs of a launch hand one another u = scale * x.A^T: 16 x kRankPad
+// entries (an fp32 value beside the mark of the launch that wrote it, one 64-bit word), then three 32-bit words: the mark
+// of the last launch that finished on this block, the CTAs that have left, the entries written.  All zero to begin with.
+constexpr int kDecExchEntries = 16 * kRankPad;
+constexpr int kDecExchStride = kDecExchEntries + 8;   // 64-bit words per block
 constexpr int kDecMaxBlocks = 8;   // parts of one decode launch at most (projections, bindings, blocks of 16 tokens)
 struct DecodeArgs {
     const void* x;
@@ -146,7 +152,7 @@ struct DecodeArgs {
     const int32_t* slot_ids;
     const int32_t* token_slots = nullptr;   // instead of segments: one slot id per row of x (then G is 1 and perm is null)
     bool by_adapter = false;                // the ids in token_slots are adapter ids, resolved through the table's device map
-    float* u;            // [16][64] fp32 scratch: scale * x.A^T, written and read by the decode kernel
+    unsigned long long* exch = nullptr;   // exchange block of the call (kDecExchStride words); null: the table's own, by order of use in the launch
     int T, d_in, d_out, G;
     int num_sms;
 };

@@ -1,19 +1,19 @@
 // lora_mixed_linear_decode_static: the decode form of the layer for callers that cannot hand the
 // library any scratch memory.  See the declaration in include/lora_mixed_linear.h.
 //
-// The decode kernel needs a little scratch between its shrink phase and its epilogue: the scaled
-// shrink result u[16][64] (fp32), which the CTAs of the grid write for one another.  The regular
-// entry point takes it from the caller's workspace.  Here it lives in a file-scope device array
-// that is part of the library image: every GPU context that loads the library carries these 4096
-// bytes until the process exits, and nothing is ever allocated or freed.
+// The decode kernel needs a little scratch between its shrink phase and its epilogue: the exchange
+// block through which the CTAs of the grid hand one another the scaled shrink result u[16][64]
+// (each fp32 value beside the mark of the launch that wrote it, then three counters).  Here it lives
+// in a file-scope device array that is part of the library image: every GPU context that loads the
+// library carries these 8448 bytes until the process exits, and nothing is ever allocated or freed.
 #include "lml_table.cuh"
 
 using namespace lml;
 
 namespace {
 
-constexpr size_t kStaticU = (size_t)kDecodeMaxT * kRankPad * sizeof(float);   // 4096 bytes
-constexpr size_t kStaticScratchBytes = 4096;
+constexpr size_t kStaticU = (size_t)kDecExchStride * sizeof(unsigned long long);   // 8256 bytes
+constexpr size_t kStaticScratchBytes = 8448;
 static_assert(kStaticU <= kStaticScratchBytes, "static scratch too small");
 
 // In host code this name is only a handle for the runtime, not a device address: the address the
@@ -52,15 +52,14 @@ extern "C" lml_status lora_mixed_linear_decode_static(lml_table* t, const void* 
 
     void* scratch = nullptr;
     if (scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
-    float* u = static_cast<float*>(scratch);
 
-    // The array keeps whatever the previous call left.  Nothing has to start at zero: the kernel
-    // writes every element of u that it later reads (all columns of a row's slot up to the next
-    // multiple of eight) before the grid-wide counter lets any CTA read it.
+    // The array starts as zeros (a file-scope object) and keeps whatever the previous call left: the
+    // block's own mark counter tells this launch's entries from those of earlier ones, whichever table
+    // they were for.
     int launches = 0;
     DecodeArgs a;
     a.x = x; a.W0 = W0; a.y = y; a.perm = perm; a.seg_offsets = seg_offsets; a.slot_ids = slot_ids;
-    a.u = G > 0 ? u : nullptr;
+    a.exch = static_cast<unsigned long long*>(scratch);
     a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
     cudaError_t e = launch_decode(t->arena, snap, a, stream, &launches);
     t->last_launches = launches;
