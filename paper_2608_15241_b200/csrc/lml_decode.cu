@@ -697,9 +697,11 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // launch's mark the table's last one, so that the next call on this table takes the next mark, and puts the
         // counter back to zero.
         if (sw == 0 && lane == 0) {
-            __threadfence();
+            // (no fence: this thread's own polls are complete, and what the other threads still read stays as it is
+            // until the next launch, which begins after this grid has finished)
             if (atomicAdd(sync_words + 1, 1u) == (unsigned)ncta - 1u) {
-                if (epoch == 0xffffffffu) {   // the marks start over: no entry may keep one of the last round
+                if (epoch == 0xffffffffu) {   // the marks start over: no entry may keep one of the last round (a thread that still
+                                              // reads then misses its entries, and its CTA computes u itself: same bits)
                     for (int i = 0; i < kDecExchEntries; ++i) u[i] = 0ull;
                     __threadfence();
                     sync_words[0] = 0u;
