@@ -70,8 +70,9 @@ constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 
 constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
 constexpr int kDecSegCache = 128;                 // segments whose offsets and slots are looked up in shared memory
 constexpr int kDecDotGroup = 4;                    // dot products of one row of x that a CTA takes together
-constexpr int kDecDotCols = 4096;                  // columns of a pass over the rows that a dot-product group needs
-constexpr int kDecDotBytes = (1 + kDecDotGroup) * kDecDotCols * 2;   // staging: one row of x, four rows of A
+constexpr int kDecDotCols = 3840;                  // columns of a pass over the rows that a dot-product group needs: a multiple of the 96 x 8
+                                                   // columns that the shrink threads take per step, so a thread sums the same chunks as in the register paths
+constexpr int kDecDotBytes = (1 + kDecDotGroup) * 4096 * 2;   // staging: one row of x, four rows of A (a pass), or the copies of B
 struct DecLookup {   // what the shrink warps work out about the call, in shared memory
     int seg[kDecSegCache + 1];
     int ids[kDecSegCache];
@@ -95,11 +96,13 @@ struct DecCtrl {
     uint64_t full[kDecStages];
     uint64_t empty[kDecStages];
     uint64_t ufull;      // the shrink warps' results (u, the slots, the copies of B) are in shared memory
+    uint64_t bfull;      // the bulk copies of B (whole rows of the compact arena) have landed
     int abort;
     int bad_offsets;
     int slot_of_row[16];
     int b_of_row[16];    // byte offset, in the staging buffer, of the B copy that serves this row of x; -1: read B from global memory
     uint8_t b_lead[16];  // 1: this row of x is the first with its slot (it stands for the slot's block of B)
+    uint8_t b_rows[16];  // 1: the block holds whole 32-byte rows of the compact arena, row after row (one bulk copy); 0: 16-byte chunks, chunk-major
 };
 static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control block");
 
@@ -205,11 +208,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
             }
             mbar_init(smem_u32(&ctrl->ufull), kDecShrinkWarps * 32);
+            mbar_init(smem_u32(&ctrl->bfull), 1);
             ctrl->abort = 0;
             ctrl->bad_offsets = 0;
             fence_mbar_init();
         }
-        if (lane < 16) { ctrl->slot_of_row[lane] = -1; ctrl->b_of_row[lane] = -1; ctrl->b_lead[lane] = 0; }
+        if (lane < 16) { ctrl->slot_of_row[lane] = -1; ctrl->b_of_row[lane] = -1; ctrl->b_lead[lane] = 0; ctrl->b_rows[lane] = 0; }
         asm volatile("bar.sync 4, %0;" ::"n"(kDecThreads) : "memory");   // the barriers are set up
         grid_launch_dependents();
         for (int round_begin = row_begin; round_begin < row_end && ok; round_begin += kDecRoundUnits * kDecUnitRows) {
@@ -451,13 +455,19 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                     lk->rank_of_row[lane] = rank;
                 }
                 // The expand reads, per distinct slot, the first ceil(rank / 8) 16-byte chunks of this CTA's
-                // rows of B.  Those go into the staging buffer, chunk-major ([chunk][row]: consecutive
-                // threads of the epilogue read consecutive 16 bytes), one block per distinct slot as long
-                // as they fit; the first row of x with a slot stands for the slot's block.
+                // rows of B.  Those go into the staging buffer, one block per distinct slot as long as they fit; the
+                // first row of x with a slot stands for the slot's block.  When the dot products will not need the
+                // staging buffer (at most two per CTA: see below), a slot of rank <= 16 comes in right here as one bulk
+                // copy of this CTA's rows of the compact arena (32 bytes each, row after row): a single instruction of
+                // this warp for all slots, where the chunk-by-chunk copies further down cost the shrink warps about
+                // 0.2 us per slot, ahead of their dot products.  The other blocks are chunk-major ([chunk][row]:
+                // consecutive threads of the epilogue read consecutive 16 bytes) and are filled by stage_b.
                 const unsigned same = __match_any_sync(0xffffffffu, slot);
                 const int first = __ffs(same) - 1;
                 const bool leader = rank > 0 && first == lane;
-                const int chunks = leader ? (row_end - row_begin) * ((rank + 7) >> 3) : 0;
+                const int rows_cta = row_end - row_begin;
+                const bool whole_rows = __shfl_sync(0xffffffffu, end, 15) <= 2 * ncta && rank <= kRankCompact;
+                const int chunks = leader ? rows_cta * (whole_rows ? kRankCompact / 8 : ((rank + 7) >> 3)) : 0;
                 int base = chunks;
 #pragma unroll
                 for (int o = 1; o < 16; o <<= 1) {
@@ -469,7 +479,17 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 if (lane < 16) {
                     ctrl->b_of_row[lane] = rank > 0 ? my_off : -1;
                     ctrl->b_lead[lane] = leader ? 1 : 0;
+                    ctrl->b_rows[lane] = rank > 0 && whole_rows && my_off >= 0 ? 1 : 0;
                 }
+                const bool bulk = leader && whole_rows && fits && lane < 16;
+                int bulk_bytes = bulk ? chunks * 16 : 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) bulk_bytes += __shfl_xor_sync(0xffffffffu, bulk_bytes, o);
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&ctrl->bfull), (uint32_t)bulk_bytes);
+                __syncwarp();
+                if (bulk)
+                    bulk_copy_g2s(smem_u32(dot_s) + (uint32_t)((base - chunks) * 16), arenaBc + ((size_t)slot * N + row_begin) * kRankCompact,
+                                  (uint32_t)(chunks * 16), smem_u32(&ctrl->bfull));
             }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
@@ -492,7 +512,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         auto stage_b = [&]() {
             const int rows_cta = row_end - row_begin;
             for (int t = 0; t < T; ++t) {
-                if (!ctrl->b_lead[t]) continue;
+                if (!ctrl->b_lead[t] || ctrl->b_rows[t]) continue;   // (whole rows came by bulk copy)
                 const int r8 = (lk->rank_of_row[t] + 7) >> 3;
                 // (ranks up to 16 are read from the compact copy of B: 32-byte rows back to back, not a quarter of a padded row each)
                 const bool compact = lk->rank_of_row[t] <= kRankCompact;
@@ -510,8 +530,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 }
             }
         };
-        // With single dot products the staging buffer is not needed for them: B can come in right away.
-        if (gsize == 1) stage_b();
+        // Single dot products and pairs keep their operands in registers; the staging buffer is not needed for them, and B
+        // can come in right away.  (Pairs through the staging buffer were measured 1.1 us slower per call at 12 and 16 tokens.)
+        const bool in_regs = gsize <= 2;
+        if (in_regs) stage_b();
         auto group = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
             const int d0 = g * gsize;
             t = 0;
@@ -603,6 +625,59 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
             return val;
         };
+        // Two dot products of one row of x (a group of two), operands in registers like the single one: each virtual thread
+        // sums the same chunks in the same order, so a dot product has the same bits whichever of the two computes it.
+        auto pair_regs = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
+            const int d0 = g * 2;
+            t = 0;
+            while (lk->dot_end[t] <= d0) ++t;
+            j0 = d0 - (t > 0 ? lk->dot_end[t - 1] : 0);
+            const int nreal = max(0, min(2, lk->rank_of_row[t] - j0));
+            float dot0 = 0.f, dot1 = 0.f;
+            if (nreal > 0) {
+                const __nv_bfloat16* xr = x + (size_t)t * K;
+                const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j0) * K;
+                constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
+                for (int kb = me * 8; kb < K; kb += kPer * kStride) {
+                    uint4 xv[kPer], av[kPer], bv[kPer];
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        const int k0 = kb + i * kStride;
+                        const bool ok_k = k0 < K;
+                        xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
+                        av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
+                        bv[i] = ok_k && nreal > 1 ? ldg_nc_v4(ar + K + k0) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kPer; ++i) {
+                        if (kb + i * kStride < K) {
+                            float p = 0.f, q = 0.f;
+                            p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
+                            p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
+                            p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
+                            p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
+                            q = fmaf(bf16_lo(xv[i].x), bf16_lo(bv[i].x), q); q = fmaf(bf16_hi(xv[i].x), bf16_hi(bv[i].x), q);
+                            q = fmaf(bf16_lo(xv[i].y), bf16_lo(bv[i].y), q); q = fmaf(bf16_hi(xv[i].y), bf16_hi(bv[i].y), q);
+                            q = fmaf(bf16_lo(xv[i].z), bf16_lo(bv[i].z), q); q = fmaf(bf16_hi(xv[i].z), bf16_hi(bv[i].z), q);
+                            q = fmaf(bf16_lo(xv[i].w), bf16_lo(bv[i].w), q); q = fmaf(bf16_hi(xv[i].w), bf16_hi(bv[i].w), q);
+                            dot0 += p;
+                            dot1 += q;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    dot0 += __shfl_xor_sync(0xffffffffu, dot0, o);
+                    dot1 += __shfl_xor_sync(0xffffffffu, dot1, o);
+                }
+                if (lane == 0) { lk->dot_part[0][sw] = dot0; lk->dot_part[1][sw] = dot1; }
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
+#pragma unroll
+            for (int i = 0; i < kDecDotGroup; ++i)
+                val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_s[ctrl->slot_of_row[t]] : 0.f;
+            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
+        };
         const long long t_shrink = clock64();
         const unsigned epoch = lk->epoch;
         if (gsize == 1) {
@@ -618,13 +693,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         for (int g = cta; g < ngroups; g += ncta) {
             float val[kDecDotGroup];
             int t, j0;
-            group(g, val, t, j0);
+            if (in_regs) pair_regs(g, val, t, j0); else group(g, val, t, j0);
             if (me == 0) {
                 for (int i = 0; i < gsize; ++i) st_relaxed_gpu_b64(u + t * kRankPad + j0 + i, pack_u(val[i], epoch));
                 red_relaxed_gpu_add(sync_words + 2, (unsigned)gsize);
             }
         }
-        if (gsize > 1) stage_b();   // the staging buffer is free now (the groups end with a barrier of these warps)
+        if (!in_regs) stage_b();   // the staging buffer is free now (the groups end with a barrier of these warps)
         // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
         // other CTAs' shares normally arrive within microseconds and are then read from global memory.
         // But this CTA never depends on them: nothing guarantees that the whole grid is resident at once
@@ -677,6 +752,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 const float val = single(d, t, j);
                 if (me == 0) u_s[t * kRankPad + j] = val;
             }
+        } else if (in_regs) {
+            for (int g = 0; g < ngroups; ++g) {
+                float val[kDecDotGroup];
+                int t, j0;
+                pair_regs(g, val, t, j0);
+                if (me == 0) for (int i = 0; i < gsize; ++i) u_s[t * kRankPad + j0 + i] = val[i];
+            }
         } else {
             cp_async_wait_all();   // the copies of B must not land on top of the groups' operands
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
@@ -689,6 +771,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             stage_b();   // the groups went through the staging buffer: bring B in once more
         }
         cp_async_wait_all();   // this thread's chunks of B have landed
+        mbar_wait_warp(smem_u32(&ctrl->bfull), 0u, abort);   // and so have the bulk copies (on a give-up the flag is up: the call reports it)
         // tell the consumers that u_s, slot_of_row, bad_offsets and the copies of B are final (each thread
         // releases what it wrote)
         if (kPutOff) mbar_arrive(smem_u32(&ctrl->ufull));   // (the consumers can test this one without waiting)
@@ -837,7 +920,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                                           ? reinterpret_cast<const uint4*>(arenaBc + ((size_t)slot * N + n) * kRankCompact)
                                           : reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
                     const int bb = ctrl->b_of_row[t];
-                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + bb) + (n - row_begin);
+                    const bool whole_rows = ctrl->b_rows[t] != 0;
+                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + bb) + (whole_rows ? (n - row_begin) * (kRankCompact / 8) : n - row_begin);
+                    const int cstep = whole_rows ? 1 : rows_cta;
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
                     auto fma8 = [&](const uint4& b, int c) {
@@ -848,7 +933,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                         d = fmaf(u1.z, bf16_lo(b.w), d); d = fmaf(u1.w, bf16_hi(b.w), d);
                     };
                     if (bb >= 0) {   // (two loops: with a select inside one loop the global loads no longer overlap)
-                        for (int c = 0; c < r8; ++c) fma8(bs[c * rows_cta], c);
+                        for (int c = 0; c < r8; ++c) fma8(bs[c * cstep], c);
                     } else {
                         for (int c = 0; c < r8; ++c) fma8(ldg_nc_v4(bp + c), c);
                     }
