@@ -30,7 +30,10 @@ cases = [wl.ragged(T=8, d_in=264, d_out=136, ranks=(4, 16, 1, 33, 64)),
          # CTAs with several rounds of rows: the expand of early rounds is put off until u is there
          wl.ragged(T=8, d_in=264, d_out=5200, ranks=(4, 16, 1, 33, 64)),
          wl.ragged(T=16, d_in=264, d_out=10360, ranks=(8, 16, 16, 64, 2), shuffled=True),
-         wl.ragged(T=3, d_in=4104, d_out=16000, ranks=(16, 16, 16, 16, 16))]
+         wl.ragged(T=3, d_in=4104, d_out=16000, ranks=(16, 16, 16, 16, 16)),
+         # rows of x wider than one pass through the staging buffer: pairs in registers, staged groups of four
+         wl.ragged(T=16, d_in=4104, d_out=512, ranks=(16, 16, 16, 16, 16)),
+         wl.ragged(T=16, d_in=8200, d_out=264, ranks=(64, 64, 33, 16, 64))]
 for i, w in enumerate(cases):
     site = Site(w)
     y, flags = site.run()
@@ -61,6 +64,6 @@ def _run(tmp_path, name, patience):
 def test_self_sufficient_path_matches_normal_path(tmp_path):
     normal = _run(tmp_path, "normal.npz", None)
     alone = _run(tmp_path, "alone.npz", 0)
-    assert sorted(normal.files) == sorted(alone.files) and len(normal.files) == 7
+    assert sorted(normal.files) == sorted(alone.files) and len(normal.files) == 9
     for k in normal.files:
         assert np.array_equal(normal[k], alone[k]), k

@@ -106,6 +106,19 @@ def test_wide_projections_take_one_launch(T):
     _check(out, sep, flags, x, W, ents, tok)
 
 
+@pytest.mark.parametrize("T,ranks", [(8, (16, 16, 16, 16)), (16, (16, 8, 16, 4)), (16, (64, 33, 64, 16))])
+def test_rows_of_x_wider_than_a_staged_pass_keep_their_bits(T, ranks):
+    """d_in beyond the width of one pass through the staging buffer.  In the one-launch call a projection has a
+    share of the SMs only, so its dot products are dealt out in larger groups than in a call of its own (singles
+    against pairs, pairs against staged groups of four): whatever the grouping, a dot product is summed in the same
+    order, and the outputs are equal bit for bit."""
+    K, Ns = 7944, (520, 264)
+    scales = [(2.0, 0.5, 1.0, 4.0), (1.0, 2.0, 0.25, 3.0)]
+    x, W, ents, tok = _case(300 + T + ranks[0], K, Ns, [ranks, ranks], scales, T, none_every=7)
+    out, sep, flags = _run_multi(K, Ns, x, W, ents, tok)
+    _check(out, sep, flags, x, W, ents, tok)
+
+
 @pytest.mark.parametrize("T", [2, 16])
 def test_four_projections_some_with_very_few_rows(T):
     """LML_MAX_PROJECTIONS projections, two of them with fewer pairs of rows than their share of the SMs."""
