@@ -295,11 +295,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     // first epilogue.
     unsigned int* sync_words = pj.sync_words;
     const bool shrinker = warp > kDecConsumers;
-    // Segments form: the lookup's loads (several small arrays) go first through the load/store path (see below).  With
-    // one slot id per row the lookup is a single load per row, and the order is not worth its price: 0.9 us on a
-    // batch in which no token is bound to an adapter.
-    if (consumer && G > 0 && token_slots == nullptr)
-        asm volatile("bar.sync 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
+    // (The consumers do not hold their loads of x back until the lookup's few loads are on their way: that order was
+    // worth 0.2 us once, and costs 0.1 - 0.4 us per call since the shrink warps no longer wait for a fence.)
     if (shrinker && G > 0) {
         const int sw = warp - kDecConsumers - 1;
         if (sw == 1) {
@@ -351,9 +348,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         if (sw == 0) {
             // One memory round trip for everything the lookup needs: the segment arrays go to shared
             // memory (all loads issued before the first is used), the search then runs there.  Calls
-            // with more segments than the cache holds search in global memory instead.  The consumer
-            // warps hold their (many) loads of x back until these few are on their way, and while they
-            // are, the slots' ranks and scales move from the kernel parameters to shared memory:
+            // with more segments than the cache holds search in global memory instead.  While the loads
+            // are on their way, the slots' ranks and scales move from the kernel parameters to shared memory:
             // indexed reads of parameters are slow the first time, and everything later reads the copy.
             const bool by_token = token_slots != nullptr;   // one slot id per row of x instead of segments
             const bool cached = !by_token && G <= kDecSegCache;
@@ -374,7 +370,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 // the ids are adapter ids: the table's device map names the serving slot (-2: none, flagged below)
                 if (adapter_map) my_token_slot = resolve_adapter(snap, adapter_map, my_token_slot);
             }
-            if (!by_token) asm volatile("bar.arrive 6, %0;" ::"n"((kDecConsumers + 1) * 32) : "memory");
             for (int sl = lane; sl < kMaxSlots; sl += 32)   // ranks only: the scales (four more lines) come by another warp
                 lk->rank_s[sl] = sl < snap.max_slots ? snap.rank[sl] : (uint8_t)0;
             if (lane == 0) lk->u_complete = 1;
