@@ -21,8 +21,10 @@
 //                       shared memory, or from one slot id per row), then compute this CTA's share of
 //                       u[row][j] = scale_s * sum_k x[row][k] A_s[j][k] (fp32).  The dot products are dealt
 //                       out over the whole grid in groups of 1, 2 or 4 columns of one row; a group's
-//                       operands are staged in shared memory by asynchronous copies (one memory round
-//                       trip per group; single dot products stay in registers).  Each result goes to
+//                       operands are all in flight at once, in registers (one memory round trip per
+//                       4608 columns).  This CTA's rows of B of the slots that the call names come
+//                       into shared memory meanwhile (rank <= 16: one bulk copy per slot, issued by
+//                       the lookup warp).  Each result goes to
 //                       the table's exchange block as one 64-bit word, the value beside this launch's
 //                       mark, followed by a plain add on a grid-wide counter (no fence anywhere); the
 //                       warps wait for the counter, then read the entries, taking only those that carry
@@ -45,6 +47,8 @@
 #include <cstdlib>
 #include "lml_internal.cuh"
 #include "lml_ptx_sm100.cuh"
+#include <type_traits>
+
 #include "lml_decode_common.cuh"
 
 namespace lml {
@@ -70,9 +74,7 @@ constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 
 constexpr int kDecUBytes = 16 * kRankPad * 4;     // shared-memory copy of u for the epilogue
 constexpr int kDecSegCache = 128;                 // segments whose offsets and slots are looked up in shared memory
 constexpr int kDecDotGroup = 4;                    // dot products of one row of x that a CTA takes together
-constexpr int kDecDotCols = 3840;                  // columns of a pass over the rows that a dot-product group needs: a multiple of the 96 x 8
-                                                   // columns that the shrink threads take per step, so a thread sums the same chunks as in the register paths
-constexpr int kDecDotBytes = (1 + kDecDotGroup) * 4096 * 2;   // staging: one row of x, four rows of A (a pass), or the copies of B
+constexpr int kDecDotBytes = 40960;                // staging buffer: this CTA's rows of B of the slots that the call names
 struct DecLookup {   // what the shrink warps work out about the call, in shared memory
     int seg[kDecSegCache + 1];
     int ids[kDecSegCache];
@@ -461,7 +463,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 const int first = __ffs(same) - 1;
                 const bool leader = rank > 0 && first == lane;
                 const int rows_cta = row_end - row_begin;
-                const bool whole_rows = __shfl_sync(0xffffffffu, end, 15) <= 2 * ncta && rank <= kRankCompact;
+                const bool whole_rows = rank <= kRankCompact;
                 const int chunks = leader ? rows_cta * (whole_rows ? kRankCompact / 8 : ((rank + 7) >> 3)) : 0;
                 int base = chunks;
 #pragma unroll
@@ -492,10 +494,11 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // shares the row of x): group g belongs to CTA g mod grid.  A dot product's arithmetic is fixed, whoever
         // computes it: 96 "virtual threads" (the three shrink warps) each sum the 8-column chunks m, m + 96,
         // m + 192, ... of the row in order, each warp adds its threads' sums up with the butterfly, and the
-        // result is (w0 + w1) + w2 times the scale.  The operands of a whole group are brought into shared
-        // memory with asynchronous 16-byte copies, all in flight at once (registers would hold a fraction of
-        // them), so a group costs one memory round trip.  A result is published as one 64-bit store (value and this
-        // launch's mark) and a relaxed add on the grid-wide counter: nobody waits for a fence.
+        // result is (w0 + w1) + w2 times the scale.  The operands of a whole group (up to six 16-byte chunks of x
+        // and of each row of A per thread and step: 4608 columns) are in flight at once, in registers, so a group costs
+        // one memory round trip per step.  (Groups staged in shared memory by asynchronous copies were measured slower:
+        // 1.1 us per call for pairs at 12 and 16 tokens, 0.6 - 2.3 us for groups of four.)  A result is published as one
+        // 64-bit store (value and this launch's mark) and a relaxed add on the grid-wide counter: nobody waits for a fence.
         const int total = lk->dot_end[15];
         // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
         // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
@@ -525,61 +528,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 }
             }
         };
-        // Single dot products and pairs keep their operands in registers; the staging buffer is not needed for them, and B
-        // can come in right away.  (Pairs through the staging buffer were measured 1.1 us slower per call at 12 and 16 tokens.)
-        const bool in_regs = gsize <= 2;
-        if (in_regs) stage_b();
-        auto group = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
-            const int d0 = g * gsize;
-            t = 0;
-            while (lk->dot_end[t] <= d0) ++t;   // which row do the group's dot products fall into
-            j0 = d0 - (t > 0 ? lk->dot_end[t - 1] : 0);
-            const int nreal = max(0, min(gsize, lk->rank_of_row[t] - j0));   // the rest are padding columns: zero
-            float acc[kDecDotGroup];
-#pragma unroll
-            for (int i = 0; i < kDecDotGroup; ++i) acc[i] = 0.f;
-            const __nv_bfloat16* xr = x + (size_t)t * K;
-            const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j0) * K;
-            for (int k_pass = 0; k_pass < K && nreal > 0; k_pass += kDecDotCols) {
-                const int chunks = min(kDecDotCols, K - k_pass) / 8;
-                for (int c = me; c < chunks; c += kDecShrinkWarps * 32) {
-                    cp_async_16(smem_u32(dot_s) + c * 16, xr + k_pass + c * 8);
-                    for (int i = 0; i < nreal; ++i)
-                        cp_async_16(smem_u32(dot_s) + (1 + i) * kDecDotCols * 2 + c * 16, ar + (size_t)i * K + k_pass + c * 8);
-                }
-                cp_async_wait_all();
-                asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // everybody's copies have landed
-                for (int c = me; c < chunks; c += kDecShrinkWarps * 32) {
-                    const uint4 xv = *reinterpret_cast<const uint4*>(dot_s + c * 16);
-#pragma unroll
-                    for (int i = 0; i < kDecDotGroup; ++i) {
-                        if (i < nreal) {
-                            const uint4 av = *reinterpret_cast<const uint4*>(dot_s + (1 + i) * kDecDotCols * 2 + c * 16);
-                            float p = 0.f;
-                            p = fmaf(bf16_lo(xv.x), bf16_lo(av.x), p); p = fmaf(bf16_hi(xv.x), bf16_hi(av.x), p);
-                            p = fmaf(bf16_lo(xv.y), bf16_lo(av.y), p); p = fmaf(bf16_hi(xv.y), bf16_hi(av.y), p);
-                            p = fmaf(bf16_lo(xv.z), bf16_lo(av.z), p); p = fmaf(bf16_hi(xv.z), bf16_hi(av.z), p);
-                            p = fmaf(bf16_lo(xv.w), bf16_lo(av.w), p); p = fmaf(bf16_hi(xv.w), bf16_hi(av.w), p);
-                            acc[i] += p;
-                        }
-                    }
-                }
-                asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the staging buffer is free again
-            }
-#pragma unroll
-            for (int i = 0; i < kDecDotGroup; ++i) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], o);
-                if (lane == 0) lk->dot_part[i][sw] = acc[i];
-            }
-            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
-#pragma unroll
-            for (int i = 0; i < kDecDotGroup; ++i)
-                val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_s[ctrl->slot_of_row[t]] : 0.f;
-            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
-        };
-        // A single dot product per CTA (few tokens, rank 16: the usual decode call) skips the staging: each
-        // virtual thread keeps its six chunks of x and of A in registers, same order, same sums.
+        stage_b();   // (the staging buffer is theirs alone: the dot products keep their operands in registers)
+        // A single dot product per CTA (few tokens, rank 16: the usual decode call).
         auto single = [&](int d, int& t, int& j) {
             t = 0;
             while (lk->dot_end[t] <= d) ++t;
@@ -620,58 +570,64 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
             return val;
         };
-        // Two dot products of one row of x (a group of two), operands in registers like the single one: each virtual thread
-        // sums the same chunks in the same order, so a dot product has the same bits whichever of the two computes it.
-        auto pair_regs = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
-            const int d0 = g * 2;
+        // A group of two or four dot products of one row of x, operands in registers like the single one: each virtual
+        // thread sums the same chunks in the same order, so a dot product has the same bits whichever path computes it.
+        auto regs_group = [&](auto ng_tag, int g, float (&val)[kDecDotGroup], int& t, int& j0) {
+            constexpr int NG = decltype(ng_tag)::value;
+            const int d0 = g * NG;
             t = 0;
             while (lk->dot_end[t] <= d0) ++t;
             j0 = d0 - (t > 0 ? lk->dot_end[t - 1] : 0);
-            const int nreal = max(0, min(2, lk->rank_of_row[t] - j0));
-            float dot0 = 0.f, dot1 = 0.f;
+            const int nreal = max(0, min(NG, lk->rank_of_row[t] - j0));
+            float dot[NG];
+#pragma unroll
+            for (int d = 0; d < NG; ++d) dot[d] = 0.f;
             if (nreal > 0) {
                 const __nv_bfloat16* xr = x + (size_t)t * K;
                 const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j0) * K;
                 constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
                 for (int kb = me * 8; kb < K; kb += kPer * kStride) {
-                    uint4 xv[kPer], av[kPer], bv[kPer];
+                    uint4 xv[kPer], av[NG][kPer];
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
                         const int k0 = kb + i * kStride;
                         const bool ok_k = k0 < K;
                         xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
-                        av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
-                        bv[i] = ok_k && nreal > 1 ? ldg_nc_v4(ar + K + k0) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int d = 0; d < NG; ++d)
+                            av[d][i] = ok_k && d < nreal ? ldg_nc_v4(ar + (size_t)d * K + k0) : make_uint4(0, 0, 0, 0);
                     }
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
                         if (kb + i * kStride < K) {
-                            float p = 0.f, q = 0.f;
-                            p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[i].x), p);
-                            p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[i].y), p);
-                            p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[i].z), p);
-                            p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[i].w), p);
-                            q = fmaf(bf16_lo(xv[i].x), bf16_lo(bv[i].x), q); q = fmaf(bf16_hi(xv[i].x), bf16_hi(bv[i].x), q);
-                            q = fmaf(bf16_lo(xv[i].y), bf16_lo(bv[i].y), q); q = fmaf(bf16_hi(xv[i].y), bf16_hi(bv[i].y), q);
-                            q = fmaf(bf16_lo(xv[i].z), bf16_lo(bv[i].z), q); q = fmaf(bf16_hi(xv[i].z), bf16_hi(bv[i].z), q);
-                            q = fmaf(bf16_lo(xv[i].w), bf16_lo(bv[i].w), q); q = fmaf(bf16_hi(xv[i].w), bf16_hi(bv[i].w), q);
-                            dot0 += p;
-                            dot1 += q;
+#pragma unroll
+                            for (int d = 0; d < NG; ++d) {
+                                float p = 0.f;
+                                p = fmaf(bf16_lo(xv[i].x), bf16_lo(av[d][i].x), p); p = fmaf(bf16_hi(xv[i].x), bf16_hi(av[d][i].x), p);
+                                p = fmaf(bf16_lo(xv[i].y), bf16_lo(av[d][i].y), p); p = fmaf(bf16_hi(xv[i].y), bf16_hi(av[d][i].y), p);
+                                p = fmaf(bf16_lo(xv[i].z), bf16_lo(av[d][i].z), p); p = fmaf(bf16_hi(xv[i].z), bf16_hi(av[d][i].z), p);
+                                p = fmaf(bf16_lo(xv[i].w), bf16_lo(av[d][i].w), p); p = fmaf(bf16_hi(xv[i].w), bf16_hi(av[d][i].w), p);
+                                dot[d] += p;
+                            }
                         }
                     }
                 }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    dot0 += __shfl_xor_sync(0xffffffffu, dot0, o);
-                    dot1 += __shfl_xor_sync(0xffffffffu, dot1, o);
+                for (int d = 0; d < NG; ++d) {
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) dot[d] += __shfl_xor_sync(0xffffffffu, dot[d], o);
+                    if (lane == 0) lk->dot_part[d][sw] = dot[d];
                 }
-                if (lane == 0) { lk->dot_part[0][sw] = dot0; lk->dot_part[1][sw] = dot1; }
             }
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
 #pragma unroll
             for (int i = 0; i < kDecDotGroup; ++i)
                 val[i] = i < nreal ? ((lk->dot_part[i][0] + lk->dot_part[i][1]) + lk->dot_part[i][2]) * lk->scale_s[ctrl->slot_of_row[t]] : 0.f;
             asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // dot_part is free again
+        };
+        auto group = [&](int g, float (&val)[kDecDotGroup], int& t, int& j0) {
+            if (gsize == 4) regs_group(std::integral_constant<int, 4>{}, g, val, t, j0);
+            else regs_group(std::integral_constant<int, 2>{}, g, val, t, j0);
         };
         const long long t_shrink = clock64();
         const unsigned epoch = lk->epoch;
@@ -688,13 +644,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         for (int g = cta; g < ngroups; g += ncta) {
             float val[kDecDotGroup];
             int t, j0;
-            if (in_regs) pair_regs(g, val, t, j0); else group(g, val, t, j0);
+            group(g, val, t, j0);
             if (me == 0) {
                 for (int i = 0; i < gsize; ++i) st_relaxed_gpu_b64(u + t * kRankPad + j0 + i, pack_u(val[i], epoch));
                 red_relaxed_gpu_add(sync_words + 2, (unsigned)gsize);
             }
         }
-        if (!in_regs) stage_b();   // the staging buffer is free now (the groups end with a barrier of these warps)
         // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
         // other CTAs' shares normally arrive within microseconds and are then read from global memory.
         // But this CTA never depends on them: nothing guarantees that the whole grid is resident at once
@@ -741,29 +696,19 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
         if (lk->u_complete) {
             // (u_s holds every column that the expand reads)
-        } else if (gsize == 1) {   // (the staging buffer may hold B rows: stay in registers)
+        } else if (gsize == 1) {
             for (int d = 0; d < total; ++d) {
                 int t, j;
                 const float val = single(d, t, j);
                 if (me == 0) u_s[t * kRankPad + j] = val;
             }
-        } else if (in_regs) {
-            for (int g = 0; g < ngroups; ++g) {
-                float val[kDecDotGroup];
-                int t, j0;
-                pair_regs(g, val, t, j0);
-                if (me == 0) for (int i = 0; i < gsize; ++i) u_s[t * kRankPad + j0 + i] = val[i];
-            }
         } else {
-            cp_async_wait_all();   // the copies of B must not land on top of the groups' operands
-            asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");
             for (int g = 0; g < ngroups; ++g) {
                 float val[kDecDotGroup];
                 int t, j0;
                 group(g, val, t, j0);
                 if (me == 0) for (int i = 0; i < gsize; ++i) u_s[t * kRankPad + j0 + i] = val[i];
             }
-            stage_b();   // the groups went through the staging buffer: bring B in once more
         }
         cp_async_wait_all();   // this thread's chunks of B have landed
         mbar_wait_warp(smem_u32(&ctrl->bfull), 0u, abort);   // and so have the bulk copies (on a give-up the flag is up: the call reports it)
