@@ -624,11 +624,11 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
         if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
         return LML_OK;
     }
-    // (measured on B200 against the GEMM path: two blocks win on every layer of a 7B-class model, 15 us against 29 us
-    // on 4096 x 4096 and 33 against 39 - 45 us on the MLP's; three win on the 4096 x 4096 layers only, 24 against 29 us;
-    // four or more lose: every block's CTAs take all of W0 in from L2)
+    // (measured on B200 against the GEMM path: two blocks win on every layer of a 7B-class model, 14 us against 29 us
+    // on 4096 x 4096 and 33 against 39 - 45 us on the MLP's; three and four win on the 4096 x 4096 layers only, 21 and
+    // 25 against 29 - 30 us; more lose: every block's CTAs take all of W0 in from L2)
     const int block_limit = t->dec_block_tokens >= 0 ? t->dec_block_tokens
-                                                     : ((long long)t->d_in * t->d_out <= (1ll << 24) ? 3 : 2) * kDecodeMaxT;
+                                                     : ((long long)t->d_in * t->d_out <= (1ll << 24) ? 4 : 2) * kDecodeMaxT;
     if (T <= block_limit) {
         // A few blocks of 16 tokens: one launch of the decode kernel with the blocks as its parts, an equal share of the
         // CTAs each.  The shares walk W0 together, so a line leaves HBM once and the other readers find it in L2; no

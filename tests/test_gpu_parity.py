@@ -211,7 +211,7 @@ def test_layer_sweep_cells_every_element(proj, T):
 
 # a few blocks of 16 tokens through the token form of the call (one launch of the decode kernel, a share of its CTAs per
 # block): every element against the oracle, output and workspace between canary bands
-@pytest.mark.parametrize("proj,T", [("q", 17), ("q", 32), ("q", 48), ("gate", 32), ("down", 31)])
+@pytest.mark.parametrize("proj,T", [("q", 17), ("q", 32), ("q", 48), ("q", 64), ("gate", 32), ("down", 31)])
 def test_layer_sweep_shapes_at_a_few_blocks_of_tokens(proj, T):
     import torch
     from gpu_util import Guarded

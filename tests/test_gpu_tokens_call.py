@@ -28,7 +28,7 @@ def _table(K, N, ranks, seed):
 
 
 @pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384),
-                                   (17, 264, 136), (24, 1032, 520), (32, 1032, 16400), (33, 1032, 16400), (48, 520, 264), (49, 520, 264), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
+                                   (17, 264, 136), (24, 1032, 520), (32, 1032, 16400), (33, 1032, 16400), (48, 520, 264), (64, 520, 264), (65, 520, 264), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
                                    (200, 1536, 520)])
 def test_tokens_call_equals_segment_then_layer(T, K, N):
     import torch
@@ -46,7 +46,7 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
     y_two = to_bits(tbl.lora_mixed_linear(x, W, so, ids, perm=perm))
     torch.cuda.synchronize()
     assert tbl.device_status() == 0
-    blocks = 16 < T <= (48 if K * N <= 1 << 24 else 32)
+    blocks = 16 < T <= (64 if K * N <= 1 << 24 else 32)
     if blocks:
         # a few blocks of 16 tokens: one launch of the decode kernel, every block's rows exactly those of a decode call
         # on that block alone; against the two-call form (the GEMM path) equal to the last place of bf16
