@@ -86,6 +86,10 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
     int u_complete;
     unsigned epoch;         // this launch's mark on the entries of u
     int pad[3];
+    // what the expand needs to know about a row of x, in one word: bit 31 the row has an adapter; bits 0-7 its slot;
+    // bits 8-11 ceil(rank / 8); bit 12 rank <= 16 (the compact arena serves it); bit 13 its block of B is in the staging
+    // buffer, at 16 x bits 16-27 bytes
+    unsigned row_info[16];
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
 constexpr int kDecDeferBytes = 2048;   // base sums of rounds whose expand is put off: 16 x 32 or 2 x (8 x 32) fp32
@@ -477,6 +481,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                     ctrl->b_of_row[lane] = rank > 0 ? my_off : -1;
                     ctrl->b_lead[lane] = leader ? 1 : 0;
                     ctrl->b_rows[lane] = rank > 0 && whole_rows && my_off >= 0 ? 1 : 0;
+                    lk->row_info[lane] = rank > 0 ? (0x80000000u | (unsigned)slot | ((unsigned)((rank + 7) >> 3) << 8) | (whole_rows ? 1u << 12 : 0u) |
+                                                     (my_off >= 0 ? (1u << 13) | ((unsigned)(my_off >> 4) << 16) : 0u))
+                                                  : 0u;
                 }
                 const bool bulk = leader && whole_rows && fits && lane < 16;
                 int bulk_bytes = bulk ? chunks * 16 : 0;
@@ -831,6 +838,29 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         // before this one has ended everywhere.  A CTA with several rounds does not wait for it: until u
         // has arrived, each thread keeps the base sums of its elements of up to kDecDefer rounds in
         // shared memory (the same thread finishes them later), and only then, or in its last round, it waits.
+        // This thread's elements of the round (token t, row j of the round) and their base sums, before any wait for u.
+        float base_v[kDecPerThread];
+        int el_t[kDecPerThread], el_j[kDecPerThread];
+        if (consumer && ok) {
+            const int per_token = nunits * kDecUnitRows;
+#pragma unroll
+            for (int i = 0; i < kDecPerThread; ++i) {
+                const int e = tid + i * kDecConsumers * 32;   // consecutive threads: consecutive rows
+                base_v[i] = 0.f;
+                el_t[i] = -1;
+                el_j[i] = 0;
+                if (e < T * per_token) {
+                    const int t = e / per_token, j = e % per_token;
+                    const int un = j / kDecUnitRows, r = j % kDecUnitRows;
+                    float v = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
+                    base_v[i] = v;
+                    el_t[i] = t;
+                    el_j[i] = j;
+                }
+            }
+        }
         if (!kPutOff) {
             if (consumer && G > 0 && !u_ready) {   // first epilogue: the shrink warps have staged u in shared memory
                 asm volatile("bar.sync 3, %0;" ::"n"((kDecConsumers + kDecShrinkWarps) * 32) : "memory");
@@ -853,48 +883,44 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             const int rows_cta = row_end - row_begin;
             // y[t][n] = base sum + u_t . B_slot[n] (the first ceil(rank / 8) chunks of the row), rounded once
             auto finish = [&](int t, int n, float v) {
-                const int slot = lora ? ctrl->slot_of_row[t] : -1;
-                if (slot >= 0) {
-                    const int r8 = (lk->rank_of_row[t] + 7) >> 3;
-                    const uint4* bp = lk->rank_of_row[t] <= kRankCompact
-                                          ? reinterpret_cast<const uint4*>(arenaBc + ((size_t)slot * N + n) * kRankCompact)
-                                          : reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
-                    const int bb = ctrl->b_of_row[t];
-                    const bool whole_rows = ctrl->b_rows[t] != 0;
-                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + bb) + (whole_rows ? (n - row_begin) * (kRankCompact / 8) : n - row_begin);
-                    const int cstep = whole_rows ? 1 : rows_cta;
+                const unsigned info = lora ? lk->row_info[t] : 0u;
+                if (info >> 31) {
+                    const int slot = (int)(info & 0xffu), r8 = (int)((info >> 8) & 0xfu);
+                    const bool compact = (info >> 12 & 1u) != 0, staged = (info >> 13 & 1u) != 0;
                     const float4* up = reinterpret_cast<const float4*>(u_s + t * kRankPad);
                     float d = 0.f;
-                    auto fma8 = [&](const uint4& b, int c) {
-                        const float4 u0 = up[2 * c], u1 = up[2 * c + 1];
+                    auto fma8 = [&](const uint4& b, const float4& u0, const float4& u1) {
                         d = fmaf(u0.x, bf16_lo(b.x), d); d = fmaf(u0.y, bf16_hi(b.x), d);
                         d = fmaf(u0.z, bf16_lo(b.y), d); d = fmaf(u0.w, bf16_hi(b.y), d);
                         d = fmaf(u1.x, bf16_lo(b.z), d); d = fmaf(u1.y, bf16_hi(b.z), d);
                         d = fmaf(u1.z, bf16_lo(b.w), d); d = fmaf(u1.w, bf16_hi(b.w), d);
                     };
-                    if (bb >= 0) {   // (two loops: with a select inside one loop the global loads no longer overlap)
-                        for (int c = 0; c < r8; ++c) fma8(bs[c * cstep], c);
+                    const uint4* bs = reinterpret_cast<const uint4*>(dot_s + ((info >> 16) & 0xfffu) * 16u);
+                    if (staged && compact) {
+                        // the usual case (whole 32-byte rows by bulk copy): everything is asked for at once, then summed in order
+                        const uint4* br = bs + (n - row_begin) * (kRankCompact / 8);
+                        const bool two = r8 > 1;
+                        const uint4 b0 = br[0];
+                        const uint4 b1 = two ? br[1] : make_uint4(0, 0, 0, 0);
+                        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float4 u0 = up[0], u1 = up[1], u2 = two ? up[2] : z, u3 = two ? up[3] : z;
+                        fma8(b0, u0, u1);
+                        if (two) fma8(b1, u2, u3);
+                    } else if (staged) {   // (two loops: with a select inside one loop the global loads no longer overlap)
+                        for (int c = 0; c < r8; ++c) fma8(bs[c * rows_cta + (n - row_begin)], up[2 * c], up[2 * c + 1]);
                     } else {
-                        for (int c = 0; c < r8; ++c) fma8(ldg_nc_v4(bp + c), c);
+                        const uint4* bp = compact ? reinterpret_cast<const uint4*>(arenaBc + ((size_t)slot * N + n) * kRankCompact)
+                                                  : reinterpret_cast<const uint4*>(arenaB + ((size_t)slot * N + n) * kRankPad);
+                        for (int c = 0; c < r8; ++c) fma8(ldg_nc_v4(bp + c), up[2 * c], up[2 * c + 1]);
                     }
                     v += d;
                 }
                 y[(size_t)t * N + n] = __float2bfloat16_rn(v);
             };
-            const int per_token = nunits * kDecUnitRows;
             if (kPutOff && G > 0 && !u_ready) {   // put this round off (a full round: the last one waits)
 #pragma unroll
-                for (int i = 0; i < kDecPerThread; ++i) {
-                    const int e = tid + i * kDecConsumers * 32;
-                    if (e < T * per_token) {
-                        const int t = e / per_token, j = e % per_token;
-                        const int un = j / kDecUnitRows, r = j % kDecUnitRows;
-                        float v = 0.f;
-#pragma unroll
-                        for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
-                        defer_s[ndefer * (kDecPerThread * kDecConsumers * 32) + e] = v;   // read back by this very thread
-                    }
-                }
+                for (int i = 0; i < kDecPerThread; ++i)
+                    if (el_t[i] >= 0) defer_s[ndefer * (kDecPerThread * kDecConsumers * 32) + tid + i * kDecConsumers * 32] = base_v[i];   // read back by this very thread
                 ++ndefer;
             } else {
                 if (kPutOff && ndefer > 0) {   // the rounds that were put off
@@ -905,15 +931,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                                    defer_s[dd * (kDecPerThread * kDecConsumers * 32) + e]);
                     ndefer = 0;
                 }
-                for (int e = tid; e < T * per_token; e += kDecConsumers * 32) {
-                    const int t = e / per_token, j = e % per_token;   // consecutive threads: consecutive n
-                    if (j >= round_rows) continue;
-                    const int un = j / kDecUnitRows, r = j % kDecUnitRows;
-                    float v = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kDecConsumers; ++w) v += slots[(un * kDecConsumers + w) * kDecSlotFloats + t * 8 + r];
-                    finish(t, round_begin + j, v);
-                }
+                for (int i = 0; i < kDecPerThread; ++i)
+                    if (el_t[i] >= 0 && el_j[i] < round_rows) finish(el_t[i], round_begin + el_j[i], base_v[i]);
             }
         }
         if (consumer) asm volatile("bar.sync 1, %0;" ::"n"(kDecConsumers * 32) : "memory");   // slots are free for the next round
