@@ -29,7 +29,7 @@
 //                       mark, followed by a plain add on a grid-wide counter (no fence anywhere); the
 //                       warps wait for the counter, then read the entries, taking only those that carry
 //                       the mark, and stage all of u in shared memory.  When the table's live
-//                       adapters are few, their rows of A are asked into L2 at kernel entry, ahead of
+//                       adapters are very few, their rows of A are asked into L2 at kernel entry, ahead of
 //                       the weight stream.  The consumers meet the shrink warps once, at their first
 //                       epilogue.  No CTA depends on the others being resident: after a bounded wait
 //                       for their shares it computes all of u itself (same arithmetic, same bits).  So
@@ -307,10 +307,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
         const int sw = warp - kDecConsumers - 1;
         if (sw == 1) {
             // Which adapters this call names is known only after the lookup below, a memory round trip
-            // from now, and their rows of A are cold: with W0 streaming at full rate a read from HBM
-            // then takes several microseconds.  So when the table's live adapters are few (their rows
-            // of A together at most a sixteenth of W0), all of them are asked into L2 right now,
-            // ahead of the weight stream, a row or two per CTA; the dot products below find them there.
+            // from now, and their rows of A are cold.  When the table's live adapters are very few (their rows
+            // of A together at most a 64th of W0), all of them are asked into L2 right now, ahead of the weight
+            // stream, a row or two per CTA.  (With a 16th as the limit this was worth 0.3 us while the chain behind
+            // the dot products was longer; now it changes nothing on a call that uses the adapters and costs
+            // 0.1 - 0.2 us on one that does not, hence the narrow rule.  Taking the block out altogether was measured
+            // too: the base-only call, which never runs it, came out 0.13 us slower, by code generation alone.)
             int rows_before = 0, my_rank[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -326,7 +328,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
             }
             const int total0 = __shfl_sync(0xffffffffu, incl0, 31);
             const int live_rows = total0 + __shfl_sync(0xffffffffu, incl1, 31);
-            if ((long long)live_rows * K * 16 <= (long long)N * K) {
+            if ((long long)live_rows * K * 64 <= (long long)N * K) {
                 // lane L of this CTA takes live row blockIdx + L * grid
                 const int i = cta + lane * ncta;
                 // find the slot holding live row i: the first whose inclusive count exceeds i
