@@ -272,13 +272,15 @@ lml_status lora_mixed_linear_backward_adapters(lml_table* t, lml_table* t_T, con
  * per row of x or -1; ids outside [-1, max_slots) or naming a free slot count as -1 and set
  * LML_FLAG_BAD_SLOT, exactly as in lml_segment_tokens.  x, W0, y as in lora_mixed_linear.
  * T <= 16: one launch; the decode kernel treats every row on its own and reads the ids itself, no
- * grouping is computed.  A few blocks of 16 tokens (T <= 32; T <= 64 where d_in * d_out <= 2^24) are
+ * grouping is computed.  A few blocks of 16 tokens (T <= 48 where d_in * d_out <= 2^24; else T <= 32 where d_in > 4096) are
  * one launch of the same kernel, an equal share of its CTAs per block: every block's rows are bit for
- * bit those of a decode call on that block, and W0 still leaves HBM once.  Larger T: the
- * segmentation pass runs into the tail of the workspace and the perm form of lora_mixed_linear
- * follows on the same stream; results are then identical to lml_segment_tokens followed by
- * lora_mixed_linear (for the blocks of 16 they agree with it to fp32 summation order and the bf16
- * rounding of u).  workspace: device, 256-byte aligned, at least
+ * bit those of a decode call on that block, and W0 still leaves HBM once.  Beyond that, up to one
+ * row tile (T <= 128): two launches, the tokens staying in their order; the first binds them and
+ * writes, per distinct slot of the batch, the slot's rows of the shrink result, the GEMM adds them
+ * slot by slot.  Larger T: the segmentation pass runs into the tail of the workspace and the perm
+ * form of lora_mixed_linear follows on the same stream; results are then identical to
+ * lml_segment_tokens followed by lora_mixed_linear (up to 128 tokens they agree with it to fp32
+ * summation order and the bf16 rounding of u).  workspace: device, 256-byte aligned, at least
  * lml_tokens_workspace_bytes(t, T) bytes.  Errors: INVALID_ARG, WORKSPACE, CUDA.
  */
 size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens);

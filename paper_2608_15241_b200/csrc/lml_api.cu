@@ -116,6 +116,8 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
                               (uint64_t)d_in * kRankPad * 2, 64, 64, 1);
     gemm_split_override(&t->split_bn, &t->split_s);   // the test knobs are read here, never on the hot path
     if (const char* e = getenv("LML_FUSE_SHRINK")) t->fuse_shrink = e[0] != '0';
+    if (const char* e = getenv("LML_ONE_TILE")) t->one_tile = e[0] != '0';
+    if (const char* e = getenv("LML_BIND_THREADS")) t->bind_threads = atoi(e);
     if (const char* e = getenv("LML_DECODE_BLOCK_TOKENS")) t->dec_block_tokens = atoi(e) < 0 ? 0 : (atoi(e) > kDecMaxBlocks * kDecodeMaxT ? kDecMaxBlocks * kDecodeMaxT : atoi(e));
     ok = ok && cudaEventCreateWithFlags(&t->ev_map, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&t->copy_in, cudaStreamNonBlocking) == cudaSuccess;
@@ -624,11 +626,12 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
         if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
         return LML_OK;
     }
-    // (measured on B200 against the GEMM path: two blocks win on every layer of a 7B-class model, 14 us against 29 us
-    // on 4096 x 4096 and 33 against 39 - 45 us on the MLP's; three and four win on the 4096 x 4096 layers only, 21 and
-    // 25 against 29 - 30 us; more lose: every block's CTAs take all of W0 in from L2)
+    // (measured on B200 against the one-tile path below, us per call at 20 / 32 / 48 / 64 tokens: 4096 x 4096 13.3 / 13.8 /
+    // 19.8 / 24.1 against 19.1 / 20.1 / 20.6 / 20.6; 11008 x 4096 33.5 / 31.5 against 29.2 / 29.7; 4096 x 11008 31.4 / 32.0
+    // against 27.4 / 35.4: every block's CTAs take all of W0 in from L2, which a wide output pays for at once)
+    const bool small_layer = (long long)t->d_in * t->d_out <= (1ll << 24);
     const int block_limit = t->dec_block_tokens >= 0 ? t->dec_block_tokens
-                                                     : ((long long)t->d_in * t->d_out <= (1ll << 24) ? 4 : 2) * kDecodeMaxT;
+                                                     : (small_layer ? 3 : (t->d_in > 4096 ? 2 : 1)) * kDecodeMaxT;
     if (T <= block_limit) {
         // A few blocks of 16 tokens: one launch of the decode kernel with the blocks as its parts, an equal share of the
         // CTAs each.  The shares walk W0 together, so a line leaves HBM once and the other readers find it in L2; no
@@ -667,6 +670,37 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
     int32_t* perm = reinterpret_cast<int32_t*>(wsb + base);
     int32_t* seg_offsets = reinterpret_cast<int32_t*>(wsb + base + round_up((size_t)T * 4 + 4, 1024));
     int32_t* seg_ids = seg_offsets + round_up((size_t)(t->max_slots + 2) * 4, 1024) / 4;
+    if (T <= kTileM && t->one_tile) {
+        // One row tile: the tokens stay where they are.  One launch binds them and writes, per distinct slot of the
+        // batch, a block of u whose rows are the slot's tokens (zeros elsewhere); the GEMM then adds block x B per
+        // slot.  No grouping, no row copy: two launches instead of four (21 against 30 us at 128 tokens on 4096 x 4096,
+        // 32 against 41 on 11008 x 4096, 38 against 46 on 4096 x 11008).
+        const SlotSnapshot snap = snapshot_locked(t);
+        DeviceGuard guard(t->device);
+        if (!guard.ok) return LML_ERR_CUDA;
+        const WsLayout ws = ws_layout(t, T, G);
+        PlanWord* plan = reinterpret_cast<PlanWord*>(wsb + ws.plan_off);
+        __nv_bfloat16* u_blocks = reinterpret_cast<__nv_bfloat16*>(wsb + ws.u_off);
+        int launches = 0;
+        cudaError_t e = launch_bind_shrink_tile(t->arena, snap, token_slots, T, t->d_in, x, seg_offsets, seg_ids, G, plan,
+                                                u_blocks, t->bind_threads > 0 ? t->bind_threads : (t->d_in > 4096 ? 1024 : 512), stream, by_adapter);
+        if (e == cudaSuccess) {
+            ++launches;
+            GemmArgs a;
+            a.fused_shrink = false;
+            a.x = x; a.x_in_place = x; a.tile_identity = nullptr; a.W0 = W0; a.y = y; a.perm = nullptr;
+            a.seg_offsets = seg_offsets; a.slot_ids = seg_ids;
+            a.plan = plan; a.u_blocks = u_blocks;
+            a.T = T; a.d_in = t->d_in; a.d_out = t->d_out; a.G = G; a.num_sms = t->num_sms;
+            a.overlap_with_previous = true;
+            a.split_bn = t->split_bn; a.split_s = t->split_s;
+            e = launch_gemm_sm100(t->arena, snap, t->tmap_B256, t->tmap_B128, t->tmap_A, &t->tmaps, a, stream);
+            if (e == cudaSuccess) ++launches;
+        }
+        t->last_launches = launches;
+        if (e != cudaSuccess) { cudaGetLastError(); return LML_ERR_CUDA; }
+        return LML_OK;
+    }
     lml_status st = segment_tokens_impl(t, token_slots, T, perm, seg_offsets, seg_ids, stream_v, by_adapter);
     if (st != LML_OK) return st;
     st = lora_mixed_linear(t, x, W0, T, seg_offsets, seg_ids, G, perm, y, workspace, base, stream_v);

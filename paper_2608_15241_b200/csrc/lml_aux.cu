@@ -256,6 +256,149 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 }
 
 // ---------------------------------------------------------------------------------------------
+// Token-form calls of at most one row tile (T <= 128) that are too long for the decode kernel: binding and shrink in
+// one launch, with no grouping and no row copy.  The GEMM adds, per LoRA piece of a row tile, the product of a whole
+// 128 x 64 block of u with the slot's B; which rows of the block are non-zero is the block's own business.  So the
+// tokens stay in their order: the distinct live slots of the batch, in ascending order, become the "segments"
+// g = 0 .. G' - 1 (segment g is given the row range [g, g + 1), the last one [G' - 1, T): ranges that lie in the
+// tile and satisfy the layer's checks; the GEMM only asks whether a range meets the tile), and block g holds
+// scale * x_t . A_slot^T in the rows t that are bound to that slot and zeros everywhere else.
+// One CTA per row of the tile: it works out the batch's slot set itself (T <= 128 ids), computes its row's dot
+// products (up to sixteen columns j at a time, one or two warps per column, each on its part of the row; the row of x
+// in shared memory when it fits) and writes its row of every block.  The GEMM that follows needs whole SMs, so it
+// runs after this kernel, not beside it: what counts is that this kernel is short.  (A small persistent grid on the
+// SMs that the GEMM leaves free was measured: beside the GEMM's stream every dependent load takes microseconds, 37
+// against 24 us per call at 128 tokens on 4096 x 4096.)
+constexpr int kBindMaxSmemCols = 20480;   // a row of x up to this width is staged in shared memory (40 KB)
+
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads) bind_shrink_tile_kernel(
+    const __grid_constant__ SlotSnapshot snap, const __nv_bfloat16* __restrict__ arenaA,
+    const int32_t* __restrict__ token_slots, int T, int K, const __nv_bfloat16* __restrict__ x,
+    int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_slot_ids, int G, PlanWord* __restrict__ plan,
+    __nv_bfloat16* __restrict__ u_blocks, uint32_t* __restrict__ status, const int32_t* __restrict__ adapter_map, int in_smem)
+{
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kCols = kWarps < 16 ? kWarps : 16;   // columns worked on side by side
+    constexpr int kParts = kWarps / kCols;             // warps per column, each on its part of the row
+    extern __shared__ uint4 bind_x_s[];
+    __shared__ unsigned mask_s[2];
+    __shared__ int my_slot_s, bad_s;
+    __shared__ float dots_s[kRankPad];
+    __shared__ float part_s[kParts][kRankPad];
+    const int row = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid < 2) mask_s[tid] = 0u;
+    if (tid == 0) { my_slot_s = -1; bad_s = 0; }
+    ptx::grid_dependency_wait();      // launched as a programmatic dependent: whatever ran before is complete now
+    ptx::grid_launch_dependents();    // the GEMM may get resident where there is room; it waits for this grid before its pieces
+    __syncthreads();
+    const int nch = K / 8;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * K);
+    if (row < T && in_smem)   // (does not depend on the binding: goes out with the ids)
+        for (int c = tid; c < nch; c += kThreads) bind_x_s[c] = __ldg(xr + c);
+    for (int i = tid; i < T; i += kThreads) {
+        int s = __ldg(token_slots + i);
+        if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
+        const bool bad_id = s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0);
+        if (bad_id) { bad_s = 1; s = -1; }
+        if (s >= 0) atomicOr(&mask_s[s >> 5], 1u << (s & 31));
+        if (i == row) my_slot_s = s;
+    }
+    __syncthreads();
+    const unsigned long long mask = (unsigned long long)mask_s[0] | ((unsigned long long)mask_s[1] << 32);
+    const int Gp = __popcll(mask);
+    if (row == 0) {
+        if (tid == 0 && bad_s) atomicOr(status, LML_FLAG_BAD_SLOT);
+        for (int g = tid; g <= G; g += kThreads) {
+            seg_offsets[g] = g == 0 ? 0 : (g < Gp ? g : T);
+            if (g < G) {
+                int slot = -1;
+                if (g < Gp) {   // the g-th live slot of the batch
+                    unsigned long long m = mask;
+                    for (int k = 0; k < g; ++k) m &= m - 1ull;
+                    slot = __ffsll((long long)m) - 1;
+                }
+                seg_slot_ids[g] = slot;
+            }
+        }
+        if (tid == 0) plan->lora_ok = 1;
+    }
+    const int my_slot = row < T ? my_slot_s : -1;
+    const int g_mine = my_slot >= 0 ? __popcll(mask & ((1ull << my_slot) - 1ull)) : -1;
+    const int rank = my_slot >= 0 ? (int)snap.rank[my_slot] : 0;
+    // this row's dot products: the warps w, w + kCols, ... take the columns j = w, w + kCols, ..., each its part of the
+    // row; a lane sums the 8-element chunks lane, lane + 32, ... of the part in order, the warp adds its lanes up with
+    // the butterfly, and the parts are added in a fixed order
+    const int part = (nch + kParts - 1) / kParts;
+    const int h = warp / kCols, c_begin = min(nch, h * part), c_end = min(nch, c_begin + part);
+    for (int j = warp % kCols; j < rank; j += kCols) {
+        const uint4* ar = reinterpret_cast<const uint4*>(arenaA + ((size_t)my_slot * kRankPad + j) * K);
+        float acc = 0.f;
+        for (int c0 = c_begin + lane; c0 < c_end; c0 += 32 * 8) {
+            uint4 av[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int c = c0 + 32 * i;
+                av[i] = c < c_end ? __ldg(ar + c) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int c = c0 + 32 * i;
+                if (c < c_end) {
+                    const uint4 xv = in_smem ? bind_x_s[c] : __ldg(xr + c);
+                    float p = 0.f;
+                    p = fmaf(bf16_lo(xv.x), bf16_lo(av[i].x), p); p = fmaf(bf16_hi(xv.x), bf16_hi(av[i].x), p);
+                    p = fmaf(bf16_lo(xv.y), bf16_lo(av[i].y), p); p = fmaf(bf16_hi(xv.y), bf16_hi(av[i].y), p);
+                    p = fmaf(bf16_lo(xv.z), bf16_lo(av[i].z), p); p = fmaf(bf16_hi(xv.z), bf16_hi(av[i].z), p);
+                    p = fmaf(bf16_lo(xv.w), bf16_lo(av[i].w), p); p = fmaf(bf16_hi(xv.w), bf16_hi(av[i].w), p);
+                    acc += p;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) part_s[h][j] = acc;
+    }
+    __syncthreads();
+    if (tid < kRankPad) {
+        float v = 0.f;
+        if (tid < rank) {
+#pragma unroll
+            for (int q = 0; q < kParts; ++q) v += part_s[q][tid];
+            v *= snap.scale[my_slot];
+        }
+        dots_s[tid] = v;
+    }
+    __syncthreads();
+    // this row of every block: the dot products in its own block, zeros in the others (pairs of columns per thread)
+    for (int i = tid; i < Gp * (kRankPad / 2); i += kThreads) {
+        const int g = i / (kRankPad / 2), c2 = i % (kRankPad / 2);
+        __nv_bfloat162 v = __floats2bfloat162_rn(0.f, 0.f);
+        if (g == g_mine) v = __floats2bfloat162_rn(dots_s[2 * c2], dots_s[2 * c2 + 1]);
+        reinterpret_cast<__nv_bfloat162*>(u_blocks + ((size_t)g * kTileM + row) * kRankPad)[c2] = v;
+    }
+}
+
+cudaError_t launch_bind_shrink_tile(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots, int T, int d_in,
+                                    const void* x, int32_t* seg_offsets, int32_t* seg_slot_ids, int G, PlanWord* plan,
+                                    void* u_blocks, int threads, cudaStream_t stream, bool by_adapter)
+{
+    const int in_smem = d_in <= kBindMaxSmemCols ? 1 : 0;   // (reading x through L1 instead was measured: 2 - 7 us slower per call)
+    const size_t smem = in_smem ? (size_t)d_in * 2 : 0;   // (at most 40 KB: no opt-in needed)
+    auto launch = [&](auto kernel, int nthreads) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        pdl_config(cfg, attr, dim3(kTileM), dim3((unsigned)nthreads), smem, stream);
+        return cudaLaunchKernelEx(&cfg, kernel, snap, (const __nv_bfloat16*)ar.A, token_slots, T, d_in,
+                                  (const __nv_bfloat16*)x, seg_offsets, seg_slot_ids, G, plan, (__nv_bfloat16*)u_blocks, ar.status,
+                                  by_adapter ? (const int32_t*)ar.adapter_map : (const int32_t*)nullptr, in_smem);
+    };
+    if (threads >= 1024) return launch(bind_shrink_tile_kernel<1024>, 1024);
+    if (threads >= 512) return launch(bind_shrink_tile_kernel<512>, 512);
+    return launch(bind_shrink_tile_kernel<256>, 256);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Row gather for the perm form of the prefill call: x_grouped[p][:] = x[perm[p]][:].
 // Batches usually arrive with each request's tokens together, so the grouping perm is the
 // identity over long stretches.  A 128-row tile whose perm is the identity is not copied: the

@@ -88,6 +88,10 @@ cudaError_t launch_shrink_pieces(const Arena& ar, const SlotSnapshot& snap, cons
                                  __nv_bfloat16* u_blocks_neg = nullptr);                              // optional second copy of the blocks, negated
 
 // tile_identity[m] = 1: tile m's perm is the identity, its rows were not copied and stay in place.
+// token-form calls of one row tile: binding and shrink in one launch, tokens in their order (see the kernel)
+cudaError_t launch_bind_shrink_tile(const Arena& ar, const SlotSnapshot& snap, const int32_t* token_slots, int T, int d_in,
+                                    const void* x, int32_t* seg_offsets, int32_t* seg_slot_ids, int G, PlanWord* plan,
+                                    void* u_blocks, int threads, cudaStream_t stream, bool by_adapter);
 cudaError_t launch_gather_rows(const void* x, const int32_t* perm, int T, int d_in, void* x_grouped,
                                int32_t* tile_identity, bool allow_skip, uint32_t* status, cudaStream_t stream);
 

@@ -28,7 +28,7 @@ def _table(K, N, ranks, seed):
 
 
 @pytest.mark.parametrize("T,K,N", [(1, 264, 136), (8, 520, 264), (16, 1024, 512), (13, 4096, 520), (300, 256, 384),
-                                   (17, 264, 136), (24, 1032, 520), (32, 1032, 16400), (33, 1032, 16400), (48, 520, 264), (64, 520, 264), (65, 520, 264), (100, 520, 264), (128, 2048, 1000), (129, 1024, 512), (256, 256, 384),
+                                   (17, 264, 136), (24, 1032, 520), (32, 1032, 16400), (33, 1032, 16400), (32, 4104, 4200), (48, 520, 264), (64, 520, 264), (65, 520, 264), (100, 520, 264), (128, 2048, 1000), (127, 1032, 264), (40, 1032, 16400), (129, 1024, 512), (256, 256, 384),
                                    (200, 1536, 520)])
 def test_tokens_call_equals_segment_then_layer(T, K, N):
     import torch
@@ -46,7 +46,9 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
     y_two = to_bits(tbl.lora_mixed_linear(x, W, so, ids, perm=perm))
     torch.cuda.synchronize()
     assert tbl.device_status() == 0
-    blocks = 16 < T <= (64 if K * N <= 1 << 24 else 32)
+    blocks = 16 < T <= (48 if K * N <= 1 << 24 else (32 if K > 4096 else 16))
+    # (the two forms differ in the bf16 rounding of u, whose size grows with the length of the dot products)
+    last_place = 2.0 ** -7 if K <= 2048 else 2.0 ** -6
     if blocks:
         # a few blocks of 16 tokens: one launch of the decode kernel, every block's rows exactly those of a decode call
         # on that block alone; against the two-call form (the GEMM path) equal to the last place of bf16
@@ -55,7 +57,13 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
             y_blk = to_bits(tbl.lora_mixed_linear_tokens(x[t0:t0 + 16].contiguous(), W, ts[t0:t0 + 16].contiguous()))
             assert np.array_equal(y_tok[t0:t0 + 16], y_blk), t0
         a, b2 = wl.bf16_bits_to_f64(y_tok), wl.bf16_bits_to_f64(y_two)
-        assert (np.abs(a - b2) <= 2.0 ** -7 * np.maximum(1.0, np.abs(b2))).all()
+        assert (np.abs(a - b2) <= last_place * np.maximum(1.0, np.abs(b2))).all()
+    elif 16 < T <= 128:
+        # one row tile: binding and shrink in one launch with the tokens in their order, then the GEMM; the shrink sums
+        # in another order than the grouped path's, so the two forms agree to the last place of bf16
+        assert launches_tok == 2
+        a, b2 = wl.bf16_bits_to_f64(y_tok), wl.bf16_bits_to_f64(y_two)
+        assert (np.abs(a - b2) <= last_place * np.maximum(1.0, np.abs(b2))).all()
     else:
         assert np.array_equal(y_tok, y_two)
     if T <= 16:
