@@ -385,8 +385,8 @@ lml_status lora_mixed_linear_decode_static(lml_table* t, const void* x, const vo
 
 /*
  * Read and clear the sticky device status word (LML_FLAG_* bits).  Synchronises `stream`.
- * Also puts the table's decode exchange blocks (values, marks, counters) back to zero, which matters only
- * after a launch that ended abnormally.
+ * When the word carries LML_FLAG_TIMEOUT (a launch gave up on a wait), the table's decode exchange blocks
+ * (values, marks, counters) are put back to zero as well; no decode call on the table may be in flight then.
  * Errors: INVALID_ARG, CUDA.
  */
 lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream);

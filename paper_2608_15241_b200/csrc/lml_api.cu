@@ -938,9 +938,13 @@ lml_status lml_device_status(lml_table* t, uint32_t* flags_out, void* stream_v)
     uint32_t v = 0;
     bool ok = cudaMemcpyAsync(&v, t->arena.status, sizeof v, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok = ok && cudaMemsetAsync(t->arena.status, 0, sizeof v, stream) == cudaSuccess;
-    // (and the decode kernel's exchange blocks start over: a launch that ended abnormally may have left its counters behind)
-    ok = ok && cudaMemsetAsync(t->arena.dec_u, 0, (size_t)kDecMaxBlocks * kDecExchStride * sizeof(unsigned long long), stream) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    if (ok && (v & LML_FLAG_TIMEOUT)) {
+        // a launch gave up on a wait: its counters may have been left behind, so the decode kernel's exchange blocks
+        // start over (only then: in normal operation nothing here touches memory that a call in flight uses)
+        ok = cudaMemsetAsync(t->arena.dec_u, 0, (size_t)kDecMaxBlocks * kDecExchStride * sizeof(unsigned long long), stream) == cudaSuccess;
+        ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    }
     if (!ok) { cudaGetLastError(); return LML_ERR_CUDA; }
     *flags_out = v;
     return LML_OK;
