@@ -816,8 +816,10 @@ def main():
                                            "cell's bound = max(bytes / measured HBM peak, flops / measured burst tensor peak) / time; "
                                            "16 adapters of rank 16, two of them in two versions (18 resident entries), Zipf(1.1) binding",
                                    "cells": run_layer_sweep(device, peaks, 200, parity=True)}
-            line["few_blocks_of_16_tokens"] = {"what": "the same sweep at 32 tokens: two blocks of 16 on the decode kernel in one launch",
-                                               "cells": run_layer_sweep(device, peaks, 200, parity=True, tokens=(32,))}
+            line["few_blocks_of_16_tokens"] = {"what": "the same sweep at 32 and 64 tokens: blocks of 16 on the decode kernel in one launch "
+                                                       "(launches_per_call 1) or, where that loses, one launch that binds the tokens in their "
+                                                       "order and computes the shrink, then the GEMM (launches_per_call 2)",
+                                               "cells": run_layer_sweep(device, peaks, 200, parity=True, tokens=(32, 64))}
         barrier()
     if rank == 0:
         print(json.dumps(line), flush=True)
