@@ -265,10 +265,14 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 // scale * x_t . A_slot^T in the rows t that are bound to that slot and zeros everywhere else.
 // One CTA per row of the tile: it works out the batch's slot set itself (T <= 128 ids), computes its row's dot
 // products (up to sixteen columns j at a time, one or two warps per column, each on its part of the row; the row of x
-// in shared memory when it fits) and writes its row of every block.  The GEMM that follows needs whole SMs, so it
-// runs after this kernel, not beside it: what counts is that this kernel is short.  (A small persistent grid on the
-// SMs that the GEMM leaves free was measured: beside the GEMM's stream every dependent load takes microseconds, 37
-// against 24 us per call at 128 tokens on 4096 x 4096.)
+// in shared memory when it fits) and writes its row of every block.  The GEMM that follows (216 KB of shared memory and
+// 18K registers per CTA) gets resident beside this kernel's CTAs, and starts on its base k-blocks, only where they leave
+// it room: 512 threads of at most 64 registers and a row of x of at most 8 KB do (d_in <= 4096); a wider row does not
+// fit beside the GEMM anyway, and 1024 threads finish it sooner.  Measured, us per call at 128 tokens on 4096 x 4096 /
+// 11008 x 4096 / 4096 x 11008: 256 threads 23.9 / 32.1 / 47.7, 512 threads 21.2 / 32.2 / 40.2, 1024 threads 24.4 / 39.6 /
+// 37.8; 512 threads with sixteen loads in flight per lane (128 registers) 25.2 / 39.9 / 40.8.  (A small persistent grid
+// on the SMs that the GEMM leaves free was measured too: beside the GEMM's stream every dependent load takes
+// microseconds, 37 against 21 us per call.)
 constexpr int kBindMaxSmemCols = 20480;   // a row of x up to this width is staged in shared memory (40 KB)
 
 template <int kThreads>
