@@ -78,7 +78,7 @@ def test_tokens_call_equals_segment_then_layer(T, K, N):
     tbl.close()
 
 
-@pytest.mark.parametrize("reps", [1, 20])
+@pytest.mark.parametrize("reps", [1, 4, 10, 20])
 def test_tokens_call_flags_ids_without_adapter(reps):
     import torch
     K, N, T = 264, 136, 8 * reps
