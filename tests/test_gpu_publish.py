@@ -25,7 +25,7 @@ def _ref(x_bits, W_bits, entries, token_entry):
                           np.asarray(token_entry, np.int32))[0]
 
 
-@pytest.mark.parametrize("T", [8, 30, 200])   # (decode kernel, two blocks of 16 on the decode kernel, GEMM path)
+@pytest.mark.parametrize("T", [8, 30, 100, 200])   # (decode kernel, two blocks of 16 on the decode kernel, one-tile path, grouped GEMM path)
 def test_publish_switches_resolution_at_a_point_of_the_stream(T):
     import torch
     from paper_2608_15241_b200 import binding as b
