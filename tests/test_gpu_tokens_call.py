@@ -2,8 +2,9 @@
 lml_segment_tokens followed by lora_mixed_linear with the perm it produced.  Both forms run the
 same arithmetic per output element, so the results must agree bit for bit; the oracle is checked
 on top.  Covers the one-launch decode form (T <= 16), the form for a few blocks of 16 tokens (the decode kernel
-again: bit for bit a decode call per block), the prefill form, ids that name no live adapter (flagged, treated
-as -1) and the all-base case."""
+again: bit for bit a decode call per block), the one-tile form (up to 128 tokens in their order: agreement with the
+two-call form to the last place), the prefill form, ids that name no live adapter (flagged, treated as -1) and the
+all-base case."""
 import numpy as np
 import pytest
 
@@ -109,4 +110,40 @@ def test_tokens_call_all_base_equals_no_segments():
     y0 = to_bits(tbl.lora_mixed_linear(x, W, None, None))
     torch.cuda.synchronize()
     assert np.array_equal(y, y0)
+    tbl.close()
+
+
+@pytest.mark.parametrize("T,K,N,n_adapters", [(40, 1032, 16400, 1),     # wide output: the one-tile path from 17 tokens on
+                                               (17, 1032, 16400, 17),    # every token its own slot
+                                               (128, 264, 136, 62)])     # a full tile, nearly every slot of a 64-slot table
+def test_one_tile_path_edge_cases(T, K, N, n_adapters):
+    """The path that keeps the tokens in their order (one launch binds them and computes the shrink, the GEMM follows):
+    a batch without any adapter, as many distinct slots as tokens, a full tile with dozens of slots."""
+    import torch
+    tbl, entries = _table(K, N, (4,) * n_adapters, seed=33)
+    slots = np.array([e[0] for e in entries], np.int32)
+    if n_adapters == 1:
+        token_slots = np.full(T, -1, np.int32)
+    else:
+        token_slots = slots[np.arange(T) % len(slots)].astype(np.int32)
+        token_slots[::7] = -1
+        if n_adapters == 17:
+            token_slots = slots[:T].copy()
+    x_bits = wl.normal_bf16(33, 1, (T, K), 1.0)
+    W_bits = wl.normal_bf16(33, 2, (N, K), 0.02)
+    x, W, ts = to_dev(x_bits), to_dev(W_bits), torch.from_numpy(token_slots).cuda()
+    y_tok = to_bits(tbl.lora_mixed_linear_tokens(x, W, ts))
+    assert tbl.last_launch_count() == 2
+    y_again = to_bits(tbl.lora_mixed_linear_tokens(x, W, ts))
+    torch.cuda.synchronize()
+    assert tbl.device_status() == 0
+    assert np.array_equal(y_tok, y_again)
+    if n_adapters == 1:
+        y0 = to_bits(tbl.lora_mixed_linear(x, W, None, None))
+        assert np.array_equal(y_tok, y0)
+    slot_to_entry = {slot: i for i, (slot, _) in enumerate(entries)}
+    seg_entry = np.array([slot_to_entry.get(int(s), -1) for s in token_slots], np.int32)
+    ref, _ = oracle.forward(x_bits, W_bits, [e for _, e in entries], np.arange(T + 1, dtype=np.int32), seg_entry)
+    cmp = oracle.compare(y_tok, ref)
+    assert cmp["ok"], cmp
     tbl.close()
