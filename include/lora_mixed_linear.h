@@ -275,12 +275,12 @@ lml_status lora_mixed_linear_backward_adapters(lml_table* t, lml_table* t_T, con
  * grouping is computed.  A few blocks of 16 tokens (T <= 48 where d_in * d_out <= 2^24; else T <= 32 where d_in > 4096) are
  * one launch of the same kernel, an equal share of its CTAs per block: every block's rows are bit for
  * bit those of a decode call on that block, and W0 still leaves HBM once.  Beyond that, up to one
- * row tile (T <= 128): two launches, the tokens staying in their order; the first binds them and
- * writes, per distinct slot of the batch, the slot's rows of the shrink result, the GEMM adds them
- * slot by slot.  Larger T: the segmentation pass runs into the tail of the workspace and the perm
- * form of lora_mixed_linear follows on the same stream; results are then identical to
- * lml_segment_tokens followed by lora_mixed_linear (up to 128 tokens they agree with it to fp32
- * summation order and the bf16 rounding of u).  workspace: device, 256-byte aligned, at least
+ * row tile (T <= 128; two tiles, T <= 256, where d_in <= 4096): two launches, the tokens staying in
+ * their order; the first binds them and writes, per row tile and distinct slot, the slot's rows of
+ * the shrink result, the GEMM adds them slot by slot.  Larger T: the segmentation pass runs into the
+ * tail of the workspace and the perm form of lora_mixed_linear follows on the same stream; results
+ * are then identical to lml_segment_tokens followed by lora_mixed_linear (on the other paths they
+ * agree with it to fp32 summation order and the bf16 rounding of u).  workspace: device, 256-byte aligned, at least
  * lml_tokens_workspace_bytes(t, T) bytes.  Errors: INVALID_ARG, WORKSPACE, CUDA.
  */
 size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens);

@@ -116,7 +116,12 @@ lml_status lml_table_create(lml_table** out, int device, int d_in, int d_out, in
                               (uint64_t)d_in * kRankPad * 2, 64, 64, 1);
     gemm_split_override(&t->split_bn, &t->split_s);   // the test knobs are read here, never on the hot path
     if (const char* e = getenv("LML_FUSE_SHRINK")) t->fuse_shrink = e[0] != '0';
-    if (const char* e = getenv("LML_ONE_TILE")) t->one_tile = e[0] != '0';
+    // (two row tiles where the rows of x are short enough for the GEMM's CTAs to get resident beside the binding kernel's:
+    // 256 tokens 29 / 45 us against 34 / 50 on the grouped path on 4096 x 4096 / 11008 x 4096; from 512 tokens on, and on
+    // 4096 x 11008 from 256 on, a piece per slot and tile costs the GEMM more than grouping the rows)
+    t->one_tile_tokens = d_in <= 4096 ? 2 * kTileM : kTileM;
+    if (const char* e = getenv("LML_ONE_TILE")) t->one_tile_tokens = e[0] != '0' ? t->one_tile_tokens : 0;
+    if (const char* e = getenv("LML_ONE_TILE_TOKENS")) t->one_tile_tokens = atoi(e) < 0 ? 0 : (atoi(e) > 8 * kTileM ? 8 * kTileM : atoi(e));
     if (const char* e = getenv("LML_BIND_THREADS")) t->bind_threads = atoi(e);
     if (const char* e = getenv("LML_DECODE_BLOCK_TOKENS")) t->dec_block_tokens = atoi(e) < 0 ? 0 : (atoi(e) > kDecMaxBlocks * kDecodeMaxT ? kDecMaxBlocks * kDecodeMaxT : atoi(e));
     ok = ok && cudaEventCreateWithFlags(&t->ev_map, cudaEventDisableTiming) == cudaSuccess;
@@ -452,13 +457,28 @@ lml_status lora_mixed_linear(lml_table* t, const void* x, const void* W0, int T,
     return LML_OK;
 }
 
+// Segments of a token-form call: one per slot and one for "none" on the grouped path; on the path that keeps the
+// tokens in their order, one per slot and row tile at most, and one more.
+static int tokens_segments(const lml_table* t, int T)
+{
+    if (T > t->one_tile_tokens) return t->max_slots + 1;
+    return ((T + kTileM - 1) / kTileM) * t->max_slots + 1;
+}
+
 size_t lml_tokens_workspace_bytes(const lml_table* t, int max_tokens)
 {
     if (!t || max_tokens < 0 || max_tokens > kMaxTokens) return 0;
-    size_t n = ws_layout(t, max_tokens, t->max_slots + 1).total;
-    n += round_up((size_t)max_tokens * 4 + 4, 1024);               // perm
-    n += 2 * round_up((size_t)(t->max_slots + 2) * 4, 1024);       // seg_offsets, seg_slot_ids
-    return n;
+    // (the largest of the layouts that a call of up to max_tokens tokens can take)
+    size_t best = 0;
+    const int candidates[2] = {max_tokens, max_tokens < t->one_tile_tokens ? max_tokens : t->one_tile_tokens};
+    for (int T : candidates) {
+        const int G = tokens_segments(t, T);
+        size_t n = ws_layout(t, T, G).total;
+        n += round_up((size_t)T * 4 + 4, 1024);               // perm
+        n += 2 * round_up((size_t)(G + 1) * 4, 1024);         // seg_offsets, seg_slot_ids
+        best = n > best ? n : best;
+    }
+    return best;
 }
 
 size_t lml_dual_workspace_bytes(const lml_table* t, int max_tokens, int max_segments)
@@ -665,12 +685,12 @@ static lml_status tokens_impl(lml_table* t, const void* x, const void* W0, int T
     }
     // Prefill: the segmentation pass writes perm and the segment arrays behind the layer's own workspace,
     // and the layer call follows on the same stream.
-    const int G = t->max_slots + 1;
+    const int G = tokens_segments(t, T);
     const size_t base = ws_layout(t, T, G).total;
     int32_t* perm = reinterpret_cast<int32_t*>(wsb + base);
     int32_t* seg_offsets = reinterpret_cast<int32_t*>(wsb + base + round_up((size_t)T * 4 + 4, 1024));
-    int32_t* seg_ids = seg_offsets + round_up((size_t)(t->max_slots + 2) * 4, 1024) / 4;
-    if (T <= kTileM && t->one_tile) {
+    int32_t* seg_ids = seg_offsets + round_up((size_t)(G + 1) * 4, 1024) / 4;
+    if (T <= t->one_tile_tokens) {
         // One row tile: the tokens stay where they are.  One launch binds them and writes, per distinct slot of the
         // batch, a block of u whose rows are the slot's tokens (zeros elsewhere); the GEMM then adds block x B per
         // slot.  No grouping, no row copy: two launches instead of four (21 against 30 us at 128 tokens on 4096 x 4096,

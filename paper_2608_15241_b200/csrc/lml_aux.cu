@@ -256,14 +256,17 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 }
 
 // ---------------------------------------------------------------------------------------------
-// Token-form calls of at most one row tile (T <= 128) that are too long for the decode kernel: binding and shrink in
+// Token-form calls of a row tile or two (T <= 128 or 256) that are too long for the decode kernel: binding and shrink in
 // one launch, with no grouping and no row copy.  The GEMM adds, per LoRA piece of a row tile, the product of a whole
 // 128 x 64 block of u with the slot's B; which rows of the block are non-zero is the block's own business.  So the
-// tokens stay in their order: the distinct live slots of the batch, in ascending order, become the "segments"
-// g = 0 .. G' - 1 (segment g is given the row range [g, g + 1), the last one [G' - 1, T): ranges that lie in the
-// tile and satisfy the layer's checks; the GEMM only asks whether a range meets the tile), and block g holds
-// scale * x_t . A_slot^T in the rows t that are bound to that slot and zeros everywhere else.
-// One CTA per row of the tile: it works out the batch's slot set itself (T <= 128 ids), computes its row's dot
+// tokens stay in their order: the distinct live slots of a tile's tokens, in ascending order, become the tile's
+// "segments" (the k-th is given the row range [128 m + k, 128 m + k + 1), the tile's last one the rest of the tile:
+// ranges that lie in their tile and satisfy the layer's checks; the GEMM only asks which tile a range meets; a tile
+// without any slot gets one segment without a slot), numbered through the tiles, and the block of segment g of tile m,
+// block m + g as on the grouped path, holds scale * x_t . A_slot^T in the tile's rows t that are bound to that slot and
+// zeros everywhere else.  (The kernel serves up to eight tiles; beyond two the GEMM's extra pieces, one per slot and
+// tile, cost more than grouping the rows: 54.9 against 48.2 us at 1024 tokens on 4096 x 4096.)
+// One CTA per row: it works out the slot sets of its tile and of the tiles before it, computes its row's dot
 // products (up to sixteen columns j at a time, one or two warps per column, each on its part of the row; the row of x
 // in shared memory when it fits) and writes its row of every block.  The GEMM that follows (216 KB of shared memory and
 // 18K registers per CTA) gets resident beside this kernel's CTAs, and starts on its base k-blocks, only where they leave
@@ -274,6 +277,7 @@ cudaError_t launch_segment_tokens(const Arena& ar, const SlotSnapshot& snap, con
 // on the SMs that the GEMM leaves free was measured too: beside the GEMM's stream every dependent load takes
 // microseconds, 37 against 21 us per call.)
 constexpr int kBindMaxSmemCols = 20480;   // a row of x up to this width is staged in shared memory (40 KB)
+constexpr int kBindMaxTiles = 8;          // row tiles of a call at most
 
 template <int kThreads>
 __global__ void __launch_bounds__(kThreads) bind_shrink_tile_kernel(
@@ -286,12 +290,13 @@ __global__ void __launch_bounds__(kThreads) bind_shrink_tile_kernel(
     constexpr int kCols = kWarps < 16 ? kWarps : 16;   // columns worked on side by side
     constexpr int kParts = kWarps / kCols;             // warps per column, each on its part of the row
     extern __shared__ uint4 bind_x_s[];
-    __shared__ unsigned mask_s[2];
+    __shared__ unsigned mask_s[kBindMaxTiles][2];
     __shared__ int my_slot_s, bad_s;
     __shared__ float dots_s[kRankPad];
     __shared__ float part_s[kParts][kRankPad];
     const int row = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid < 2) mask_s[tid] = 0u;
+    const int tile = row / kTileM, r_in_tile = row % kTileM, num_m = (T + kTileM - 1) / kTileM;
+    if (tid < 2 * kBindMaxTiles) (&mask_s[0][0])[tid] = 0u;
     if (tid == 0) { my_slot_s = -1; bad_s = 0; }
     ptx::grid_dependency_wait();      // launched as a programmatic dependent: whatever ran before is complete now
     ptx::grid_launch_dependents();    // the GEMM may get resident where there is room; it waits for this grid before its pieces
@@ -300,32 +305,45 @@ __global__ void __launch_bounds__(kThreads) bind_shrink_tile_kernel(
     const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * K);
     if (row < T && in_smem)   // (does not depend on the binding: goes out with the ids)
         for (int c = tid; c < nch; c += kThreads) bind_x_s[c] = __ldg(xr + c);
-    for (int i = tid; i < T; i += kThreads) {
+    // the slot sets of this row's tile and of the tiles before it (their sizes place this tile's segments and blocks)
+    const bool closes = tile == num_m - 1 && r_in_tile == 0;   // the CTA that also closes the segment arrays
+    const int ids_end = min(T, (tile + 1) * kTileM);
+    for (int i = tid; i < ids_end; i += kThreads) {
         int s = __ldg(token_slots + i);
         if (adapter_map) s = resolve_adapter(snap, adapter_map, s);
         const bool bad_id = s < -1 || s >= snap.max_slots || (s >= 0 && snap.rank[s] == 0);
         if (bad_id) { bad_s = 1; s = -1; }
-        if (s >= 0) atomicOr(&mask_s[s >> 5], 1u << (s & 31));
+        if (s >= 0) atomicOr(&mask_s[i / kTileM][s >> 5], 1u << (s & 31));
         if (i == row) my_slot_s = s;
     }
     __syncthreads();
-    const unsigned long long mask = (unsigned long long)mask_s[0] | ((unsigned long long)mask_s[1] << 32);
+    // A tile's segments: one per distinct live slot of the tile, in ascending order; a tile without any gets one
+    // segment without a slot, so that every tile's rows belong to segments of its own.
+    auto tile_mask = [&](int m) { return (unsigned long long)mask_s[m][0] | ((unsigned long long)mask_s[m][1] << 32); };
+    int base = 0;   // segments of the tiles before this one
+    for (int m = 0; m < tile; ++m) base += max(1, __popcll(tile_mask(m)));
+    const unsigned long long mask = tile_mask(tile);
     const int Gp = __popcll(mask);
-    if (row == 0) {
-        if (tid == 0 && bad_s) atomicOr(status, LML_FLAG_BAD_SLOT);
-        for (int g = tid; g <= G; g += kThreads) {
-            seg_offsets[g] = g == 0 ? 0 : (g < Gp ? g : T);
-            if (g < G) {
-                int slot = -1;
-                if (g < Gp) {   // the g-th live slot of the batch
-                    unsigned long long m = mask;
-                    for (int k = 0; k < g; ++k) m &= m - 1ull;
-                    slot = __ffsll((long long)m) - 1;
-                }
-                seg_slot_ids[g] = slot;
+    if (r_in_tile == 0) {
+        if (tid == 0 && bad_s && closes) atomicOr(status, LML_FLAG_BAD_SLOT);   // (this CTA has seen every id)
+        const int nseg = max(1, Gp);
+        for (int k = tid; k < nseg; k += kThreads) {
+            int slot = -1;
+            if (k < Gp) {   // the k-th live slot of the tile
+                unsigned long long mm = mask;
+                for (int q = 0; q < k; ++q) mm &= mm - 1ull;
+                slot = __ffsll((long long)mm) - 1;
             }
+            seg_offsets[base + k] = tile * kTileM + k;
+            seg_slot_ids[base + k] = slot;
         }
-        if (tid == 0) plan->lora_ok = 1;
+        if (closes) {
+            for (int g = base + nseg + tid; g <= G; g += kThreads) {
+                seg_offsets[g] = T;
+                if (g < G) seg_slot_ids[g] = -1;
+            }
+            if (tid == 0) plan->lora_ok = 1;
+        }
     }
     const int my_slot = row < T ? my_slot_s : -1;
     const int g_mine = my_slot >= 0 ? __popcll(mask & ((1ull << my_slot) - 1ull)) : -1;
@@ -379,7 +397,7 @@ __global__ void __launch_bounds__(kThreads) bind_shrink_tile_kernel(
         const int g = i / (kRankPad / 2), c2 = i % (kRankPad / 2);
         __nv_bfloat162 v = __floats2bfloat162_rn(0.f, 0.f);
         if (g == g_mine) v = __floats2bfloat162_rn(dots_s[2 * c2], dots_s[2 * c2 + 1]);
-        reinterpret_cast<__nv_bfloat162*>(u_blocks + ((size_t)g * kTileM + row) * kRankPad)[c2] = v;
+        reinterpret_cast<__nv_bfloat162*>(u_blocks + ((size_t)(tile + base + g) * kTileM + r_in_tile) * kRankPad)[c2] = v;
     }
 }
 
@@ -392,7 +410,7 @@ cudaError_t launch_bind_shrink_tile(const Arena& ar, const SlotSnapshot& snap, c
     auto launch = [&](auto kernel, int nthreads) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[1];
-        pdl_config(cfg, attr, dim3(kTileM), dim3((unsigned)nthreads), smem, stream);
+        pdl_config(cfg, attr, dim3((unsigned)(((T + kTileM - 1) / kTileM) * kTileM)), dim3((unsigned)nthreads), smem, stream);
         return cudaLaunchKernelEx(&cfg, kernel, snap, (const __nv_bfloat16*)ar.A, token_slots, T, d_in,
                                   (const __nv_bfloat16*)x, seg_offsets, seg_slot_ids, G, plan, (__nv_bfloat16*)u_blocks, ar.status,
                                   by_adapter ? (const int32_t*)ar.adapter_map : (const int32_t*)nullptr, in_smem);

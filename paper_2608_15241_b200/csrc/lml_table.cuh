@@ -22,7 +22,7 @@ struct lml_table {
     bool fuse_shrink = true;            // LML_FUSE_SHRINK=0 when the table was created: always the separate shrink kernel (a test knob)
     lml::TmapCache tmaps;               // tensor maps of the caller's buffers seen so far
     int bind_threads = 0;               // LML_BIND_THREADS as it stood when the table was created (0: the library chooses; a test knob)
-    bool one_tile = true;               // LML_ONE_TILE=0 when the table was created: token-form calls of up to 128 tokens take the grouped path (a test knob)
+    int one_tile_tokens = lml::kTileM;  // token-form calls of up to this many tokens (beyond the decode kernel's range) keep the tokens in their order: one or two row tiles, set when the table is created; LML_ONE_TILE=0 or LML_ONE_TILE_TOKENS=n at that time change it (test knobs)
     int dec_block_tokens = -1;          // token-form calls of up to this many tokens run as blocks of 16 on the decode kernel; -1: the library's own limit (LML_DECODE_BLOCK_TOKENS as it stood when the table was created)
     int split_bn = -1, split_s = -1;    // LML_GEMM_SPLIT as it stood when the table was created (-1: not set)
     // Retiring a serving entry clears its word of the device map with a kernel on a stream; the event marks

@@ -242,7 +242,7 @@ def test_layer_sweep_shapes_at_a_few_blocks_of_tokens(proj, T):
 # up to one row tile through the token form of the call beyond the blocks' range: the tokens stay in their order, one
 # launch binds them and writes the shrink result slot by slot, the GEMM follows (two launches): every element against
 # the oracle, output and workspace between canary bands
-@pytest.mark.parametrize("proj,T", [("q", 49), ("q", 64), ("q", 128), ("gate", 17), ("gate", 32), ("gate", 128), ("down", 33), ("down", 127)])
+@pytest.mark.parametrize("proj,T", [("q", 49), ("q", 64), ("q", 128), ("q", 129), ("q", 256), ("gate", 17), ("gate", 32), ("gate", 128), ("gate", 200), ("down", 33), ("down", 127)])
 def test_layer_sweep_shapes_in_one_row_tile_through_the_token_form(proj, T):
     import torch
     from gpu_util import Guarded
