@@ -67,7 +67,8 @@ constexpr int kDecChunksPerSpan = kDecSpan / kDecChunk;             // 4
 constexpr int kDecStepsPerChunk = kDecChunk / 32 / kDecConsumers;   // 8 k-steps per warp and stage
 constexpr int kDecRowPitch = kDecChunk * 2 + 16; // bytes; one 16-byte chunk more than a multiple of 128: a quarter-warp's reads (2 rows x 4 lanes, 32 bytes apart) cover all banks
 constexpr int kDecStageBytes = kDecUnitRows * kDecRowPitch;
-constexpr int kDecStages = 4;
+constexpr int kDecStages = 4;                    // ring stages of a call with adapters
+constexpr int kDecStagesBase = 5;                // of a call without any (see DecCfg)
 constexpr int kDecRoundUnits = 4;                // units (= 32 rows) reduced together
 constexpr int kDecSlotFloats = 16 * kDecUnitRows;   // [token][row] partial sums of one warp for one unit
 constexpr int kDecSlotBytes = kDecRoundUnits * kDecConsumers * kDecSlotFloats * 4;
@@ -93,14 +94,23 @@ struct DecLookup {   // what the shrink warps work out about the call, in shared
 };
 constexpr int kDecSegBytes = (int)sizeof(DecLookup);
 constexpr int kDecDeferBytes = 2048;   // base sums of rounds whose expand is put off: 16 x 32 or 2 x (8 x 32) fp32
-constexpr int kDecSmemBytes = 128 + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8 + kDecDotBytes + kDecDeferBytes;
+constexpr int kDecCtrlBytes = 320;
+// A call without any adapter (G == 0) has no use for the staging buffer of B and takes a fifth ring stage instead: the
+// deeper ring is worth 0.5 us on a 4096 x 4096 layer (8.24 -> 7.73 us).  With adapters a fifth stage loses (8.63 against
+// 8.39 us even where the blocks of B still fit): the shrink warps' cold loads queue up behind whatever the ring has asked for.
+template <bool kBase> struct DecCfg {
+    static constexpr int kStages = kBase ? kDecStagesBase : kDecStages;
+    static constexpr int kDotBytes = kBase ? 0 : kDecDotBytes;
+    static constexpr int kSmemBytes = 128 + kStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + kDecCtrlBytes + kDecSegBytes + 8 + kDotBytes + kDecDeferBytes;
+};
+constexpr int kDecSmemBytes = DecCfg<false>::kSmemBytes;
 // 196 KB is also the largest shared-memory carve-out that leaves the SM a useful L1 for the loads of x:
 // one step more and the base-only call is 0.8 us slower.
-static_assert(kDecSmemBytes + 1024 <= 200704, "shared memory budget");   // the system keeps 1 KB per CTA for itself
+static_assert(kDecSmemBytes + 1024 <= 200704 && DecCfg<true>::kSmemBytes + 1024 <= 200704, "shared memory budget");   // the system keeps 1 KB per CTA for itself
 
 struct DecCtrl {
-    uint64_t full[kDecStages];
-    uint64_t empty[kDecStages];
+    uint64_t full[kDecStagesBase];
+    uint64_t empty[kDecStagesBase];
     uint64_t ufull;      // the shrink warps' results (u, the slots, the copies of B) are in shared memory
     uint64_t bfull;      // the bulk copies of B (whole rows of the compact arena) have landed
     int abort;
@@ -110,7 +120,7 @@ struct DecCtrl {
     uint8_t b_lead[16];  // 1: this row of x is the first with its slot (it stands for the slot's block of B)
     uint8_t b_rows[16];  // 1: the block holds whole 32-byte rows of the compact arena, row after row (one bulk copy); 0: 16-byte chunks, chunk-major
 };
-static_assert(sizeof(DecCtrl) <= 256 && (kDecSegBytes + 8) % 16 == 0, "control block");
+static_assert(sizeof(DecCtrl) <= kDecCtrlBytes && kDecStagesBase >= kDecStages && (kDecSegBytes + 8) % 16 == 0, "control block");
 
 // kTwo false: T <= 8, the second half of the 16-row MMA operand is zero and needs no registers.
 // kMulti: the CTAs have more than one round of rows; compiled with the code that saves reloads of x between rounds.
@@ -149,7 +159,7 @@ template <int kP> struct DecLaunch {
     int T, K, P, patience;
 };
 
-template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1>
+template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1, bool kBase = false>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __grid_constant__ DecLaunch<kP> prm)
 {
     int pi = 0;
@@ -171,17 +181,18 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     const int32_t* __restrict__ token_slots = pj.token_slots;
     const int32_t* __restrict__ adapter_map = pj.adapter_map;
     uint32_t* status = pj.status;
-    const int T = kP == 1 ? prm.T : pj.T, K = prm.K, N = pj.N, G = pj.G, patience = prm.patience;
+    constexpr int kS = DecCfg<kBase>::kStages, kDotBytes = DecCfg<kBase>::kDotBytes;
+    const int T = kP == 1 ? prm.T : pj.T, K = prm.K, N = pj.N, G = kBase ? 0 : pj.G, patience = prm.patience;
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
     const uint32_t ring = (raw + 127u) & ~127u;
     uint8_t* base_ptr = dec_smem_raw + (ring - raw);
-    float* slots = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes);   // [stage][warp][token][row]
-    float* u_s = reinterpret_cast<float*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes);   // [16][64]
-    DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes);
-    DecLookup* lk = reinterpret_cast<DecLookup*>(base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256);
-    uint8_t* dot_s = base_ptr + kDecStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + 256 + kDecSegBytes + 8;   // 16-byte aligned
-    float* defer_s = reinterpret_cast<float*>(dot_s + kDecDotBytes);
+    float* slots = reinterpret_cast<float*>(base_ptr + kS * kDecStageBytes);   // [stage][warp][token][row]
+    float* u_s = reinterpret_cast<float*>(base_ptr + kS * kDecStageBytes + kDecSlotBytes);   // [16][64]
+    DecCtrl* ctrl = reinterpret_cast<DecCtrl*>(base_ptr + kS * kDecStageBytes + kDecSlotBytes + kDecUBytes);
+    DecLookup* lk = reinterpret_cast<DecLookup*>(base_ptr + kS * kDecStageBytes + kDecSlotBytes + kDecUBytes + kDecCtrlBytes);
+    uint8_t* dot_s = base_ptr + kS * kDecStageBytes + kDecSlotBytes + kDecUBytes + kDecCtrlBytes + kDecSegBytes + 8;   // 16-byte aligned
+    float* defer_s = reinterpret_cast<float*>(dot_s + kDotBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // this CTA's rows: a contiguous, balanced range
@@ -209,7 +220,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     // for free stages.
     if (producer) {
         if (lane == 0) {
-            for (int s = 0; s < kDecStages; ++s) {
+            for (int s = 0; s < kS; ++s) {
                 mbar_init(smem_u32(&ctrl->full[s]), 1);
                 mbar_init(smem_u32(&ctrl->empty[s]), kDecConsumers);
             }
@@ -244,7 +255,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                             bulk_copy_g2s(ring + stage * kDecStageBytes + lane * kDecRowPitch,
                                           W0 + (size_t)(r0 + lane) * K + k_begin + kc * kDecChunk,
                                           (uint32_t)(cols * 2), smem_u32(&ctrl->full[stage]));
-                        if (++stage == kDecStages) { stage = 0; phase ^= 1u; }
+                        if (++stage == kS) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
@@ -477,7 +488,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                     const int v = __shfl_up_sync(0xffffffffu, base, o);
                     if (lane >= o) base += v;
                 }
-                const int fits = base * 16 <= kDecDotBytes;   // (inclusive end of this block)
+                const int fits = base * 16 <= kDotBytes;   // (inclusive end of this block)
                 const int my_off = __shfl_sync(0xffffffffu, fits ? (base - chunks) * 16 : -1, first);
                 if (lane < 16) {
                     ctrl->b_of_row[lane] = rank > 0 ? my_off : -1;
@@ -812,7 +823,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                                 }
                                 __syncwarp();
                                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[stage]));
-                                if (++stage == kDecStages) { stage = 0; phase ^= 1u; }
+                                if (++stage == kS) { stage = 0; phase ^= 1u; }
                             }
                         }
                     }
@@ -963,6 +974,11 @@ cudaError_t decode_init()
     set(decode_main_kernel<true, false, false, 1>);  set(decode_main_kernel<true, true, false, 1>);  set(decode_main_kernel<true, true, true, 1>);
     set(decode_main_kernel<false, false, false, kDecMaxProj>); set(decode_main_kernel<false, true, false, kDecMaxProj>); set(decode_main_kernel<false, true, true, kDecMaxProj>);
     set(decode_main_kernel<true, false, false, kDecMaxProj>);  set(decode_main_kernel<true, true, false, kDecMaxProj>);  set(decode_main_kernel<true, true, true, kDecMaxProj>);
+    auto set_base = [&](auto kernel) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<true>::kSmemBytes);
+    };
+    set_base(decode_main_kernel<false, false, false, 1, true>); set_base(decode_main_kernel<false, true, false, 1, true>);
+    set_base(decode_main_kernel<true, false, false, 1, true>);  set_base(decode_main_kernel<true, true, false, 1, true>);
     return e;
 }
 
@@ -1008,6 +1024,13 @@ cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_
     const bool multi = rows_per_cta > kDecRoundUnits * kDecUnitRows;
     const bool put_off = multi && adapters;
     auto launch = [&](auto kernel) { return cudaLaunchKernelEx(&cfg, kernel, prm); };
+    if constexpr (kP == 1) {
+        if (!adapters) {   // no adapter anywhere in the call: the build with the deeper ring and no staging buffer
+            cfg.dynamicSmemBytes = DecCfg<true>::kSmemBytes;
+            if (max_T > 8) return multi ? launch(decode_main_kernel<true, true, false, 1, true>) : launch(decode_main_kernel<true, false, false, 1, true>);
+            return multi ? launch(decode_main_kernel<false, true, false, 1, true>) : launch(decode_main_kernel<false, false, false, 1, true>);
+        }
+    }
     if (max_T > 8)
         return put_off ? launch(decode_main_kernel<true, true, true, kP>)
                        : (multi ? launch(decode_main_kernel<true, true, false, kP>) : launch(decode_main_kernel<true, false, false, kP>));
