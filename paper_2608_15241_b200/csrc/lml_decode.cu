@@ -468,13 +468,39 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                     lk->dot_end[lane] = end;
                     lk->rank_of_row[lane] = rank;
                 }
+            }
+        }
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
+        // The dot products are dealt out in groups of one, two or four columns j of one row of x (a group
+        // shares the row of x): group g belongs to CTA g mod grid.  A dot product's arithmetic is fixed, whoever
+        // computes it: 96 "virtual threads" (the three shrink warps) each sum the 8-column chunks m, m + 96,
+        // m + 192, ... of the row in order, each warp adds its threads' sums up with the butterfly, and the
+        // result is (w0 + w1) + w2 times the scale.  The operands of a whole group (up to six 16-byte chunks of x
+        // and of each row of A per thread and step: 4608 columns) are in flight at once, in registers, so a group costs
+        // one memory round trip per step.  (Groups staged in shared memory by asynchronous copies were measured slower:
+        // 1.1 us per call for pairs at 12 and 16 tokens, 0.6 - 2.3 us for groups of four.)  A result is published as one
+        // 64-bit store (value and this launch's mark) and a relaxed add on the grid-wide counter: nobody waits for a fence.
+        const int total = lk->dot_end[15];
+        // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
+        // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
+        const int gsize = total <= ncta ? 1 : (total <= 2 * ncta ? 2 : kDecDotGroup);
+        const int ngroups = total / gsize;
+        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+        // Where the expand will find its B operand: worked out by the first shrink warp in the shadow of its first dot
+        // product's loads (0.6 us of single-warp work that nothing ahead of the epilogue waits for; CTAs without a dot
+        // product of their own do it after the others').
+        bool booked = false;
+        auto book_once = [&]() {   // (called by whole warps only: the first shrink warp shuffles in here)
+            if (sw == 0 && !booked) {
+                __syncwarp();
+                const int slot = lane < T ? ctrl->slot_of_row[lane] : -1;
+                const int rank = slot >= 0 ? (int)lk->rank_s[slot] : 0;
                 // The expand reads, per distinct slot, the first ceil(rank / 8) 16-byte chunks of this CTA's
                 // rows of B.  Those go into the staging buffer, one block per distinct slot as long as they fit; the
-                // first row of x with a slot stands for the slot's block.  When the dot products will not need the
-                // staging buffer (at most two per CTA: see below), a slot of rank <= 16 comes in right here as one bulk
-                // copy of this CTA's rows of the compact arena (32 bytes each, row after row): a single instruction of
-                // this warp for all slots, where the chunk-by-chunk copies further down cost the shrink warps about
-                // 0.2 us per slot, ahead of their dot products.  The other blocks are chunk-major ([chunk][row]:
+                // first row of x with a slot stands for the slot's block.  A slot of rank <= 16 comes in right here as
+                // one bulk copy of this CTA's rows of the compact arena (32 bytes each, row after row): a single
+                // instruction of this warp for all slots, where the chunk-by-chunk copies further down cost the shrink
+                // warps about 0.2 us per slot.  The other blocks are chunk-major ([chunk][row]:
                 // consecutive threads of the epilogue read consecutive 16 bytes) and are filled by stage_b.
                 const unsigned same = __match_any_sync(0xffffffffu, slot);
                 const int first = __ffs(same) - 1;
@@ -508,23 +534,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                     bulk_copy_g2s(smem_u32(dot_s) + (uint32_t)((base - chunks) * 16), arenaBc + ((size_t)slot * N + row_begin) * kRankCompact,
                                   (uint32_t)(chunks * 16), smem_u32(&ctrl->bfull));
             }
-        }
-        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the slots are known
-        // The dot products are dealt out in groups of one, two or four columns j of one row of x (a group
-        // shares the row of x): group g belongs to CTA g mod grid.  A dot product's arithmetic is fixed, whoever
-        // computes it: 96 "virtual threads" (the three shrink warps) each sum the 8-column chunks m, m + 96,
-        // m + 192, ... of the row in order, each warp adds its threads' sums up with the butterfly, and the
-        // result is (w0 + w1) + w2 times the scale.  The operands of a whole group (up to six 16-byte chunks of x
-        // and of each row of A per thread and step: 4608 columns) are in flight at once, in registers, so a group costs
-        // one memory round trip per step.  (Groups staged in shared memory by asynchronous copies were measured slower:
-        // 1.1 us per call for pairs at 12 and 16 tokens, 0.6 - 2.3 us for groups of four.)  A result is published as one
-        // 64-bit store (value and this launch's mark) and a relaxed add on the grid-wide counter: nobody waits for a fence.
-        const int total = lk->dot_end[15];
-        // Group size: the smallest of 1, 2, 4 that gives every CTA at most one group (a group costs a memory
-        // round trip, but also (1 + size) x 8 KB through the load path of its CTA), else 4.
-        const int gsize = total <= ncta ? 1 : (total <= 2 * ncta ? 2 : kDecDotGroup);
-        const int ngroups = total / gsize;
-        const int me = tid - (kDecConsumers + 1) * 32;   // 0 .. 95
+            booked = true;
+        };
         // Brings the blocks of B into the staging buffer (16-byte asynchronous copies, all in flight at
         // once); blocks that did not fit are asked into L2 and read from there by the epilogue.
         auto stage_b = [&]() {
@@ -548,7 +559,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 }
             }
         };
-        stage_b();   // (the staging buffer is theirs alone: the dot products keep their operands in registers)
         // A single dot product per CTA (few tokens, rank 16: the usual decode call).
         auto single = [&](int d, int& t, int& j) {
             t = 0;
@@ -560,7 +570,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j) * K;
                 constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
                 float dot = 0.f;
-                for (int kb = me * 8; kb < K; kb += kPer * kStride) {
+                for (int kb = me * 8, step = 0; step == 0 || kb < K; kb += kPer * kStride, ++step) {   // (every thread takes the first step: see book_once)
                     uint4 xv[kPer], av[kPer];
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
@@ -569,6 +579,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                         xv[i] = ok_k ? ldg_nc_v4(xr + k0) : make_uint4(0, 0, 0, 0);
                         av[i] = ok_k ? ldg_nc_v4(ar + k0) : make_uint4(0, 0, 0, 0);
                     }
+                    book_once();   // (while the loads are on their way)
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
                         if (kb + i * kStride < K) {
@@ -606,7 +617,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 const __nv_bfloat16* xr = x + (size_t)t * K;
                 const __nv_bfloat16* ar = arenaA + ((size_t)ctrl->slot_of_row[t] * kRankPad + j0) * K;
                 constexpr int kPer = 6, kStride = kDecShrinkWarps * 32 * 8;
-                for (int kb = me * 8; kb < K; kb += kPer * kStride) {
+                for (int kb = me * 8, step = 0; step == 0 || kb < K; kb += kPer * kStride, ++step) {   // (every thread takes the first step: see book_once)
                     uint4 xv[kPer], av[NG][kPer];
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
@@ -617,6 +628,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                         for (int d = 0; d < NG; ++d)
                             av[d][i] = ok_k && d < nreal ? ldg_nc_v4(ar + (size_t)d * K + k0) : make_uint4(0, 0, 0, 0);
                     }
+                    book_once();   // (while the loads are on their way)
 #pragma unroll
                     for (int i = 0; i < kPer; ++i) {
                         if (kb + i * kStride < K) {
@@ -670,6 +682,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
                 red_relaxed_gpu_add(sync_words + 2, (unsigned)gsize);
             }
         }
+        book_once();   // (a CTA without a dot product of its own, or whose group had only padding columns)
+        asm volatile("bar.sync 2, %0;" ::"n"(kDecShrinkWarps * 32) : "memory");   // the blocks of B are placed
+        stage_b();     // the chunk-by-chunk copies (ranks above 16); the staging buffer is theirs alone
         // Collect all of u in shared memory for the consumers' epilogue, off their critical path.  The
         // other CTAs' shares normally arrive within microseconds and are then read from global memory.
         // But this CTA never depends on them: nothing guarantees that the whole grid is resident at once
