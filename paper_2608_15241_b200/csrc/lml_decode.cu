@@ -98,15 +98,22 @@ constexpr int kDecCtrlBytes = 320;
 // A call without any adapter (G == 0) has no use for the staging buffer of B and takes a fifth ring stage instead: the
 // deeper ring is worth 0.5 us on a 4096 x 4096 layer (8.24 -> 7.73 us).  With adapters a fifth stage loses (8.63 against
 // 8.39 us even where the blocks of B still fit): the shrink warps' cold loads queue up behind whatever the ring has asked for.
-template <bool kBase> struct DecCfg {
-    static constexpr int kStages = kBase ? kDecStagesBase : kDecStages;
-    static constexpr int kDotBytes = kBase ? 0 : kDecDotBytes;
+// The third build lies between the two: five stages and what is left of the carve-out, 10.5 KB, as staging buffer, for
+// calls whose blocks of B are sure to fit in that (few tokens or few rows per CTA; the launcher works out the worst
+// case from the table's ranks): 8.20 -> 8.07 us on decode_q_proj.  Where the blocks do not fit, the fifth stage costs
+// more than it brings (9.4 -> 10.4 us at 16 tokens and 11 slots), hence the choice per call.
+constexpr int kDecVarFull = 0, kDecVarBase = 1, kDecVarSmall = 2;
+constexpr int kDecDotBytesSmall = 10496;
+template <int kVar> struct DecCfg {
+    static constexpr int kStages = kVar == kDecVarFull ? kDecStages : kDecStagesBase;
+    static constexpr int kDotBytes = kVar == kDecVarFull ? kDecDotBytes : (kVar == kDecVarBase ? 0 : kDecDotBytesSmall);
     static constexpr int kSmemBytes = 128 + kStages * kDecStageBytes + kDecSlotBytes + kDecUBytes + kDecCtrlBytes + kDecSegBytes + 8 + kDotBytes + kDecDeferBytes;
 };
-constexpr int kDecSmemBytes = DecCfg<false>::kSmemBytes;
+constexpr int kDecSmemBytes = DecCfg<kDecVarFull>::kSmemBytes;
 // 196 KB is also the largest shared-memory carve-out that leaves the SM a useful L1 for the loads of x:
 // one step more and the base-only call is 0.8 us slower.
-static_assert(kDecSmemBytes + 1024 <= 200704 && DecCfg<true>::kSmemBytes + 1024 <= 200704, "shared memory budget");   // the system keeps 1 KB per CTA for itself
+static_assert(kDecSmemBytes + 1024 <= 200704 && DecCfg<kDecVarBase>::kSmemBytes + 1024 <= 200704 &&
+              DecCfg<kDecVarSmall>::kSmemBytes + 1024 <= 200704 && kDecDotBytesSmall % 16 == 0, "shared memory budget");   // the system keeps 1 KB per CTA for itself
 
 struct DecCtrl {
     uint64_t full[kDecStagesBase];
@@ -159,7 +166,7 @@ template <int kP> struct DecLaunch {
     int T, K, P, patience;
 };
 
-template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1, bool kBase = false>
+template <bool kTwo, bool kMulti, bool kPutOff, int kP = 1, int kVar = kDecVarFull>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __grid_constant__ DecLaunch<kP> prm)
 {
     int pi = 0;
@@ -181,7 +188,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_main_kernel(const __gri
     const int32_t* __restrict__ token_slots = pj.token_slots;
     const int32_t* __restrict__ adapter_map = pj.adapter_map;
     uint32_t* status = pj.status;
-    constexpr int kS = DecCfg<kBase>::kStages, kDotBytes = DecCfg<kBase>::kDotBytes;
+    constexpr bool kBase = kVar == kDecVarBase;
+    constexpr int kS = DecCfg<kVar>::kStages, kDotBytes = DecCfg<kVar>::kDotBytes;
     const int T = kP == 1 ? prm.T : pj.T, K = prm.K, N = pj.N, G = kBase ? 0 : pj.G, patience = prm.patience;
     extern __shared__ uint8_t dec_smem_raw[];
     const uint32_t raw = smem_u32(dec_smem_raw);
@@ -993,10 +1001,15 @@ cudaError_t decode_init()
     set(decode_main_kernel<false, false, false, kDecMaxProj>); set(decode_main_kernel<false, true, false, kDecMaxProj>); set(decode_main_kernel<false, true, true, kDecMaxProj>);
     set(decode_main_kernel<true, false, false, kDecMaxProj>);  set(decode_main_kernel<true, true, false, kDecMaxProj>);  set(decode_main_kernel<true, true, true, kDecMaxProj>);
     auto set_base = [&](auto kernel) {
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<true>::kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<kDecVarBase>::kSmemBytes);
     };
-    set_base(decode_main_kernel<false, false, false, 1, true>); set_base(decode_main_kernel<false, true, false, 1, true>);
-    set_base(decode_main_kernel<true, false, false, 1, true>);  set_base(decode_main_kernel<true, true, false, 1, true>);
+    set_base(decode_main_kernel<false, false, false, 1, kDecVarBase>); set_base(decode_main_kernel<false, true, false, 1, kDecVarBase>);
+    set_base(decode_main_kernel<true, false, false, 1, kDecVarBase>);  set_base(decode_main_kernel<true, true, false, 1, kDecVarBase>);
+    auto set_small = [&](auto kernel) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<kDecVarSmall>::kSmemBytes);
+    };
+    set_small(decode_main_kernel<false, false, false, 1, kDecVarSmall>); set_small(decode_main_kernel<false, true, true, 1, kDecVarSmall>);
+    set_small(decode_main_kernel<true, false, false, 1, kDecVarSmall>);  set_small(decode_main_kernel<true, true, true, 1, kDecVarSmall>);
     return e;
 }
 
@@ -1027,7 +1040,8 @@ void fill_proj(DecProj& pj, const Arena& ar, const DecodeArgs& a)
 // several rounds (x is kept between rounds), and with several rounds and adapters (the expand of early rounds is put
 // off until u has arrived).
 template <int kP>
-cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_cta, bool adapters, int max_T, cudaStream_t stream)
+cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_cta, bool adapters, int max_T, cudaStream_t stream,
+                               bool small_blocks = false)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -1044,9 +1058,14 @@ cudaError_t launch_decode_grid(const DecLaunch<kP>& prm, int grid, int rows_per_
     auto launch = [&](auto kernel) { return cudaLaunchKernelEx(&cfg, kernel, prm); };
     if constexpr (kP == 1) {
         if (!adapters) {   // no adapter anywhere in the call: the build with the deeper ring and no staging buffer
-            cfg.dynamicSmemBytes = DecCfg<true>::kSmemBytes;
-            if (max_T > 8) return multi ? launch(decode_main_kernel<true, true, false, 1, true>) : launch(decode_main_kernel<true, false, false, 1, true>);
-            return multi ? launch(decode_main_kernel<false, true, false, 1, true>) : launch(decode_main_kernel<false, false, false, 1, true>);
+            cfg.dynamicSmemBytes = DecCfg<kDecVarBase>::kSmemBytes;
+            if (max_T > 8) return multi ? launch(decode_main_kernel<true, true, false, 1, kDecVarBase>) : launch(decode_main_kernel<true, false, false, 1, kDecVarBase>);
+            return multi ? launch(decode_main_kernel<false, true, false, 1, kDecVarBase>) : launch(decode_main_kernel<false, false, false, 1, kDecVarBase>);
+        }
+        if (small_blocks) {   // the blocks of B are sure to fit in the small staging buffer: the build with the deeper ring
+            cfg.dynamicSmemBytes = DecCfg<kDecVarSmall>::kSmemBytes;
+            if (max_T > 8) return multi ? launch(decode_main_kernel<true, true, true, 1, kDecVarSmall>) : launch(decode_main_kernel<true, false, false, 1, kDecVarSmall>);
+            return multi ? launch(decode_main_kernel<false, true, true, 1, kDecVarSmall>) : launch(decode_main_kernel<false, false, false, 1, kDecVarSmall>);
         }
     }
     if (max_T > 8)
@@ -1070,7 +1089,20 @@ cudaError_t launch_decode(const Arena& ar, const SlotSnapshot& snap, const Decod
     prm.proj[0].cta_begin = 0; prm.proj[0].cta_count = grid;
     prm.x = (const __nv_bfloat16*)a.x;
     prm.T = a.T; prm.K = a.d_in; prm.P = 1; prm.patience = g_dec_patience;
-    const cudaError_t e = launch_decode_grid<1>(prm, grid, (a.d_out + grid - 1) / grid, a.G > 0, a.T, stream);
+    // Worst case of what the expand's copies of B take per CTA: a block per distinct slot (at most one per token, and no
+    // more than the table has live), the widest block that any live slot can have.
+    const int rows_per_cta = (a.d_out + grid - 1) / grid;
+    int live = 0, widest = 0;
+    for (int sl = 0; sl < snap.max_slots && sl < kMaxSlots; ++sl) {
+        const int r = snap.rank[sl];
+        if (r == 0) continue;
+        ++live;
+        const int per_row = r <= kRankCompact ? kRankCompact * 2 : ((r + 7) >> 3) * 16;
+        widest = per_row > widest ? per_row : widest;
+    }
+    const int blocks = a.T < live ? a.T : live;
+    const bool small_blocks = a.G > 0 && (long long)blocks * rows_per_cta * widest <= kDecDotBytesSmall;
+    const cudaError_t e = launch_decode_grid<1>(prm, grid, rows_per_cta, a.G > 0, a.T, stream, small_blocks);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
